@@ -1,0 +1,165 @@
+"""Pins of the oracle's reduction evaluator (O2): special cases with a plain definition."""
+import numpy as np
+import pytest
+
+from oracle import rd_oracle as O
+
+f32 = np.float32
+
+
+def schedules(p, sizes, A=3, B=1, G=1):
+    """Every tree schedule for (p, sizes) as (name, events)."""
+    out = [("uni", O.uni_greedy(p, sizes, A, B, G)[0]),
+           ("pipe", O.pipeline(p, sizes, A, B, G, False)[0]),
+           ("binary", O.binary(p, sizes, A, B, G, True)[0]),
+           ("binomial", O.binomial(p, sizes, A, B, G)[0])]
+    if p >= 2:
+        out.append(("bi", O.bi_greedy(p, sizes, A, B, G)[0]))
+    return out
+
+
+def seg_off(sizes):
+    return np.concatenate([[0], np.cumsum(sizes)])
+
+
+@pytest.mark.parametrize("p", [2, 3, 8, 13, 64])
+def test_integer_results_do_not_depend_on_the_order(p):
+    rng = np.random.default_rng(p)
+    sizes = [5, 5, 5, 2]
+    n = sum(sizes)
+    x = rng.integers(-2**31, 2**31, size=(p, n), dtype=np.int64).astype(np.int32)   # wraps on purpose
+    want_sum = x.astype(np.int64).sum(axis=0).astype(np.uint64).astype(np.uint32).view(np.int32) \
+        if False else (x.astype(np.int64).sum(axis=0) & 0xFFFFFFFF).astype(np.uint32).view(np.int32)
+    want_max = x.max(axis=0)
+    for name, ev in schedules(p, sizes):
+        assert (O.reduce(ev, x, seg_off(sizes), "sum") == want_sum).all(), name
+        assert (O.reduce(ev, x, seg_off(sizes), "max") == want_max).all(), name
+    if p & (p - 1) == 0:
+        ev, off, _ = O.butterfly(p, n, 4, 3, 1, 1)
+        assert (O.reduce(ev, x, off, "sum") == want_sum).all()
+        assert (O.reduce(ev, x, off, "max") == want_max).all()
+
+
+@pytest.mark.parametrize("p", [2, 5, 16, 33])
+def test_fp32_max_is_the_maximum(p):
+    rng = np.random.default_rng(100 + p)
+    sizes = [7, 7, 3]
+    x = rng.standard_normal((p, 17)).astype(f32)
+    for name, ev in schedules(p, sizes):
+        assert (O.reduce(ev, x, seg_off(sizes), "max") == x.max(axis=0)).all(), name
+
+
+def test_fp32_max_keeps_the_held_value_on_ties():
+    """incoming > held ? incoming : held -- with +0 and -0 the held one survives."""
+    x = np.array([[0.0], [-0.0]], dtype=f32)           # root holds +0, receives -0
+    ev, _ = O.uni_greedy(2, [1], 1, 1, 1)
+    assert np.signbit(O.reduce(ev, x, [0, 1], "max"))[0] == False
+    x = np.array([[-0.0], [0.0]], dtype=f32)           # root holds -0, receives +0: not greater
+    assert np.signbit(O.reduce(ev, x, [0, 1], "max"))[0] == True
+
+
+def test_fp32_sum_two_processes_is_one_add():
+    rng = np.random.default_rng(7)
+    x = (rng.standard_normal((2, 1000)) * 10.0 ** rng.integers(-8, 8, size=(2, 1000))).astype(f32)
+    ev, _ = O.uni_greedy(2, [600, 400], 1, 1, 1)
+    assert (O.reduce(ev, x, [0, 600, 1000], "sum") == x[0] + x[1]).all()
+
+
+@pytest.mark.parametrize("p", [3, 4, 9, 32])
+def test_fp32_sum_pipeline_is_a_running_sum_from_the_far_end(p):
+    """Process k combines what it holds with what k+1 sends: x_0 + (x_1 + (... + x_{p-1}))."""
+    rng = np.random.default_rng(p)
+    x = (rng.standard_normal((p, 64)) * 10.0 ** rng.integers(-4, 5, size=(p, 64))).astype(f32)
+    want = x[p - 1].copy()
+    for k in range(p - 2, -1, -1):
+        want = (x[k] + want).astype(f32)
+    for bidir in (False, True):
+        ev, _ = O.pipeline(p, [16] * 4, 2, 1, 1, bidir)
+        assert (O.reduce(ev, x, [0, 16, 32, 48, 64], "sum") == want).all()
+
+
+def test_fp32_sum_binomial_and_binary_association():
+    """Association order matters in fp32.  p = 4, each tree written out from its definition:
+    binomial  round 0: 1->0, 3->2; round 1: 2->0         =>  (x0 + x1) + (x2 + x3)
+    pipeline  3->2->1->0                                  =>  x0 + (x1 + (x2 + x3))
+    binary    heap order, left child first: 3->1, 1->0, 2->0  =>  (x0 + (x1 + x3)) + x2
+    and on inputs with a wide exponent range the three differ from each other."""
+    rng = np.random.default_rng(11)
+    n = 256
+    x = (rng.standard_normal((4, n)) * 10.0 ** rng.integers(-6, 7, size=(4, n))).astype(f32)
+    x0, x1, x2, x3 = x
+    forms = {
+        "binomial": ((x0 + x1).astype(f32) + (x2 + x3).astype(f32)).astype(f32),
+        "pipeline": (x0 + (x1 + (x2 + x3).astype(f32)).astype(f32)).astype(f32),
+        "binary": ((x0 + (x1 + x3).astype(f32)).astype(f32) + x2).astype(f32),
+    }
+    got = {
+        "binomial": O.reduce(O.binomial(4, [n], 1, 1, 1)[0], x, [0, n], "sum"),
+        "pipeline": O.reduce(O.pipeline(4, [n], 1, 1, 1, False)[0], x, [0, n], "sum"),
+        "binary": O.reduce(O.binary(4, [n], 1, 1, 1, False)[0], x, [0, n], "sum"),
+    }
+    for a in forms:
+        assert (got[a] == forms[a]).all(), a
+        for b in forms:
+            if a != b:
+                assert (got[a] != forms[b]).any(), (a, b)
+    # a hand-checkable instance: 2^24 + 1 + 1 + 1
+    big, one = f32(2.0 ** 24), f32(1.0)
+    y = np.array([[big], [one], [one], [one]], dtype=f32)
+    assert O.reduce(O.binomial(4, [1], 1, 1, 1)[0], y, [0, 1], "sum")[0] == f32(2.0 ** 24 + 2)   # (2^24+1 -> 2^24) + 2
+    assert O.reduce(O.pipeline(4, [1], 1, 1, 1, False)[0], y, [0, 1], "sum")[0] == f32(2.0 ** 24 + 4)  # 2^24 + 3 -> even
+
+
+def test_fp32_sum_butterfly_association():
+    """p = 4: chunk c is reduced by V(c) = (x_c + x_{c^2}) + (x_{c^1} + x_{c^3})."""
+    rng = np.random.default_rng(3)
+    n = 8
+    x = (rng.standard_normal((4, n)) * 10.0 ** rng.integers(-6, 7, size=(4, n))).astype(f32)
+    ev, off, _ = O.butterfly(4, n, 4, 1, 1, 1)
+    got = O.reduce(ev, x, off, "sum")
+    assert list(off) == [0, 2, 4, 6, 8]
+    for c in range(4):
+        sl = slice(off[c], off[c + 1])
+        want = (x[c, sl] + x[c ^ 2, sl]).astype(f32) + (x[c ^ 1, sl] + x[c ^ 3, sl]).astype(f32)
+        assert (got[sl] == want.astype(f32)).all()
+
+
+@pytest.mark.parametrize("p,dist", [(8, "normal"), (64, "normal"), (256, "uniform")])
+def test_fp32_sum_is_close_to_fp64(p, dist):
+    """Any association of p fp32 numbers is within (p-1) * 2^-24 * sum|x_i| of the exact sum."""
+    rng = np.random.default_rng(p)
+    sizes = [100, 100, 56]
+    n = 256
+    x = (rng.standard_normal((p, n)) if dist == "normal" else rng.uniform(-1, 1, (p, n))).astype(f32)
+    ref, mag = O.reference_f64(x, "sum")
+    assert np.allclose(ref, x.astype(np.float64).sum(axis=0), rtol=1e-13, atol=1e-13)
+    assert np.allclose(mag, np.abs(x.astype(np.float64)).sum(axis=0), rtol=1e-13)
+    for name, ev in schedules(p, sizes):
+        got = O.reduce(ev, x, seg_off(sizes), "sum").astype(np.float64)
+        assert (np.abs(got - ref) <= (p - 1) * 2.0 ** -24 * mag).all(), name
+        assert (np.abs(got - ref) <= 1e-5 * mag).all(), name
+
+
+def test_segments_use_their_own_trees():
+    """Uni-greedy builds a different tree per segment: replaying segment j's events on segment k's data
+    must in general change fp32 bits, while each segment alone matches a replay restricted to it."""
+    p, sizes = 16, [8, 8, 8, 8]
+    rng = np.random.default_rng(0)
+    x = (rng.standard_normal((p, 32)) * 10.0 ** rng.integers(-3, 4, size=(p, 32))).astype(f32)
+    ev, _ = O.uni_greedy(p, sizes, 2, 0, 1)
+    full = O.reduce(ev, x, seg_off(sizes), "sum")
+    for j in range(4):
+        only = ev[ev["seg"] == j].copy()
+        only["seg"] = 0
+        part = O.reduce(only, x[:, 8 * j:8 * j + 8].copy(), [0, 8], "sum")
+        assert (part == full[8 * j:8 * j + 8]).all()
+
+
+def test_empty_segments_and_single_process():
+    x = np.arange(12, dtype=np.int32).reshape(1, 12)
+    ev, _ = O.uni_greedy(1, [4, 8], 1, 1, 1)
+    assert len(ev) == 0
+    assert (O.reduce(ev, x, [0, 4, 12], "sum") == x[0]).all()
+    x = np.ones((4, 3), dtype=np.int32)
+    ev, off, _ = O.butterfly(4, 3, 4, 1, 1, 1)          # fewer elements than processes: empty chunks
+    assert (O.reduce(ev, x, off, "sum") == 4).all()
