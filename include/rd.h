@@ -1,0 +1,227 @@
+/*
+ * rd.h -- C ABI of the schedule-exact pipelined reduction library (librd.so).
+ *
+ * The library reduces the messages of p "processes" (p buffers of n 4-byte
+ * elements in the memory of ONE GPU) into a root buffer, combining entry-wise
+ * in exactly the order a reduction schedule fixes.  Schedules follow
+ * Lowery & Langou, "A Greedy Algorithm for Optimally Pipelining a Reduction":
+ * uni-greedy (Algorithm 1), bi-greedy (Algorithm 2), and the algorithms the
+ * paper compares them with: binomial, pipeline, binary tree (Section IV) and
+ * the reduce-scatter/gather butterfly (Section III).
+ *
+ * Conventions
+ *   - Every function returns RD_OK (0) or a negative rd_status_t; nothing
+ *     aborts, nothing throws across this boundary, and output arguments are
+ *     left untouched on failure.
+ *   - Processes are numbered 0..p-1 and the root is process 0 (the paper's
+ *     implementation makes the same restriction, Fig. 2 caption).
+ *   - Sizes called "bytes" are bytes; "elems" are 4-byte elements.
+ *   - "host" / "device" in a comment says where a pointer must point.
+ *   - Times of the linear model (Section II): a message of b bytes costs
+ *     alpha + beta*b, combining it costs gamma*b.  Internally time is an exact
+ *     integer count of `tick` seconds, so that equal times are decided the
+ *     same way everywhere: t_comm = round(alpha/tick) + round(beta/tick)*b,
+ *     t_comp = round(gamma/tick)*b.
+ *   - Thread safety: distinct schedules may be used from distinct threads.
+ *     One schedule may be used by one thread at a time.
+ */
+#ifndef RD_H_
+#define RD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define RD_API __attribute__((visibility("default")))
+#else
+#define RD_API
+#endif
+
+typedef struct rd_schedule rd_schedule_t; /* opaque; owns its host and device tables */
+
+typedef enum {
+    RD_OK = 0,
+    RD_ERR_INVALID_ARG = -1,   /* null pointer, p < 1, size not a multiple of 4, unknown enum, ...      */
+    RD_ERR_UNSUPPORTED = -2,   /* a combination the method does not define (see rd_schedule_create)     */
+    RD_ERR_NOMEM = -3,         /* host or device allocation failed                                      */
+    RD_ERR_CUDA = -4,          /* a CUDA runtime call failed (including: no device, no driver)          */
+    RD_ERR_TIMEOUT = -5,       /* a bounded wait inside the schedule-faithful kernel gave up            */
+    RD_ERR_SIZE_MISMATCH = -6, /* n_elems * 4 differs from the schedule's message size                  */
+    RD_ERR_INTERNAL = -7,      /* a generated schedule failed the library's own consistency check       */
+    RD_ERR_TOO_SMALL = -8      /* an output array passed by the caller is too short                     */
+} rd_status_t;
+
+typedef enum {
+    RD_UNI_GREEDY = 0, /* Algorithm 1; unidirectional ports only                                 */
+    RD_BI_GREEDY = 1,  /* Algorithm 2; bidirectional ports only                                  */
+    RD_BINOMIAL = 2,   /* Section IV; either port model                                          */
+    RD_PIPELINE = 3,   /* Section IV; either port model                                          */
+    RD_BINARY = 4,     /* Section IV; either port model                                          */
+    RD_BUTTERFLY = 5   /* Section III (reduce-scatter/gather); bidirectional, p a power of two   */
+} rd_algo_t;
+
+typedef enum { RD_PORT_UNI = 0, RD_PORT_BI = 1 } rd_port_t;   /* Section II */
+typedef enum { RD_SUM = 0, RD_MAX = 1 } rd_op_t;
+typedef enum { RD_INT32 = 0, RD_FP32 = 1 } rd_dtype_t;
+typedef enum { RD_EXEC_TREE = 0, RD_EXEC_FAITHFUL = 1 } rd_exec_t;
+
+/* Linear model of Section II.  alpha in seconds, beta and gamma in seconds per
+ * byte, tick = seconds per integer time unit (0 selects 1e-15).  alpha/tick,
+ * beta/tick and gamma/tick are rounded to the nearest integer.               */
+typedef struct { double alpha, beta, gamma, tick; } rd_model_t;
+
+/* One send/receive pair (Section V: reduce(X, S, a, b, t)): process src sends
+ * segment seg to process dst starting at tick t_start.  kind 0: dst combines
+ * what it holds (left operand) with what arrives; kind 1: dst only stores it
+ * (gather phase of the butterfly).  For the butterfly a "segment" is the final
+ * chunk of the message that one process owns after the reduce-scatter.        */
+typedef struct { int32_t seg, src, dst, kind; int64_t t_start; } rd_event_t;
+
+/* Filled by rd_reduce when requested.  Asking for it makes the call wait for
+ * the kernel.                                                                 */
+typedef struct {
+    double kernel_ms;      /* device time of the kernel(s), CUDA events                       */
+    double gbytes_per_s;   /* (p*m + m) bytes / kernel time, in 1e9 bytes per second          */
+    double makespan_ns;    /* faithful mode: first action start to the root's last combine    */
+    double predicted_s;    /* the schedule's completion time under the linear model           */
+    uint64_t bytes_moved;  /* p*m + m                                                         */
+    int32_t device_status; /* faithful mode: 0, or RD_ERR_TIMEOUT                             */
+    int32_t n_launches;    /* kernels launched by this call                                   */
+} rd_stats_t;
+
+/*
+ * rd_schedule_create -- Sections II, IV, V (Algorithm 1), VI (Algorithm 2), III.
+ * Generates the schedule for p processes and a message of msg_bytes per
+ * process, cut into equal segments of seg_bytes with a possibly smaller last
+ * one (Section II), and compiles it into per-segment combine programs.  Host
+ * work only: no CUDA call is made, so it works without a GPU.
+ *   out        host; receives the new schedule; release with rd_destroy.
+ *   algo/port  legal pairs: uni-greedy + UNI; bi-greedy + BI; butterfly + BI;
+ *              binomial, pipeline, binary + either.  Others: RD_ERR_UNSUPPORTED.
+ *   p          1..4096.  Butterfly: a power of two, else RD_ERR_UNSUPPORTED.
+ *   msg_bytes  multiple of 4; may be 0.
+ *   seg_bytes  multiple of 4, 0 < seg_bytes; values above msg_bytes mean one
+ *              segment.  0 selects the segment size rd_optimal_segment gives.
+ *              Ignored by the butterfly, which halves the message instead.
+ *              Binomial: the paper uses one segment (seg_bytes = 0 gives
+ *              that); several segments are reduced one after the other, each
+ *              by the same tree.
+ *   model      host; must not be NULL.
+ */
+RD_API int rd_schedule_create(rd_schedule_t **out, rd_algo_t algo, rd_port_t port, int p,
+                       size_t msg_bytes, size_t seg_bytes, const rd_model_t *model);
+
+/*
+ * rd_schedule_create_segments -- Section VIII (unequal segmentation).
+ * As rd_schedule_create, with the q segment sizes given one by one (each a
+ * positive multiple of 4 bytes; their sum is the message size).  Algorithm 1
+ * is defined for any segmentation; the lock-step algorithms use the largest
+ * segment as their round length.  Not available for the butterfly.
+ *   seg_bytes  host array of q sizes.
+ */
+RD_API int rd_schedule_create_segments(rd_schedule_t **out, rd_algo_t algo, rd_port_t port, int p,
+                                const size_t *seg_bytes, size_t q, const rd_model_t *model);
+
+/*
+ * rd_optimal_segment -- Table I and Table III (s_opt rows), Section VII.
+ * The equal segment size, in bytes (multiple of 4, 4 <= s <= msg_bytes), that
+ * minimises the schedule's completion time under `model`: the closed forms of
+ * the tables for pipeline, binary and bi-greedy (the better of the two
+ * integer segment counts around the real optimum; the whole message when the
+ * formula's denominator is not positive), the whole message for binomial, a
+ * search over powers of two for uni-greedy (the paper's tuning protocol), and
+ * the whole message for the butterfly (it ignores the value).
+ */
+RD_API int rd_optimal_segment(rd_algo_t algo, rd_port_t port, int p, size_t msg_bytes,
+                       const rd_model_t *model, size_t *seg_bytes_out);
+
+/* rd_schedule_info -- Section V: the completion time is the final state of the
+ * root.  Any output pointer may be NULL.  q is the number of segments (for the
+ * butterfly: p chunks), n_events the number of send/receive pairs
+ * ((p-1)*q for the tree schedules), predicted_ticks / predicted_seconds the
+ * completion time under the model, stack_depth the number of partial results
+ * the combine programs keep besides the running one.                          */
+RD_API int rd_schedule_info(const rd_schedule_t *s, int *p, size_t *q, size_t *n_events,
+                     double *predicted_seconds, int64_t *predicted_ticks, int *stack_depth);
+
+/* rd_schedule_events -- copies the n_events pairs into buf (host, capacity cap
+ * entries) ordered by (t_start, seg, src, dst).  RD_ERR_TOO_SMALL if cap is
+ * too small.                                                                  */
+RD_API int rd_schedule_events(const rd_schedule_t *s, rd_event_t *buf, size_t cap);
+
+/* rd_schedule_segments -- writes the q+1 segment boundaries in elements into
+ * off (host, capacity cap entries): segment j is elements [off[j], off[j+1]). */
+RD_API int rd_schedule_segments(const rd_schedule_t *s, uint64_t *off, size_t cap);
+
+/*
+ * rd_schedule_program -- the compiled combine program of one segment (what the
+ * tree kernel interprets), for inspection and for checking it on the host.
+ * Writes its p operations to ops (host, capacity cap) and returns RD_OK, or
+ * RD_ERR_TOO_SMALL.  An operation is a 32-bit word:
+ *   bits  0-11  process whose element is loaded
+ *   bits 12-13  0 LOAD      top = x
+ *               1 PUSH_LOAD push top; top = x
+ *               2 ACC_IN    top = combine(held = top, incoming = x)
+ *               3 ACC_HELD  top = combine(held = x,   incoming = top)
+ *   bits 14-17  npop: number of pops that follow
+ *   bits 18-29  bit k = role of the k-th pop: 1: top = combine(held = popped, incoming = top)
+ *                                              0: top = combine(held = top, incoming = popped)
+ * combine(held, incoming) = held + incoming, or incoming > held ? incoming : held.
+ * After the last operation top is the root's value (Section IV: the receiver
+ * combines its segment with the one received).
+ */
+RD_API int rd_schedule_program(const rd_schedule_t *s, size_t seg, uint32_t *ops, size_t cap);
+
+/*
+ * rd_reduce -- the reduction itself (Section III "Reduce"; Section IV).
+ *   d_inputs  HOST array of p DEVICE pointers; d_inputs[i] is process i's
+ *             message of n_elems elements.  Never written.
+ *   d_out     DEVICE; n_elems elements; receives what the root holds at the
+ *             end.  May alias d_inputs[0] in tree mode only.
+ *   n_elems   must equal the schedule's msg_bytes / 4 (RD_ERR_SIZE_MISMATCH).
+ *   exec      RD_EXEC_TREE: one kernel evaluates, per element, the segment's
+ *             combine program in registers; asynchronous on cuda_stream.
+ *             RD_EXEC_FAITHFUL: a persistent kernel in which groups of thread
+ *             blocks play the processes and hand partial segments to each
+ *             other through device memory, action by action; the call waits
+ *             for it and reports its makespan.  Needs scratch memory, which
+ *             the schedule allocates on first use and keeps.
+ *   cuda_stream  a cudaStream_t (NULL = the legacy default stream).
+ *   stats     host, or NULL.
+ * The first call on a schedule uploads its tables to the current device
+ * (allocates device memory, synchronises); rd_schedule_upload does the same
+ * ahead of time.  Buffers must be 4-byte aligned; 16-byte aligned buffers and
+ * segment sizes that are multiples of 16 bytes take the 128-bit path.
+ */
+RD_API int rd_reduce(rd_schedule_t *s, const void *const *d_inputs, void *d_out, size_t n_elems,
+              rd_dtype_t dtype, rd_op_t op, rd_exec_t exec, void *cuda_stream, rd_stats_t *stats);
+
+/* rd_schedule_upload -- copies the schedule's tables to the current device now. */
+RD_API int rd_schedule_upload(rd_schedule_t *s);
+
+/*
+ * rd_reduce_host -- rd_reduce (tree mode) for messages that live in HOST memory.
+ *   h_inputs  HOST array of p HOST pointers (pinned memory makes the copies
+ *             asynchronous); h_out HOST, n_elems elements.
+ *   d_staging DEVICE; (p + 1) * n_elems elements of scratch owned by the
+ *             caller: the p messages are copied there, reduced, and the
+ *             result copied back.  The call returns after the result is in
+ *             h_out.
+ */
+RD_API int rd_reduce_host(rd_schedule_t *s, const void *const *h_inputs, void *h_out, void *d_staging,
+                   size_t n_elems, rd_dtype_t dtype, rd_op_t op, void *cuda_stream);
+
+/* rd_destroy -- frees the schedule and its device tables.  NULL is allowed. */
+RD_API void rd_destroy(rd_schedule_t *s);
+
+/* rd_strerror -- static, never NULL. */
+RD_API const char *rd_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RD_H_ */

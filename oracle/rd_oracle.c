@@ -132,7 +132,8 @@ int orc_uni_greedy(int p, int q, const int64_t *sizes, int64_t A, int64_t B, int
 int orc_bi_greedy(int p, int q, const int64_t *sizes, int64_t A, int64_t B, int64_t G,
                   int unit_step, orc_event_t *events, int64_t *completion)
 {
-    if (p < 2 || q < 1 || !sizes) return ORC_BAD_ARG;
+    if (p < 1 || q < 1 || !sizes) return ORC_BAD_ARG;
+    if (p == 1) { if (completion) *completion = 0; return ORC_OK; }   /* nothing to send */
     int64_t *S = calloc((size_t)p, 8), *R = calloc((size_t)p, 8);
     int64_t *C1 = calloc((size_t)p, 8), *C2 = calloc((size_t)p, 8);
     int64_t *M = calloc((size_t)p * (size_t)q, 8);
@@ -255,9 +256,16 @@ done:
 
 /* ------------------------------------------------------------------------- */
 /* The three standard algorithms of Section IV as lock-step rounds of length */
-/* alpha + beta*s + gamma*s (s = sizes[0], the full segment size), which is  */
-/* how Tables I and III count them.  bidir = 0: unidirectional ports.        */
+/* alpha + beta*s + gamma*s (s = the largest segment, i.e. the full segment  */
+/* size of an equi-segmentation), which is how Tables I and III count them.  */
+/* bidir = 0: unidirectional ports.                                          */
 /* ------------------------------------------------------------------------- */
+static int64_t round_length(int q, const int64_t *sizes, int64_t A, int64_t B, int64_t G)
+{
+    int64_t s = 0;
+    for (int j = 0; j < q; j++) if (sizes[j] > s) s = sizes[j];
+    return t_comm(A, B, s) + t_comp(G, s);
+}
 
 /* Binomial: with n processes left, floor(n/2) send and floor(n/2) receive,
  * ceil(n/2) remain.  Round r: every k with k mod 2^(r+1) = 2^r sends to
@@ -269,7 +277,7 @@ int orc_binomial(int p, int q, const int64_t *sizes, int64_t A, int64_t B, int64
 {
     if (p < 1 || q < 1 || !sizes) return ORC_BAD_ARG;
     int L = orc_ceil_log2(p);
-    int64_t round_len = t_comm(A, B, sizes[0]) + t_comp(G, sizes[0]);
+    int64_t round_len = round_length(q, sizes, A, B, G);
     size_t ne = 0;
     for (int j = 0; j < q; j++) {
         for (int r = 0; r < L; r++) {
@@ -294,7 +302,7 @@ int orc_pipeline(int p, int q, const int64_t *sizes, int64_t A, int64_t B, int64
                  orc_event_t *events, int64_t *completion)
 {
     if (p < 1 || q < 1 || !sizes) return ORC_BAD_ARG;
-    int64_t round_len = t_comm(A, B, sizes[0]) + t_comp(G, sizes[0]);
+    int64_t round_len = round_length(q, sizes, A, B, G);
     int stride = bidir ? 1 : 2;
     size_t ne = 0;
     for (int i = 0; i < q; i++) {
@@ -322,7 +330,7 @@ int orc_binary(int p, int q, const int64_t *sizes, int64_t A, int64_t B, int64_t
 {
     if (p < 1 || q < 1 || !sizes) return ORC_BAD_ARG;
     int D = orc_ceil_log2((int64_t)p + 1) - 1;
-    int64_t round_len = t_comm(A, B, sizes[0]) + t_comp(G, sizes[0]);
+    int64_t round_len = round_length(q, sizes, A, B, G);
     int stride = bidir ? 2 : 4;
     size_t ne = 0;
     int64_t rounds = 0;

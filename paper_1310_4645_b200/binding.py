@@ -1,0 +1,211 @@
+"""Thin ctypes binding of librd.so: the same names as include/rd.h, argument marshalling only.
+
+Nothing is computed here.  When the shared library is missing (not built) every call fails with
+an ImportError-derived exception: there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "librd.so")
+
+RD_OK = 0
+RD_ERR_INVALID_ARG, RD_ERR_UNSUPPORTED, RD_ERR_NOMEM, RD_ERR_CUDA = -1, -2, -3, -4
+RD_ERR_TIMEOUT, RD_ERR_SIZE_MISMATCH, RD_ERR_INTERNAL, RD_ERR_TOO_SMALL = -5, -6, -7, -8
+RD_UNI_GREEDY, RD_BI_GREEDY, RD_BINOMIAL, RD_PIPELINE, RD_BINARY, RD_BUTTERFLY = range(6)
+RD_PORT_UNI, RD_PORT_BI = 0, 1
+RD_SUM, RD_MAX = 0, 1
+RD_INT32, RD_FP32 = 0, 1
+RD_EXEC_TREE, RD_EXEC_FAITHFUL = 0, 1
+
+ALGOS = {"uni_greedy": RD_UNI_GREEDY, "bi_greedy": RD_BI_GREEDY, "binomial": RD_BINOMIAL,
+         "pipeline": RD_PIPELINE, "binary": RD_BINARY, "butterfly": RD_BUTTERFLY}
+
+EXPORTS = ("rd_schedule_create", "rd_schedule_create_segments", "rd_optimal_segment", "rd_schedule_info",
+           "rd_schedule_events", "rd_schedule_segments", "rd_schedule_program", "rd_reduce",
+           "rd_schedule_upload", "rd_reduce_host", "rd_destroy", "rd_strerror")
+
+
+class rd_model_t(C.Structure):
+    _fields_ = [("alpha", C.c_double), ("beta", C.c_double), ("gamma", C.c_double), ("tick", C.c_double)]
+
+
+class rd_stats_t(C.Structure):
+    _fields_ = [("kernel_ms", C.c_double), ("gbytes_per_s", C.c_double), ("makespan_ns", C.c_double),
+                ("predicted_s", C.c_double), ("bytes_moved", C.c_uint64), ("device_status", C.c_int32),
+                ("n_launches", C.c_int32)]
+
+
+EVENT_DTYPE = np.dtype(
+    [("seg", "<i4"), ("src", "<i4"), ("dst", "<i4"), ("kind", "<i4"), ("t_start", "<i8")], align=True)
+
+
+class RdError(RuntimeError):
+    def __init__(self, status, what):
+        self.status = status
+        super().__init__("%s: %s (%d)" % (what, rd_strerror(status), status))
+
+
+class LibraryMissing(ImportError):
+    pass
+
+
+_lib = None
+
+
+def lib():
+    """The loaded library.  Raises LibraryMissing when librd.so has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise LibraryMissing("librd.so not found at %s: build it with `python -m paper_1310_4645_b200.build`"
+                                 % LIB_PATH)
+        L = C.CDLL(LIB_PATH)
+        vp, sz, i32 = C.c_void_p, C.c_size_t, C.c_int
+        L.rd_schedule_create.argtypes = [C.POINTER(vp), i32, i32, i32, sz, sz, C.POINTER(rd_model_t)]
+        L.rd_schedule_create_segments.argtypes = [C.POINTER(vp), i32, i32, i32, C.POINTER(sz), sz, C.POINTER(rd_model_t)]
+        L.rd_optimal_segment.argtypes = [i32, i32, i32, sz, C.POINTER(rd_model_t), C.POINTER(sz)]
+        L.rd_schedule_info.argtypes = [vp, C.POINTER(i32), C.POINTER(sz), C.POINTER(sz), C.POINTER(C.c_double),
+                                       C.POINTER(C.c_int64), C.POINTER(i32)]
+        L.rd_schedule_events.argtypes = [vp, vp, sz]
+        L.rd_schedule_segments.argtypes = [vp, vp, sz]
+        L.rd_schedule_program.argtypes = [vp, sz, vp, sz]
+        L.rd_reduce.argtypes = [vp, C.POINTER(vp), vp, sz, i32, i32, i32, vp, C.POINTER(rd_stats_t)]
+        L.rd_schedule_upload.argtypes = [vp]
+        L.rd_reduce_host.argtypes = [vp, C.POINTER(vp), vp, vp, sz, i32, i32, vp]
+        L.rd_destroy.argtypes = [vp]
+        L.rd_destroy.restype = None
+        L.rd_strerror.argtypes = [i32]
+        L.rd_strerror.restype = C.c_char_p
+        for name in EXPORTS:
+            if name not in ("rd_destroy", "rd_strerror"):
+                getattr(L, name).restype = i32
+        _lib = L
+    return _lib
+
+
+def rd_strerror(status: int) -> str:
+    return lib().rd_strerror(int(status)).decode()
+
+
+def _check(status, what):
+    if status != RD_OK:
+        raise RdError(status, what)
+
+
+def _model(alpha, beta, gamma, tick=0.0):
+    return rd_model_t(float(alpha), float(beta), float(gamma), float(tick))
+
+
+def rd_schedule_create(algo, port, p, msg_bytes, seg_bytes, alpha, beta, gamma, tick=0.0):
+    """Returns an opaque schedule handle (int).  Release with rd_destroy."""
+    h = C.c_void_p()
+    m = _model(alpha, beta, gamma, tick)
+    _check(lib().rd_schedule_create(C.byref(h), int(algo), int(port), int(p), int(msg_bytes), int(seg_bytes),
+                                    C.byref(m)), "rd_schedule_create")
+    return h.value
+
+
+def rd_schedule_create_segments(algo, port, p, seg_bytes, alpha, beta, gamma, tick=0.0):
+    h = C.c_void_p()
+    m = _model(alpha, beta, gamma, tick)
+    arr = (C.c_size_t * len(seg_bytes))(*[int(s) for s in seg_bytes])
+    _check(lib().rd_schedule_create_segments(C.byref(h), int(algo), int(port), int(p), arr, len(seg_bytes),
+                                             C.byref(m)), "rd_schedule_create_segments")
+    return h.value
+
+
+def rd_optimal_segment(algo, port, p, msg_bytes, alpha, beta, gamma, tick=0.0) -> int:
+    out = C.c_size_t(0)
+    m = _model(alpha, beta, gamma, tick)
+    _check(lib().rd_optimal_segment(int(algo), int(port), int(p), int(msg_bytes), C.byref(m), C.byref(out)),
+           "rd_optimal_segment")
+    return out.value
+
+
+def rd_schedule_info(h) -> dict:
+    p, q, ne, sec, ticks, depth = C.c_int(), C.c_size_t(), C.c_size_t(), C.c_double(), C.c_int64(), C.c_int()
+    _check(lib().rd_schedule_info(h, C.byref(p), C.byref(q), C.byref(ne), C.byref(sec), C.byref(ticks),
+                                  C.byref(depth)), "rd_schedule_info")
+    return dict(p=p.value, q=q.value, n_events=ne.value, predicted_seconds=sec.value,
+                predicted_ticks=ticks.value, stack_depth=depth.value)
+
+
+def rd_schedule_events(h) -> np.ndarray:
+    n = rd_schedule_info(h)["n_events"]
+    ev = np.zeros(n, dtype=EVENT_DTYPE)
+    _check(lib().rd_schedule_events(h, ev.ctypes.data, n), "rd_schedule_events")
+    return ev
+
+
+def rd_schedule_segments(h) -> np.ndarray:
+    q = rd_schedule_info(h)["q"]
+    off = np.zeros(q + 1, dtype=np.uint64)
+    _check(lib().rd_schedule_segments(h, off.ctypes.data, q + 1), "rd_schedule_segments")
+    return off
+
+
+def rd_schedule_program(h, seg) -> np.ndarray:
+    p = rd_schedule_info(h)["p"]
+    ops = np.zeros(p, dtype=np.uint32)
+    _check(lib().rd_schedule_program(h, int(seg), ops.ctypes.data, p), "rd_schedule_program")
+    return ops
+
+
+def rd_schedule_upload(h) -> None:
+    _check(lib().rd_schedule_upload(h), "rd_schedule_upload")
+
+
+def _dtype_code(t):
+    import torch
+    if t.dtype == torch.int32:
+        return RD_INT32
+    if t.dtype == torch.float32:
+        return RD_FP32
+    raise TypeError("int32 or float32 expected, got %s" % t.dtype)
+
+
+def rd_reduce(h, inputs, out, op, exec_mode=RD_EXEC_TREE, stream=None, want_stats=False):
+    """inputs: list of p CUDA tensors (or one [p, n] tensor); out: CUDA tensor of n elements.
+    stream: a torch.cuda.Stream (default: the current one).  Returns rd_stats_t or None."""
+    import torch
+    rows = [inputs[i] for i in range(len(inputs))]
+    n = out.numel()
+    for r in rows:
+        if not r.is_cuda or not r.is_contiguous() or r.numel() != n or r.dtype != out.dtype:
+            raise ValueError("every input must be a contiguous CUDA tensor with the output's dtype and length")
+    if not out.is_cuda or not out.is_contiguous():
+        raise ValueError("out must be a contiguous CUDA tensor")
+    ptrs = (C.c_void_p * len(rows))(*[r.data_ptr() for r in rows])
+    s = stream if stream is not None else torch.cuda.current_stream(out.device)
+    stats = rd_stats_t() if want_stats else None
+    with torch.cuda.device(out.device):
+        _check(lib().rd_reduce(h, ptrs, out.data_ptr(), n, _dtype_code(out), int(op), int(exec_mode),
+                               s.cuda_stream, C.byref(stats) if want_stats else None), "rd_reduce")
+    return stats
+
+
+def rd_reduce_host(h, inputs, out, staging, op, stream=None):
+    """inputs: list of p host tensors (pinned for asynchronous copies); out: host tensor;
+    staging: CUDA tensor of (p + 1) * n elements."""
+    import torch
+    rows = [inputs[i] for i in range(len(inputs))]
+    n = out.numel()
+    for r in rows:
+        if r.is_cuda or not r.is_contiguous() or r.numel() != n or r.dtype != out.dtype:
+            raise ValueError("every input must be a contiguous host tensor with the output's dtype and length")
+    if staging.numel() < (len(rows) + 1) * n or staging.dtype != out.dtype or not staging.is_cuda:
+        raise ValueError("staging must be a CUDA tensor of (p + 1) * n elements")
+    ptrs = (C.c_void_p * len(rows))(*[r.data_ptr() for r in rows])
+    s = stream if stream is not None else torch.cuda.current_stream(staging.device)
+    with torch.cuda.device(staging.device):
+        _check(lib().rd_reduce_host(h, ptrs, out.data_ptr(), staging.data_ptr(), n, _dtype_code(out), int(op),
+                                    s.cuda_stream), "rd_reduce_host")
+
+
+def rd_destroy(h) -> None:
+    lib().rd_destroy(h)

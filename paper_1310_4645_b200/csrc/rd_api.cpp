@@ -1,0 +1,400 @@
+// The C ABI (see include/rd.h): argument checking, schedule objects, device tables, launches.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <map>
+#include <new>
+#include <vector>
+
+#include "rd.h"
+#include "rd_internal.h"
+#include "rd_kernels.h"
+
+using namespace rd;
+
+namespace {
+
+constexpr int kPtrRing = 8;   // pointer tables in flight for p > kPackedPtrs
+
+struct DeviceTables {
+    int device = -1;
+    int sm_count = 0;
+    uint32_t *ops = nullptr;
+    std::map<int, std::pair<TileDesc *, uint32_t>> tiles;   // vector width -> (device table, count)
+    // pointer tables for large p: pinned host ring + device ring, one event per slot
+    void **h_ring = nullptr;
+    void **d_ring = nullptr;
+    cudaEvent_t ring_done[kPtrRing] = {};
+    int ring_next = 0;
+    cudaEvent_t ev_start = nullptr, ev_stop = nullptr;
+};
+
+}  // namespace
+
+struct rd_schedule {
+    rd_algo_t algo;
+    rd_port_t port;
+    int p;
+    size_t msg_bytes;
+    rd_model_t model;
+    Ticks ticks;
+    std::vector<int64_t> seg_bytes;
+    Schedule sched;
+    Programs progs;
+    DeviceTables dev;
+};
+
+namespace {
+
+int make_ticks(const rd_model_t *m, Ticks &t)
+{
+    if (!m) return RD_ERR_INVALID_ARG;
+    const double tick = m->tick > 0 ? m->tick : 1e-15;
+    if (!(m->alpha >= 0) || !(m->beta >= 0) || !(m->gamma >= 0) || !std::isfinite(tick)) return RD_ERR_INVALID_ARG;
+    const double a = m->alpha / tick, b = m->beta / tick, g = m->gamma / tick;
+    if (!(a < 4e18) || !(b < 4e18) || !(g < 4e18)) return RD_ERR_INVALID_ARG;
+    t.A = llround(a); t.B = llround(b); t.G = llround(g); t.tick = tick;
+    return RD_OK;
+}
+
+bool legal_pair(rd_algo_t algo, rd_port_t port)
+{
+    switch (algo) {
+    case RD_UNI_GREEDY: return port == RD_PORT_UNI;
+    case RD_BI_GREEDY: case RD_BUTTERFLY: return port == RD_PORT_BI;
+    case RD_BINOMIAL: case RD_PIPELINE: case RD_BINARY: return port == RD_PORT_UNI || port == RD_PORT_BI;
+    }
+    return false;
+}
+
+int build(rd_schedule_t **out, rd_algo_t algo, rd_port_t port, int p, std::vector<int64_t> seg_bytes,
+          size_t msg_bytes, const rd_model_t *model)
+{
+    if (!out || !model) return RD_ERR_INVALID_ARG;
+    if (int(algo) < 0 || int(algo) > RD_BUTTERFLY || (port != RD_PORT_UNI && port != RD_PORT_BI)) return RD_ERR_INVALID_ARG;
+    if (p < 1 || p > kMaxProcs) return RD_ERR_INVALID_ARG;
+    if (!legal_pair(algo, port)) return RD_ERR_UNSUPPORTED;
+    Ticks ticks;
+    if (int rc = make_ticks(model, ticks)) return rc;
+    // the largest time that can occur must stay far from int64 overflow
+    {
+        const long double worst = ((long double)ticks.A + ((long double)ticks.B + ticks.G) * (long double)msg_bytes) *
+                                  ((long double)p + 2.0L * (long double)(seg_bytes.size() + 1)) * 4.0L;
+        if (worst > 4.0e18L) return RD_ERR_INVALID_ARG;
+    }
+    rd_schedule *s = new (std::nothrow) rd_schedule();
+    if (!s) return RD_ERR_NOMEM;
+    int rc = RD_OK;
+    try {
+        s->algo = algo; s->port = port; s->p = p; s->msg_bytes = msg_bytes; s->model = *model; s->ticks = ticks;
+        s->seg_bytes = std::move(seg_bytes);
+        const bool bidir = port == RD_PORT_BI;
+        switch (algo) {
+        case RD_UNI_GREEDY: rc = gen_uni_greedy(p, s->seg_bytes, ticks, s->sched, true); break;
+        case RD_BI_GREEDY: rc = gen_bi_greedy(p, s->seg_bytes, ticks, s->sched, true); break;
+        case RD_BINOMIAL: rc = gen_binomial(p, s->seg_bytes, ticks, s->sched); break;
+        case RD_PIPELINE: rc = gen_pipeline(p, s->seg_bytes, ticks, bidir, s->sched); break;
+        case RD_BINARY: rc = gen_binary(p, s->seg_bytes, ticks, bidir, s->sched); break;
+        case RD_BUTTERFLY: rc = gen_butterfly(p, msg_bytes / 4, ticks, s->sched); break;
+        }
+        if (rc == RD_OK) rc = compile_programs(p, s->sched.seg_off.size() - 1, s->sched.events, s->progs);
+    } catch (const std::bad_alloc &) {
+        rc = RD_ERR_NOMEM;
+    }
+    if (rc != RD_OK) { delete s; return rc; }
+    *out = s;
+    return RD_OK;
+}
+
+void release_device(DeviceTables &d)
+{
+    if (d.device < 0) return;
+    int prev = -1;
+    cudaGetDevice(&prev);
+    cudaSetDevice(d.device);
+    cudaFree(d.ops);
+    for (auto &kv : d.tiles) cudaFree(kv.second.first);
+    if (d.h_ring) cudaFreeHost(d.h_ring);
+    cudaFree(d.d_ring);
+    for (auto &e : d.ring_done) if (e) cudaEventDestroy(e);
+    if (d.ev_start) cudaEventDestroy(d.ev_start);
+    if (d.ev_stop) cudaEventDestroy(d.ev_stop);
+    if (prev >= 0) cudaSetDevice(prev);
+    d = DeviceTables();
+}
+
+int upload(rd_schedule *s)
+{
+    DeviceTables &d = s->dev;
+    int cur = -1;
+    if (cudaGetDevice(&cur) != cudaSuccess) return RD_ERR_CUDA;
+    if (d.device == cur) return RD_OK;
+    if (d.device >= 0) release_device(d);
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, cur) != cudaSuccess) return RD_ERR_CUDA;
+    d.sm_count = prop.multiProcessorCount;
+    const size_t opBytes = std::max<size_t>(s->progs.ops.size(), 1) * sizeof(uint32_t);
+    if (cudaMalloc(reinterpret_cast<void **>(&d.ops), opBytes) != cudaSuccess) return RD_ERR_NOMEM;
+    d.device = cur;
+    if (!s->progs.ops.empty() &&
+        cudaMemcpy(d.ops, s->progs.ops.data(), s->progs.ops.size() * sizeof(uint32_t), cudaMemcpyHostToDevice) != cudaSuccess)
+        return RD_ERR_CUDA;
+    if (cudaEventCreate(&d.ev_start) != cudaSuccess || cudaEventCreate(&d.ev_stop) != cudaSuccess) return RD_ERR_CUDA;
+    if (s->p > kPackedPtrs) {
+        const size_t bytes = size_t(kPtrRing) * size_t(s->p) * sizeof(void *);
+        if (cudaHostAlloc(reinterpret_cast<void **>(&d.h_ring), bytes, cudaHostAllocDefault) != cudaSuccess) return RD_ERR_NOMEM;
+        if (cudaMalloc(reinterpret_cast<void **>(&d.d_ring), bytes) != cudaSuccess) return RD_ERR_NOMEM;
+        for (auto &e : d.ring_done)
+            if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return RD_ERR_CUDA;
+    }
+    return RD_OK;
+}
+
+// Tiles of the tree kernel for one vector width: runs of at most `cap` elements inside a segment.
+int tiles_for(rd_schedule *s, int vec, const TileDesc **tiles, uint32_t *count)
+{
+    DeviceTables &d = s->dev;
+    auto it = d.tiles.find(vec);
+    if (it == d.tiles.end()) {
+        const uint32_t cap = tree_tile_elems(vec);
+        std::vector<TileDesc> host;
+        const std::vector<uint64_t> &off = s->sched.seg_off;
+        for (size_t j = 0; j + 1 < off.size(); j++)
+            for (uint64_t e = off[j]; e < off[j + 1]; e += cap)
+                host.push_back(TileDesc{e, uint32_t(std::min<uint64_t>(cap, off[j + 1] - e)), s->progs.seg_prog[j]});
+        if (host.size() > 0xFFFFFFFFull) return RD_ERR_UNSUPPORTED;
+        TileDesc *dev = nullptr;
+        if (cudaMalloc(reinterpret_cast<void **>(&dev), std::max<size_t>(host.size(), 1) * sizeof(TileDesc)) != cudaSuccess)
+            return RD_ERR_NOMEM;
+        if (!host.empty() &&
+            cudaMemcpy(dev, host.data(), host.size() * sizeof(TileDesc), cudaMemcpyHostToDevice) != cudaSuccess) {
+            cudaFree(dev);
+            return RD_ERR_CUDA;
+        }
+        it = d.tiles.emplace(vec, std::make_pair(dev, uint32_t(host.size()))).first;
+    }
+    *tiles = it->second.first;
+    *count = it->second.second;
+    return RD_OK;
+}
+
+int reduce_tree(rd_schedule *s, const void *const *d_inputs, void *d_out, size_t n, rd_dtype_t dtype, rd_op_t op,
+                cudaStream_t stream, rd_stats_t *stats)
+{
+    DeviceTables &d = s->dev;
+    // 128-bit path: every buffer 16-byte aligned and every segment boundary a multiple of 4 elements
+    bool wide = (reinterpret_cast<uintptr_t>(d_out) & 15u) == 0;
+    for (int i = 0; i < s->p && wide; i++) wide = (reinterpret_cast<uintptr_t>(d_inputs[i]) & 15u) == 0;
+    for (size_t j = 0; j < s->sched.seg_off.size() && wide; j++) wide = (s->sched.seg_off[j] & 3u) == 0;
+    TreeLaunch l{};
+    l.vec = wide ? 4 : 1;
+    if (int rc = tiles_for(s, l.vec, &l.tiles, &l.n_tiles)) return rc;
+    l.host_ptrs = d_inputs;
+    l.dev_ptr_table = nullptr;
+    if (s->p > kPackedPtrs) {
+        const int slot = d.ring_next;
+        d.ring_next = (d.ring_next + 1) % kPtrRing;
+        if (cudaEventSynchronize(d.ring_done[slot]) != cudaSuccess) return RD_ERR_CUDA;   // previous user of the slot
+        void **h = d.h_ring + size_t(slot) * size_t(s->p), **dv = d.d_ring + size_t(slot) * size_t(s->p);
+        std::memcpy(h, d_inputs, size_t(s->p) * sizeof(void *));
+        if (cudaMemcpyAsync(dv, h, size_t(s->p) * sizeof(void *), cudaMemcpyHostToDevice, stream) != cudaSuccess) return RD_ERR_CUDA;
+        l.dev_ptr_table = dv;
+    }
+    l.out = d_out; l.ops = d.ops; l.p = s->p; l.stack_depth = s->progs.stack_depth;
+    l.dtype = int(dtype); l.op = int(op); l.sm_count = d.sm_count; l.stream = stream;
+    if (stats && cudaEventRecord(d.ev_start, stream) != cudaSuccess) return RD_ERR_CUDA;
+    if (launch_tree(l) != 0) return RD_ERR_CUDA;
+    if (s->p > kPackedPtrs) {
+        const int slot = (d.ring_next + kPtrRing - 1) % kPtrRing;
+        if (cudaEventRecord(d.ring_done[slot], stream) != cudaSuccess) return RD_ERR_CUDA;
+    }
+    if (stats) {
+        if (cudaEventRecord(d.ev_stop, stream) != cudaSuccess) return RD_ERR_CUDA;
+        if (cudaEventSynchronize(d.ev_stop) != cudaSuccess) return RD_ERR_CUDA;
+        float ms = 0;
+        if (cudaEventElapsedTime(&ms, d.ev_start, d.ev_stop) != cudaSuccess) return RD_ERR_CUDA;
+        std::memset(stats, 0, sizeof(*stats));
+        stats->kernel_ms = ms;
+        stats->bytes_moved = uint64_t(s->p + 1) * uint64_t(n) * 4u;
+        stats->gbytes_per_s = ms > 0 ? double(stats->bytes_moved) / (double(ms) * 1e6) : 0.0;
+        stats->predicted_s = double(s->sched.completion) * s->ticks.tick;
+        stats->n_launches = l.n_tiles ? 1 : 0;
+    }
+    return RD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int rd_schedule_create(rd_schedule_t **out, rd_algo_t algo, rd_port_t port, int p, size_t msg_bytes, size_t seg_bytes,
+                       const rd_model_t *model)
+{
+    if (!out || !model || (msg_bytes & 3u) || (seg_bytes & 3u)) return RD_ERR_INVALID_ARG;
+    if (p < 1 || p > kMaxProcs) return RD_ERR_INVALID_ARG;
+    if (int(algo) < 0 || int(algo) > RD_BUTTERFLY || (port != RD_PORT_UNI && port != RD_PORT_BI)) return RD_ERR_INVALID_ARG;
+    if (!legal_pair(algo, port)) return RD_ERR_UNSUPPORTED;
+    if (algo == RD_BUTTERFLY && (p & (p - 1)) != 0) return RD_ERR_UNSUPPORTED;
+    if (seg_bytes == 0) {
+        Ticks t;
+        if (int rc = make_ticks(model, t)) return rc;
+        if (int rc = optimal_segment(algo, port, p, msg_bytes, t, &seg_bytes)) return rc;
+    }
+    std::vector<int64_t> segs;
+    try {
+        if (algo != RD_BUTTERFLY) {
+            if (seg_bytes > msg_bytes) seg_bytes = msg_bytes;
+            if (msg_bytes > 0 && (msg_bytes + seg_bytes - 1) / seg_bytes > (size_t(1) << 22)) return RD_ERR_INVALID_ARG;
+            for (size_t done = 0; done < msg_bytes; done += seg_bytes)
+                segs.push_back(int64_t(std::min(seg_bytes, msg_bytes - done)));
+        }
+    } catch (const std::bad_alloc &) {
+        return RD_ERR_NOMEM;
+    }
+    return build(out, algo, port, p, std::move(segs), msg_bytes, model);
+}
+
+int rd_schedule_create_segments(rd_schedule_t **out, rd_algo_t algo, rd_port_t port, int p, const size_t *seg_bytes,
+                                size_t q, const rd_model_t *model)
+{
+    if (!out || !model || (!seg_bytes && q > 0)) return RD_ERR_INVALID_ARG;
+    if (algo == RD_BUTTERFLY) return RD_ERR_UNSUPPORTED;
+    if (q > (size_t(1) << 22)) return RD_ERR_INVALID_ARG;
+    std::vector<int64_t> segs;
+    size_t total = 0;
+    try {
+        for (size_t j = 0; j < q; j++) {
+            if (seg_bytes[j] == 0 || (seg_bytes[j] & 3u)) return RD_ERR_INVALID_ARG;
+            segs.push_back(int64_t(seg_bytes[j]));
+            total += seg_bytes[j];
+        }
+    } catch (const std::bad_alloc &) {
+        return RD_ERR_NOMEM;
+    }
+    return build(out, algo, port, p, std::move(segs), total, model);
+}
+
+int rd_optimal_segment(rd_algo_t algo, rd_port_t port, int p, size_t msg_bytes, const rd_model_t *model, size_t *seg_bytes_out)
+{
+    if (!model || !seg_bytes_out || (msg_bytes & 3u) || p < 1 || p > kMaxProcs) return RD_ERR_INVALID_ARG;
+    if (int(algo) < 0 || int(algo) > RD_BUTTERFLY || (port != RD_PORT_UNI && port != RD_PORT_BI)) return RD_ERR_INVALID_ARG;
+    if (!legal_pair(algo, port)) return RD_ERR_UNSUPPORTED;
+    Ticks t;
+    if (int rc = make_ticks(model, t)) return rc;
+    size_t s = 0;
+    try {
+        if (int rc = optimal_segment(algo, port, p, msg_bytes, t, &s)) return rc;
+    } catch (const std::bad_alloc &) {
+        return RD_ERR_NOMEM;
+    }
+    *seg_bytes_out = s;
+    return RD_OK;
+}
+
+int rd_schedule_info(const rd_schedule_t *s, int *p, size_t *q, size_t *n_events, double *predicted_seconds,
+                     int64_t *predicted_ticks, int *stack_depth)
+{
+    if (!s) return RD_ERR_INVALID_ARG;
+    if (p) *p = s->p;
+    if (q) *q = s->sched.seg_off.size() - 1;
+    if (n_events) *n_events = s->sched.events.size();
+    if (predicted_seconds) *predicted_seconds = double(s->sched.completion) * s->ticks.tick;
+    if (predicted_ticks) *predicted_ticks = s->sched.completion;
+    if (stack_depth) *stack_depth = s->progs.stack_depth;
+    return RD_OK;
+}
+
+int rd_schedule_events(const rd_schedule_t *s, rd_event_t *buf, size_t cap)
+{
+    if (!s || (!buf && cap > 0)) return RD_ERR_INVALID_ARG;
+    if (cap < s->sched.events.size()) return RD_ERR_TOO_SMALL;
+    if (!s->sched.events.empty()) std::memcpy(buf, s->sched.events.data(), s->sched.events.size() * sizeof(rd_event_t));
+    return RD_OK;
+}
+
+int rd_schedule_segments(const rd_schedule_t *s, uint64_t *off, size_t cap)
+{
+    if (!s || !off) return RD_ERR_INVALID_ARG;
+    if (cap < s->sched.seg_off.size()) return RD_ERR_TOO_SMALL;
+    std::memcpy(off, s->sched.seg_off.data(), s->sched.seg_off.size() * sizeof(uint64_t));
+    return RD_OK;
+}
+
+int rd_schedule_program(const rd_schedule_t *s, size_t seg, uint32_t *ops, size_t cap)
+{
+    if (!s || !ops || seg >= s->progs.seg_prog.size()) return RD_ERR_INVALID_ARG;
+    if (cap < size_t(s->p)) return RD_ERR_TOO_SMALL;
+    std::memcpy(ops, s->progs.ops.data() + s->progs.seg_prog[seg], size_t(s->p) * sizeof(uint32_t));
+    return RD_OK;
+}
+
+int rd_schedule_upload(rd_schedule_t *s)
+{
+    if (!s) return RD_ERR_INVALID_ARG;
+    return upload(s);
+}
+
+int rd_reduce(rd_schedule_t *s, const void *const *d_inputs, void *d_out, size_t n_elems, rd_dtype_t dtype, rd_op_t op,
+              rd_exec_t exec, void *cuda_stream, rd_stats_t *stats)
+{
+    if (!s || !d_inputs || (dtype != RD_INT32 && dtype != RD_FP32) || (op != RD_SUM && op != RD_MAX)) return RD_ERR_INVALID_ARG;
+    if (exec != RD_EXEC_TREE && exec != RD_EXEC_FAITHFUL) return RD_ERR_INVALID_ARG;
+    if (n_elems * 4 != s->msg_bytes) return RD_ERR_SIZE_MISMATCH;
+    if (n_elems > 0 && !d_out) return RD_ERR_INVALID_ARG;
+    for (int i = 0; i < s->p; i++)
+        if ((n_elems > 0 && !d_inputs[i]) || (reinterpret_cast<uintptr_t>(d_inputs[i]) & 3u)) return RD_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(d_out) & 3u) return RD_ERR_INVALID_ARG;
+    if (int rc = upload(s)) return rc;
+    if (exec == RD_EXEC_FAITHFUL) return RD_ERR_UNSUPPORTED;
+    return reduce_tree(s, d_inputs, d_out, n_elems, dtype, op, static_cast<cudaStream_t>(cuda_stream), stats);
+}
+
+int rd_reduce_host(rd_schedule_t *s, const void *const *h_inputs, void *h_out, void *d_staging, size_t n_elems,
+                   rd_dtype_t dtype, rd_op_t op, void *cuda_stream)
+{
+    if (!s || !h_inputs || (n_elems > 0 && (!h_out || !d_staging))) return RD_ERR_INVALID_ARG;
+    if (n_elems * 4 != s->msg_bytes) return RD_ERR_SIZE_MISMATCH;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    std::vector<const void *> dptr;
+    try { dptr.resize(size_t(s->p)); } catch (const std::bad_alloc &) { return RD_ERR_NOMEM; }
+    char *base = static_cast<char *>(d_staging);
+    for (int i = 0; i < s->p; i++) {
+        if (n_elems > 0 && !h_inputs[i]) return RD_ERR_INVALID_ARG;
+        dptr[size_t(i)] = base + size_t(i) * n_elems * 4;
+        if (n_elems > 0 &&
+            cudaMemcpyAsync(base + size_t(i) * n_elems * 4, h_inputs[i], n_elems * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+            return RD_ERR_CUDA;
+    }
+    void *d_out = base + size_t(s->p) * n_elems * 4;
+    if (int rc = rd_reduce(s, dptr.data(), d_out, n_elems, dtype, op, RD_EXEC_TREE, cuda_stream, nullptr)) return rc;
+    if (n_elems > 0 && cudaMemcpyAsync(h_out, d_out, n_elems * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return RD_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return RD_ERR_CUDA;
+    return RD_OK;
+}
+
+void rd_destroy(rd_schedule_t *s)
+{
+    if (!s) return;
+    release_device(s->dev);
+    delete s;
+}
+
+const char *rd_strerror(int status)
+{
+    switch (status) {
+    case RD_OK: return "success";
+    case RD_ERR_INVALID_ARG: return "invalid argument";
+    case RD_ERR_UNSUPPORTED: return "combination not supported";
+    case RD_ERR_NOMEM: return "out of memory";
+    case RD_ERR_CUDA: return "CUDA runtime call failed";
+    case RD_ERR_TIMEOUT: return "a bounded wait in the schedule-faithful kernel gave up";
+    case RD_ERR_SIZE_MISMATCH: return "n_elems does not match the schedule's message size";
+    case RD_ERR_INTERNAL: return "generated schedule failed the consistency check";
+    case RD_ERR_TOO_SMALL: return "output array too small";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

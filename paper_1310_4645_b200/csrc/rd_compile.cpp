@@ -1,0 +1,153 @@
+// From a schedule's send/receive pairs to what the kernels execute.
+//
+// Tree mode: per segment the pairs define one binary expression over the p inputs ("the receiving
+// processor combines its segment with the segment received", Section IV).  The expression is built
+// by replaying the pairs symbolically, then flattened into a program for a one-accumulator stack
+// machine; operand roles (held / incoming) are kept in every operation so the evaluation order can
+// be chosen freely (deepest subtree first, which keeps the stack at most log2 p deep).
+//
+// Faithful mode: per process the ordered list of its own sends and receives.
+#include <algorithm>
+#include <cstring>
+#include <string>
+#include <unordered_map>
+
+#include "rd_internal.h"
+
+namespace rd {
+
+namespace {
+
+struct Node { int32_t held, incoming; };   // children; ids < p are the processes' own data
+
+struct Flattener {
+    int p;
+    const std::vector<Node> &nodes;        // nodes[k] is expression p + k
+    const std::vector<int> &need;          // stack entries needed to evaluate expression id
+    std::vector<uint32_t> &ops;
+
+    bool leaf(int id) const { return id < p; }
+    void emit(uint32_t kind, int proc) { ops.push_back(uint32_t(proc) | (kind << kIdxBits)); }
+    int addPop(bool poppedIsHeld)
+    {
+        uint32_t &w = ops.back();
+        const uint32_t n = (w >> (kIdxBits + 2)) & 0xF;
+        if (n >= uint32_t(kMaxPops)) return RD_ERR_INTERNAL;
+        if (poppedIsHeld) w |= uint32_t(1) << (kIdxBits + 6 + n);
+        w = (w & ~(uint32_t(0xF) << (kIdxBits + 2))) | ((n + 1) << (kIdxBits + 2));
+        return RD_OK;
+    }
+    int gen(int id, bool pushFirst)
+    {
+        if (leaf(id)) { emit(pushFirst ? OP_PUSH_LOAD : OP_LOAD, id); return RD_OK; }
+        const Node &n = nodes[size_t(id - p)];
+        if (leaf(n.held) && leaf(n.incoming)) {
+            emit(pushFirst ? OP_PUSH_LOAD : OP_LOAD, n.held);
+            emit(OP_ACC_IN, n.incoming);
+            return RD_OK;
+        }
+        if (leaf(n.incoming)) {
+            if (int rc = gen(n.held, pushFirst)) return rc;
+            emit(OP_ACC_IN, n.incoming);
+            return RD_OK;
+        }
+        if (leaf(n.held)) {
+            if (int rc = gen(n.incoming, pushFirst)) return rc;
+            emit(OP_ACC_HELD, n.held);
+            return RD_OK;
+        }
+        const bool heldFirst = need[size_t(n.held)] >= need[size_t(n.incoming)];
+        if (int rc = gen(heldFirst ? n.held : n.incoming, pushFirst)) return rc;
+        if (int rc = gen(heldFirst ? n.incoming : n.held, true)) return rc;
+        return addPop(heldFirst);
+    }
+};
+
+}  // namespace
+
+int compile_programs(int p, size_t q, const std::vector<rd_event_t> &events, Programs &out)
+{
+    if (p < 1 || p > kMaxProcs) return RD_ERR_INVALID_ARG;
+    out.ops.clear();
+    out.seg_prog.assign(q, 0);
+    out.stack_depth = 0;
+    out.n_distinct = 0;
+    // bucket the pairs by segment, keeping their start-time order
+    std::vector<size_t> first(q + 1, 0);
+    for (const rd_event_t &e : events) {
+        if (e.seg < 0 || size_t(e.seg) >= q) return RD_ERR_INTERNAL;
+        first[size_t(e.seg) + 1]++;
+    }
+    for (size_t j = 0; j < q; j++) first[j + 1] += first[j];
+    std::vector<rd_event_t> bySeg(events.size());
+    {
+        std::vector<size_t> fill(first.begin(), first.end() - 1);
+        for (const rd_event_t &e : events) bySeg[fill[size_t(e.seg)]++] = e;
+    }
+    std::unordered_map<std::string, uint32_t> seen;
+    std::vector<Node> nodes;
+    const size_t P = size_t(p);
+    std::vector<int> expr(P, 0), need, leafSeen(P, 0);
+    std::vector<uint32_t> prog;
+    std::vector<int> walk;
+    for (size_t j = 0; j < q; j++) {
+        nodes.clear();
+        for (int i = 0; i < p; i++) expr[size_t(i)] = i;
+        for (size_t k = first[j]; k < first[j + 1]; k++) {
+            const rd_event_t &e = bySeg[k];
+            if (e.src < 0 || e.src >= p || e.dst < 0 || e.dst >= p || e.src == e.dst) return RD_ERR_INTERNAL;
+            if (e.kind == 0) {
+                nodes.push_back(Node{expr[size_t(e.dst)], expr[size_t(e.src)]});
+                expr[size_t(e.dst)] = p + int(nodes.size()) - 1;
+            } else {
+                expr[size_t(e.dst)] = expr[size_t(e.src)];
+            }
+        }
+        const int root = expr[0];
+        // every process's data must enter the root's expression exactly once
+        std::fill(leafSeen.begin(), leafSeen.end(), 0);
+        walk.assign(1, root);
+        size_t leaves = 0;
+        while (!walk.empty()) {
+            const int id = walk.back(); walk.pop_back();
+            if (id < p) { if (leafSeen[size_t(id)]++) return RD_ERR_INTERNAL; leaves++; continue; }
+            walk.push_back(nodes[size_t(id - p)].held);
+            walk.push_back(nodes[size_t(id - p)].incoming);
+            if (leaves + walk.size() > size_t(2 * p)) return RD_ERR_INTERNAL;
+        }
+        if (leaves != size_t(p)) return RD_ERR_INTERNAL;
+        // stack need, children before parents (a node only refers to older expressions)
+        need.assign(size_t(p) + nodes.size(), 0);
+        for (size_t k = 0; k < nodes.size(); k++) {
+            const Node &n = nodes[k];
+            const bool lh = n.held < p, li = n.incoming < p;
+            int v;
+            if (lh && li) v = 0;
+            else if (li) v = need[size_t(n.held)];
+            else if (lh) v = need[size_t(n.incoming)];
+            else {
+                const int a = std::max(need[size_t(n.held)], need[size_t(n.incoming)]);
+                const int b = std::min(need[size_t(n.held)], need[size_t(n.incoming)]);
+                v = std::max(a, b + 1);
+            }
+            need[size_t(p) + k] = v;
+        }
+        prog.clear();
+        Flattener fl{p, nodes, need, prog};
+        if (int rc = fl.gen(root, false)) return rc;
+        if (prog.size() != size_t(p)) return RD_ERR_INTERNAL;
+        if (need[size_t(root)] > kMaxPops) return RD_ERR_INTERNAL;
+        out.stack_depth = std::max(out.stack_depth, need[size_t(root)]);
+        std::string key(reinterpret_cast<const char *>(prog.data()), prog.size() * sizeof(uint32_t));
+        auto it = seen.find(key);
+        if (it == seen.end()) {
+            it = seen.emplace(std::move(key), uint32_t(out.ops.size())).first;
+            out.ops.insert(out.ops.end(), prog.begin(), prog.end());
+            out.n_distinct++;
+        }
+        out.seg_prog[j] = it->second;
+    }
+    return RD_OK;
+}
+
+}  // namespace rd

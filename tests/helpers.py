@@ -1,0 +1,73 @@
+"""Shared helpers of the tests (no method arithmetic of the library, no oracle internals)."""
+import numpy as np
+
+import paper_1310_4645_b200 as rd
+from oracle import rd_oracle as O
+
+TICK = 1e-15
+ORDER = ["t_start", "seg", "src", "dst"]
+
+
+def ticks(alpha, beta, gamma, tick=TICK):
+    return int(round(alpha / tick)), int(round(beta / tick)), int(round(gamma / tick))
+
+
+def oracle_schedule(algo, port, p, msg_bytes, seg_bytes, alpha, beta, gamma, sizes=None):
+    """(events sorted like the library's export, segment offsets in elements, completion ticks)."""
+    A, B, G = ticks(alpha, beta, gamma)
+    bidir = port == rd.RD_PORT_BI
+    if algo == rd.RD_BUTTERFLY:
+        ev, off, comp = O.butterfly(p, msg_bytes // 4, 4, A, B, G)
+        return np.sort(ev, order=ORDER), off, comp
+    if sizes is None:
+        sizes = O.equal_sizes(msg_bytes, min(seg_bytes, msg_bytes)) if msg_bytes else []
+    if algo == rd.RD_UNI_GREEDY:
+        ev, comp = O.uni_greedy(p, sizes, A, B, G)
+    elif algo == rd.RD_BI_GREEDY:
+        ev, comp = O.bi_greedy(p, sizes, A, B, G)
+    elif algo == rd.RD_BINOMIAL:
+        ev, comp = O.binomial(p, sizes, A, B, G)
+    elif algo == rd.RD_PIPELINE:
+        ev, comp = O.pipeline(p, sizes, A, B, G, bidir)
+    elif algo == rd.RD_BINARY:
+        ev, comp = O.binary(p, sizes, A, B, G, bidir)
+    else:
+        raise ValueError(algo)
+    off = np.concatenate([[0], np.cumsum(np.asarray(sizes, dtype=np.int64) // 4)])
+    return np.sort(ev, order=ORDER), off, comp
+
+
+def run_program(ops, x, op):
+    """Reference interpreter of one compiled combine program (format documented in include/rd.h).
+    x: [p, len] array; returns the root's value.  Written from the header's description only."""
+    x = np.asarray(x)
+
+    def combine(held, incoming):
+        if op == "sum":
+            if x.dtype == np.int32:
+                return (held.astype(np.int64) + incoming.astype(np.int64)).astype(np.uint64).astype(np.uint32) \
+                    .view(np.int32) if False else ((held.view(np.uint32) + incoming.view(np.uint32)).view(np.int32))
+            return (held + incoming).astype(np.float32)
+        return np.where(incoming > held, incoming, held)
+
+    stack, top = [], None
+    loads = 0
+    for w in ops:
+        w = int(w)
+        proc, kind, npop, roles = w & 0xFFF, (w >> 12) & 3, (w >> 14) & 0xF, w >> 18
+        v = x[proc]
+        loads += 1
+        if kind == 0:
+            top = v.copy()
+        elif kind == 1:
+            stack.append(top)
+            top = v.copy()
+        elif kind == 2:
+            top = combine(top, v)
+        else:
+            top = combine(v, top)
+        for k in range(npop):
+            y = stack.pop()
+            top = combine(y, top) if (roles >> k) & 1 else combine(top, y)
+    assert not stack and loads == x.shape[0]
+    return top

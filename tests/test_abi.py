@@ -1,0 +1,121 @@
+"""The C ABI: the library loads, exports what include/rd.h declares, and rejects bad arguments
+(no GPU needed: nothing here launches a kernel)."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+import paper_1310_4645_b200 as rd
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+MODEL = (2e-6, 1e-10, 5e-11)
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "rd.h")).read()
+    return sorted(set(re.findall(r"RD_API\s+[\w\s\*]*?\b(rd_\w+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = declared_functions()
+    assert len(names) >= 12 and set(names) == set(rd.EXPORTS)
+    L = C.CDLL(rd.LIB_PATH)
+    for n in names:
+        assert getattr(L, n) is not None
+
+
+def test_only_the_abi_is_exported():
+    """Internal C++ symbols stay hidden: the dynamic symbol table's rd:: / rd_ definitions are the ABI."""
+    out = os.popen("nm -D --defined-only %s" % rd.LIB_PATH).read()
+    mine = [ln.split()[-1] for ln in out.splitlines() if " T " in ln and ("rd" in ln.split()[-1])]
+    assert sorted(m for m in mine if m.startswith("rd_")) == sorted(rd.EXPORTS)
+    assert not [m for m in mine if m.startswith("_ZN2rd")]
+
+
+def test_strerror():
+    assert rd.rd_strerror(0) == "success"
+    for code in range(-8, 0):
+        assert rd.rd_strerror(code) and rd.rd_strerror(code) != "unknown status"
+    assert rd.rd_strerror(-99) == "unknown status"
+
+
+def status_of(fn, *a):
+    with pytest.raises(rd.RdError) as e:
+        fn(*a)
+    return e.value.status
+
+
+def test_create_rejects_bad_arguments():
+    f = rd.rd_schedule_create
+    assert status_of(f, rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, 0, 64, 16, *MODEL) == rd.RD_ERR_INVALID_ARG
+    assert status_of(f, rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, 5000, 64, 16, *MODEL) == rd.RD_ERR_INVALID_ARG
+    assert status_of(f, rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, 4, 66, 16, *MODEL) == rd.RD_ERR_INVALID_ARG
+    assert status_of(f, rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, 4, 64, 18, *MODEL) == rd.RD_ERR_INVALID_ARG
+    assert status_of(f, 17, rd.RD_PORT_UNI, 4, 64, 16, *MODEL) == rd.RD_ERR_INVALID_ARG
+    assert status_of(f, rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, 4, 64, 16, -1.0, 1e-10, 0) == rd.RD_ERR_INVALID_ARG
+    # pairs the method does not define
+    assert status_of(f, rd.RD_UNI_GREEDY, rd.RD_PORT_BI, 4, 64, 16, *MODEL) == rd.RD_ERR_UNSUPPORTED
+    assert status_of(f, rd.RD_BI_GREEDY, rd.RD_PORT_UNI, 4, 64, 16, *MODEL) == rd.RD_ERR_UNSUPPORTED
+    assert status_of(f, rd.RD_BUTTERFLY, rd.RD_PORT_UNI, 4, 64, 16, *MODEL) == rd.RD_ERR_UNSUPPORTED
+    assert status_of(f, rd.RD_BUTTERFLY, rd.RD_PORT_BI, 6, 64, 16, *MODEL) == rd.RD_ERR_UNSUPPORTED
+    assert status_of(rd.rd_schedule_create_segments, rd.RD_BUTTERFLY, rd.RD_PORT_BI, 4, [32, 32], *MODEL) \
+        == rd.RD_ERR_UNSUPPORTED
+    assert status_of(rd.rd_schedule_create_segments, rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, 4, [32, 0], *MODEL) \
+        == rd.RD_ERR_INVALID_ARG
+    # null pointers straight through ctypes
+    L = rd.lib()
+    m = rd.rd_model_t(*MODEL, 0.0)
+    assert L.rd_schedule_create(None, 0, 0, 4, 64, 16, C.byref(m)) == rd.RD_ERR_INVALID_ARG
+    h = C.c_void_p(0x1234)
+    assert L.rd_schedule_create(C.byref(h), 0, 0, 4, 64, 16, None) == rd.RD_ERR_INVALID_ARG
+    assert h.value == 0x1234            # untouched on failure
+    L.rd_destroy(None)                  # allowed
+
+
+def test_info_events_segments_program_capacity_checks():
+    h = rd.rd_schedule_create(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, 8, 16384, 2048, *MODEL)
+    try:
+        info = rd.rd_schedule_info(h)
+        assert info["p"] == 8 and info["q"] == 8 and info["n_events"] == 56
+        L = rd.lib()
+        buf = np.zeros(10, dtype=rd.EVENT_DTYPE)
+        assert L.rd_schedule_events(h, buf.ctypes.data, 10) == rd.RD_ERR_TOO_SMALL
+        off = np.zeros(4, dtype=np.uint64)
+        assert L.rd_schedule_segments(h, off.ctypes.data, 4) == rd.RD_ERR_TOO_SMALL
+        ops = np.zeros(4, dtype=np.uint32)
+        assert L.rd_schedule_program(h, 0, ops.ctypes.data, 4) == rd.RD_ERR_TOO_SMALL
+        assert L.rd_schedule_program(h, 8, ops.ctypes.data, 4) == rd.RD_ERR_INVALID_ARG
+        assert (rd.rd_schedule_segments(h) == np.arange(9) * 512).all()
+        # argument checks of rd_reduce come before any CUDA call
+        ptrs = (C.c_void_p * 8)(*([0x1000] * 8))
+        assert L.rd_reduce(h, ptrs, 0x2000, 100, rd.RD_INT32, rd.RD_SUM, rd.RD_EXEC_TREE, None, None) \
+            == rd.RD_ERR_SIZE_MISMATCH
+        assert L.rd_reduce(h, ptrs, 0x2000, 4096, 7, rd.RD_SUM, rd.RD_EXEC_TREE, None, None) == rd.RD_ERR_INVALID_ARG
+        assert L.rd_reduce(h, ptrs, None, 4096, rd.RD_INT32, rd.RD_SUM, rd.RD_EXEC_TREE, None, None) \
+            == rd.RD_ERR_INVALID_ARG
+        ptrs[3] = 0x1002                 # misaligned input
+        assert L.rd_reduce(h, ptrs, 0x2000, 4096, rd.RD_INT32, rd.RD_SUM, rd.RD_EXEC_TREE, None, None) \
+            == rd.RD_ERR_INVALID_ARG
+    finally:
+        rd.rd_destroy(h)
+
+
+def test_missing_library_fails_loudly(monkeypatch):
+    import paper_1310_4645_b200.binding as b
+    monkeypatch.setattr(b, "_lib", None)
+    monkeypatch.setattr(b, "LIB_PATH", "/nonexistent/librd.so")
+    with pytest.raises(ImportError):
+        b.rd_schedule_create(0, 0, 4, 64, 16, *MODEL)
+
+
+def test_empty_message_and_single_process():
+    h = rd.rd_schedule_create(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, 4, 0, 16, *MODEL)
+    assert rd.rd_schedule_info(h)["q"] == 0 and rd.rd_schedule_info(h)["n_events"] == 0
+    rd.rd_destroy(h)
+    h = rd.rd_schedule_create(rd.RD_PIPELINE, rd.RD_PORT_BI, 1, 64, 16, *MODEL)
+    info = rd.rd_schedule_info(h)
+    assert info["q"] == 4 and info["n_events"] == 0 and info["predicted_ticks"] == 0
+    assert list(rd.rd_schedule_program(h, 2)) == [0]      # LOAD process 0
+    rd.rd_destroy(h)

@@ -1,0 +1,183 @@
+"""Parity of the tree kernel with the oracle, element by element, through the C ABI (GPU)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_1310_4645_b200 as rd
+from paper_1310_4645_b200.inputs import make_inputs, WORKLOADS
+from oracle import rd_oracle as O
+from helpers import oracle_schedule
+
+pytestmark = pytest.mark.gpu
+
+M1 = (2e-6, 1e-10, 5e-11)
+SCHEDULES = [("uni_greedy", rd.RD_UNI_GREEDY, rd.RD_PORT_UNI), ("bi_greedy", rd.RD_BI_GREEDY, rd.RD_PORT_BI),
+             ("binomial", rd.RD_BINOMIAL, rd.RD_PORT_UNI), ("pipeline", rd.RD_PIPELINE, rd.RD_PORT_UNI),
+             ("binary", rd.RD_BINARY, rd.RD_PORT_BI), ("butterfly", rd.RD_BUTTERFLY, rd.RD_PORT_BI)]
+OPS = {"sum": rd.RD_SUM, "max": rd.RD_MAX}
+
+
+def gpu_reduce(algo, port, x_dev, seg_bytes, op, model=M1, out=None, rows=None):
+    p, n = x_dev.shape
+    h = rd.rd_schedule_create(algo, port, p, 4 * n, seg_bytes, *model)
+    try:
+        out = torch.full((n,), 77, dtype=x_dev.dtype, device=x_dev.device) if out is None else out
+        rd.rd_reduce(h, rows if rows is not None else x_dev, out, OPS[op])
+        torch.cuda.synchronize()
+    finally:
+        rd.rd_destroy(h)
+    return out
+
+
+def check(algo, port, x_dev, seg_bytes, op, model=M1):
+    p, n = x_dev.shape
+    got = gpu_reduce(algo, port, x_dev, seg_bytes, op, model).cpu().numpy()
+    x = x_dev.cpu().numpy()
+    ev, off, _ = oracle_schedule(algo, port, p, 4 * n, seg_bytes if seg_bytes else 4 * n, *model)
+    want = O.reduce(ev, x, off, op)
+    assert got.tobytes() == want.tobytes()
+    return got, x
+
+
+# (p, n, segment elements): several tiles (2048 elements each on the 128-bit path), ragged tails,
+# segments shorter and longer than a tile, non-power-of-two process counts
+SHAPES = [(8, 4096, 512), (5, 10000, 2500), (13, 3 * 2048 + 36, 2048 + 520), (64, 8192, 1024), (2, 4100, 4100),
+          (33, 6000, 1000), (16, 128, 8), (1, 5000, 1000)]
+
+
+@pytest.mark.parametrize("name,algo,port", SCHEDULES)
+@pytest.mark.parametrize("dist,op", [("int_pm2p20", "sum"), ("int_pm2p20", "max"), ("normal", "sum"), ("normal", "max")])
+def test_parity_small_shapes(name, algo, port, dist, op):
+    for p, n, seg in SHAPES:
+        if algo == rd.RD_BUTTERFLY and p & (p - 1):
+            continue
+        x = make_inputs(p, n, dist, seed=p * 1000 + n, device="cuda")
+        if dist == "normal":
+            x *= 10.0 ** torch.randint(-4, 5, x.shape, device="cuda", generator=torch.Generator("cuda").manual_seed(1))
+        check(algo, port, x, 4 * seg, op)
+
+
+def test_config1_bit_exact_and_order_free():
+    """p = 8, 4096 int32, 8 segments of 512, uni-greedy, wrapping sum."""
+    w = WORKLOADS["config1"]
+    x = make_inputs(w["p"], w["n"], w["dist"], w["seed"], device="cuda")
+    got, xh = check(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, x, w["seg_bytes"], "sum", (w["alpha"], w["beta"], w["gamma"]))
+    assert (got == xh.astype(np.int64).sum(axis=0).astype(np.int32)).all()
+
+
+def test_int32_sum_wraps():
+    x = torch.full((8, 4096), 2**30, dtype=torch.int32, device="cuda")
+    got, _ = check(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, x, 2048, "sum")
+    assert (got == 0).all()            # 8 * 2^30 = 2^33 = 0 mod 2^32
+
+
+@pytest.mark.parametrize("name,algo,port", SCHEDULES)
+def test_element_path_for_unaligned_segments_and_buffers(name, algo, port):
+    """Segment sizes that are not multiples of 16 bytes, and buffers that start 4 bytes off a 16-byte
+    boundary, take the one-element-per-lane path."""
+    p, n = 8, 3003
+    x = make_inputs(p, n, "normal", seed=5, device="cuda")
+    check(algo, port, x, 4 * 333, "sum")
+    # misaligned views: row i starts at element 1 of a longer buffer
+    big = make_inputs(p, n + 1, "normal", seed=6, device="cuda")
+    rows = [big[i, 1:] for i in range(p)]
+    assert rows[0].data_ptr() % 16 == 4
+    out_big = torch.zeros(n + 1, dtype=torch.float32, device="cuda")
+    gpu_reduce(algo, port, big[:, 1:], 4 * 1024, "sum", out=out_big[1:], rows=rows)
+    ev, off, _ = oracle_schedule(algo, port, p, 4 * n, 4 * 1024, *M1)
+    want = O.reduce(ev, big[:, 1:].cpu().numpy().copy(), off, "sum")
+    assert out_big[1:].cpu().numpy().tobytes() == want.tobytes()
+    assert out_big[0].item() == 0.0                                    # nothing written before the view
+
+
+def test_signed_zero_and_inf_follow_the_held_incoming_rule():
+    p, n = 16, 4096
+    g = torch.Generator("cuda").manual_seed(3)
+    choices = torch.tensor([0.0, -0.0, 1.0, -1.0, float("inf"), -float("inf")], device="cuda")
+    x = choices[torch.randint(0, 6, (p, n), device="cuda", generator=g)].contiguous()
+    for name, algo, port in SCHEDULES:
+        check(algo, port, x, 4 * 512, "max")
+    x = choices[torch.randint(0, 5, (p, n), device="cuda", generator=g)].contiguous()     # no -inf: inf - inf is NaN
+    for name, algo, port in SCHEDULES:
+        check(algo, port, x, 4 * 512, "sum")
+
+
+def test_denormals_are_not_flushed():
+    p, n = 4, 2048
+    x = torch.full((p, n), 1e-45, dtype=torch.float32, device="cuda")       # smallest subnormal
+    got, _ = check(rd.RD_BINOMIAL, rd.RD_PORT_UNI, x, 0, "sum")
+    assert (got == np.float32(4e-45)).all() and got[0] > 0
+
+
+def test_output_may_alias_the_roots_input():
+    p, n = 8, 8192
+    x = make_inputs(p, n, "normal", seed=9, device="cuda")
+    keep = x.clone()
+    gpu_reduce(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, x, 4096, "sum", out=x[0])
+    ev, off, _ = oracle_schedule(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, p, 4 * n, 4096, *M1)
+    want = O.reduce(ev, keep.cpu().numpy(), off, "sum")
+    assert x[0].cpu().numpy().tobytes() == want.tobytes()
+    assert torch.equal(x[1:], keep[1:])                                # inputs are never written
+
+
+def test_many_processes_use_the_pointer_table():
+    """More processes than fit in the kernel's parameter block."""
+    p, n = 300, 4096
+    x = make_inputs(p, n, "uniform_pm1", seed=2, device="cuda")
+    for _ in range(3):                                                 # cycles the table slots
+        check(rd.RD_BI_GREEDY, rd.RD_PORT_BI, x, 4096, "sum")
+    p, n = 1024, 2048
+    x = make_inputs(p, n, "uniform_pm1", seed=2, device="cuda")
+    check(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, x, 2048, "sum")
+    check(rd.RD_BUTTERFLY, rd.RD_PORT_BI, x, 0, "max")
+
+
+def test_empty_message_and_stats():
+    x = torch.zeros((4, 0), dtype=torch.float32, device="cuda")
+    h = rd.rd_schedule_create(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, 4, 0, 16, *M1)
+    rd.rd_reduce(h, x, torch.zeros(0, device="cuda"), rd.RD_SUM)
+    rd.rd_destroy(h)
+    x = make_inputs(8, 1 << 16, "normal", seed=1, device="cuda")
+    out = torch.empty(1 << 16, device="cuda")
+    h = rd.rd_schedule_create(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, 8, 4 << 16, 4096, *M1)
+    st = rd.rd_reduce(h, x, out, rd.RD_SUM, want_stats=True)
+    assert st.kernel_ms > 0 and st.bytes_moved == 9 * (4 << 16) and st.n_launches == 1
+    assert abs(st.predicted_s - rd.rd_schedule_info(h)["predicted_seconds"]) < 1e-12
+    with pytest.raises(rd.RdError) as e:
+        rd.rd_reduce(h, x[:, :100].contiguous(), out[:100], rd.RD_SUM)
+    assert e.value.status == rd.RD_ERR_SIZE_MISMATCH
+    rd.rd_destroy(h)
+
+
+def test_reduce_host_round_trip():
+    p, n = 8, 10000
+    x = make_inputs(p, n, "normal", seed=4, device="cpu").pin_memory()
+    out = torch.empty(n, dtype=torch.float32).pin_memory()
+    staging = torch.empty((p + 1) * n, dtype=torch.float32, device="cuda")
+    h = rd.rd_schedule_create(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, p, 4 * n, 4000, *M1)
+    rd.rd_reduce_host(h, x, out, staging, rd.RD_SUM)
+    rd.rd_destroy(h)
+    ev, off, _ = oracle_schedule(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, p, 4 * n, 4000, *M1)
+    assert out.numpy().tobytes() == O.reduce(ev, x.numpy(), off, "sum").tobytes()
+
+
+@pytest.mark.parametrize("name,algo,port", SCHEDULES[:5])
+def test_config2_shape_full_size(name, algo, port):
+    """p = 64, n = 2^20 fp32 N(0,1), 16 KB segments: bit-exact against the oracle on every element of
+    sampled segments, and within 1e-5 * sum|x_i| of the fp64 sum everywhere."""
+    w = WORKLOADS["config2"]
+    model = (w["alpha"], w["beta"], w["gamma"])
+    x = make_inputs(w["p"], w["n"], w["dist"], w["seed"], device="cuda")
+    got = gpu_reduce(algo, port, x, w["seg_bytes"], "sum", model).cpu().numpy()
+    xh = x.cpu().numpy()
+    ev, off, _ = oracle_schedule(algo, port, w["p"], 4 * w["n"], w["seg_bytes"], *model)
+    q = len(off) - 1
+    for j in sorted(set([0, 1, q // 3, q // 2, q - 2, q - 1])):
+        sel = ev[ev["seg"] == j].copy()
+        sel["seg"] = 0
+        sl = slice(int(off[j]), int(off[j + 1]))
+        want = O.reduce(sel, np.ascontiguousarray(xh[:, sl]), [0, sl.stop - sl.start], "sum")
+        assert got[sl].tobytes() == want.tobytes(), j
+    ref, mag = O.reference_f64(xh, "sum")
+    assert (np.abs(got.astype(np.float64) - ref) <= 1e-5 * mag).all()
+    assert np.abs(got - ref).max() / np.abs(ref).max() <= 1e-5
