@@ -1,0 +1,376 @@
+#!/usr/bin/env python
+"""Throughput of the schedule-exact reduction on B200: `python bench.py --gpus N --steps K --warmup W`.
+
+A step is one pass of the reduction path over one batch of synthetic inputs: for every schedule the
+workload names, one tree-mode rd_reduce of the p resident messages (fp32) into the root buffer.
+The schedules themselves (cost model, event generation, combine programs) are plans built once and
+reused; their build time is reported beside the throughput.  Metric: reduction GB/s, counting
+p*m input bytes plus m output bytes per reduction.
+
+One JSON line is printed by rank 0.  With N > 1 every rank runs an independent replica on its own
+GPU (the path needs no exchange between GPUs); times are taken on the device and the slowest rank
+counts.  `--impl reference` times the plain CPU checker instead, on rank 0 only.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+TICK = 1e-15
+# schedules per workload: (label, algo name, bidirectional ports)
+WORKLOAD_SCHEDULES = {
+    "config1": [("uni_greedy", "uni_greedy", False)],
+    "config2": [("uni_greedy", "uni_greedy", False), ("binomial", "binomial", False),
+                ("pipeline", "pipeline", False), ("binary", "binary", False)],
+    "config3": [("bi_greedy", "bi_greedy", True), ("butterfly", "butterfly", True), ("binomial", "binomial", True),
+                ("pipeline", "pipeline", True), ("binary", "binary", True)],
+    "config4": [("uni_greedy", "uni_greedy", False), ("bi_greedy", "bi_greedy", True)],
+}
+WORKLOAD_OPS = {"config1": ["sum"], "config2": ["sum"], "config3": ["sum"], "config4": ["sum", "max"]}
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, copy read+write)"
+    except Exception:
+        return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs (read only)."""
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.reasons, self.max_mhz = index, [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+            "hw_power_brake": getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80),
+        }
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.02)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(s)}
+
+
+def visible_gpu_index(local_rank):
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+def oracle_events(rdmod, algo_name, bidir, p, msg_bytes, seg_bytes, model):
+    """Events, offsets for the CPU checker (used by the reference arm and the cpu_baseline leg only)."""
+    import numpy as np
+    from oracle import rd_oracle as O
+    A, B, G = (int(round(v / TICK)) for v in model)
+    if algo_name == "butterfly":
+        ev, off, _ = O.butterfly(p, msg_bytes // 4, 4, A, B, G)
+        return ev, off
+    sizes = O.equal_sizes(msg_bytes, min(seg_bytes, msg_bytes))
+    if algo_name == "uni_greedy":
+        ev, _ = O.uni_greedy(p, sizes, A, B, G)
+    elif algo_name == "bi_greedy":
+        ev, _ = O.bi_greedy(p, sizes, A, B, G)
+    elif algo_name == "binomial":
+        ev, _ = O.binomial(p, sizes, A, B, G)
+    elif algo_name == "pipeline":
+        ev, _ = O.pipeline(p, sizes, A, B, G, bidir)
+    else:
+        ev, _ = O.binary(p, sizes, A, B, G, bidir)
+    off = np.concatenate([[0], np.cumsum(np.asarray(sizes, dtype=np.int64) // 4)])
+    return ev, off
+
+
+def cpu_pass(w, wname, x_host, budget_s, max_passes):
+    """Times the CPU checker's reduction on the workload (or a slab of whole segments of it when one pass
+    would exceed the budget).  Returns (GB/s, description, cores)."""
+    import numpy as np
+    from oracle import rd_oracle as O
+    p, n = x_host.shape
+    model = (w["alpha"], w["beta"], w["gamma"])
+    plans = []
+    for label, algo_name, bidir in WORKLOAD_SCHEDULES[wname]:
+        ev, off = oracle_events(None, algo_name, bidir, p, 4 * n, w["seg_bytes"], model)
+        plans.append((ev, off))
+    bytes_per_pass = len(plans) * len(WORKLOAD_OPS[wname]) * (p + 1) * n * 4
+    t_total, passes = 0.0, 0
+    while passes < max_passes and (passes == 0 or t_total < budget_s):
+        t0 = time.perf_counter()
+        for ev, off in plans:
+            for op in WORKLOAD_OPS[wname]:
+                O.reduce(ev, x_host, off, op)
+        t_total += time.perf_counter() - t0
+        passes += 1
+    return bytes_per_pass * passes / t_total / 1e9, passes, t_total
+
+
+def host_slab(w, wname, max_bytes):
+    """Host copy of the workload, or of its first whole segments when it exceeds max_bytes."""
+    from paper_1310_4645_b200.inputs import make_inputs
+    p, n = w["p"], w["n"]
+    seg = w["seg_bytes"] // 4
+    if p * n * 4 > max_bytes:
+        n = max(seg, (max_bytes // (4 * p)) // seg * seg)
+    return make_inputs(p, n, w["dist"], w["seed"], device="cpu"), n
+
+
+def run_reference(args, wname, w):
+    """The CPU checker as it stands, timed on the host cores: one step = one pass over a bounded slab."""
+    import torch
+    x, n = host_slab(w, wname, 1 << 30)
+    xh = x.numpy()
+    slab = dict(w, n=n)
+    for _ in range(args.warmup):
+        cpu_pass(slab, wname, xh, 0.0, 1)
+    t0 = time.perf_counter()
+    gb = 0.0
+    for _ in range(args.steps):
+        v, passes, dt = cpu_pass(slab, wname, xh, 0.0, 1)
+        gb += v * dt
+    dt = time.perf_counter() - t0
+    value = gb / dt
+    sample = "each step: every schedule x op of the workload on the first %d of %d elements per process" % (n, w["n"])
+    line = {"impl": "reference", "metric": "reduction_throughput", "value": value, "unit": "GB/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": wname, "p": w["p"], "n_elems": w["n"], "segment_bytes": w["seg_bytes"],
+                       "schedules": [s[0] for s in WORKLOAD_SCHEDULES[wname]], "ops": WORKLOAD_OPS[wname]},
+            "cpu_baseline": {"value": value, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="config2", choices=sorted(WORKLOAD_SCHEDULES))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    from paper_1310_4645_b200.inputs import make_inputs, WORKLOADS
+    wname = args.workload
+    w = WORKLOADS[wname]
+
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        args.steps = args.steps if args.steps is not None else 5
+        args.warmup = args.warmup if args.warmup is not None else 1
+        run_reference(args, wname, w)
+        return 0
+
+    import torch
+    import paper_1310_4645_b200 as rd
+
+    p, n = w["p"], w["n"]
+    bytes_per_reduce = (p + 1) * n * 4
+    # default step count: about a second of timed work
+    if args.steps is None:
+        args.steps = max(20, int(1.0 / (len(WORKLOAD_SCHEDULES[wname]) * len(WORKLOAD_OPS[wname]) * bytes_per_reduce / 5e12)))
+    if args.warmup is None:
+        args.warmup = max(3, args.steps // 20)
+    if args.warmup < 3:
+        args.warmup = 3
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist_on = world > 1
+    if dist_on:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    model = (w["alpha"], w["beta"], w["gamma"])
+    # arenas: the kernel never reads the arena the previous launch read, and two arenas together exceed L2
+    n_arenas = 3 if p * n * 4 <= (1 << 30) else 1
+    arenas = [make_inputs(p, n, w["dist"], w["seed"] + 1000 * a, device=str(dev)) for a in range(n_arenas)]
+    out = torch.empty(n, dtype=torch.float32, device=dev)
+    tables = [rd.PointerTable(a) for a in arenas]
+
+    t0 = time.perf_counter()
+    plans = []
+    for label, algo_name, bidir in WORKLOAD_SCHEDULES[wname]:
+        h = rd.rd_schedule_create(rd.ALGOS[algo_name], rd.RD_PORT_BI if bidir else rd.RD_PORT_UNI, p, 4 * n,
+                                  w["seg_bytes"], *model)
+        plans.append((label, h))
+    create_ms = (time.perf_counter() - t0) * 1e3
+    for _, h in plans:
+        rd.rd_schedule_upload(h)
+    ops = [rd.RD_SUM if o == "sum" else rd.RD_MAX for o in WORKLOAD_OPS[wname]]
+    launches_per_step = len(plans) * len(ops)
+
+    counter = [0]
+
+    def step():
+        for _, h in plans:
+            for op in ops:
+                rd.rd_reduce(h, tables[counter[0] % n_arenas], out, op)
+                counter[0] += 1
+
+    def barrier():
+        if dist_on:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(visible_gpu_index(local_rank))
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1)
+    if dist_on:
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    total_bytes = world * args.steps * launches_per_step * bytes_per_reduce
+    value = total_bytes / (ms * 1e-3) / 1e9
+
+    # per-schedule throughput (same launches, timed one schedule at a time)
+    per_schedule = {}
+    for label, h in plans:
+        for opname, op in zip(WORKLOAD_OPS[wname], ops):
+            reps = max(5, args.steps // 2)
+            for _ in range(3):
+                rd.rd_reduce(h, tables[counter[0] % n_arenas], out, op); counter[0] += 1
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(reps):
+                rd.rd_reduce(h, tables[counter[0] % n_arenas], out, op); counter[0] += 1
+            b.record()
+            torch.cuda.synchronize()
+            per_schedule["%s/%s" % (label, opname)] = round(bytes_per_reduce * reps / (a.elapsed_time(b) * 1e-3) / 1e9, 1)
+
+    # end to end: host buffers in, host result out, through rd_reduce_host
+    e2e = None
+    if not args.no_e2e:
+        e2e_n_plans = plans
+        host_bytes = p * n * 4
+        if host_bytes <= (8 << 30):
+            hx = arenas[0].cpu().pin_memory()
+            hout = torch.empty(n, dtype=torch.float32).pin_memory()
+            staging = torch.empty((p + 1) * n, dtype=torch.float32, device=dev)
+            e_steps = max(3, min(args.steps, int(2.0 / (launches_per_step * host_bytes / 40e9)) or 1))
+            for _, h in e2e_n_plans:
+                rd.rd_reduce_host(h, hx, hout, staging, ops[0])
+            barrier()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(e_steps):
+                for _, h in e2e_n_plans:
+                    for op in ops:
+                        rd.rd_reduce_host(h, hx, hout, staging, op)
+            b.record()
+            barrier()
+            e_ms = a.elapsed_time(b)
+            if dist_on:
+                t = torch.tensor([e_ms], device=dev, dtype=torch.float64)
+                dist.all_reduce(t, op=dist.ReduceOp.MAX)
+                e_ms = float(t.item())
+            e2e = {"value": world * e_steps * launches_per_step * bytes_per_reduce / (e_ms * 1e-3) / 1e9, "unit": "GB/s",
+                   "h2d_bytes_per_step": launches_per_step * host_bytes, "d2h_bytes_per_step": launches_per_step * n * 4,
+                   "steps": e_steps}
+            del hx, hout, staging
+
+    if rank == 0:
+        peak, peak_src = measured_peak()
+        ms_per_launch = ms / (args.steps * launches_per_step)
+        achieved = bytes_per_reduce / (ms_per_launch * 1e-3) / 1e9
+        cpu = None
+        if not args.no_cpu_baseline and world == 1:
+            x, n_s = host_slab(w, wname, 1 << 30)
+            v, passes, dt = cpu_pass(dict(w, n=n_s), wname, x.numpy(), 10.0, 200)
+            cpu = {"value": v, "unit": "GB/s", "cores": 1, "kind": "oracle",
+                   "sample": "%d passes over every schedule x op on %d of %d elements per process (%.1f s)"
+                             % (passes, n_s, n, dt)}
+        line = {
+            "metric": "reduction_throughput", "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": wname, "p": p, "n_elems": n, "segment_bytes": w["seg_bytes"],
+                       "schedules": [s[0] for s in WORKLOAD_SCHEDULES[wname]], "ops": WORKLOAD_OPS[wname],
+                       "bytes_counted": "p*m + m per reduction",
+                       "l2": "inputs rotate over %d arenas of %.0f MiB each (> L2 between reuses)" % (n_arenas, p * n * 4 / 2**20)
+                             if n_arenas > 1 else "inputs (%.1f GiB) exceed L2" % (p * n * 4 / 2**30),
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": None, "peak_source": peak_src, "kernel": "rd_tree_kernel",
+                         "frac_of_nominal_8000": achieved / 8000.0},
+            "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": args.steps * launches_per_step, "clocks": clocks,
+            "per_schedule_gbs": per_schedule, "schedule_create_ms": create_ms,
+            "percent_of_peak": {"measured_copy": 100 * value / peak, "nominal_8TBs": 100 * value / 8000.0},
+        }
+        print(json.dumps(line), flush=True)
+    for _, h in plans:
+        rd.rd_destroy(h)
+    if dist_on:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -5,4 +5,4 @@ The package is a thin binding over librd.so (CUDA kernels + C ABI, built in-tree
 CPU path: calls raise when the library is missing.
 """
 from .binding import *  # noqa: F401,F403
-from .binding import lib, LIB_PATH, EXPORTS, ALGOS, RdError, LibraryMissing, rd_model_t, rd_stats_t  # noqa: F401
+from .binding import lib, LIB_PATH, EXPORTS, ALGOS, RdError, LibraryMissing, rd_model_t, rd_stats_t, PointerTable  # noqa: F401

@@ -169,41 +169,72 @@ def _dtype_code(t):
     raise TypeError("int32 or float32 expected, got %s" % t.dtype)
 
 
+class PointerTable:
+    """The host array of p device (or host) pointers rd_reduce takes, built once and reusable.
+
+    `inputs` is either one contiguous [p, n] tensor (row i = process i) or a sequence of p contiguous
+    1-D tensors.  The table keeps the tensors alive."""
+
+    def __init__(self, inputs):
+        import torch
+        if isinstance(inputs, torch.Tensor):
+            if inputs.dim() != 2 or not inputs.is_contiguous():
+                raise ValueError("a [p, n] contiguous tensor is expected")
+            self.p, self.n = int(inputs.shape[0]), int(inputs.shape[1])
+            addr = inputs.data_ptr() + np.arange(self.p, dtype=np.uint64) * np.uint64(self.n * inputs.element_size())
+            self.dtype, self.is_cuda, self.device = inputs.dtype, inputs.is_cuda, inputs.device
+        else:
+            rows = list(inputs)
+            if not rows:
+                raise ValueError("at least one process is needed")
+            self.p, self.n = len(rows), int(rows[0].numel())
+            for r in rows:
+                if not r.is_contiguous() or r.numel() != self.n or r.dtype != rows[0].dtype or r.is_cuda != rows[0].is_cuda:
+                    raise ValueError("every input must be contiguous, of the same length, dtype and placement")
+            addr = np.array([r.data_ptr() for r in rows], dtype=np.uint64)
+            self.dtype, self.is_cuda, self.device = rows[0].dtype, rows[0].is_cuda, rows[0].device
+        self._keep = inputs
+        self._addr = np.ascontiguousarray(addr)
+        self.array = C.cast(self._addr.ctypes.data, C.POINTER(C.c_void_p))
+
+
 def rd_reduce(h, inputs, out, op, exec_mode=RD_EXEC_TREE, stream=None, want_stats=False):
-    """inputs: list of p CUDA tensors (or one [p, n] tensor); out: CUDA tensor of n elements.
-    stream: a torch.cuda.Stream (default: the current one).  Returns rd_stats_t or None."""
+    """inputs: a PointerTable, a [p, n] CUDA tensor or a list of p CUDA tensors; out: CUDA tensor of n
+    elements.  stream: a torch.cuda.Stream (default: the current one).  Returns rd_stats_t or None."""
     import torch
-    rows = [inputs[i] for i in range(len(inputs))]
+    tab = inputs if isinstance(inputs, PointerTable) else PointerTable(inputs)
     n = out.numel()
-    for r in rows:
-        if not r.is_cuda or not r.is_contiguous() or r.numel() != n or r.dtype != out.dtype:
-            raise ValueError("every input must be a contiguous CUDA tensor with the output's dtype and length")
+    if not tab.is_cuda or tab.n != n or tab.dtype != out.dtype:
+        raise ValueError("every input must be a contiguous CUDA tensor with the output's dtype and length")
     if not out.is_cuda or not out.is_contiguous():
         raise ValueError("out must be a contiguous CUDA tensor")
-    ptrs = (C.c_void_p * len(rows))(*[r.data_ptr() for r in rows])
     s = stream if stream is not None else torch.cuda.current_stream(out.device)
     stats = rd_stats_t() if want_stats else None
-    with torch.cuda.device(out.device):
-        _check(lib().rd_reduce(h, ptrs, out.data_ptr(), n, _dtype_code(out), int(op), int(exec_mode),
+    prev = torch.cuda.current_device()
+    if out.device.index != prev:
+        torch.cuda.set_device(out.device)
+    try:
+        _check(lib().rd_reduce(h, tab.array, out.data_ptr(), n, _dtype_code(out), int(op), int(exec_mode),
                                s.cuda_stream, C.byref(stats) if want_stats else None), "rd_reduce")
+    finally:
+        if out.device.index != prev:
+            torch.cuda.set_device(prev)
     return stats
 
 
 def rd_reduce_host(h, inputs, out, staging, op, stream=None):
-    """inputs: list of p host tensors (pinned for asynchronous copies); out: host tensor;
-    staging: CUDA tensor of (p + 1) * n elements."""
+    """inputs: a PointerTable, a [p, n] host tensor or a list of p host tensors (pinned memory makes the
+    copies asynchronous); out: host tensor; staging: CUDA tensor of (p + 1) * n elements."""
     import torch
-    rows = [inputs[i] for i in range(len(inputs))]
+    tab = inputs if isinstance(inputs, PointerTable) else PointerTable(inputs)
     n = out.numel()
-    for r in rows:
-        if r.is_cuda or not r.is_contiguous() or r.numel() != n or r.dtype != out.dtype:
-            raise ValueError("every input must be a contiguous host tensor with the output's dtype and length")
-    if staging.numel() < (len(rows) + 1) * n or staging.dtype != out.dtype or not staging.is_cuda:
+    if tab.is_cuda or tab.n != n or tab.dtype != out.dtype or out.is_cuda:
+        raise ValueError("inputs and out must be contiguous host tensors of the same dtype and length")
+    if staging.numel() < (tab.p + 1) * n or staging.dtype != out.dtype or not staging.is_cuda:
         raise ValueError("staging must be a CUDA tensor of (p + 1) * n elements")
-    ptrs = (C.c_void_p * len(rows))(*[r.data_ptr() for r in rows])
     s = stream if stream is not None else torch.cuda.current_stream(staging.device)
     with torch.cuda.device(staging.device):
-        _check(lib().rd_reduce_host(h, ptrs, out.data_ptr(), staging.data_ptr(), n, _dtype_code(out), int(op),
+        _check(lib().rd_reduce_host(h, tab.array, out.data_ptr(), staging.data_ptr(), n, _dtype_code(out), int(op),
                                     s.cuda_stream), "rd_reduce_host")
 
 

@@ -21,8 +21,14 @@ constexpr int kPtrRing = 8;   // pointer tables in flight for p > kPackedPtrs
 struct DeviceTables {
     int device = -1;
     int sm_count = 0;
+    int smem_per_sm = 0;
     uint32_t *ops = nullptr;
     std::map<int, std::pair<TileDesc *, uint32_t>> tiles;   // vector width -> (device table, count)
+    // streaming (128-bit) path: tiles grouped per CTA, every CTA the same number of elements
+    uint32_t *cta_first = nullptr;
+    uint32_t n_ctas = 0;
+    int stages = 0;
+    int *status = nullptr;                                  // device word written by a kernel that gave up a wait
     // pointer tables for large p: pinned host ring + device ring, one event per slot
     void **h_ring = nullptr;
     void **d_ring = nullptr;
@@ -115,6 +121,8 @@ void release_device(DeviceTables &d)
     cudaGetDevice(&prev);
     cudaSetDevice(d.device);
     cudaFree(d.ops);
+    cudaFree(d.cta_first);
+    cudaFree(d.status);
     for (auto &kv : d.tiles) cudaFree(kv.second.first);
     if (d.h_ring) cudaFreeHost(d.h_ring);
     cudaFree(d.d_ring);
@@ -142,6 +150,9 @@ int upload(rd_schedule *s)
         cudaMemcpy(d.ops, s->progs.ops.data(), s->progs.ops.size() * sizeof(uint32_t), cudaMemcpyHostToDevice) != cudaSuccess)
         return RD_ERR_CUDA;
     if (cudaEventCreate(&d.ev_start) != cudaSuccess || cudaEventCreate(&d.ev_stop) != cudaSuccess) return RD_ERR_CUDA;
+    if (cudaMalloc(reinterpret_cast<void **>(&d.status), sizeof(int)) != cudaSuccess) return RD_ERR_NOMEM;
+    if (cudaMemset(d.status, 0, sizeof(int)) != cudaSuccess) return RD_ERR_CUDA;
+    d.smem_per_sm = int(prop.sharedMemPerMultiprocessor);
     if (s->p > kPackedPtrs) {
         const size_t bytes = size_t(kPtrRing) * size_t(s->p) * sizeof(void *);
         if (cudaHostAlloc(reinterpret_cast<void **>(&d.h_ring), bytes, cudaHostAllocDefault) != cudaSuccess) return RD_ERR_NOMEM;
@@ -152,28 +163,64 @@ int upload(rd_schedule *s)
     return RD_OK;
 }
 
-// Tiles of the tree kernel for one vector width: runs of at most `cap` elements inside a segment.
+// Tiles of the element-path kernel: runs of at most `cap` elements inside a segment.
+int upload_tiles(DeviceTables &d, int key, const std::vector<TileDesc> &host)
+{
+    if (host.size() > 0xFFFFFFFFull) return RD_ERR_UNSUPPORTED;
+    TileDesc *dev = nullptr;
+    if (cudaMalloc(reinterpret_cast<void **>(&dev), std::max<size_t>(host.size(), 1) * sizeof(TileDesc)) != cudaSuccess)
+        return RD_ERR_NOMEM;
+    if (!host.empty() && cudaMemcpy(dev, host.data(), host.size() * sizeof(TileDesc), cudaMemcpyHostToDevice) != cudaSuccess) {
+        cudaFree(dev);
+        return RD_ERR_CUDA;
+    }
+    d.tiles.emplace(key, std::make_pair(dev, uint32_t(host.size())));
+    return RD_OK;
+}
+
 int tiles_for(rd_schedule *s, int vec, const TileDesc **tiles, uint32_t *count)
 {
     DeviceTables &d = s->dev;
     auto it = d.tiles.find(vec);
     if (it == d.tiles.end()) {
-        const uint32_t cap = tree_tile_elems(vec);
-        std::vector<TileDesc> host;
         const std::vector<uint64_t> &off = s->sched.seg_off;
-        for (size_t j = 0; j + 1 < off.size(); j++)
-            for (uint64_t e = off[j]; e < off[j + 1]; e += cap)
-                host.push_back(TileDesc{e, uint32_t(std::min<uint64_t>(cap, off[j + 1] - e)), s->progs.seg_prog[j]});
-        if (host.size() > 0xFFFFFFFFull) return RD_ERR_UNSUPPORTED;
-        TileDesc *dev = nullptr;
-        if (cudaMalloc(reinterpret_cast<void **>(&dev), std::max<size_t>(host.size(), 1) * sizeof(TileDesc)) != cudaSuccess)
-            return RD_ERR_NOMEM;
-        if (!host.empty() &&
-            cudaMemcpy(dev, host.data(), host.size() * sizeof(TileDesc), cudaMemcpyHostToDevice) != cudaSuccess) {
-            cudaFree(dev);
-            return RD_ERR_CUDA;
+        std::vector<TileDesc> host;
+        if (vec == 4) {
+            // Streaming path.  The message is cut into one contiguous range per CTA, all of the same
+            // length up to one granule of 128 elements, so that every CTA moves the same number of
+            // bytes; a range is then cut at segment boundaries and at the stage capacity.
+            int ctasPerSm = 1;
+            stream_shape(s->progs.stack_depth, d.smem_per_sm, &ctasPerSm, &d.stages);
+            const uint64_t n = off.empty() ? 0 : off.back();
+            const uint64_t granule = 128, granules = (n + granule - 1) / granule;
+            const uint64_t ctas = std::min<uint64_t>(uint64_t(d.sm_count) * uint64_t(ctasPerSm), std::max<uint64_t>(granules, 1));
+            const uint32_t cap = tree_tile_elems(4);
+            std::vector<uint32_t> first(size_t(ctas) + 1, 0);
+            size_t seg = 0;
+            for (uint64_t c = 0; c < ctas; c++) {
+                const uint64_t lo = std::min(n, granules * c / ctas * granule), hi = std::min(n, granules * (c + 1) / ctas * granule);
+                first[size_t(c)] = uint32_t(host.size());
+                uint64_t e = lo;
+                while (e < hi) {
+                    while (seg + 1 < off.size() && off[seg + 1] <= e) seg++;
+                    const uint64_t end = std::min<uint64_t>(std::min<uint64_t>(hi, off[seg + 1]), e + cap);
+                    host.push_back(TileDesc{e, uint32_t(end - e), s->progs.seg_prog[seg]});
+                    e = end;
+                }
+            }
+            first[size_t(ctas)] = uint32_t(host.size());
+            if (cudaMalloc(reinterpret_cast<void **>(&d.cta_first), first.size() * sizeof(uint32_t)) != cudaSuccess) return RD_ERR_NOMEM;
+            if (cudaMemcpy(d.cta_first, first.data(), first.size() * sizeof(uint32_t), cudaMemcpyHostToDevice) != cudaSuccess)
+                return RD_ERR_CUDA;
+            d.n_ctas = uint32_t(ctas);
+        } else {
+            const uint32_t cap = tree_tile_elems(vec);
+            for (size_t j = 0; j + 1 < off.size(); j++)
+                for (uint64_t e = off[j]; e < off[j + 1]; e += cap)
+                    host.push_back(TileDesc{e, uint32_t(std::min<uint64_t>(cap, off[j + 1] - e)), s->progs.seg_prog[j]});
         }
-        it = d.tiles.emplace(vec, std::make_pair(dev, uint32_t(host.size()))).first;
+        if (int rc = upload_tiles(d, vec, host)) return rc;
+        it = d.tiles.find(vec);
     }
     *tiles = it->second.first;
     *count = it->second.second;
@@ -204,8 +251,9 @@ int reduce_tree(rd_schedule *s, const void *const *d_inputs, void *d_out, size_t
     }
     l.out = d_out; l.ops = d.ops; l.p = s->p; l.stack_depth = s->progs.stack_depth;
     l.dtype = int(dtype); l.op = int(op); l.sm_count = d.sm_count; l.stream = stream;
+    l.cta_first = d.cta_first; l.n_ctas = d.n_ctas; l.stages = d.stages; l.status = d.status; l.device = d.device;
     if (stats && cudaEventRecord(d.ev_start, stream) != cudaSuccess) return RD_ERR_CUDA;
-    if (launch_tree(l) != 0) return RD_ERR_CUDA;
+    if ((wide ? launch_tree_stream(l) : launch_tree(l)) != 0) return RD_ERR_CUDA;
     if (s->p > kPackedPtrs) {
         const int slot = (d.ring_next + kPtrRing - 1) % kPtrRing;
         if (cudaEventRecord(d.ring_done[slot], stream) != cudaSuccess) return RD_ERR_CUDA;
@@ -221,6 +269,10 @@ int reduce_tree(rd_schedule *s, const void *const *d_inputs, void *d_out, size_t
         stats->gbytes_per_s = ms > 0 ? double(stats->bytes_moved) / (double(ms) * 1e6) : 0.0;
         stats->predicted_s = double(s->sched.completion) * s->ticks.tick;
         stats->n_launches = l.n_tiles ? 1 : 0;
+        int st = 0;
+        if (cudaMemcpy(&st, d.status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return RD_ERR_CUDA;
+        stats->device_status = st;
+        if (st != 0) return RD_ERR_TIMEOUT;
     }
     return RD_OK;
 }

@@ -165,6 +165,203 @@ rd_tree_kernel(const __grid_constant__ TreeParams<PACKED> a)
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Streaming variant (128-bit path).  One producer thread per CTA walks (tile, operation) pairs in
+// program order and issues one bulk asynchronous copy (cp.async.bulk, global -> shared, completion
+// counted in bytes on an mbarrier) per operand tile into a ring of shared-memory stages; it runs
+// ahead across tile boundaries, so the number of bytes in flight per SM is set by the ring size,
+// not by registers or scoreboards.  256 consumer threads take the stages in the same order, each
+// reading its two 128-bit vectors of the stage, and execute the program on them.
+// Every wait is bounded: on expiry the thread records an error code and the CTA winds down (the
+// producer first waits, again bounded, for the copies it has issued).
+// ---------------------------------------------------------------------------------------------
+constexpr int kStageElems = 2048;                       // elements per stage = per tile (8 KB)
+constexpr int kStageBytes = kStageElems * 4;
+constexpr int kConsumers = 256;
+constexpr int kStreamThreads = kConsumers + 32;
+constexpr long long kWaitCycles = 4000000000ll;         // a wait gives up after about two seconds of SM clock
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return uint32_t(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait; false when it gave up or another thread of the CTA already did.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long start = clock64();
+    while (clock64() - start < kWaitCycles) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+    }
+    return false;
+}
+__device__ __forceinline__ void bulk_load(void *smem_dst, const void *gmem_src, uint32_t bytes, uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_addr(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+
+template <bool PACKED> struct StreamParams {
+    TreeParams<PACKED> t;
+    const uint32_t *cta_first;   // per CTA: first tile; n_ctas + 1 entries
+    int *status;                 // device word: 0, or the first error code
+    int stages, depth;
+};
+
+template <int DT, int OPR, bool PACKED>
+__global__ void __launch_bounds__(kStreamThreads, 2)
+rd_tree_stream_kernel(const __grid_constant__ StreamParams<PACKED> a)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const int S = a.stages;
+    uint4 *ring = reinterpret_cast<uint4 *>(smem_raw);                                      // [S][512]
+    uint4 *stack = reinterpret_cast<uint4 *>(smem_raw + size_t(S) * kStageBytes);            // [depth][2][256]
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem_raw + size_t(S + a.depth) * kStageBytes);
+    uint64_t *empty = full + S;
+    __shared__ int abort_flag;
+    const uint32_t tid = threadIdx.x;
+    const int p = a.t.p;
+    const uint32_t tile0 = a.cta_first[blockIdx.x], tile1 = a.cta_first[blockIdx.x + 1];
+
+    if (tid == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < S; s++) { mbar_init(full + s, 1); mbar_init(empty + s, kConsumers / 32); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (tid >= kConsumers) {
+        // ------------------------------------------------------------------ producer (one lane)
+        if (tid != kConsumers) return;
+        int stage = 0;
+        uint32_t phase = 0;
+        uint32_t issued = 0;
+        bool ok = true;
+        for (uint32_t tile = tile0; tile < tile1 && ok; tile++) {
+            const TileDesc td = a.t.tiles[tile];
+            const uint32_t *prog = a.t.ops + td.prog;
+            const uint32_t bytes = td.len * 4u;
+            for (int i = 0; i < p; i++) {
+                if (issued >= uint32_t(S) && !mbar_wait(empty + stage, phase ^ 1u, &abort_flag)) { ok = false; break; }
+                const uint32_t *src = a.t.input(__ldg(prog + i) & kIdxMask) + td.elem_off;
+                mbar_expect_tx(full + stage, bytes);
+                bulk_load(ring + size_t(stage) * (kStageBytes / 16), src, bytes, full + stage);
+                issued++;
+                if (++stage == S) { stage = 0; phase ^= 1u; }
+            }
+        }
+        if (!ok) {
+            if (!abort_flag) { atomicCAS(a.status, 0, -5); abort_flag = 1; }
+            // leave only after the copies already issued have landed (bounded)
+            const uint32_t pending = issued < uint32_t(S) ? issued : uint32_t(S);
+            for (uint32_t k = 0; k < pending; k++) {
+                // stage issued k+1 copies ago
+                int st = stage - 1 - int(k);
+                uint32_t ph = phase;
+                while (st < 0) { st += S; ph ^= 1u; }
+                const long long start = clock64();
+                while (!mbar_try_wait(full + st, ph) && clock64() - start < kWaitCycles) {}
+            }
+        }
+        return;
+    }
+
+    // ---------------------------------------------------------------------- consumers
+    const uint32_t lane = tid & 31u;
+    int stage = 0;
+    uint32_t phase = 0;
+    for (uint32_t tile = tile0; tile < tile1; tile++) {
+        const TileDesc td = a.t.tiles[tile];
+        const uint32_t *prog = a.t.ops + td.prog;
+        const bool live0 = tid * 4u < td.len, live1 = (kConsumers + tid) * 4u < td.len;
+        Vec<4> top0, top1;
+#pragma unroll
+        for (int v = 0; v < 4; v++) { top0.w[v] = 0; top1.w[v] = 0; }
+        int sp = 0;
+        uint32_t w = __ldg(prog);
+        for (int i = 0; i < p; i++) {
+            const uint32_t wn = (i + 1 < p) ? __ldg(prog + i + 1) : 0u;
+            if (!mbar_wait(full + stage, phase, &abort_flag)) {
+                if (!abort_flag) { atomicCAS(a.status, 0, -5); abort_flag = 1; }
+                return;
+            }
+            const uint4 *st = ring + size_t(stage) * (kStageBytes / 16);
+            uint4 r0 = make_uint4(0, 0, 0, 0), r1 = make_uint4(0, 0, 0, 0);
+            if (live0) r0 = st[tid];
+            if (live1) r1 = st[kConsumers + tid];
+            Vec<4> x0, x1;
+            x0.w[0] = r0.x; x0.w[1] = r0.y; x0.w[2] = r0.z; x0.w[3] = r0.w;
+            x1.w[0] = r1.x; x1.w[1] = r1.y; x1.w[2] = r1.z; x1.w[3] = r1.w;
+            const uint32_t kind = (w >> kIdxBits) & 3u;
+            if (kind == 1u) {
+                stack[(sp * 2 + 0) * kConsumers + tid] = make_uint4(top0.w[0], top0.w[1], top0.w[2], top0.w[3]);
+                stack[(sp * 2 + 1) * kConsumers + tid] = make_uint4(top1.w[0], top1.w[1], top1.w[2], top1.w[3]);
+                sp++;
+            }
+            if (kind <= 1u) {
+                top0 = x0; top1 = x1;
+            } else if (kind == 2u || OPR == OPR_SUM) {
+#pragma unroll
+                for (int v = 0; v < 4; v++) {
+                    top0.w[v] = combine<DT, OPR>(top0.w[v], x0.w[v]);
+                    top1.w[v] = combine<DT, OPR>(top1.w[v], x1.w[v]);
+                }
+            } else {
+#pragma unroll
+                for (int v = 0; v < 4; v++) {
+                    top0.w[v] = combine<DT, OPR>(x0.w[v], top0.w[v]);
+                    top1.w[v] = combine<DT, OPR>(x1.w[v], top1.w[v]);
+                }
+            }
+            // the stage's data is in registers: hand the stage back to the producer
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty + stage);
+            if (++stage == S) { stage = 0; phase ^= 1u; }
+            uint32_t npop = (w >> (kIdxBits + 2)) & 0xFu;
+            uint32_t roles = w >> (kIdxBits + 6);
+            while (npop--) {
+                sp--;
+                const bool poppedHeld = (roles & 1u) != 0;
+                roles >>= 1;
+                const uint4 y0 = stack[(sp * 2 + 0) * kConsumers + tid], y1 = stack[(sp * 2 + 1) * kConsumers + tid];
+                const uint32_t ya[4] = {y0.x, y0.y, y0.z, y0.w}, yb[4] = {y1.x, y1.y, y1.z, y1.w};
+#pragma unroll
+                for (int v = 0; v < 4; v++) {
+                    if (poppedHeld || OPR == OPR_SUM) {
+                        top0.w[v] = combine<DT, OPR>(ya[v], top0.w[v]);
+                        top1.w[v] = combine<DT, OPR>(yb[v], top1.w[v]);
+                    } else {
+                        top0.w[v] = combine<DT, OPR>(top0.w[v], ya[v]);
+                        top1.w[v] = combine<DT, OPR>(top1.w[v], yb[v]);
+                    }
+                }
+            }
+            w = wn;
+        }
+        uint32_t *dst = a.t.out + td.elem_off;
+        if (live0) store_stream<4>(dst + tid * 4u, top0);
+        if (live1) store_stream<4>(dst + (kConsumers + tid) * 4u, top1);
+    }
+}
+
 constexpr int kU = 2;   // vectors per thread per operation
 constexpr int kK = 4;   // operations fetched ahead
 
@@ -202,9 +399,67 @@ cudaError_t launch_dtop(const TreeLaunch &l)
     return packed ? launch_one<DT, OPR, 1, true>(l) : launch_one<DT, OPR, 1, false>(l);
 }
 
+template <int DT, int OPR, bool PACKED>
+cudaError_t launch_stream(const TreeLaunch &l)
+{
+    StreamParams<PACKED> prm;
+    if constexpr (PACKED) {
+        for (int i = 0; i < kPackedPtrs; i++) prm.t.in.ptr[i] = i < l.p ? static_cast<const uint32_t *>(l.host_ptrs[i]) : nullptr;
+    } else {
+        prm.t.in.table = reinterpret_cast<const uint32_t *const *>(l.dev_ptr_table);
+    }
+    prm.t.out = static_cast<uint32_t *>(l.out);
+    prm.t.tiles = l.tiles; prm.t.ops = l.ops; prm.t.n_tiles = l.n_tiles; prm.t.p = l.p;
+    prm.cta_first = l.cta_first; prm.status = l.status;
+    prm.stages = l.stages; prm.depth = l.stack_depth > 0 ? l.stack_depth : 1;
+    auto kernel = rd_tree_stream_kernel<DT, OPR, PACKED>;
+    const size_t smem = stream_smem_bytes(prm.stages, prm.depth);
+    static size_t configured[64] = {};     // per device: largest dynamic shared memory size opted into so far
+    const int dv = l.device & 63;
+    if (smem > configured[dv]) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+        if (e != cudaSuccess) return e;
+        configured[dv] = smem;
+    }
+    kernel<<<l.n_ctas, kStreamThreads, smem, static_cast<cudaStream_t>(l.stream)>>>(prm);
+    return cudaGetLastError();
+}
+
+template <int DT, int OPR>
+cudaError_t launch_stream_dtop(const TreeLaunch &l)
+{
+    return l.p <= kPackedPtrs ? launch_stream<DT, OPR, true>(l) : launch_stream<DT, OPR, false>(l);
+}
+
 }  // namespace
 
-uint32_t tree_tile_elems(int vec) { return uint32_t(kTreeThreads) * kU * uint32_t(vec); }
+uint32_t tree_tile_elems(int vec) { return vec == 4 ? uint32_t(kStageElems) : uint32_t(kTreeThreads) * kU * uint32_t(vec); }
+
+size_t stream_smem_bytes(int stages, int depth)
+{
+    return size_t(stages + depth) * kStageBytes + size_t(2 * stages) * sizeof(uint64_t);
+}
+
+void stream_shape(int stack_depth, int smem_per_sm, int *ctas_per_sm, int *stages)
+{
+    const int depth = stack_depth > 0 ? stack_depth : 1;
+    // two CTAs per SM when each still gets at least 6 stages, otherwise one
+    for (int ctas = 2; ctas >= 1; ctas--) {
+        const int budget = smem_per_sm / ctas - 2048;                 // leave room for the per-CTA reserve and statics
+        int s = (budget - depth * kStageBytes - 512) / kStageBytes;
+        if (s > 24) s = 24;
+        if (s >= 6 || ctas == 1) { *ctas_per_sm = ctas; *stages = s < 2 ? 2 : s; return; }
+    }
+}
+
+int launch_tree_stream(const TreeLaunch &l)
+{
+    if (l.n_tiles == 0 || l.n_ctas == 0) return 0;
+    cudaError_t e;
+    if (l.dtype == DT_INT32) e = l.op == OPR_SUM ? launch_stream_dtop<DT_INT32, OPR_SUM>(l) : launch_stream_dtop<DT_INT32, OPR_MAX>(l);
+    else e = l.op == OPR_SUM ? launch_stream_dtop<DT_FP32, OPR_SUM>(l) : launch_stream_dtop<DT_FP32, OPR_MAX>(l);
+    return int(e);
+}
 
 int launch_tree(const TreeLaunch &l)
 {

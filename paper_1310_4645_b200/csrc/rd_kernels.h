@@ -2,6 +2,7 @@
 #ifndef RD_KERNELS_H_
 #define RD_KERNELS_H_
 
+#include <cstddef>
 #include <cstdint>
 
 namespace rd {
@@ -28,13 +29,23 @@ struct TreeLaunch {
     int dtype, op;                    // rd_dtype_t, rd_op_t
     int vec;                          // 4: 128-bit path, 1: element path
     int sm_count;
+    int device;
     void *stream;
+    // streaming variant only
+    const uint32_t *cta_first;        // device: n_ctas + 1 offsets into tiles
+    uint32_t n_ctas;
+    int stages;
+    int *status;                      // device word
 };
 
 // Elements one tile may hold for the given vector width.
 uint32_t tree_tile_elems(int vec);
 // Launches the tree kernel; returns a cudaError_t value (0 = success).
 int launch_tree(const TreeLaunch &a);
+// Streaming variant (128-bit path): shape for a stack depth and the SM's shared memory, launch.
+void stream_shape(int stack_depth, int smem_per_sm, int *ctas_per_sm, int *stages);
+size_t stream_smem_bytes(int stages, int depth);
+int launch_tree_stream(const TreeLaunch &a);
 
 }  // namespace rd
 #endif

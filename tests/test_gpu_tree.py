@@ -104,9 +104,10 @@ def test_signed_zero_and_inf_follow_the_held_incoming_rule():
 
 def test_denormals_are_not_flushed():
     p, n = 4, 2048
-    x = torch.full((p, n), 1e-45, dtype=torch.float32, device="cuda")       # smallest subnormal
+    tiny = np.float32(2.0 ** -149)                                             # smallest subnormal
+    x = torch.full((p, n), float(tiny), dtype=torch.float32, device="cuda")
     got, _ = check(rd.RD_BINOMIAL, rd.RD_PORT_UNI, x, 0, "sum")
-    assert (got == np.float32(4e-45)).all() and got[0] > 0
+    assert (got == np.float32(2.0 ** -147)).all() and got[0] > 0
 
 
 def test_output_may_alias_the_roots_input():
