@@ -28,6 +28,7 @@ struct DeviceTables {
     uint32_t *cta_first = nullptr;
     uint32_t n_ctas = 0;
     int stages = 0;
+    int stage_elems = 0;
     int *status = nullptr;                                  // device word written by a kernel that gave up a wait
     // pointer tables for large p: pinned host ring + device ring, one event per slot
     void **h_ring = nullptr;
@@ -189,12 +190,13 @@ int tiles_for(rd_schedule *s, int vec, const TileDesc **tiles, uint32_t *count)
             // Streaming path.  The message is cut into one contiguous range per CTA, all of the same
             // length up to one granule of 128 elements, so that every CTA moves the same number of
             // bytes; a range is then cut at segment boundaries and at the stage capacity.
-            int ctasPerSm = 1;
-            stream_shape(s->progs.stack_depth, d.smem_per_sm, &ctasPerSm, &d.stages);
             const uint64_t n = off.empty() ? 0 : off.back();
+            d.stage_elems = stream_stage_elems(n / (uint64_t(d.sm_count) * 2) + 1);
+            int ctasPerSm = 1;
+            stream_shape(s->progs.stack_depth, d.smem_per_sm, d.stage_elems, &ctasPerSm, &d.stages);
             const uint64_t granule = 128, granules = (n + granule - 1) / granule;
             const uint64_t ctas = std::min<uint64_t>(uint64_t(d.sm_count) * uint64_t(ctasPerSm), std::max<uint64_t>(granules, 1));
-            const uint32_t cap = tree_tile_elems(4);
+            const uint32_t cap = uint32_t(d.stage_elems);
             std::vector<uint32_t> first(size_t(ctas) + 1, 0);
             size_t seg = 0;
             for (uint64_t c = 0; c < ctas; c++) {
@@ -203,9 +205,15 @@ int tiles_for(rd_schedule *s, int vec, const TileDesc **tiles, uint32_t *count)
                 uint64_t e = lo;
                 while (e < hi) {
                     while (seg + 1 < off.size() && off[seg + 1] <= e) seg++;
-                    const uint64_t end = std::min<uint64_t>(std::min<uint64_t>(hi, off[seg + 1]), e + cap);
-                    host.push_back(TileDesc{e, uint32_t(end - e), s->progs.seg_prog[seg]});
-                    e = end;
+                    // the part of the range inside this segment, in equal tiles of at most one stage
+                    const uint64_t pieceEnd = std::min<uint64_t>(hi, off[seg + 1]);
+                    const uint64_t parts = (pieceEnd - e + cap - 1) / cap;
+                    const uint64_t each = ((pieceEnd - e + parts - 1) / parts + 31) / 32 * 32;
+                    while (e < pieceEnd) {
+                        const uint64_t end = std::min<uint64_t>(pieceEnd, e + each);
+                        host.push_back(TileDesc{e, uint32_t(end - e), s->progs.seg_prog[seg]});
+                        e = end;
+                    }
                 }
             }
             first[size_t(ctas)] = uint32_t(host.size());
@@ -251,7 +259,7 @@ int reduce_tree(rd_schedule *s, const void *const *d_inputs, void *d_out, size_t
     }
     l.out = d_out; l.ops = d.ops; l.p = s->p; l.stack_depth = s->progs.stack_depth;
     l.dtype = int(dtype); l.op = int(op); l.sm_count = d.sm_count; l.stream = stream;
-    l.cta_first = d.cta_first; l.n_ctas = d.n_ctas; l.stages = d.stages; l.status = d.status; l.device = d.device;
+    l.cta_first = d.cta_first; l.n_ctas = d.n_ctas; l.stages = d.stages; l.stage_elems = d.stage_elems; l.status = d.status; l.device = d.device;
     if (stats && cudaEventRecord(d.ev_start, stream) != cudaSuccess) return RD_ERR_CUDA;
     if ((wide ? launch_tree_stream(l) : launch_tree(l)) != 0) return RD_ERR_CUDA;
     if (s->p > kPackedPtrs) {

@@ -166,19 +166,22 @@ rd_tree_kernel(const __grid_constant__ TreeParams<PACKED> a)
 }
 
 // ---------------------------------------------------------------------------------------------
-// Streaming variant (128-bit path).  One producer thread per CTA walks (tile, operation) pairs in
-// program order and issues one bulk asynchronous copy (cp.async.bulk, global -> shared, completion
-// counted in bytes on an mbarrier) per operand tile into a ring of shared-memory stages; it runs
-// ahead across tile boundaries, so the number of bytes in flight per SM is set by the ring size,
-// not by registers or scoreboards.  256 consumer threads take the stages in the same order, each
-// reading its two 128-bit vectors of the stage, and execute the program on them.
-// Every wait is bounded: on expiry the thread records an error code and the CTA winds down (the
-// producer first waits, again bounded, for the copies it has issued).
+// Streaming variant (128-bit path).  Two producer threads per CTA (one per producer warp) walk the
+// CTA's (tile, operation) pairs in program order and issue one bulk asynchronous copy
+// (cp.async.bulk, global -> shared, completion counted in bytes on an mbarrier) per operand tile
+// into a ring of shared-memory stages; they run ahead across tile boundaries, so the number of
+// bytes in flight per SM is set by the ring, not by registers or scoreboards.  256 consumer
+// threads take the stages in the same order, each reading its (up to) two 128-bit vectors of the
+// stage, and execute the program on them.  The stage size is a launch parameter (up to 2048
+// elements).
+// Every wait is bounded: on expiry the thread records an error code and the CTA winds down (a
+// producer lane first waits, again bounded, for the copy it has in flight).
 // ---------------------------------------------------------------------------------------------
-constexpr int kStageElems = 2048;                       // elements per stage = per tile (8 KB)
-constexpr int kStageBytes = kStageElems * 4;
+constexpr int kMaxStageElems = 2048;                    // largest stage = largest tile (8 KB)
+constexpr int kMaxStages = 32;
 constexpr int kConsumers = 256;
-constexpr int kStreamThreads = kConsumers + 32;
+constexpr int kProducers = 2;                            // producer warps per CTA (one active lane each)
+constexpr int kStreamThreads = kConsumers + 32 * kProducers;
 constexpr long long kWaitCycles = 4000000000ll;         // a wait gives up after about two seconds of SM clock
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p) { return uint32_t(__cvta_generic_to_shared(p)); }
@@ -223,7 +226,7 @@ template <bool PACKED> struct StreamParams {
     TreeParams<PACKED> t;
     const uint32_t *cta_first;   // per CTA: first tile; n_ctas + 1 entries
     int *status;                 // device word: 0, or the first error code
-    int stages, depth;
+    int stages, depth, stage_elems;
 };
 
 template <int DT, int OPR, bool PACKED>
@@ -232,9 +235,12 @@ rd_tree_stream_kernel(const __grid_constant__ StreamParams<PACKED> a)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int S = a.stages;
-    uint4 *ring = reinterpret_cast<uint4 *>(smem_raw);                                      // [S][512]
-    uint4 *stack = reinterpret_cast<uint4 *>(smem_raw + size_t(S) * kStageBytes);            // [depth][2][256]
-    uint64_t *full = reinterpret_cast<uint64_t *>(smem_raw + size_t(S + a.depth) * kStageBytes);
+    const uint32_t stageVecs = uint32_t(a.stage_elems) / 4u;                                 // 128-bit vectors per stage
+    uint4 *ring = reinterpret_cast<uint4 *>(smem_raw);                                       // [S][stageVecs]
+    const bool two = a.stage_elems > 4 * kConsumers;                                         // a second vector per thread
+    const uint32_t levelVecs = two ? 2u * kConsumers : uint32_t(kConsumers);
+    uint4 *stack = ring + size_t(S) * stageVecs;                                              // [depth][1 or 2][256]
+    uint64_t *full = reinterpret_cast<uint64_t *>(stack + size_t(a.depth) * levelVecs);
     uint64_t *empty = full + S;
     __shared__ int abort_flag;
     const uint32_t tid = threadIdx.x;
@@ -249,36 +255,44 @@ rd_tree_stream_kernel(const __grid_constant__ StreamParams<PACKED> a)
     __syncthreads();
 
     if (tid >= kConsumers) {
-        // ------------------------------------------------------------------ producer (one lane)
-        if (tid != kConsumers) return;
-        int stage = 0;
-        uint32_t phase = 0;
-        uint32_t issued = 0;
-        bool ok = true;
-        for (uint32_t tile = tile0; tile < tile1 && ok; tile++) {
-            const TileDesc td = a.t.tiles[tile];
-            const uint32_t *prog = a.t.ops + td.prog;
-            const uint32_t bytes = td.len * 4u;
-            for (int i = 0; i < p; i++) {
-                if (issued >= uint32_t(S) && !mbar_wait(empty + stage, phase ^ 1u, &abort_flag)) { ok = false; break; }
-                const uint32_t *src = a.t.input(__ldg(prog + i) & kIdxMask) + td.elem_off;
-                mbar_expect_tx(full + stage, bytes);
-                bulk_load(ring + size_t(stage) * (kStageBytes / 16), src, bytes, full + stage);
-                issued++;
-                if (++stage == S) { stage = 0; phase ^= 1u; }
-            }
+        // ------------------------------------------------------------------ producers
+        // One lane in each of the kProducers producer warps.  Producer j owns the steps j, j + P,
+        // j + 2P, ... of this CTA's sequence of (tile, operation) pairs and issues them in order:
+        // stages are released by the consumers in that same order, so a producer never waits for a
+        // stage while a later one of its own is already free.  Being alone in its warp, a producer
+        // polls without divergence; the table look-ups of a step are issued before its wait.
+        if ((tid & 31u) != 0) return;
+        const int P = kProducers < S ? kProducers : S;
+        const int j = int(tid - kConsumers) / 32;
+        if (j >= P) return;
+        uint32_t tile = tile0;
+        int i = j;
+        while (i >= p && tile < tile1) { i -= p; tile++; }
+        int stage = j % S;
+        uint32_t laps = 0;                      // times this producer has gone round the ring
+        uint32_t cur = 0xFFFFFFFFu;
+        TileDesc td = TileDesc{0, 0, 0};
+        bool ok = true, any = false;
+        int lastStage = 0;
+        uint32_t lastLap = 0;
+        while (tile < tile1) {
+            if (tile != cur) { td = a.t.tiles[tile]; cur = tile; }
+            const uint32_t *src = a.t.input(__ldg(a.t.ops + td.prog + i) & kIdxMask) + td.elem_off;
+            if (laps >= 1u && !mbar_wait(empty + stage, (laps - 1u) & 1u, &abort_flag)) { ok = false; break; }
+            mbar_expect_tx(full + stage, td.len * 4u);
+            bulk_load(ring + size_t(stage) * stageVecs, src, td.len * 4u, full + stage);
+            any = true; lastStage = stage; lastLap = laps;
+            i += P;
+            while (i >= p && tile < tile1) { i -= p; tile++; }
+            stage += P;
+            if (stage >= S) { stage -= S; laps++; }
         }
         if (!ok) {
             if (!abort_flag) { atomicCAS(a.status, 0, -5); abort_flag = 1; }
-            // leave only after the copies already issued have landed (bounded)
-            const uint32_t pending = issued < uint32_t(S) ? issued : uint32_t(S);
-            for (uint32_t k = 0; k < pending; k++) {
-                // stage issued k+1 copies ago
-                int st = stage - 1 - int(k);
-                uint32_t ph = phase;
-                while (st < 0) { st += S; ph ^= 1u; }
+            // leave only after this producer's last copy has landed (bounded); its earlier ones were consumed
+            if (any) {
                 const long long start = clock64();
-                while (!mbar_try_wait(full + st, ph) && clock64() - start < kWaitCycles) {}
+                while (!mbar_try_wait(full + lastStage, lastLap & 1u) && clock64() - start < kWaitCycles) {}
             }
         }
         return;
@@ -303,7 +317,7 @@ rd_tree_stream_kernel(const __grid_constant__ StreamParams<PACKED> a)
                 if (!abort_flag) { atomicCAS(a.status, 0, -5); abort_flag = 1; }
                 return;
             }
-            const uint4 *st = ring + size_t(stage) * (kStageBytes / 16);
+            const uint4 *st = ring + size_t(stage) * stageVecs;
             uint4 r0 = make_uint4(0, 0, 0, 0), r1 = make_uint4(0, 0, 0, 0);
             if (live0) r0 = st[tid];
             if (live1) r1 = st[kConsumers + tid];
@@ -312,8 +326,8 @@ rd_tree_stream_kernel(const __grid_constant__ StreamParams<PACKED> a)
             x1.w[0] = r1.x; x1.w[1] = r1.y; x1.w[2] = r1.z; x1.w[3] = r1.w;
             const uint32_t kind = (w >> kIdxBits) & 3u;
             if (kind == 1u) {
-                stack[(sp * 2 + 0) * kConsumers + tid] = make_uint4(top0.w[0], top0.w[1], top0.w[2], top0.w[3]);
-                stack[(sp * 2 + 1) * kConsumers + tid] = make_uint4(top1.w[0], top1.w[1], top1.w[2], top1.w[3]);
+                stack[sp * levelVecs + tid] = make_uint4(top0.w[0], top0.w[1], top0.w[2], top0.w[3]);
+                if (two) stack[sp * levelVecs + kConsumers + tid] = make_uint4(top1.w[0], top1.w[1], top1.w[2], top1.w[3]);
                 sp++;
             }
             if (kind <= 1u) {
@@ -341,7 +355,8 @@ rd_tree_stream_kernel(const __grid_constant__ StreamParams<PACKED> a)
                 sp--;
                 const bool poppedHeld = (roles & 1u) != 0;
                 roles >>= 1;
-                const uint4 y0 = stack[(sp * 2 + 0) * kConsumers + tid], y1 = stack[(sp * 2 + 1) * kConsumers + tid];
+                const uint4 y0 = stack[sp * levelVecs + tid];
+                const uint4 y1 = two ? stack[sp * levelVecs + kConsumers + tid] : make_uint4(0, 0, 0, 0);
                 const uint32_t ya[4] = {y0.x, y0.y, y0.z, y0.w}, yb[4] = {y1.x, y1.y, y1.z, y1.w};
 #pragma unroll
                 for (int v = 0; v < 4; v++) {
@@ -411,9 +426,9 @@ cudaError_t launch_stream(const TreeLaunch &l)
     prm.t.out = static_cast<uint32_t *>(l.out);
     prm.t.tiles = l.tiles; prm.t.ops = l.ops; prm.t.n_tiles = l.n_tiles; prm.t.p = l.p;
     prm.cta_first = l.cta_first; prm.status = l.status;
-    prm.stages = l.stages; prm.depth = l.stack_depth > 0 ? l.stack_depth : 1;
+    prm.stages = l.stages; prm.depth = l.stack_depth > 0 ? l.stack_depth : 1; prm.stage_elems = l.stage_elems;
     auto kernel = rd_tree_stream_kernel<DT, OPR, PACKED>;
-    const size_t smem = stream_smem_bytes(prm.stages, prm.depth);
+    const size_t smem = stream_smem_bytes(prm.stages, prm.depth, prm.stage_elems);
     static size_t configured[64] = {};     // per device: largest dynamic shared memory size opted into so far
     const int dv = l.device & 63;
     if (smem > configured[dv]) {
@@ -433,22 +448,34 @@ cudaError_t launch_stream_dtop(const TreeLaunch &l)
 
 }  // namespace
 
-uint32_t tree_tile_elems(int vec) { return vec == 4 ? uint32_t(kStageElems) : uint32_t(kTreeThreads) * kU * uint32_t(vec); }
+uint32_t tree_tile_elems(int vec) { return uint32_t(kTreeThreads) * kU * uint32_t(vec); }
 
-size_t stream_smem_bytes(int stages, int depth)
+// One stack level holds one 128-bit vector per consumer thread, two when a stage has more than 1024 elements.
+static int stack_level_bytes(int stage_elems) { return (stage_elems > 4 * kConsumers ? 2 : 1) * kConsumers * 16; }
+
+size_t stream_smem_bytes(int stages, int depth, int stage_elems)
 {
-    return size_t(stages + depth) * kStageBytes + size_t(2 * stages) * sizeof(uint64_t);
+    return size_t(stages) * size_t(stage_elems) * 4 + size_t(depth) * stack_level_bytes(stage_elems) + size_t(2 * stages) * sizeof(uint64_t);
 }
 
-void stream_shape(int stack_depth, int smem_per_sm, int *ctas_per_sm, int *stages)
+int stream_stage_elems(uint64_t elems_per_cta)
+{
+    // Measured on B200: the time per bulk copy hardly depends on its size up to 8 KB, so smaller
+    // stages only lower the throughput, also for small messages.  The kernel accepts 512 and 1024.
+    (void)elems_per_cta;
+    return kMaxStageElems;
+}
+
+void stream_shape(int stack_depth, int smem_per_sm, int stage_elems, int *ctas_per_sm, int *stages)
 {
     const int depth = stack_depth > 0 ? stack_depth : 1;
-    // two CTAs per SM when each still gets at least 6 stages, otherwise one
+    const int stageBytes = stage_elems * 4;
+    // two CTAs per SM when each still gets at least 48 KB of ring, otherwise one
     for (int ctas = 2; ctas >= 1; ctas--) {
         const int budget = smem_per_sm / ctas - 2048;                 // leave room for the per-CTA reserve and statics
-        int s = (budget - depth * kStageBytes - 512) / kStageBytes;
-        if (s > 24) s = 24;
-        if (s >= 6 || ctas == 1) { *ctas_per_sm = ctas; *stages = s < 2 ? 2 : s; return; }
+        int s = (budget - depth * stack_level_bytes(stage_elems) - 512) / stageBytes;
+        if (s > kMaxStages) s = kMaxStages;
+        if (s * stageBytes >= 48 * 1024 || ctas == 1) { *ctas_per_sm = ctas; *stages = s < 2 ? 2 : s; return; }
     }
 }
 

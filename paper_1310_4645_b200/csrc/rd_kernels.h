@@ -35,16 +35,19 @@ struct TreeLaunch {
     const uint32_t *cta_first;        // device: n_ctas + 1 offsets into tiles
     uint32_t n_ctas;
     int stages;
+    int stage_elems;
     int *status;                      // device word
 };
 
-// Elements one tile may hold for the given vector width.
+// Elements one tile of the element-path kernel may hold for the given vector width.
 uint32_t tree_tile_elems(int vec);
 // Launches the tree kernel; returns a cudaError_t value (0 = success).
 int launch_tree(const TreeLaunch &a);
-// Streaming variant (128-bit path): shape for a stack depth and the SM's shared memory, launch.
-void stream_shape(int stack_depth, int smem_per_sm, int *ctas_per_sm, int *stages);
-size_t stream_smem_bytes(int stages, int depth);
+// Streaming variant (128-bit path): stage size for a CTA's share of the message, ring shape for a
+// stack depth and the SM's shared memory, launch.
+int stream_stage_elems(uint64_t elems_per_cta);
+void stream_shape(int stack_depth, int smem_per_sm, int stage_elems, int *ctas_per_sm, int *stages);
+size_t stream_smem_bytes(int stages, int depth, int stage_elems);
 int launch_tree_stream(const TreeLaunch &a);
 
 }  // namespace rd
