@@ -199,6 +199,7 @@ def main():
     ap.add_argument("--workload", default="config2", choices=sorted(WORKLOAD_SCHEDULES))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-large", action="store_true", help="skip the extra large-message (config4) measurement")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -336,8 +337,47 @@ def main():
                    "steps": e_steps}
             del hx, hout, staging
 
+    # the large-message workload (1 GiB per process), measured beside the main one when it fits
+    large = None
+    if not args.no_large and world == 1 and wname != "config4":
+        del arenas, tables
+        torch.cuda.empty_cache()
+        free_b, _ = torch.cuda.mem_get_info(dev)
+        w4 = WORKLOADS["config4"]
+        need = (w4["p"] + 1) * w4["n"] * 4
+        if free_b > need + (4 << 30):
+            x4 = make_inputs(w4["p"], w4["n"], w4["dist"], w4["seed"], device=str(dev))
+            t4 = rd.PointerTable(x4)
+            out4 = torch.empty(w4["n"], dtype=torch.float32, device=dev)
+            m4 = (w4["alpha"], w4["beta"], w4["gamma"])
+            res, tot_ms, tot_b = {}, 0.0, 0
+            for label, algo_name, bidir in WORKLOAD_SCHEDULES["config4"]:
+                h4 = rd.rd_schedule_create(rd.ALGOS[algo_name], rd.RD_PORT_BI if bidir else rd.RD_PORT_UNI, w4["p"],
+                                           4 * w4["n"], w4["seg_bytes"], *m4)
+                for opname in WORKLOAD_OPS["config4"]:
+                    op = rd.RD_SUM if opname == "sum" else rd.RD_MAX
+                    for _ in range(3):
+                        rd.rd_reduce(h4, t4, out4, op)
+                    torch.cuda.synchronize()
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record()
+                    for _ in range(10):
+                        rd.rd_reduce(h4, t4, out4, op)
+                    b.record()
+                    torch.cuda.synchronize()
+                    res["%s/%s" % (label, opname)] = round(need * 10 / (a.elapsed_time(b) * 1e-3) / 1e9, 1)
+                    tot_ms += a.elapsed_time(b); tot_b += need * 10
+                rd.rd_destroy(h4)
+            large = {"workload": "config4", "p": w4["p"], "n_elems": w4["n"], "segment_bytes": w4["seg_bytes"],
+                     "value": tot_b / (tot_ms * 1e-3) / 1e9, "unit": "GB/s", "per_schedule_gbs": res,
+                     "l2": "inputs (32 GiB) exceed L2"}
+            del x4, out4, t4
+
     if rank == 0:
         peak, peak_src = measured_peak()
+        if large:
+            large["frac_of_measured_peak"] = large["value"] / peak
+            large["frac_of_nominal_8000"] = large["value"] / 8000.0
         ms_per_launch = ms / (args.steps * launches_per_step)
         achieved = bytes_per_reduce / (ms_per_launch * 1e-3) / 1e9
         cpu = None
@@ -358,10 +398,10 @@ def main():
                              if n_arenas > 1 else "inputs (%.1f GiB) exceed L2" % (p * n * 4 / 2**30),
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": None, "peak_source": peak_src, "kernel": "rd_tree_kernel",
+                         "traffic": None, "peak_source": peak_src, "kernel": "rd_tree_stream_kernel",
                          "frac_of_nominal_8000": achieved / 8000.0},
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": args.steps * launches_per_step, "clocks": clocks,
-            "per_schedule_gbs": per_schedule, "schedule_create_ms": create_ms,
+            "per_schedule_gbs": per_schedule, "schedule_create_ms": create_ms, "large_message": large,
             "percent_of_peak": {"measured_copy": 100 * value / peak, "nominal_8TBs": 100 * value / 8000.0},
         }
         print(json.dumps(line), flush=True)

@@ -205,16 +205,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
                  : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait; false when it gave up or another thread of the CTA already did.
+// Bounded wait; false when it gave up or another thread of the CTA already did.  try_wait suspends
+// the thread in hardware for a while, so the loop turns slowly; the clock and the abort flag are
+// only looked at every 64 turns.
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    const long long start = clock64();
-    while (clock64() - start < kWaitCycles) {
+    long long start = 0;
+    for (uint32_t turns = 1;; turns++) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
+        if ((turns & 63u) == 0u) {
+            if (*abort_flag) return false;
+            const long long now = clock64();
+            if (start == 0) start = now;
+            else if (now - start > kWaitCycles) return false;
+        }
     }
-    return false;
 }
 __device__ __forceinline__ void bulk_load(void *smem_dst, const void *gmem_src, uint32_t bytes, uint64_t *bar)
 {
