@@ -215,6 +215,51 @@ RD_API int rd_schedule_upload(rd_schedule_t *s);
 RD_API int rd_reduce_host(rd_schedule_t *s, const void *const *h_inputs, void *h_out, void *d_staging,
                    size_t n_elems, rd_dtype_t dtype, rd_op_t op, void *cuda_stream);
 
+/*
+ * rd_schedule_set_wait_budget -- the longest a block of the schedule-faithful kernel waits for
+ * another process before it gives up (default 2 s, at most 60 s).  When a wait runs out the
+ * kernel ends by itself, rd_reduce returns RD_ERR_TIMEOUT and the schedule stays usable.  The
+ * paper has no counterpart: its processes block in MPI_Recv.
+ */
+RD_API int rd_schedule_set_wait_budget(rd_schedule_t *s, double seconds);
+
+/*
+ * rd_schedule_trace -- measured times of the last schedule-faithful rd_reduce, to set against
+ * the model's alpha + beta*s (+ gamma*s) per pair (Section V).  For every send/receive pair, in
+ * the order of rd_schedule_events, three values in nanoseconds of the GPU's global timer, taken by
+ * the receiver's first block: when the receiver was ready for the pair, when the sender's data
+ * became available to it, and when the combined segment was written.
+ *   t_ns  host; 3 * n_events values; cap_events = capacity in pairs (RD_ERR_TOO_SMALL).
+ * RD_ERR_UNSUPPORTED before any schedule-faithful run.
+ */
+RD_API int rd_schedule_trace(const rd_schedule_t *s, uint64_t *t_ns, size_t cap_events);
+
+/*
+ * rd_schedule_faithful_shape -- how the schedule-faithful kernel will run this schedule on the
+ * current device: thread blocks per process, scratch slots per process (Section V: a process that
+ * has received but not yet sent a segment must keep its partial result; uni-greedy needs one such
+ * buffer, bi-greedy more, Section VI-B) and the bytes of scratch the schedule allocates for them.
+ * Allocates that scratch if it has not been allocated yet.  Any output pointer may be NULL.
+ */
+RD_API int rd_schedule_faithful_shape(rd_schedule_t *s, int *blocks_per_process, int *slots_per_process,
+                                      size_t *scratch_bytes);
+
+/*
+ * rd_schedule_actions -- what one process does in the schedule-faithful execution: its own sends
+ * and receives in start-time order (Section IV: sending and receiving processors are paired; after
+ * a processor sends a segment it is reduced for it).  Host work only.  Each action is 8 int32:
+ *   seg, peer, kind (0 receive and combine, 1 receive and store, 2 send),
+ *   slot (where this process keeps its value of the segment: >= 0 scratch slot, -1 its input,
+ *   -2 the output buffer), peer_slot (receive: the same for the sender), first (receive: 1 when
+ *   the held operand is this process's own input), event (index of the pair in
+ *   rd_schedule_events), wait_event (receive into a recycled slot: the pair that must have been
+ *   taken before the slot is overwritten, else -1).
+ *   buf host, capacity cap_actions actions; n_actions / slots_per_process may be NULL.
+ * RD_ERR_TOO_SMALL leaves buf untouched but still reports n_actions.
+ */
+RD_API int rd_schedule_actions(const rd_schedule_t *s, int process, int32_t *buf, size_t cap_actions,
+                               size_t *n_actions, int *slots_per_process);
+
 /* rd_destroy -- frees the schedule and its device tables.  NULL is allowed. */
 RD_API void rd_destroy(rd_schedule_t *s);
 

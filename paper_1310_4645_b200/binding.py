@@ -27,7 +27,8 @@ ALGOS = {"uni_greedy": RD_UNI_GREEDY, "bi_greedy": RD_BI_GREEDY, "binomial": RD_
 
 EXPORTS = ("rd_schedule_create", "rd_schedule_create_segments", "rd_optimal_segment", "rd_schedule_info",
            "rd_schedule_events", "rd_schedule_segments", "rd_schedule_program", "rd_reduce",
-           "rd_schedule_upload", "rd_reduce_host", "rd_destroy", "rd_strerror")
+           "rd_schedule_upload", "rd_reduce_host", "rd_destroy", "rd_strerror", "rd_schedule_set_wait_budget",
+           "rd_schedule_trace", "rd_schedule_faithful_shape", "rd_schedule_actions")
 
 
 class rd_model_t(C.Structure):
@@ -77,6 +78,10 @@ def lib():
         L.rd_reduce.argtypes = [vp, C.POINTER(vp), vp, sz, i32, i32, i32, vp, C.POINTER(rd_stats_t)]
         L.rd_schedule_upload.argtypes = [vp]
         L.rd_reduce_host.argtypes = [vp, C.POINTER(vp), vp, vp, sz, i32, i32, vp]
+        L.rd_schedule_set_wait_budget.argtypes = [vp, C.c_double]
+        L.rd_schedule_trace.argtypes = [vp, vp, sz]
+        L.rd_schedule_faithful_shape.argtypes = [vp, C.POINTER(i32), C.POINTER(i32), C.POINTER(sz)]
+        L.rd_schedule_actions.argtypes = [vp, i32, vp, sz, C.POINTER(sz), C.POINTER(i32)]
         L.rd_destroy.argtypes = [vp]
         L.rd_destroy.restype = None
         L.rd_strerror.argtypes = [i32]
@@ -236,6 +241,39 @@ def rd_reduce_host(h, inputs, out, staging, op, stream=None):
     with torch.cuda.device(staging.device):
         _check(lib().rd_reduce_host(h, tab.array, out.data_ptr(), staging.data_ptr(), n, _dtype_code(out), int(op),
                                     s.cuda_stream), "rd_reduce_host")
+
+
+def rd_schedule_set_wait_budget(h, seconds) -> None:
+    _check(lib().rd_schedule_set_wait_budget(h, float(seconds)), "rd_schedule_set_wait_budget")
+
+
+def rd_schedule_trace(h) -> np.ndarray:
+    """[n_events, 3] uint64 nanoseconds: receiver ready, data available, combine written."""
+    n = rd_schedule_info(h)["n_events"]
+    t = np.zeros((n, 3), dtype=np.uint64)
+    _check(lib().rd_schedule_trace(h, t.ctypes.data, n), "rd_schedule_trace")
+    return t
+
+
+def rd_schedule_faithful_shape(h) -> dict:
+    b, s, sc = C.c_int(), C.c_int(), C.c_size_t()
+    _check(lib().rd_schedule_faithful_shape(h, C.byref(b), C.byref(s), C.byref(sc)), "rd_schedule_faithful_shape")
+    return dict(blocks_per_process=b.value, slots_per_process=s.value, scratch_bytes=sc.value)
+
+
+ACTION_FIELDS = ("seg", "peer", "kind", "slot", "peer_slot", "first", "event", "wait_event")
+
+
+def rd_schedule_actions(h, process):
+    """(actions as an [n, 8] int32 array with columns ACTION_FIELDS, scratch slots per process)."""
+    n, slots = C.c_size_t(), C.c_int()
+    rc = lib().rd_schedule_actions(h, int(process), None, 0, C.byref(n), C.byref(slots))
+    if rc not in (RD_OK, RD_ERR_TOO_SMALL):
+        raise RdError(rc, "rd_schedule_actions")
+    buf = np.zeros((n.value, 8), dtype=np.int32)
+    _check(lib().rd_schedule_actions(h, int(process), buf.ctypes.data, n.value, C.byref(n), C.byref(slots)),
+           "rd_schedule_actions")
+    return buf, slots.value
 
 
 def rd_destroy(h) -> None:

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librd.so")
-SOURCES = ["rd_api.cpp", "rd_sched.cpp", "rd_compile.cpp", "rd_kernels.cu"]
+SOURCES = ["rd_api.cpp", "rd_sched.cpp", "rd_compile.cpp", "rd_kernels.cu", "rd_faithful.cu"]
 HEADERS = ["rd_internal.h", "rd_kernels.h"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -36,6 +36,20 @@ struct DeviceTables {
     cudaEvent_t ring_done[kPtrRing] = {};
     int ring_next = 0;
     cudaEvent_t ev_start = nullptr, ev_stop = nullptr;
+    // schedule-faithful execution (allocated on its first use)
+    bool faithful_ready = false;
+    FaithfulAction *f_actions = nullptr;
+    uint32_t *f_first = nullptr;
+    uint64_t *f_seg_off = nullptr;
+    uint32_t *f_flags = nullptr;            // posted, then taken: 2 * n_events * lanes words
+    unsigned long long *f_trace = nullptr, *f_block_times = nullptr;
+    uint32_t *f_scratch = nullptr;
+    const uint32_t **f_inputs = nullptr;
+    int *f_abort = nullptr;
+    int f_lanes = 0, f_slots = 0;
+    uint64_t f_slot_elems = 0;
+    uint32_t f_epoch = 0;
+    bool f_traced = false;
 };
 
 }  // namespace
@@ -50,6 +64,7 @@ struct rd_schedule {
     std::vector<int64_t> seg_bytes;
     Schedule sched;
     Programs progs;
+    double wait_budget_s = 2.0;             // bound of one wait inside the faithful kernel
     DeviceTables dev;
 };
 
@@ -130,6 +145,8 @@ void release_device(DeviceTables &d)
     for (auto &e : d.ring_done) if (e) cudaEventDestroy(e);
     if (d.ev_start) cudaEventDestroy(d.ev_start);
     if (d.ev_stop) cudaEventDestroy(d.ev_stop);
+    cudaFree(d.f_actions); cudaFree(d.f_first); cudaFree(d.f_seg_off); cudaFree(d.f_flags); cudaFree(d.f_trace);
+    cudaFree(d.f_block_times); cudaFree(d.f_scratch); cudaFree(d.f_inputs); cudaFree(d.f_abort);
     if (prev >= 0) cudaSetDevice(prev);
     d = DeviceTables();
 }
@@ -285,6 +302,127 @@ int reduce_tree(rd_schedule *s, const void *const *d_inputs, void *d_out, size_t
     return RD_OK;
 }
 
+
+template <typename T> int dev_alloc(T **ptr, size_t count)
+{
+    return cudaMalloc(reinterpret_cast<void **>(ptr), std::max<size_t>(count, 1) * sizeof(T)) == cudaSuccess ? RD_OK : RD_ERR_NOMEM;
+}
+
+// Device tables and scratch of the schedule-faithful execution, built on its first use.
+int prepare_faithful(rd_schedule *s)
+{
+    DeviceTables &d = s->dev;
+    if (d.faithful_ready) return RD_OK;
+    ActionLists lists;
+    const size_t q = s->sched.seg_off.size() - 1;
+    if (int rc = build_actions(s->p, q, s->sched.events, lists)) return rc;
+    // all blocks have to be resident together: lanes per process from the least occupant variant
+    int perSm = 1 << 30;
+    for (int dt = 0; dt < 2; dt++)
+        for (int op = 0; op < 2; op++)
+            for (int wide = 0; wide < 2; wide++) {
+                int b = 0;
+                if (faithful_blocks_per_sm(dt, op, wide != 0, &b) != 0) return RD_ERR_CUDA;
+                perSm = std::min(perSm, b);
+            }
+    const long long capacity = (long long)perSm * d.sm_count;
+    if (capacity < s->p) return RD_ERR_UNSUPPORTED;
+    d.f_lanes = int(std::min<long long>(16, capacity / s->p));
+    d.f_slots = std::max(lists.slots_per_proc, 1);
+    uint64_t longest = 0;
+    for (size_t j = 0; j < q; j++) longest = std::max(longest, s->sched.seg_off[j + 1] - s->sched.seg_off[j]);
+    d.f_slot_elems = (longest + 3) / 4 * 4;
+    const size_t nEvents = s->sched.events.size();
+    std::vector<FaithfulAction> acts(lists.actions.size());
+    for (size_t k = 0; k < acts.size(); k++) {
+        const Action &a = lists.actions[k];
+        acts[k] = FaithfulAction{a.seg, a.peer, a.kind, a.slot, a.peer_slot, a.first, a.event, a.wait_event};
+    }
+    if (dev_alloc(&d.f_actions, acts.size()) || dev_alloc(&d.f_first, lists.first.size()) ||
+        dev_alloc(&d.f_seg_off, s->sched.seg_off.size()) || dev_alloc(&d.f_flags, 2 * nEvents * size_t(d.f_lanes)) ||
+        dev_alloc(&d.f_trace, 3 * nEvents) || dev_alloc(&d.f_block_times, 2 * size_t(s->p) * size_t(d.f_lanes)) ||
+        dev_alloc(&d.f_inputs, size_t(s->p)) || dev_alloc(&d.f_abort, 1) ||
+        dev_alloc(&d.f_scratch, size_t(s->p) * size_t(d.f_slots) * size_t(d.f_slot_elems)))
+        return RD_ERR_NOMEM;
+    bool ok = true;
+    ok = ok && (acts.empty() || cudaMemcpy(d.f_actions, acts.data(), acts.size() * sizeof(FaithfulAction), cudaMemcpyHostToDevice) == cudaSuccess);
+    ok = ok && cudaMemcpy(d.f_first, lists.first.data(), lists.first.size() * sizeof(uint32_t), cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemcpy(d.f_seg_off, s->sched.seg_off.data(), s->sched.seg_off.size() * sizeof(uint64_t), cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemset(d.f_flags, 0, std::max<size_t>(2 * nEvents * size_t(d.f_lanes), 1) * sizeof(uint32_t)) == cudaSuccess;
+    ok = ok && cudaMemset(d.f_trace, 0, std::max<size_t>(3 * nEvents, 1) * sizeof(unsigned long long)) == cudaSuccess;
+    ok = ok && cudaMemset(d.f_abort, 0, sizeof(int)) == cudaSuccess;
+    if (!ok) return RD_ERR_CUDA;
+    d.f_epoch = 0;
+    d.faithful_ready = true;
+    return RD_OK;
+}
+
+int reduce_faithful(rd_schedule *s, const void *const *d_inputs, void *d_out, size_t n, rd_dtype_t dtype, rd_op_t op,
+                    cudaStream_t stream, rd_stats_t *stats)
+{
+    DeviceTables &d = s->dev;
+    rd_stats_t st;
+    std::memset(&st, 0, sizeof(st));
+    st.bytes_moved = uint64_t(s->p + 1) * uint64_t(n) * 4u;
+    st.predicted_s = double(s->sched.completion) * s->ticks.tick;
+    if (n == 0) { if (stats) *stats = st; return RD_OK; }
+    if (cudaEventRecord(d.ev_start, stream) != cudaSuccess) return RD_ERR_CUDA;
+    if (s->p == 1) {
+        // a single process holds the result already
+        if (d_out != d_inputs[0] && cudaMemcpyAsync(d_out, d_inputs[0], n * 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+            return RD_ERR_CUDA;
+    } else {
+        if (int rc = prepare_faithful(s)) return rc;
+        bool wide = (reinterpret_cast<uintptr_t>(d_out) & 15u) == 0;
+        for (int i = 0; i < s->p && wide; i++) wide = (reinterpret_cast<uintptr_t>(d_inputs[i]) & 15u) == 0;
+        for (size_t j = 0; j < s->sched.seg_off.size() && wide; j++) wide = (s->sched.seg_off[j] & 3u) == 0;
+        if (cudaMemcpyAsync(d.f_inputs, d_inputs, size_t(s->p) * sizeof(void *), cudaMemcpyHostToDevice, stream) != cudaSuccess)
+            return RD_ERR_CUDA;
+        if (++d.f_epoch == 0) d.f_epoch = 1;
+        const size_t nEvents = s->sched.events.size();
+        FaithfulParams prm{};
+        prm.inputs = reinterpret_cast<const uint32_t *const *>(d.f_inputs);
+        prm.out = static_cast<uint32_t *>(d_out);
+        prm.scratch = d.f_scratch; prm.actions = d.f_actions; prm.first = d.f_first; prm.seg_off = d.f_seg_off;
+        prm.posted = d.f_flags; prm.taken = d.f_flags + nEvents * size_t(d.f_lanes);
+        prm.trace = d.f_trace; prm.block_times = d.f_block_times; prm.status = d.status; prm.abort_flag = d.f_abort;
+        int khz = 0;
+        cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, d.device);
+        prm.wait_cycles = (long long)(s->wait_budget_s * double(khz > 0 ? khz : 1000000) * 1e3);
+        prm.epoch = d.f_epoch; prm.n_procs = s->p; prm.lanes = d.f_lanes; prm.slots = d.f_slots;
+        prm.slot_elems = d.f_slot_elems; prm.blocking_send = s->port == RD_PORT_UNI ? 1 : 0;
+        if (launch_faithful(prm, int(dtype), int(op), wide, stream) != 0) return RD_ERR_CUDA;
+        st.n_launches = 1;
+        d.f_traced = true;
+    }
+    if (cudaEventRecord(d.ev_stop, stream) != cudaSuccess || cudaEventSynchronize(d.ev_stop) != cudaSuccess) return RD_ERR_CUDA;
+    float ms = 0;
+    if (cudaEventElapsedTime(&ms, d.ev_start, d.ev_stop) != cudaSuccess) return RD_ERR_CUDA;
+    st.kernel_ms = ms;
+    st.gbytes_per_s = ms > 0 ? double(st.bytes_moved) / (double(ms) * 1e6) : 0.0;
+    if (s->p > 1) {
+        int status = 0;
+        if (cudaMemcpy(&status, d.status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return RD_ERR_CUDA;
+        st.device_status = status;
+        if (status != 0) {
+            // leave the flags usable for the next call: new epoch, cleared status and abort flag
+            cudaMemset(d.status, 0, sizeof(int));
+            cudaMemset(d.f_abort, 0, sizeof(int));
+            if (stats) *stats = st;
+            return RD_ERR_TIMEOUT;
+        }
+        std::vector<unsigned long long> bt(2 * size_t(s->p) * size_t(d.f_lanes));
+        if (cudaMemcpy(bt.data(), d.f_block_times, bt.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost) != cudaSuccess)
+            return RD_ERR_CUDA;
+        unsigned long long begin = ~0ull, end = 0;
+        for (size_t b = 0; b < bt.size() / 2; b++) begin = std::min(begin, bt[2 * b]);
+        for (int g = 0; g < d.f_lanes; g++) end = std::max(end, bt[2 * size_t(g) + 1]);     // the root's blocks
+        st.makespan_ns = end > begin ? double(end - begin) : 0.0;
+    }
+    if (stats) *stats = st;
+    return RD_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -407,7 +545,8 @@ int rd_reduce(rd_schedule_t *s, const void *const *d_inputs, void *d_out, size_t
         if ((n_elems > 0 && !d_inputs[i]) || (reinterpret_cast<uintptr_t>(d_inputs[i]) & 3u)) return RD_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(d_out) & 3u) return RD_ERR_INVALID_ARG;
     if (int rc = upload(s)) return rc;
-    if (exec == RD_EXEC_FAITHFUL) return RD_ERR_UNSUPPORTED;
+    if (exec == RD_EXEC_FAITHFUL)
+        return reduce_faithful(s, d_inputs, d_out, n_elems, dtype, op, static_cast<cudaStream_t>(cuda_stream), stats);
     return reduce_tree(s, d_inputs, d_out, n_elems, dtype, op, static_cast<cudaStream_t>(cuda_stream), stats);
 }
 
@@ -431,6 +570,61 @@ int rd_reduce_host(rd_schedule_t *s, const void *const *h_inputs, void *h_out, v
     if (int rc = rd_reduce(s, dptr.data(), d_out, n_elems, dtype, op, RD_EXEC_TREE, cuda_stream, nullptr)) return rc;
     if (n_elems > 0 && cudaMemcpyAsync(h_out, d_out, n_elems * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return RD_ERR_CUDA;
     if (cudaStreamSynchronize(stream) != cudaSuccess) return RD_ERR_CUDA;
+    return RD_OK;
+}
+
+int rd_schedule_set_wait_budget(rd_schedule_t *s, double seconds)
+{
+    if (!s || !(seconds > 0) || !(seconds <= 60.0)) return RD_ERR_INVALID_ARG;
+    s->wait_budget_s = seconds;
+    return RD_OK;
+}
+
+int rd_schedule_trace(const rd_schedule_t *s, uint64_t *t_ns, size_t cap_events)
+{
+    if (!s || !t_ns) return RD_ERR_INVALID_ARG;
+    const size_t n = s->sched.events.size();
+    if (cap_events < n) return RD_ERR_TOO_SMALL;
+    if (!s->dev.f_traced) return RD_ERR_UNSUPPORTED;
+    if (n > 0 && cudaMemcpy(t_ns, s->dev.f_trace, 3 * n * sizeof(uint64_t), cudaMemcpyDeviceToHost) != cudaSuccess) return RD_ERR_CUDA;
+    return RD_OK;
+}
+
+int rd_schedule_faithful_shape(rd_schedule_t *s, int *blocks_per_process, int *slots_per_process, size_t *scratch_bytes)
+{
+    if (!s) return RD_ERR_INVALID_ARG;
+    if (s->p < 2) {
+        if (blocks_per_process) *blocks_per_process = 0;
+        if (slots_per_process) *slots_per_process = 0;
+        if (scratch_bytes) *scratch_bytes = 0;
+        return RD_OK;
+    }
+    if (int rc = upload(s)) return rc;
+    if (int rc = prepare_faithful(s)) return rc;
+    if (blocks_per_process) *blocks_per_process = s->dev.f_lanes;
+    if (slots_per_process) *slots_per_process = s->dev.f_slots;
+    if (scratch_bytes) *scratch_bytes = size_t(s->p) * size_t(s->dev.f_slots) * size_t(s->dev.f_slot_elems) * 4;
+    return RD_OK;
+}
+
+int rd_schedule_actions(const rd_schedule_t *s, int process, int32_t *buf, size_t cap_actions, size_t *n_actions, int *slots_per_process)
+{
+    if (!s || process < 0 || process >= s->p || (!buf && cap_actions > 0)) return RD_ERR_INVALID_ARG;
+    ActionLists lists;
+    try {
+        if (int rc = build_actions(s->p, s->sched.seg_off.size() - 1, s->sched.events, lists)) return rc;
+    } catch (const std::bad_alloc &) {
+        return RD_ERR_NOMEM;
+    }
+    const uint32_t k0 = lists.first[size_t(process)], k1 = lists.first[size_t(process) + 1];
+    if (n_actions) *n_actions = k1 - k0;
+    if (slots_per_process) *slots_per_process = lists.slots_per_proc;
+    if (cap_actions < k1 - k0) return RD_ERR_TOO_SMALL;
+    for (uint32_t k = k0; k < k1; k++) {
+        const Action &a = lists.actions[k];
+        const int32_t v[8] = {a.seg, a.peer, a.kind, a.slot, a.peer_slot, a.first, a.event, a.wait_event};
+        std::memcpy(buf + size_t(k - k0) * 8, v, sizeof(v));
+    }
     return RD_OK;
 }
 

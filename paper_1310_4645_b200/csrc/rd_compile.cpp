@@ -150,4 +150,77 @@ int compile_programs(int p, size_t q, const std::vector<rd_event_t> &events, Pro
     return RD_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Schedule-faithful execution: every process gets the list of its own sends and receives in
+// start-time order (a send before a receive that starts at the same tick: with two ports a send
+// is only a posting).  A process keeps its partial result of a segment in a scratch slot from its
+// first receive of the segment until the send of that segment has been taken by the receiver;
+// slots are recycled first-freed-first once the freeing send lies in the past of the schedule, and
+// a receive into a recycled slot names the send whose completion it has to see first.  The root accumulates straight into the output buffer.
+// ---------------------------------------------------------------------------------------------
+int build_actions(int p, size_t q, const std::vector<rd_event_t> &events, ActionLists &out)
+{
+    const size_t P = size_t(p);
+    out.actions.clear();
+    out.first.assign(P + 1, 0);
+    out.slots_per_proc = 0;
+    for (const rd_event_t &e : events) { out.first[size_t(e.src) + 1]++; out.first[size_t(e.dst) + 1]++; }
+    for (size_t i = 0; i < P; i++) out.first[i + 1] += out.first[i];
+    out.actions.resize(out.first[P]);
+    // events are ordered by start time; two passes keep "sends first" among equal times
+    std::vector<uint32_t> fill(out.first.begin(), out.first.end() - 1);
+    for (size_t k = 0; k < events.size();) {
+        size_t k1 = k;
+        while (k1 < events.size() && events[k1].t_start == events[k].t_start) k1++;
+        for (size_t e = k; e < k1; e++) {
+            Action a{events[e].seg, events[e].dst, 2, -1, -1, 0, int32_t(e), -1};
+            out.actions[fill[size_t(events[e].src)]++] = a;
+        }
+        for (size_t e = k; e < k1; e++) {
+            Action a{events[e].seg, events[e].src, events[e].kind == 0 ? 0 : 1, -1, -1, 0, int32_t(e), -1};
+            out.actions[fill[size_t(events[e].dst)]++] = a;
+        }
+        k = k1;
+    }
+    // slots, process by process
+    std::vector<int32_t> senderSlot(events.size(), -1);
+    std::vector<int32_t> cur(q), arrivals(q);
+    std::vector<std::pair<int32_t, int32_t>> freed;     // (slot, send that must be taken), oldest first
+    for (size_t i = 0; i < P; i++) {
+        std::fill(cur.begin(), cur.end(), -1);
+        std::fill(arrivals.begin(), arrivals.end(), 0);
+        freed.clear();
+        size_t freedHead = 0;
+        int used = 0;
+        for (uint32_t k = out.first[i]; k < out.first[i + 1]; k++) {
+            Action &a = out.actions[k];
+            const size_t j = size_t(a.seg);
+            if (a.kind == 2) {
+                a.slot = i == 0 ? -2 : cur[j];
+                if (i == 0 && arrivals[j] == 0) a.slot = -1;          // the root forwards its own input
+                senderSlot[size_t(a.event)] = a.slot;
+                if (a.slot >= 0) { freed.push_back(std::make_pair(a.slot, a.event)); cur[j] = -1; }
+                arrivals[j] = 0;
+            } else {
+                a.first = arrivals[j] == 0 ? 1 : 0;
+                arrivals[j]++;
+                if (i == 0) { a.slot = -2; continue; }
+                if (cur[j] < 0) {
+                    // recycle only a slot whose send started earlier than this receive: the schedule
+                    // itself then expects it to be over; otherwise take a fresh one
+                    if (freedHead < freed.size() &&
+                        events[size_t(freed[freedHead].second)].t_start < events[size_t(a.event)].t_start) {
+                        cur[j] = freed[freedHead].first; a.wait_event = freed[freedHead].second; freedHead++;
+                    } else cur[j] = used++;
+                }
+                a.slot = cur[j];
+            }
+        }
+        out.slots_per_proc = std::max(out.slots_per_proc, used);
+    }
+    for (Action &a : out.actions)
+        if (a.kind != 2) a.peer_slot = senderSlot[size_t(a.event)];
+    return RD_OK;
+}
+
 }  // namespace rd

@@ -1,0 +1,199 @@
+// Schedule-faithful execution on sm_100a: groups of thread blocks play the processes.
+//
+// Process i is played by G thread blocks ("lanes"); lane g owns the same 1/G share of every
+// segment, so the G lanes are G independent copies of the whole p-process system working on
+// disjoint element ranges and never synchronise with each other.  Each block walks its process's
+// action list in order:
+//   send     post a flag for the pair (release), so that the receiver may read the value this
+//            process holds for the segment (its input, or its partial result in a scratch slot);
+//            with one port per process the sender then waits until the receiver has taken it.
+//   receive  wait for the sender's flag (acquire), read the sender's value, combine it with the value
+//            held here (held operand first) or just store it, write the result to this process's
+//            slot (the root: to the output), then raise the pair's "taken" flag.
+// Flags carry the launch's epoch number, so they never need clearing.  Every wait is bounded by a
+// clock budget: when it runs out the block records RD_ERR_TIMEOUT, raises a global abort flag that
+// all other waits watch, and leaves; nothing traps and nothing spins forever.
+// All blocks must be resident at once (cooperative launch).
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "rd_kernels.h"
+
+namespace rd {
+
+namespace {
+
+enum { DT_INT32 = 0, DT_FP32 = 1 };
+enum { OPR_SUM = 0, OPR_MAX = 1 };
+
+template <int DT, int OPR> __device__ __forceinline__ uint32_t combine(uint32_t held, uint32_t in)
+{
+    if (DT == DT_INT32) {
+        if (OPR == OPR_SUM) return held + in;
+        return (int32_t(in) > int32_t(held)) ? in : held;
+    } else {
+        const float h = __uint_as_float(held), i = __uint_as_float(in);
+        if (OPR == OPR_SUM) return __float_as_uint(__fadd_rn(h, i));
+        return (i > h) ? in : held;
+    }
+}
+
+__device__ __forceinline__ unsigned long long now_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ uint32_t load_acquire(const uint32_t *p)
+{
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void store_release(uint32_t *p, uint32_t v)
+{
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+// Thread 0 waits until *flag == epoch; everybody learns the outcome.  False: gave up or aborted.
+__device__ __forceinline__ bool wait_flag(const uint32_t *flag, uint32_t epoch, const FaithfulParams &a, int *sh_ok)
+{
+    if (threadIdx.x == 0) {
+        int ok = 1;
+        if (load_acquire(flag) != epoch) {
+            const long long start = clock64();
+            uint32_t turns = 0;
+            while (load_acquire(flag) != epoch) {
+                __nanosleep(40);
+                if ((++turns & 15u) == 0u) {
+                    if (*reinterpret_cast<volatile int *>(a.abort_flag) != 0) { ok = 0; break; }
+                    if (clock64() - start > a.wait_cycles) {
+                        atomicCAS(a.status, 0, -5);
+                        atomicExch(a.abort_flag, 1);
+                        ok = 0;
+                        break;
+                    }
+                }
+            }
+        }
+        *sh_ok = ok;
+    }
+    __syncthreads();
+    const bool ok = *sh_ok != 0;
+    __syncthreads();
+    return ok;
+}
+
+template <int DT, int OPR, int V>
+__global__ void __launch_bounds__(kFaithfulThreads, 8)
+rd_faithful_kernel(const FaithfulParams a)
+{
+    __shared__ int sh_ok;
+    const int proc = int(blockIdx.x) / a.lanes, lane = int(blockIdx.x) % a.lanes;
+    const uint32_t k0 = a.first[proc], k1 = a.first[proc + 1];
+    const uint32_t *mine = a.inputs[proc];
+    unsigned long long t_begin = 0, t_end = 0;
+    if (threadIdx.x == 0) t_begin = now_ns();
+    bool alive = true;
+    for (uint32_t k = k0; k < k1 && alive; k++) {
+        const FaithfulAction act = a.actions[k];
+        uint32_t *posted = a.posted + size_t(act.event) * a.lanes + lane;
+        uint32_t *taken = a.taken + size_t(act.event) * a.lanes + lane;
+        if (act.kind == 2) {
+            // everything this block wrote for the segment is ordered before the flag
+            __syncthreads();
+            if (threadIdx.x == 0) { __threadfence(); store_release(posted, a.epoch); }
+            if (a.blocking_send) alive = wait_flag(taken, a.epoch, a, &sh_ok);
+            continue;
+        }
+        unsigned long long t_ready = 0, t_start = 0;
+        if (threadIdx.x == 0 && lane == 0) t_ready = now_ns();
+        if (act.wait_event >= 0)
+            alive = wait_flag(a.taken + size_t(act.wait_event) * a.lanes + lane, a.epoch, a, &sh_ok);
+        if (alive) alive = wait_flag(posted, a.epoch, a, &sh_ok);
+        if (!alive) break;
+        if (threadIdx.x == 0 && lane == 0) t_start = now_ns();
+        // this lane's share of the segment, in whole vectors
+        const uint64_t seg_lo = a.seg_off[act.seg], seg_len = a.seg_off[act.seg + 1] - seg_lo;
+        const uint64_t units = (seg_len + V - 1) / V;
+        const uint64_t lo = units * uint64_t(lane) / uint64_t(a.lanes) * V;
+        uint64_t hi = units * uint64_t(lane + 1) / uint64_t(a.lanes) * V;
+        if (hi > seg_len) hi = seg_len;
+        const uint32_t *src = act.peer_slot >= 0 ? a.scratch + (size_t(act.peer) * a.slots + size_t(act.peer_slot)) * a.slot_elems
+                              : act.peer_slot == -1 ? a.inputs[act.peer] + seg_lo : a.out + seg_lo;
+        uint32_t *dst = act.slot >= 0 ? a.scratch + (size_t(proc) * a.slots + size_t(act.slot)) * a.slot_elems : a.out + seg_lo;
+        const uint32_t *held = act.first ? mine + seg_lo : dst;
+        const bool store_only = act.kind == 1;
+        for (uint64_t e = lo + uint64_t(threadIdx.x) * V; e < hi; e += uint64_t(kFaithfulThreads) * V) {
+            if (V == 4) {
+                const uint4 in = __ldcg(reinterpret_cast<const uint4 *>(src + e));
+                uint4 r = in;
+                if (!store_only) {
+                    const uint4 h = __ldcg(reinterpret_cast<const uint4 *>(held + e));
+                    r.x = combine<DT, OPR>(h.x, in.x); r.y = combine<DT, OPR>(h.y, in.y);
+                    r.z = combine<DT, OPR>(h.z, in.z); r.w = combine<DT, OPR>(h.w, in.w);
+                }
+                __stcg(reinterpret_cast<uint4 *>(dst + e), r);
+            } else {
+                const uint32_t in = __ldcg(src + e);
+                const uint32_t r = store_only ? in : combine<DT, OPR>(__ldcg(held + e), in);
+                __stcg(dst + e, r);
+            }
+        }
+        // the sender's value has been read: tell it
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            __threadfence();
+            store_release(taken, a.epoch);
+            t_end = now_ns();
+            if (lane == 0) {
+                a.trace[size_t(act.event) * 3 + 0] = t_ready;
+                a.trace[size_t(act.event) * 3 + 1] = t_start;
+                a.trace[size_t(act.event) * 3 + 2] = t_end;
+            }
+        }
+    }
+    if (threadIdx.x == 0) {
+        if (t_end == 0) t_end = now_ns();
+        a.block_times[size_t(blockIdx.x) * 2 + 0] = t_begin;
+        a.block_times[size_t(blockIdx.x) * 2 + 1] = t_end;
+    }
+}
+
+template <int DT, int OPR>
+cudaError_t launch_dtop(const FaithfulParams &prm, bool wide, cudaStream_t stream, bool occupancy_only, int *blocks_per_sm)
+{
+    const void *fn = wide ? reinterpret_cast<const void *>(rd_faithful_kernel<DT, OPR, 4>)
+                          : reinterpret_cast<const void *>(rd_faithful_kernel<DT, OPR, 1>);
+    if (occupancy_only) {
+        return wide ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, rd_faithful_kernel<DT, OPR, 4>, kFaithfulThreads, 0)
+                    : cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, rd_faithful_kernel<DT, OPR, 1>, kFaithfulThreads, 0);
+    }
+    FaithfulParams copy = prm;
+    void *args[] = {&copy};
+    return cudaLaunchCooperativeKernel(fn, dim3(unsigned(prm.n_procs * prm.lanes)), dim3(kFaithfulThreads), args, 0, stream);
+}
+
+cudaError_t dispatch(const FaithfulParams &prm, int dtype, int op, bool wide, cudaStream_t stream, bool occ, int *bps)
+{
+    if (dtype == DT_INT32) return op == OPR_SUM ? launch_dtop<DT_INT32, OPR_SUM>(prm, wide, stream, occ, bps)
+                                                 : launch_dtop<DT_INT32, OPR_MAX>(prm, wide, stream, occ, bps);
+    return op == OPR_SUM ? launch_dtop<DT_FP32, OPR_SUM>(prm, wide, stream, occ, bps)
+                         : launch_dtop<DT_FP32, OPR_MAX>(prm, wide, stream, occ, bps);
+}
+
+}  // namespace
+
+int faithful_blocks_per_sm(int dtype, int op, bool wide, int *blocks_per_sm)
+{
+    FaithfulParams dummy{};
+    return int(dispatch(dummy, dtype, op, wide, nullptr, true, blocks_per_sm));
+}
+
+int launch_faithful(const FaithfulParams &prm, int dtype, int op, bool wide, void *stream)
+{
+    return int(dispatch(prm, dtype, op, wide, static_cast<cudaStream_t>(stream), false, nullptr));
+}
+
+}  // namespace rd

@@ -51,19 +51,20 @@ int compile_programs(int p, size_t q, const std::vector<rd_event_t> &events, Pro
 
 // One step of a process in the schedule-faithful execution.
 struct Action {
-    int32_t seg;        // segment (index into seg_off)
-    int32_t peer;       // the other process
-    int32_t kind;       // 0 receive+combine, 1 receive+store, 2 send
-    int32_t slot;       // partial-result slot of this process used by the action (-1: its own input / the output)
-    int32_t peer_slot;  // receive: slot of the sender holding the data (-1: the sender's input)
-    int32_t first;      // receive: 1 when this is the first arrival of the segment (held operand = own input)
-    int32_t seq;        // send: 1-based number of this send among the sender's sends; receive: the matching number
-    int32_t wait_ack;   // receive: number of own sends that must have been taken before the slot may be overwritten
+    int32_t seg;         // segment (index into seg_off)
+    int32_t peer;        // the other process
+    int32_t kind;        // 0 receive and combine, 1 receive and store, 2 send
+    int32_t slot;        // where this process keeps its value of the segment: >= 0 a scratch slot,
+                         // -1 its own input (a send of a segment it never received), -2 the output (root)
+    int32_t peer_slot;   // receive: where the sender keeps the value it sends (same encoding)
+    int32_t first;       // receive: 1 when the held operand is the process's own input
+    int32_t event;       // index of the send/receive pair in the schedule's event list (its flags)
+    int32_t wait_event;  // receive into a recycled slot: the pair that must have been taken first, or -1
 };
 struct ActionLists {
-    std::vector<Action> actions;      // all processes back to back
+    std::vector<Action> actions;      // all processes back to back, each in start-time order
     std::vector<uint32_t> first;      // p+1 offsets
-    int slots_per_proc = 0;
+    int slots_per_proc = 0;           // scratch slots (of one largest segment each) a process needs
 };
 int build_actions(int p, size_t q, const std::vector<rd_event_t> &events, ActionLists &out);
 

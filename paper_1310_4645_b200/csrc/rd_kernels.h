@@ -50,5 +50,35 @@ void stream_shape(int stack_depth, int smem_per_sm, int stage_elems, int *ctas_p
 size_t stream_smem_bytes(int stages, int depth, int stage_elems);
 int launch_tree_stream(const TreeLaunch &a);
 
+// ---- schedule-faithful execution (rd_faithful.cu)
+constexpr int kFaithfulThreads = 128;
+
+struct FaithfulAction {            // device copy of one step of a process (see rd::Action)
+    int32_t seg, peer, kind, slot, peer_slot, first, event, wait_event;
+};
+
+struct FaithfulParams {
+    const uint32_t *const *inputs;   // device table of the p input pointers
+    uint32_t *out;
+    uint32_t *scratch;               // [p][slots][slot_elems]
+    const FaithfulAction *actions;   // all processes back to back
+    const uint32_t *first;           // p+1 offsets into actions
+    const uint64_t *seg_off;         // q+1 segment boundaries, elements
+    uint32_t *posted, *taken;        // [n_events][lanes], hold the epoch of the launch that raised them
+    unsigned long long *trace;       // [n_events][3]: receiver ready, transfer start, combine end (ns), lane 0 only
+    unsigned long long *block_times; // [blocks][2]: first action start, last action end (ns)
+    int *status;                     // 0 or RD_ERR_TIMEOUT
+    int *abort_flag;
+    long long wait_cycles;           // budget of one wait, SM clock cycles
+    uint32_t epoch;
+    int n_procs, lanes, slots;
+    uint64_t slot_elems;
+    int blocking_send;               // 1: a send waits until it has been taken (one port per process)
+};
+
+// Resident blocks per SM of the kernel variant (0 = success), and the cooperative launch itself.
+int faithful_blocks_per_sm(int dtype, int op, bool wide, int *blocks_per_sm);
+int launch_faithful(const FaithfulParams &prm, int dtype, int op, bool wide, void *stream);
+
 }  // namespace rd
 #endif
