@@ -256,6 +256,11 @@ RD_API int rd_schedule_faithful_shape(rd_schedule_t *s, int *blocks_per_process,
  *   taken before the slot is overwritten, else -1).
  *   buf host, capacity cap_actions actions; n_actions / slots_per_process may be NULL.
  * RD_ERR_TOO_SMALL leaves buf untouched but still reports n_actions.
+ * On the GPU a process is played by G thread blocks that never synchronise with each other; block
+ * g works on offsets [U*g/G, U*(g+1)/G) * v of every segment, clipped to the segment's length,
+ * with v = 4 elements on the 128-bit path (else 1) and U = ceil(L / v) for the largest segment
+ * length L rounded up to a multiple of 4: the same offsets for every segment, so that blocks which
+ * are at different points of the schedule never meet in a scratch slot.
  */
 RD_API int rd_schedule_actions(const rd_schedule_t *s, int process, int32_t *buf, size_t cap_actions,
                                size_t *n_actions, int *slots_per_process);

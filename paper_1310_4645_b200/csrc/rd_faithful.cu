@@ -1,8 +1,9 @@
 // Schedule-faithful execution on sm_100a: groups of thread blocks play the processes.
 //
-// Process i is played by G thread blocks ("lanes"); lane g owns the same 1/G share of every
-// segment, so the G lanes are G independent copies of the whole p-process system working on
-// disjoint element ranges and never synchronise with each other.  Each block walks its process's
+// Process i is played by G thread blocks ("lanes"); lane g owns the same range of offsets of every
+// segment (1/G of the largest segment, clipped), so the G lanes are G independent copies of the
+// whole p-process system working on disjoint parts of the message and of the scratch slots, and
+// never synchronise with each other.  Each block walks its process's
 // action list in order:
 //   send     post a flag for the pair (release), so that the receiver may read the value this
 //            process holds for the segment (its input, or its partial result in a scratch slot);
@@ -114,11 +115,15 @@ rd_faithful_kernel(const FaithfulParams a)
         if (alive) alive = wait_flag(posted, a.epoch, a, &sh_ok);
         if (!alive) break;
         if (threadIdx.x == 0 && lane == 0) t_start = now_ns();
-        // this lane's share of the segment, in whole vectors
+        // This lane's share: the same offsets of EVERY segment (a fixed 1/G of the slot, clipped to the
+        // segment's length).  Lanes run independently of each other and share the slots, so a lane
+        // that is already re-using a slot for a later, shorter segment must never touch offsets that
+        // belong to another lane's share of the segment still held there.
         const uint64_t seg_lo = a.seg_off[act.seg], seg_len = a.seg_off[act.seg + 1] - seg_lo;
-        const uint64_t units = (seg_len + V - 1) / V;
-        const uint64_t lo = units * uint64_t(lane) / uint64_t(a.lanes) * V;
+        const uint64_t units = (a.slot_elems + V - 1) / V;
+        uint64_t lo = units * uint64_t(lane) / uint64_t(a.lanes) * V;
         uint64_t hi = units * uint64_t(lane + 1) / uint64_t(a.lanes) * V;
+        if (lo > seg_len) lo = seg_len;
         if (hi > seg_len) hi = seg_len;
         const uint32_t *src = act.peer_slot >= 0 ? a.scratch + (size_t(act.peer) * a.slots + size_t(act.peer_slot)) * a.slot_elems
                               : act.peer_slot == -1 ? a.inputs[act.peer] + seg_lo : a.out + seg_lo;

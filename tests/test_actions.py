@@ -14,8 +14,19 @@ CASES = [(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI), (rd.RD_BI_GREEDY, rd.RD_PORT_BI), (
          (rd.RD_BINARY, rd.RD_PORT_BI), (rd.RD_BUTTERFLY, rd.RD_PORT_BI)]
 
 
-def emulate(h, x, op, blocking_send, rng):
-    """Runs every process's action list; processes advance in random order, one action at a time."""
+def lane_range(longest, lanes, g, seg_len, v=4):
+    """Offsets of a segment that block g of a process's G blocks works on (rule stated in include/rd.h)."""
+    slot_elems = (longest + 3) // 4 * 4
+    units = -(-slot_elems // v)
+    lo, hi = units * g // lanes * v, units * (g + 1) // lanes * v
+    return min(lo, seg_len), min(hi, seg_len)
+
+
+def emulate(h, x, op, blocking_send, rng, lanes=1):
+    """Runs every process's action list; the (process, lane) agents advance in random order, one action at
+    a time.  Lanes have their own flags but share the scratch slots, as on the GPU."""
+    if lanes > 1:
+        return emulate_lanes(h, x, op, blocking_send, rng, lanes)
     p, n = x.shape
     off = rd.rd_schedule_segments(h).astype(np.int64)
     lists, slots = [], 0
@@ -90,6 +101,100 @@ def emulate(h, x, op, blocking_send, rng):
         assert progressed, "dead-lock in the action lists"
     assert posted.all() and taken.all()
     return out, slots
+
+
+def emulate_lanes(h, x, op, blocking_send, rng, lanes):
+    p, n = x.shape
+    off = rd.rd_schedule_segments(h).astype(np.int64)
+    lists = [rd.rd_schedule_actions(h, i)[0] for i in range(p)]
+    slots = rd.rd_schedule_actions(h, 0)[1]
+    longest = int(np.diff(off).max())
+    scratch = np.zeros((p, max(slots, 1), (longest + 3) // 4 * 4), dtype=x.dtype)
+    owner = np.full(scratch.shape, -1, dtype=np.int64)      # segment whose value an offset of a slot holds
+    out = np.zeros(n, dtype=x.dtype)
+    n_events = rd.rd_schedule_info(h)["n_events"]
+    posted = np.zeros((n_events, lanes), dtype=bool)
+    taken = np.zeros((n_events, lanes), dtype=bool)
+    pc = np.zeros((p, lanes), dtype=np.int64)
+    waiting = np.full((p, lanes), -1, dtype=np.int64)
+    # let some lanes run far ahead of others: a lane is only scheduled with its own probability
+    speed = rng.uniform(0.05, 1.0, size=lanes)
+
+    def combine(held, inc):
+        if op == "sum":
+            if x.dtype == np.int32:
+                return (held.view(np.uint32) + inc.view(np.uint32)).view(np.int32)
+            return (held + inc).astype(np.float32)
+        return np.where(inc > held, inc, held)
+
+    agents = [(i, g) for i in range(p) for g in range(lanes)]
+    idle_rounds = 0
+    while any(pc[i, g] < len(lists[i]) or waiting[i, g] >= 0 for i, g in agents):
+        progressed = False
+        for k in rng.permutation(len(agents)):
+            i, g = agents[k]
+            if rng.random() > speed[g]:
+                continue
+            if waiting[i, g] >= 0:
+                if not taken[waiting[i, g], g]:
+                    continue
+                waiting[i, g] = -1
+                progressed = True
+            if pc[i, g] >= len(lists[i]):
+                continue
+            seg, peer, kind, slot, peer_slot, first, ev, wait_ev = (int(v) for v in lists[i][pc[i, g]])
+            base, seg_len = off[seg], off[seg + 1] - off[seg]
+            lo, hi = lane_range(longest, lanes, g, seg_len)
+            if kind == 2:
+                posted[ev, g] = True
+                if blocking_send:
+                    waiting[i, g] = ev
+                pc[i, g] += 1
+                progressed = True
+                continue
+            if (wait_ev >= 0 and not taken[wait_ev, g]) or not posted[ev, g]:
+                continue
+            if peer_slot >= 0:
+                assert (owner[peer, peer_slot, lo:hi] == seg).all(), "the sender's slot holds another segment here"
+                inc = scratch[peer, peer_slot, lo:hi].copy()
+            else:
+                inc = (x[peer, base + lo:base + hi] if peer_slot == -1 else out[base + lo:base + hi]).copy()
+            if first:
+                held = x[i, base + lo:base + hi]
+            elif slot >= 0:
+                assert (owner[i, slot, lo:hi] == seg).all(), "own slot holds another segment here"
+                held = scratch[i, slot, lo:hi]
+            else:
+                held = out[base + lo:base + hi]
+            res = inc if kind == 1 else combine(held, inc)
+            if slot >= 0:
+                scratch[i, slot, lo:hi] = res
+                owner[i, slot, lo:hi] = seg
+            else:
+                out[base + lo:base + hi] = res
+            taken[ev, g] = True
+            pc[i, g] += 1
+            progressed = True
+        idle_rounds = 0 if progressed else idle_rounds + 1
+        assert idle_rounds < 200, "dead-lock in the action lists"
+    return out, slots
+
+
+@pytest.mark.parametrize("algo,port", CASES)
+def test_lanes_that_drift_apart_never_meet_in_a_slot(algo, port):
+    """Unequal segments (a short last one), several blocks per process running at very different speeds."""
+    p, n, seg = 13 if algo != rd.RD_BUTTERFLY else 8, 618, 257
+    rng = np.random.default_rng(algo)
+    x = (rng.standard_normal((p, n)) * 10.0 ** rng.integers(-4, 5, size=(p, n))).astype(np.float32)
+    h = rd.rd_schedule_create(algo, port, p, 4 * n, 4 * 256 if algo != rd.RD_BUTTERFLY else 0, *M1)
+    try:
+        ev, off, _ = oracle_schedule(algo, port, p, 4 * n, 4 * 256 if algo != rd.RD_BUTTERFLY else 4 * n, *M1)
+        want = O.reduce(ev, x, off, "sum")
+        for trial in range(4):
+            got, _ = emulate(h, x, "sum", port == rd.RD_PORT_UNI, np.random.default_rng(100 + trial), lanes=5)
+            assert got.tobytes() == want.tobytes()
+    finally:
+        rd.rd_destroy(h)
 
 
 @pytest.mark.parametrize("algo,port", CASES)
