@@ -52,7 +52,8 @@ typedef enum {
     RD_ERR_TIMEOUT = -5,       /* a bounded wait inside the schedule-faithful kernel gave up            */
     RD_ERR_SIZE_MISMATCH = -6, /* n_elems * 4 differs from the schedule's message size                  */
     RD_ERR_INTERNAL = -7,      /* a generated schedule failed the library's own consistency check       */
-    RD_ERR_TOO_SMALL = -8      /* an output array passed by the caller is too short                     */
+    RD_ERR_TOO_SMALL = -8,     /* an output array passed by the caller is too short                     */
+    RD_ERR_TOO_LARGE = -9      /* rd_reduce_faithful_static: more scratch needed than its fixed array has */
 } rd_status_t;
 
 typedef enum {
@@ -264,6 +265,40 @@ RD_API int rd_schedule_faithful_shape(rd_schedule_t *s, int *blocks_per_process,
  */
 RD_API int rd_schedule_actions(const rd_schedule_t *s, int process, int32_t *buf, size_t cap_actions,
                                size_t *n_actions, int *slots_per_process);
+
+/*
+ * rd_reduce_faithful_static -- the schedule-faithful reduction for callers that must not allocate
+ * device memory.  (The paper has no counterpart; this exists for the library's users.)
+ *
+ * Who needs it: code that runs after a framework has claimed all device memory for its own pool
+ * (an inference server, a training job sized to the last byte) and would get cudaErrorMemoryAllocation
+ * from any cudaMalloc; code in a latency-critical loop, where an allocation may take the driver's
+ * global lock and stall every stream; code that is not allowed to change the process's memory
+ * footprint at run time.  rd_reduce in RD_EXEC_FAITHFUL mode allocates its tables, flags and partial
+ * result slots with cudaMalloc on first use; this entry point instead keeps all of that in one
+ * device array of 32 MiB that is part of the library image (every GPU that loads librd.so holds
+ * these 32 MiB until the process exits).  It calls no cudaMalloc / cudaFree and nothing that
+ * allocates device memory; it does not touch the device tables rd_reduce keeps for the schedule.
+ *
+ * Arguments and result are those of rd_reduce(..., RD_EXEC_FAITHFUL, ...): same kernel, same bits.
+ * stats (host, may be NULL): makespan_ns, predicted_s, bytes_moved, device_status, n_launches;
+ * kernel_ms and gbytes_per_s are derived from the makespan.  The call returns when the result is
+ * in d_out.
+ *
+ * Limits and rules
+ *   - The schedule's tables (32 bytes per action, two actions per send/receive pair), 8 bytes of
+ *     flags per pair and block, 24 bytes of time stamps per pair, and p x slots x largest-segment
+ *     bytes of partial results must fit in the 32 MiB together: otherwise RD_ERR_TOO_LARGE and
+ *     nothing is launched.  (Example: p = 64, 256 segments of 16 KiB, uni-greedy: about 5 MiB.)
+ *   - The first call on a device looks up the array's device address (the device must be current);
+ *     make that first call outside any stream capture.
+ *   - All calls, of all schedules and threads, share the one array, and it still holds the previous
+ *     call's contents: the entry point clears the flags, status words and time stamps itself at the
+ *     start of every call, but two calls that overlap on the GPU (different streams or threads)
+ *     corrupt each other.  Issue them one after the other.
+ */
+RD_API int rd_reduce_faithful_static(rd_schedule_t *s, const void *const *d_inputs, void *d_out, size_t n_elems,
+                                     rd_dtype_t dtype, rd_op_t op, void *cuda_stream, rd_stats_t *stats);
 
 /* rd_destroy -- frees the schedule and its device tables.  NULL is allowed. */
 RD_API void rd_destroy(rd_schedule_t *s);

@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(_HERE, "librd.so")
 RD_OK = 0
 RD_ERR_INVALID_ARG, RD_ERR_UNSUPPORTED, RD_ERR_NOMEM, RD_ERR_CUDA = -1, -2, -3, -4
 RD_ERR_TIMEOUT, RD_ERR_SIZE_MISMATCH, RD_ERR_INTERNAL, RD_ERR_TOO_SMALL = -5, -6, -7, -8
+RD_ERR_TOO_LARGE = -9
 RD_UNI_GREEDY, RD_BI_GREEDY, RD_BINOMIAL, RD_PIPELINE, RD_BINARY, RD_BUTTERFLY = range(6)
 RD_PORT_UNI, RD_PORT_BI = 0, 1
 RD_SUM, RD_MAX = 0, 1
@@ -28,7 +29,7 @@ ALGOS = {"uni_greedy": RD_UNI_GREEDY, "bi_greedy": RD_BI_GREEDY, "binomial": RD_
 EXPORTS = ("rd_schedule_create", "rd_schedule_create_segments", "rd_optimal_segment", "rd_schedule_info",
            "rd_schedule_events", "rd_schedule_segments", "rd_schedule_program", "rd_reduce",
            "rd_schedule_upload", "rd_reduce_host", "rd_destroy", "rd_strerror", "rd_schedule_set_wait_budget",
-           "rd_schedule_trace", "rd_schedule_faithful_shape", "rd_schedule_actions")
+           "rd_schedule_trace", "rd_schedule_faithful_shape", "rd_schedule_actions", "rd_reduce_faithful_static")
 
 
 class rd_model_t(C.Structure):
@@ -82,6 +83,7 @@ def lib():
         L.rd_schedule_trace.argtypes = [vp, vp, sz]
         L.rd_schedule_faithful_shape.argtypes = [vp, C.POINTER(i32), C.POINTER(i32), C.POINTER(sz)]
         L.rd_schedule_actions.argtypes = [vp, i32, vp, sz, C.POINTER(sz), C.POINTER(i32)]
+        L.rd_reduce_faithful_static.argtypes = [vp, C.POINTER(vp), vp, sz, i32, i32, vp, C.POINTER(rd_stats_t)]
         L.rd_destroy.argtypes = [vp]
         L.rd_destroy.restype = None
         L.rd_strerror.argtypes = [i32]
@@ -224,6 +226,26 @@ def rd_reduce(h, inputs, out, op, exec_mode=RD_EXEC_TREE, stream=None, want_stat
     finally:
         if out.device.index != prev:
             torch.cuda.set_device(prev)
+    return stats
+
+
+def rd_reduce_faithful_static(h, inputs, out, op, stream=None, want_stats=False):
+    """The schedule-faithful reduction without any device allocation (scratch in the library's fixed
+    32 MiB device array).  Same arguments as rd_reduce; see include/rd.h for who needs this and for the
+    rules (one call at a time, first call per device outside stream capture)."""
+    import torch
+    tab = inputs if isinstance(inputs, PointerTable) else PointerTable(inputs)
+    n = out.numel()
+    if not tab.is_cuda or tab.n != n or tab.dtype != out.dtype:
+        raise ValueError("every input must be a contiguous CUDA tensor with the output's dtype and length")
+    if not out.is_cuda or not out.is_contiguous():
+        raise ValueError("out must be a contiguous CUDA tensor")
+    s = stream if stream is not None else torch.cuda.current_stream(out.device)
+    stats = rd_stats_t() if want_stats else None
+    with torch.cuda.device(out.device):
+        _check(lib().rd_reduce_faithful_static(h, tab.array, out.data_ptr(), n, _dtype_code(out), int(op),
+                                               s.cuda_stream, C.byref(stats) if want_stats else None),
+               "rd_reduce_faithful_static")
     return stats
 
 

@@ -628,6 +628,73 @@ int rd_schedule_actions(const rd_schedule_t *s, int process, int32_t *buf, size_
     return RD_OK;
 }
 
+int rd_reduce_faithful_static(rd_schedule_t *s, const void *const *d_inputs, void *d_out, size_t n_elems, rd_dtype_t dtype,
+                              rd_op_t op, void *cuda_stream, rd_stats_t *stats)
+{
+    if (!s || !d_inputs || (dtype != RD_INT32 && dtype != RD_FP32) || (op != RD_SUM && op != RD_MAX)) return RD_ERR_INVALID_ARG;
+    if (n_elems * 4 != s->msg_bytes) return RD_ERR_SIZE_MISMATCH;
+    if (n_elems > 0 && !d_out) return RD_ERR_INVALID_ARG;
+    for (int i = 0; i < s->p; i++)
+        if ((n_elems > 0 && !d_inputs[i]) || (reinterpret_cast<uintptr_t>(d_inputs[i]) & 3u)) return RD_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(d_out) & 3u) return RD_ERR_INVALID_ARG;
+    rd_stats_t st;
+    std::memset(&st, 0, sizeof(st));
+    st.bytes_moved = uint64_t(s->p + 1) * uint64_t(n_elems) * 4u;
+    st.predicted_s = double(s->sched.completion) * s->ticks.tick;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (n_elems == 0) { if (stats) *stats = st; return RD_OK; }
+    if (s->p == 1) {
+        if (d_out != d_inputs[0] && cudaMemcpyAsync(d_out, d_inputs[0], n_elems * 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+            return RD_ERR_CUDA;
+        if (cudaStreamSynchronize(stream) != cudaSuccess) return RD_ERR_CUDA;
+        if (stats) *stats = st;
+        return RD_OK;
+    }
+    try {
+        ActionLists lists;
+        const size_t q = s->sched.seg_off.size() - 1;
+        if (int rc = build_actions(s->p, q, s->sched.events, lists)) return rc;
+        std::vector<FaithfulAction> acts(lists.actions.size());
+        for (size_t k = 0; k < acts.size(); k++) {
+            const Action &a = lists.actions[k];
+            acts[k] = FaithfulAction{a.seg, a.peer, a.kind, a.slot, a.peer_slot, a.first, a.event, a.wait_event};
+        }
+        uint64_t longest = 0;
+        for (size_t j = 0; j < q; j++) longest = std::max(longest, s->sched.seg_off[j + 1] - s->sched.seg_off[j]);
+        std::vector<unsigned long long> times(2 * size_t(s->p) * 16);
+        bool wide = (reinterpret_cast<uintptr_t>(d_out) & 15u) == 0;
+        for (int i = 0; i < s->p && wide; i++) wide = (reinterpret_cast<uintptr_t>(d_inputs[i]) & 15u) == 0;
+        for (size_t j = 0; j < s->sched.seg_off.size() && wide; j++) wide = (s->sched.seg_off[j] & 3u) == 0;
+        StaticRun r{};
+        r.p = s->p;
+        r.h_actions = acts.data(); r.n_actions = acts.size();
+        r.h_first = lists.first.data();
+        r.h_seg_off = s->sched.seg_off.data(); r.n_seg_off = s->sched.seg_off.size();
+        r.h_inputs = d_inputs; r.d_out = d_out;
+        r.n_events = s->sched.events.size();
+        r.slots = std::max(lists.slots_per_proc, 1);
+        r.slot_elems = (longest + 3) / 4 * 4;
+        r.blocking_send = s->port == RD_PORT_UNI ? 1 : 0;
+        r.dtype = int(dtype); r.op = int(op); r.wide = wide;
+        r.wait_seconds = s->wait_budget_s;
+        r.stream = cuda_stream;
+        r.h_block_times = times.data();
+        const int rc = faithful_static_run(r);
+        if (rc == 2) return RD_ERR_TOO_LARGE;
+        if (rc == 3) return RD_ERR_UNSUPPORTED;
+        if (rc != 0) return RD_ERR_CUDA;
+        st.device_status = r.device_status;
+        st.makespan_ns = r.makespan_ns;
+        st.kernel_ms = r.makespan_ns * 1e-6;
+        st.gbytes_per_s = r.makespan_ns > 0 ? double(st.bytes_moved) / r.makespan_ns : 0.0;
+        st.n_launches = 1;
+        if (stats) *stats = st;
+        return r.device_status != 0 ? RD_ERR_TIMEOUT : RD_OK;
+    } catch (const std::bad_alloc &) {
+        return RD_ERR_NOMEM;
+    }
+}
+
 void rd_destroy(rd_schedule_t *s)
 {
     if (!s) return;
@@ -647,6 +714,7 @@ const char *rd_strerror(int status)
     case RD_ERR_SIZE_MISMATCH: return "n_elems does not match the schedule's message size";
     case RD_ERR_INTERNAL: return "generated schedule failed the consistency check";
     case RD_ERR_TOO_SMALL: return "output array too small";
+    case RD_ERR_TOO_LARGE: return "the schedule needs more scratch than the built-in device array holds";
     }
     return "unknown status";
 }

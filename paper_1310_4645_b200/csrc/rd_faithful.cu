@@ -201,4 +201,109 @@ int launch_faithful(const FaithfulParams &prm, int dtype, int op, bool wide, voi
     return int(dispatch(prm, dtype, op, wide, static_cast<cudaStream_t>(stream), false, nullptr));
 }
 
+// ---------------------------------------------------------------------------------------------
+// The same kernel for callers that cannot allocate device memory: every table, flag and partial
+// result lives in one file-scope device array of fixed size instead of cudaMalloc'ed buffers.
+// In host code the array's name only stands for the symbol; the device address is asked for once
+// per device (cudaGetSymbolAddress, with that device current) and handed to the kernel as ordinary
+// pointers.  All calls share the array and it keeps what the last call left in it, so the flags,
+// the status words and the time stamps are cleared at the start of every call.
+// ---------------------------------------------------------------------------------------------
+constexpr size_t kStaticScratchBytes = size_t(32) << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+namespace {
+
+unsigned char *g_static_base[64] = {};   // per device: address of g_static_scratch once looked up
+
+size_t carve(size_t &cursor, size_t bytes)
+{
+    const size_t at = cursor;
+    cursor += (bytes + 255) / 256 * 256;
+    return at;
+}
+
+}  // namespace
+
+size_t faithful_static_capacity() { return kStaticScratchBytes; }
+
+int faithful_static_run(StaticRun &r)
+{
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return 1;
+    if (!g_static_base[device]) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return 1;
+        g_static_base[device] = static_cast<unsigned char *>(ptr);
+    }
+    unsigned char *base = g_static_base[device];
+    // blocks per process: everything must be resident at once
+    int perSm = 0, sms = 0, khz = 0;
+    if (dispatch(FaithfulParams{}, r.dtype, r.op, r.wide, nullptr, true, &perSm) != cudaSuccess) return 1;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) return 1;
+    if (cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, device) != cudaSuccess) return 1;
+    const long long capacity = (long long)perSm * sms;
+    if (capacity < r.p) return 3;
+    const int lanes = int(capacity / r.p < 16 ? capacity / r.p : 16);
+    // carve the array
+    size_t cursor = 0;
+    const size_t oActions = carve(cursor, r.n_actions * sizeof(FaithfulAction));
+    const size_t oFirst = carve(cursor, size_t(r.p + 1) * sizeof(uint32_t));
+    const size_t oSegOff = carve(cursor, r.n_seg_off * sizeof(uint64_t));
+    const size_t oInputs = carve(cursor, size_t(r.p) * sizeof(void *));
+    const size_t flagBytes = 2 * r.n_events * size_t(lanes) * sizeof(uint32_t);
+    const size_t oFlags = carve(cursor, flagBytes);
+    const size_t traceBytes = 3 * r.n_events * sizeof(unsigned long long);
+    const size_t oTrace = carve(cursor, traceBytes);
+    const size_t timeBytes = 2 * size_t(r.p) * size_t(lanes) * sizeof(unsigned long long);
+    const size_t oTimes = carve(cursor, timeBytes);
+    const size_t oStatus = carve(cursor, 2 * sizeof(int));
+    const size_t oSlots = carve(cursor, size_t(r.p) * size_t(r.slots) * size_t(r.slot_elems) * sizeof(uint32_t));
+    r.needed_bytes = cursor;
+    if (cursor > kStaticScratchBytes) return 2;
+    cudaStream_t stream = static_cast<cudaStream_t>(r.stream);
+    bool ok = true;
+    ok = ok && cudaMemcpyAsync(base + oActions, r.h_actions, r.n_actions * sizeof(FaithfulAction), cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(base + oFirst, r.h_first, size_t(r.p + 1) * sizeof(uint32_t), cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(base + oSegOff, r.h_seg_off, r.n_seg_off * sizeof(uint64_t), cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(base + oInputs, r.h_inputs, size_t(r.p) * sizeof(void *), cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    // what must start at zero: flags (the array still holds the previous call's), status, abort flag, time stamps
+    ok = ok && cudaMemsetAsync(base + oFlags, 0, flagBytes > 0 ? flagBytes : 4, stream) == cudaSuccess;
+    ok = ok && cudaMemsetAsync(base + oTrace, 0, traceBytes > 0 ? traceBytes : 8, stream) == cudaSuccess;
+    ok = ok && cudaMemsetAsync(base + oStatus, 0, 2 * sizeof(int), stream) == cudaSuccess;
+    if (!ok) return 1;
+    FaithfulParams prm{};
+    prm.inputs = reinterpret_cast<const uint32_t *const *>(base + oInputs);
+    prm.out = static_cast<uint32_t *>(r.d_out);
+    prm.scratch = reinterpret_cast<uint32_t *>(base + oSlots);
+    prm.actions = reinterpret_cast<const FaithfulAction *>(base + oActions);
+    prm.first = reinterpret_cast<const uint32_t *>(base + oFirst);
+    prm.seg_off = reinterpret_cast<const uint64_t *>(base + oSegOff);
+    prm.posted = reinterpret_cast<uint32_t *>(base + oFlags);
+    prm.taken = prm.posted + r.n_events * size_t(lanes);
+    prm.trace = reinterpret_cast<unsigned long long *>(base + oTrace);
+    prm.block_times = reinterpret_cast<unsigned long long *>(base + oTimes);
+    prm.status = reinterpret_cast<int *>(base + oStatus);
+    prm.abort_flag = prm.status + 1;
+    prm.wait_cycles = (long long)(r.wait_seconds * double(khz > 0 ? khz : 1000000) * 1e3);
+    prm.epoch = 1;
+    prm.n_procs = r.p; prm.lanes = lanes; prm.slots = r.slots; prm.slot_elems = r.slot_elems;
+    prm.blocking_send = r.blocking_send;
+    if (dispatch(prm, r.dtype, r.op, r.wide, stream, false, nullptr) != cudaSuccess) return 1;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return 1;
+    int status[2] = {0, 0};
+    if (cudaMemcpy(status, base + oStatus, sizeof(status), cudaMemcpyDeviceToHost) != cudaSuccess) return 1;
+    r.device_status = status[0];
+    r.lanes = lanes;
+    r.makespan_ns = 0.0;
+    if (status[0] == 0 && r.h_block_times) {
+        if (cudaMemcpy(r.h_block_times, base + oTimes, timeBytes, cudaMemcpyDeviceToHost) != cudaSuccess) return 1;
+        unsigned long long begin = ~0ull, end = 0;
+        for (size_t b = 0; b < size_t(r.p) * size_t(lanes); b++) if (r.h_block_times[2 * b] < begin) begin = r.h_block_times[2 * b];
+        for (int g = 0; g < lanes; g++) if (r.h_block_times[2 * size_t(g) + 1] > end) end = r.h_block_times[2 * size_t(g) + 1];
+        r.makespan_ns = end > begin ? double(end - begin) : 0.0;
+    }
+    return 0;
+}
+
 }  // namespace rd

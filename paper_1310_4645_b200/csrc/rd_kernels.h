@@ -80,5 +80,30 @@ struct FaithfulParams {
 int faithful_blocks_per_sm(int dtype, int op, bool wide, int *blocks_per_sm);
 int launch_faithful(const FaithfulParams &prm, int dtype, int op, bool wide, void *stream);
 
+// ---- the same kernel run entirely out of a fixed device array (no device allocation)
+struct StaticRun {
+    // in
+    int p;
+    const FaithfulAction *h_actions; size_t n_actions;   // host
+    const uint32_t *h_first;                              // host, p + 1
+    const uint64_t *h_seg_off; size_t n_seg_off;          // host
+    const void *const *h_inputs;                          // host array of p device pointers
+    void *d_out;
+    size_t n_events;
+    int slots; uint64_t slot_elems;
+    int blocking_send, dtype, op;
+    bool wide;
+    double wait_seconds;
+    void *stream;
+    unsigned long long *h_block_times;                    // host scratch, 2 * p * 16 values
+    // out
+    size_t needed_bytes;
+    int device_status, lanes;
+    double makespan_ns;
+};
+size_t faithful_static_capacity();
+// 0 done, 1 a CUDA call failed, 2 the schedule needs more than the array holds, 3 too many processes to be resident
+int faithful_static_run(StaticRun &r);
+
 }  // namespace rd
 #endif
