@@ -200,6 +200,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-large", action="store_true", help="skip the extra large-message (config4) measurement")
+    ap.add_argument("--no-faithful", action="store_true", help="skip the schedule-faithful makespan measurement")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -337,6 +338,26 @@ def main():
                    "steps": e_steps}
             del hx, hout, staging
 
+    # schedule-faithful execution: measured makespan of every schedule beside the linear model's prediction
+    faithful = None
+    if not args.no_faithful and world == 1 and p > 1:
+        rows = {}
+        for label, h in plans:
+            spans = []
+            for rep in range(7):
+                st = rd.rd_reduce(h, tables[rep % n_arenas], out, ops[0], exec_mode=rd.RD_EXEC_FAITHFUL, want_stats=True)
+                if rep >= 2:
+                    spans.append(st.makespan_ns)
+            spans.sort()
+            shape = rd.rd_schedule_faithful_shape(h)
+            rows[label] = {"measured_us": spans[len(spans) // 2] / 1e3, "best_us": spans[0] / 1e3,
+                           "predicted_us": rd.rd_schedule_info(h)["predicted_seconds"] * 1e6,
+                           "blocks_per_process": shape["blocks_per_process"], "slots_per_process": shape["slots_per_process"]}
+        by_model = sorted(rows, key=lambda k: rows[k]["predicted_us"])
+        by_gpu = sorted(rows, key=lambda k: rows[k]["measured_us"])
+        faithful = {"schedules": rows, "rank_by_model": by_model, "rank_measured": by_gpu,
+                    "ranks_agree": by_model == by_gpu, "fastest_agrees": by_model[0] == by_gpu[0]}
+
     # the large-message workload (1 GiB per process), measured beside the main one when it fits
     large = None
     if not args.no_large and world == 1 and wname != "config4":
@@ -401,7 +422,7 @@ def main():
                          "traffic": None, "peak_source": peak_src, "kernel": "rd_tree_stream_kernel",
                          "frac_of_nominal_8000": achieved / 8000.0},
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": args.steps * launches_per_step, "clocks": clocks,
-            "per_schedule_gbs": per_schedule, "schedule_create_ms": create_ms, "large_message": large,
+            "per_schedule_gbs": per_schedule, "schedule_create_ms": create_ms, "large_message": large, "faithful": faithful,
             "percent_of_peak": {"measured_copy": 100 * value / peak, "nominal_8TBs": 100 * value / 8000.0},
         }
         print(json.dumps(line), flush=True)
