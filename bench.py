@@ -37,6 +37,23 @@ WORKLOAD_SCHEDULES = {
 WORKLOAD_OPS = {"config1": ["sum"], "config2": ["sum"], "config3": ["sum"], "config4": ["sum", "max"]}
 
 
+# DRAM bytes per launch of the tree kernel from one ncu capture (profiles/rd_tree_stream_kernel_config2.md):
+# dram__bytes_read.sum + dram__bytes_write.sum, mean of three launches.  Reported only while the kernel
+# source is the one that was profiled.
+NCU_TRAFFIC = {"workload": "config2", "bytes_per_launch": 274.4e6,
+               "kernel_sha256": "edf7693b791db6f6b010ed9ae97d4bfe6accefad333ddcb98011795718e0eac8"}
+
+
+def profiled_traffic(wname):
+    import hashlib
+    try:
+        with open(os.path.join(ROOT, "paper_1310_4645_b200", "csrc", "rd_kernels.cu"), "rb") as f:
+            same = hashlib.sha256(f.read()).hexdigest() == NCU_TRAFFIC["kernel_sha256"]
+    except OSError:
+        same = False
+    return NCU_TRAFFIC["bytes_per_launch"] if same and wname == NCU_TRAFFIC["workload"] else None
+
+
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -419,7 +436,8 @@ def main():
                              if n_arenas > 1 else "inputs (%.1f GiB) exceed L2" % (p * n * 4 / 2**30),
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": None, "peak_source": peak_src, "kernel": "rd_tree_stream_kernel",
+                         "traffic": profiled_traffic(wname), "traffic_unit": "bytes per launch", "algorithmic_bytes": bytes_per_reduce,
+                         "peak_source": peak_src, "kernel": "rd_tree_stream_kernel",
                          "frac_of_nominal_8000": achieved / 8000.0},
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": args.steps * launches_per_step, "clocks": clocks,
             "per_schedule_gbs": per_schedule, "schedule_create_ms": create_ms, "large_message": large, "faithful": faithful,
