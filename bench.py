@@ -114,6 +114,22 @@ class ClockSampler(threading.Thread):
                 "samples": len(s)}
 
 
+def max_over_ranks(value, device=None):
+    """The largest `value` over all ranks of the default process group (the slowest rank sets the time)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_throughput(bytes_per_rank, ms, world):
+    """Whole-job GB/s of `world` independent replicas that each moved bytes_per_rank in at most ms."""
+    return world * bytes_per_rank / (ms * 1e-3) / 1e9
+
+
 def visible_gpu_index(local_rank):
     vis = os.environ.get("CUDA_VISIBLE_DEVICES")
     if vis:
@@ -300,13 +316,8 @@ def main():
     e1.record()
     barrier()
     clocks = sampler.stop()
-    ms = e0.elapsed_time(e1)
-    if dist_on:
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    total_bytes = world * args.steps * launches_per_step * bytes_per_reduce
-    value = total_bytes / (ms * 1e-3) / 1e9
+    ms = max_over_ranks(e0.elapsed_time(e1), dev)
+    value = replica_throughput(args.steps * launches_per_step * bytes_per_reduce, ms, world)
 
     # per-schedule throughput (same launches, timed one schedule at a time)
     per_schedule = {}
@@ -345,12 +356,8 @@ def main():
                         rd.rd_reduce_host(h, hx, hout, staging, op)
             b.record()
             barrier()
-            e_ms = a.elapsed_time(b)
-            if dist_on:
-                t = torch.tensor([e_ms], device=dev, dtype=torch.float64)
-                dist.all_reduce(t, op=dist.ReduceOp.MAX)
-                e_ms = float(t.item())
-            e2e = {"value": world * e_steps * launches_per_step * bytes_per_reduce / (e_ms * 1e-3) / 1e9, "unit": "GB/s",
+            e_ms = max_over_ranks(a.elapsed_time(b), dev)
+            e2e = {"value": replica_throughput(e_steps * launches_per_step * bytes_per_reduce, e_ms, world), "unit": "GB/s",
                    "h2d_bytes_per_step": launches_per_step * host_bytes, "d2h_bytes_per_step": launches_per_step * n * 4,
                    "steps": e_steps}
             del hx, hout, staging
