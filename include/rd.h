@@ -195,8 +195,9 @@ RD_API int rd_schedule_program(const rd_schedule_t *s, size_t seg, uint32_t *ops
  *   stats     host, or NULL.
  * The first call on a schedule uploads its tables to the current device
  * (allocates device memory, synchronises); rd_schedule_upload does the same
- * ahead of time.  Buffers must be 4-byte aligned; 16-byte aligned buffers and
- * segment sizes that are multiples of 16 bytes take the 128-bit path.
+ * ahead of time.  Buffers must be 4-byte aligned; 16-byte aligned buffers of a
+ * multiple of 4 elements take the 128-bit streaming path (segments may start
+ * and end anywhere), anything else a slower element-wise path.
  */
 RD_API int rd_reduce(rd_schedule_t *s, const void *const *d_inputs, void *d_out, size_t n_elems,
               rd_dtype_t dtype, rd_op_t op, rd_exec_t exec, void *cuda_stream, rd_stats_t *stats);

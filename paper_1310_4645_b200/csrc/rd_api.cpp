@@ -222,15 +222,19 @@ int tiles_for(rd_schedule *s, int vec, const TileDesc **tiles, uint32_t *count)
                 uint64_t e = lo;
                 while (e < hi) {
                     while (seg + 1 < off.size() && off[seg + 1] <= e) seg++;
-                    // the part of the range inside this segment, in equal tiles of at most one stage
+                    // The part of the range inside this segment, in equal tiles of at most one stage.  Tiles are
+                    // whole 128-bit vectors of the buffers: where the segment starts or ends inside a vector
+                    // the tile is padded to the vector and remembers how many elements are not its own.
                     const uint64_t pieceEnd = std::min<uint64_t>(hi, off[seg + 1]);
-                    const uint64_t parts = (pieceEnd - e + cap - 1) / cap;
-                    const uint64_t each = ((pieceEnd - e + parts - 1) / parts + 31) / 32 * 32;
-                    while (e < pieceEnd) {
-                        const uint64_t end = std::min<uint64_t>(pieceEnd, e + each);
-                        host.push_back(TileDesc{e, uint32_t(end - e), s->progs.seg_prog[seg]});
-                        e = end;
+                    const uint64_t ps = e & ~uint64_t(3), pe = (pieceEnd + 3) & ~uint64_t(3);
+                    const uint64_t parts = (pe - ps + cap - 1) / cap;
+                    const uint64_t each = std::min<uint64_t>(cap, ((pe - ps + parts - 1) / parts + 31) / 32 * 32);
+                    for (uint64_t ts = ps; ts < pe; ts += each) {
+                        const uint64_t te = std::min<uint64_t>(pe, ts + each);
+                        const uint32_t head = ts < e ? uint32_t(e - ts) : 0u, tail = te > pieceEnd ? uint32_t(te - pieceEnd) : 0u;
+                        host.push_back(TileDesc{ts, uint32_t(te - ts) | (head << 16) | (tail << 18), s->progs.seg_prog[seg]});
                     }
+                    e = pieceEnd;
                 }
             }
             first[size_t(ctas)] = uint32_t(host.size());
@@ -256,10 +260,9 @@ int reduce_tree(rd_schedule *s, const void *const *d_inputs, void *d_out, size_t
                 cudaStream_t stream, rd_stats_t *stats)
 {
     DeviceTables &d = s->dev;
-    // 128-bit path: every buffer 16-byte aligned and every segment boundary a multiple of 4 elements
-    bool wide = (reinterpret_cast<uintptr_t>(d_out) & 15u) == 0;
+    // 128-bit path: every buffer 16-byte aligned and a whole number of vectors (segments may start anywhere)
+    bool wide = (reinterpret_cast<uintptr_t>(d_out) & 15u) == 0 && (n & 3u) == 0;
     for (int i = 0; i < s->p && wide; i++) wide = (reinterpret_cast<uintptr_t>(d_inputs[i]) & 15u) == 0;
-    for (size_t j = 0; j < s->sched.seg_off.size() && wide; j++) wide = (s->sched.seg_off[j] & 3u) == 0;
     TreeLaunch l{};
     l.vec = wide ? 4 : 1;
     if (int rc = tiles_for(s, l.vec, &l.tiles, &l.n_tiles)) return rc;

@@ -228,6 +228,17 @@ __device__ __forceinline__ void bulk_load(void *smem_dst, const void *gmem_src, 
                  ::"r"(smem_addr(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
 }
 
+constexpr uint32_t kLenMask = 0xFFFFu;   // TileDesc::len: bits 0-15 padded length, 16-17 elements to skip at the head, 18-19 at the tail
+
+// Stores a 4-element vector, or only elements [skip_head, 4 - skip_tail) of it.
+__device__ __forceinline__ void store_part(uint32_t *p, const Vec<4> &v, uint32_t skip_head, uint32_t skip_tail)
+{
+    if ((skip_head | skip_tail) == 0u) { store_stream<4>(p, v); return; }
+#pragma unroll
+    for (uint32_t e = 0; e < 4u; e++)
+        if (e >= skip_head && e < 4u - skip_tail) __stcs(p + e, v.w[e]);
+}
+
 template <bool PACKED> struct StreamParams {
     TreeParams<PACKED> t;
     const uint32_t *cta_first;   // per CTA: first tile; n_ctas + 1 entries
@@ -285,8 +296,8 @@ rd_tree_stream_kernel(const __grid_constant__ StreamParams<PACKED> a)
             if (tile != cur) { td = a.t.tiles[tile]; cur = tile; }
             const uint32_t *src = a.t.input(__ldg(a.t.ops + td.prog + i) & kIdxMask) + td.elem_off;
             if (laps >= 1u && !mbar_wait(empty + stage, (laps - 1u) & 1u, &abort_flag)) { ok = false; break; }
-            mbar_expect_tx(full + stage, td.len * 4u);
-            bulk_load(ring + size_t(stage) * stageVecs, src, td.len * 4u, full + stage);
+            mbar_expect_tx(full + stage, (td.len & kLenMask) * 4u);
+            bulk_load(ring + size_t(stage) * stageVecs, src, (td.len & kLenMask) * 4u, full + stage);
             any = true; lastStage = stage; lastLap = laps;
             i += P;
             while (i >= p && tile < tile1) { i -= p; tile++; }
@@ -311,7 +322,8 @@ rd_tree_stream_kernel(const __grid_constant__ StreamParams<PACKED> a)
     for (uint32_t tile = tile0; tile < tile1; tile++) {
         const TileDesc td = a.t.tiles[tile];
         const uint32_t *prog = a.t.ops + td.prog;
-        const bool live0 = tid * 4u < td.len, live1 = (kConsumers + tid) * 4u < td.len;
+        const uint32_t len = td.len & kLenMask;                       // padded to whole 128-bit vectors
+        const bool live0 = tid * 4u < len, live1 = (kConsumers + tid) * 4u < len;
         Vec<4> top0, top1;
 #pragma unroll
         for (int v = 0; v < 4; v++) { top0.w[v] = 0; top1.w[v] = 0; }
@@ -377,9 +389,12 @@ rd_tree_stream_kernel(const __grid_constant__ StreamParams<PACKED> a)
             }
             w = wn;
         }
+        // A segment may begin or end inside a vector: the tile then starts / ends with a vector whose other
+        // elements belong to the neighbouring segment (another tile writes those); only this tile's are stored.
         uint32_t *dst = a.t.out + td.elem_off;
-        if (live0) store_stream<4>(dst + tid * 4u, top0);
-        if (live1) store_stream<4>(dst + (kConsumers + tid) * 4u, top1);
+        const uint32_t head = (td.len >> 16) & 3u, tail = (td.len >> 18) & 3u, lastVec = len / 4u - 1u;
+        if (live0) store_part(dst + tid * 4u, top0, tid == 0 ? head : 0u, tid == lastVec ? tail : 0u);
+        if (live1) store_part(dst + (kConsumers + tid) * 4u, top1, 0u, kConsumers + tid == lastVec ? tail : 0u);
     }
 }
 

@@ -1,0 +1,133 @@
+"""Sweep of the tree-mode reduction over process counts, message sizes, element types, operations and
+schedules, every schedule at its own optimal segment size (the paper tunes each algorithm's segment
+size before comparing, Sections V-B and VII).
+
+    python -m paper_1310_4645_b200.sweep --out sweep.jsonl [--max-total-gib 64] [--reps 5]
+
+For every case one JSON line: shape, segment size chosen, the schedule's predicted completion time
+under the linear model, measured microseconds and GB/s ((p+1)*m bytes per reduction), and whether the
+result passed its check (int32 and fp32 max: exact against torch's order-free result; fp32 sum:
+|r - r64| <= 1e-5 * sum|x| against an fp64 sum, on the whole message or on sampled slices of it).
+Inputs: uniform random numbers from seed 4 (int32 in [-2^20, 2^20], fp32 in [-1, 1)), one arena per
+element type, every case a view of its first p*n elements.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import sys
+import time
+
+import torch
+
+from . import binding as rd
+
+ALPHA, BETA, GAMMA = 2e-6, 1e-10, 5e-11
+SCHEDULES = [("uni_greedy", rd.RD_UNI_GREEDY, rd.RD_PORT_UNI), ("bi_greedy", rd.RD_BI_GREEDY, rd.RD_PORT_BI),
+             ("binomial", rd.RD_BINOMIAL, rd.RD_PORT_UNI), ("pipeline", rd.RD_PIPELINE, rd.RD_PORT_UNI),
+             ("binary", rd.RD_BINARY, rd.RD_PORT_UNI), ("butterfly", rd.RD_BUTTERFLY, rd.RD_PORT_BI)]
+
+
+def fill_arena(n_elems, dtype, dev):
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(4)
+    arena = torch.empty(n_elems, dtype=dtype, device=dev)
+    step = 1 << 28
+    for lo in range(0, n_elems, step):
+        part = arena[lo:lo + step]
+        if dtype == torch.int32:
+            part.random_(-(1 << 20), (1 << 20) + 1, generator=gen)
+        else:
+            part.uniform_(-1.0, 1.0, generator=gen)
+    return arena
+
+
+def check(x, out, op, max_check_elems=1 << 22):
+    """Order-free check on the whole message when small, else on the first, middle and last slices."""
+    p, n = x.shape
+    per = max(1, max_check_elems // p)
+    spans = [(0, n)] if n <= 3 * per else [(0, per), ((n - per) // 2, (n - per) // 2 + per), (n - per, n)]
+    for lo, hi in spans:
+        xs, o = x[:, lo:hi], out[lo:hi]
+        if op == "max":
+            if not torch.equal(o, xs.amax(dim=0)):
+                return False
+        elif x.dtype == torch.int32:
+            want = xs.to(torch.int64).sum(dim=0)
+            want = ((want + (1 << 31)) % (1 << 32) - (1 << 31)).to(torch.int32)
+            if not torch.equal(o, want):
+                return False
+        else:
+            ref = xs.to(torch.float64).sum(dim=0)
+            mag = xs.to(torch.float64).abs().sum(dim=0)
+            if not bool(((o.to(torch.float64) - ref).abs() <= 1e-5 * mag).all()):
+                return False
+    return True
+
+
+def main(argv=None):
+    ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
+    ap.add_argument("--out", default="-")
+    ap.add_argument("--max-total-gib", type=float, default=64.0, help="skip cases whose p*m exceeds this")
+    ap.add_argument("--reps", type=int, default=5)
+    ap.add_argument("--p", type=int, nargs="*", default=[2 ** k for k in range(1, 11)])
+    ap.add_argument("--min-log2-bytes", type=int, default=3)
+    ap.add_argument("--max-log2-bytes", type=int, default=26)
+    args = ap.parse_args(argv)
+    dev = torch.device("cuda", torch.cuda.current_device())
+    sink = sys.stdout if args.out == "-" else open(args.out, "w")
+    sizes = [1 << k for k in range(args.min_log2_bytes, args.max_log2_bytes + 1)]
+    limit = int(args.max_total_gib * (1 << 30))
+    biggest = max(p * m for p in args.p for m in sizes if p * m <= limit)
+    arenas = {"int32": fill_arena(biggest // 4, torch.int32, dev), "fp32": fill_arena(biggest // 4, torch.float32, dev)}
+    out_buf = {"int32": torch.empty(max(sizes) // 4, dtype=torch.int32, device=dev),
+               "fp32": torch.empty(max(sizes) // 4, dtype=torch.float32, device=dev)}
+    n_cases = n_bad = 0
+    t_start = time.time()
+    for p in args.p:
+        for m in sizes:
+            if p * m > limit:
+                continue
+            n = m // 4
+            for name, algo, port in SCHEDULES:
+                t0 = time.perf_counter()
+                seg = rd.rd_optimal_segment(algo, port, p, m, ALPHA, BETA, GAMMA)
+                h = rd.rd_schedule_create(algo, port, p, m, seg, ALPHA, BETA, GAMMA)
+                create_ms = (time.perf_counter() - t0) * 1e3
+                info = rd.rd_schedule_info(h)
+                rd.rd_schedule_upload(h)
+                try:
+                    for dt in ("int32", "fp32"):
+                        x = arenas[dt][: p * n].view(p, n)
+                        out = out_buf[dt][:n]
+                        tab = rd.PointerTable(x)
+                        for op, opc in (("sum", rd.RD_SUM), ("max", rd.RD_MAX)):
+                            rd.rd_reduce(h, tab, out, opc)
+                            ok = check(x, out, op)
+                            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                            a.record()
+                            for _ in range(args.reps):
+                                rd.rd_reduce(h, tab, out, opc)
+                            b.record()
+                            torch.cuda.synchronize()
+                            us = a.elapsed_time(b) * 1e3 / args.reps
+                            rec = {"p": p, "msg_bytes": m, "dtype": dt, "op": op, "schedule": name, "seg_bytes": seg,
+                                   "q": info["q"], "predicted_us": info["predicted_seconds"] * 1e6, "measured_us": us,
+                                   "gbs": (p + 1) * m / us / 1e3, "ok": ok, "create_ms": create_ms,
+                                   "cache": "L2 resident (inputs re-read every repetition)" if p * m < (96 << 20) else "HBM"}
+                            sink.write(json.dumps(rec) + "\n")
+                            n_cases += 1
+                            n_bad += 0 if ok else 1
+                finally:
+                    rd.rd_destroy(h)
+        sink.flush()
+    summary = {"summary": True, "cases": n_cases, "failed_checks": n_bad, "seconds": time.time() - t_start}
+    sink.write(json.dumps(summary) + "\n")
+    if sink is not sys.stdout:
+        sink.close()
+        print(json.dumps(summary))
+    return 1 if n_bad else 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -42,7 +42,9 @@ def check(algo, port, x_dev, seg_bytes, op, model=M1):
 # (p, n, segment elements): several tiles (2048 elements each on the 128-bit path), ragged tails,
 # segments shorter and longer than a tile, non-power-of-two process counts
 SHAPES = [(8, 4096, 512), (5, 10000, 2500), (13, 3 * 2048 + 36, 2048 + 520), (64, 8192, 1024), (2, 4100, 4100),
-          (33, 6000, 1000), (16, 128, 8), (1, 5000, 1000)]
+          (33, 6000, 1000), (16, 128, 8), (1, 5000, 1000),
+          # segments that start and end inside a 128-bit vector (the message itself is whole vectors)
+          (8, 3000, 333), (16, 4100, 4100), (13, 6180, 999), (4, 64, 3), (8, 4096, 6), (32, 8192, 2049)]
 
 
 @pytest.mark.parametrize("name,algo,port", SCHEDULES)
