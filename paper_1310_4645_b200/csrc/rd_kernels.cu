@@ -270,6 +270,11 @@ rd_tree_stream_kernel(const __grid_constant__ StreamParams<PACKED> a)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    // Programmatic dependent launch: the next launch on the stream may begin its own set-up (barriers, table
+    // look-ups above) while this grid is still running; before it touches message data it waits here for
+    // the grid before it to have finished completely.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     if (tid >= kConsumers) {
         // ------------------------------------------------------------------ producers
@@ -457,8 +462,14 @@ cudaError_t launch_stream(const TreeLaunch &l)
         if (e != cudaSuccess) return e;
         configured[dv] = smem;
     }
-    kernel<<<l.n_ctas, kStreamThreads, smem, static_cast<cudaStream_t>(l.stream)>>>(prm);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(l.n_ctas); cfg.blockDim = dim3(kStreamThreads); cfg.dynamicSmemBytes = smem;
+    cfg.stream = static_cast<cudaStream_t>(l.stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, prm);
 }
 
 template <int DT, int OPR>
