@@ -131,3 +131,15 @@ def test_faithful_and_tree_agree_on_config2_and_makespans_are_reported():
         rd.rd_destroy(h)
         assert torch.equal(a.view(torch.int32), b.view(torch.int32))
         assert st.makespan_ns > 0
+
+
+def test_calibration_tool_fits_positive_parameters(capsys):
+    """The fitted latency and inverse bandwidth are positive and uni-greedy is the model's favourite."""
+    import json
+    from paper_1310_4645_b200 import calibrate
+    assert calibrate.main(["--p", "8", "--msg-bytes", str(1 << 20)]) == 0
+    d = json.loads(capsys.readouterr().out)
+    assert d["fitted"]["alpha_s"] > 0 and d["fitted"]["beta_s_per_byte"] > 0
+    assert set(d["schedules"]) == {"uni_greedy", "binomial", "pipeline", "binary"}
+    assert d["rank_by_model"][0] == "uni_greedy"          # Theorem 5: optimal among in-order one-port schedules
+    assert all(v["measured_us"] > 0 for v in d["schedules"].values())
