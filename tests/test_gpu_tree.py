@@ -184,3 +184,26 @@ def test_config2_shape_full_size(name, algo, port):
     ref, mag = O.reference_f64(xh, "sum")
     assert (np.abs(got.astype(np.float64) - ref) <= 1e-5 * mag).all()
     assert np.abs(got - ref).max() / np.abs(ref).max() <= 1e-5
+
+
+@pytest.mark.parametrize("mode", [rd.RD_EXEC_TREE, rd.RD_EXEC_FAITHFUL])
+def test_unequal_segmentation_end_to_end(mode):
+    """Section VIII: segments of different sizes, e.g. (5,3,2) and (3,2,2,2,1) tenths of the message;
+    both kernels execute the uni-greedy / bi-greedy / pipeline schedules built for them, bit for bit."""
+    from helpers import ticks
+    p = 12
+    for parts in ((5, 3, 2), (3, 2, 2, 2, 1), (2, 2, 1, 1, 1, 1, 1, 1), (10,)):
+        unit = 412                                           # elements per tenth: segments are not vector aligned
+        sizes = [4 * unit * k for k in parts]
+        n = unit * 10
+        x = make_inputs(p, n, "normal", seed=sum(parts) + len(parts), device="cuda")
+        x *= 10.0 ** torch.randint(-4, 5, x.shape, device="cuda", generator=torch.Generator("cuda").manual_seed(2))
+        for algo, port in ((rd.RD_UNI_GREEDY, rd.RD_PORT_UNI), (rd.RD_BI_GREEDY, rd.RD_PORT_BI), (rd.RD_PIPELINE, rd.RD_PORT_BI)):
+            h = rd.rd_schedule_create_segments(algo, port, p, sizes, *M1)
+            out = torch.empty(n, device="cuda")
+            rd.rd_reduce(h, x, out, rd.RD_SUM, exec_mode=mode)
+            torch.cuda.synchronize()
+            rd.rd_destroy(h)
+            ev, off, _ = oracle_schedule(algo, port, p, 4 * n, 0, *M1, sizes=sizes)
+            want = O.reduce(ev, x.cpu().numpy(), off, "sum")
+            assert out.cpu().numpy().tobytes() == want.tobytes(), (parts, algo)
