@@ -301,6 +301,21 @@ RD_API int rd_schedule_actions(const rd_schedule_t *s, int process, int32_t *buf
 RD_API int rd_reduce_faithful_static(rd_schedule_t *s, const void *const *d_inputs, void *d_out, size_t n_elems,
                                      rd_dtype_t dtype, rd_op_t op, void *cuda_stream, rd_stats_t *stats);
 
+/*
+ * rd_search_segmentation -- Section VIII (unequal segmentation) for uni-greedy, which is optimal for
+ * any given segmentation (Theorem 5) but whose best segmentation need not be an equal one.  Starts from
+ * every best equi-segmentation in multiples of unit_bytes and moves one unit at a time between segments
+ * (or splits one off), looking two moves ahead when no single move helps, while the completion time
+ * under `model` gets shorter; the paper observes that the optimum usually lies one or two such moves
+ * from the best equi-segmentation.  Host work only.
+ *   msg_bytes  a multiple of unit_bytes; unit_bytes a multiple of 4; at most 4096 units.
+ *   seg_bytes  host, capacity cap sizes; q_out receives the number of segments (also when cap is too
+ *              small: RD_ERR_TOO_SMALL); predicted_ticks (may be NULL) the completion time.
+ * Feed the result to rd_schedule_create_segments.
+ */
+RD_API int rd_search_segmentation(int p, size_t msg_bytes, size_t unit_bytes, const rd_model_t *model,
+                                  size_t *seg_bytes, size_t cap, size_t *q_out, int64_t *predicted_ticks);
+
 /* rd_destroy -- frees the schedule and its device tables.  NULL is allowed. */
 RD_API void rd_destroy(rd_schedule_t *s);
 

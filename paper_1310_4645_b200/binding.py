@@ -29,7 +29,7 @@ ALGOS = {"uni_greedy": RD_UNI_GREEDY, "bi_greedy": RD_BI_GREEDY, "binomial": RD_
 EXPORTS = ("rd_schedule_create", "rd_schedule_create_segments", "rd_optimal_segment", "rd_schedule_info",
            "rd_schedule_events", "rd_schedule_segments", "rd_schedule_program", "rd_reduce",
            "rd_schedule_upload", "rd_reduce_host", "rd_destroy", "rd_strerror", "rd_schedule_set_wait_budget",
-           "rd_schedule_trace", "rd_schedule_faithful_shape", "rd_schedule_actions", "rd_reduce_faithful_static")
+           "rd_schedule_trace", "rd_schedule_faithful_shape", "rd_schedule_actions", "rd_reduce_faithful_static", "rd_search_segmentation")
 
 
 class rd_model_t(C.Structure):
@@ -84,6 +84,8 @@ def lib():
         L.rd_schedule_faithful_shape.argtypes = [vp, C.POINTER(i32), C.POINTER(i32), C.POINTER(sz)]
         L.rd_schedule_actions.argtypes = [vp, i32, vp, sz, C.POINTER(sz), C.POINTER(i32)]
         L.rd_reduce_faithful_static.argtypes = [vp, C.POINTER(vp), vp, sz, i32, i32, vp, C.POINTER(rd_stats_t)]
+        L.rd_search_segmentation.argtypes = [i32, sz, sz, C.POINTER(rd_model_t), C.POINTER(sz), sz, C.POINTER(sz),
+                                             C.POINTER(C.c_int64)]
         L.rd_destroy.argtypes = [vp]
         L.rd_destroy.restype = None
         L.rd_strerror.argtypes = [i32]
@@ -296,6 +298,17 @@ def rd_schedule_actions(h, process):
     _check(lib().rd_schedule_actions(h, int(process), buf.ctypes.data, n.value, C.byref(n), C.byref(slots)),
            "rd_schedule_actions")
     return buf, slots.value
+
+
+def rd_search_segmentation(p, msg_bytes, unit_bytes, alpha, beta, gamma, tick=0.0):
+    """(segment sizes in bytes, predicted completion ticks) of the local search around the best equi-segmentation."""
+    m = _model(alpha, beta, gamma, tick)
+    cap = int(msg_bytes) // int(unit_bytes) if unit_bytes else 0
+    arr = (C.c_size_t * max(cap, 1))()
+    q, ticks = C.c_size_t(), C.c_int64()
+    _check(lib().rd_search_segmentation(int(p), int(msg_bytes), int(unit_bytes), C.byref(m), arr, cap, C.byref(q),
+                                        C.byref(ticks)), "rd_search_segmentation")
+    return [int(arr[j]) for j in range(q.value)], ticks.value
 
 
 def rd_destroy(h) -> None:

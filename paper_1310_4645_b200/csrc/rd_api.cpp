@@ -698,6 +698,26 @@ int rd_reduce_faithful_static(rd_schedule_t *s, const void *const *d_inputs, voi
     }
 }
 
+int rd_search_segmentation(int p, size_t msg_bytes, size_t unit_bytes, const rd_model_t *model, size_t *seg_bytes, size_t cap,
+                           size_t *q_out, int64_t *predicted_ticks)
+{
+    if (!model || !q_out || (!seg_bytes && cap > 0) || p < 1 || p > kMaxProcs) return RD_ERR_INVALID_ARG;
+    Ticks t;
+    if (int rc = make_ticks(model, t)) return rc;
+    try {
+        std::vector<int64_t> best;
+        int64_t ticks = 0;
+        if (int rc = search_segmentation(p, msg_bytes, unit_bytes, t, best, &ticks)) return rc;
+        *q_out = best.size();
+        if (predicted_ticks) *predicted_ticks = ticks;
+        if (cap < best.size()) return RD_ERR_TOO_SMALL;
+        for (size_t j = 0; j < best.size(); j++) seg_bytes[j] = size_t(best[j]);
+    } catch (const std::bad_alloc &) {
+        return RD_ERR_NOMEM;
+    }
+    return RD_OK;
+}
+
 void rd_destroy(rd_schedule_t *s)
 {
     if (!s) return;

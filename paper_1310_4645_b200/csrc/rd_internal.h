@@ -34,6 +34,7 @@ int gen_butterfly(int p, uint64_t n_elems, const Ticks &c, Schedule &out);
 void sort_events(std::vector<rd_event_t> &ev);
 int optimal_segment(rd_algo_t algo, rd_port_t port, int p, size_t msg_bytes, const Ticks &c, size_t *out);
 int ceil_log2(uint64_t v);
+int search_segmentation(int p, size_t msg_bytes, size_t unit, const Ticks &c, std::vector<int64_t> &best, int64_t *bestTicks);
 
 // ---- rd_compile.cpp: events -> per-segment combine trees -> interpreter programs
 constexpr int kIdxBits = 12;           // process index field of an operation word

@@ -337,4 +337,78 @@ int optimal_segment(rd_algo_t algo, rd_port_t port, int p, size_t m, const Ticks
     return RD_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Section VIII: unequal segmentation for uni-greedy.  Start from the best equi-segmentation in
+// multiples of `unit` bytes and move one unit at a time from one segment to another while that
+// shortens the completion time (the paper observes that the optimum is usually one or two such moves
+// away from the best equi-segmentation).
+// ---------------------------------------------------------------------------------------------
+static void neighbours(const std::vector<int64_t> &seg, int64_t unit, std::vector<std::vector<int64_t>> &out)
+{
+    for (size_t i = 0; i < seg.size(); i++) {
+        for (size_t j = 0; j < seg.size(); j++) {              // one unit from segment i to segment j
+            if (i == j) continue;
+            std::vector<int64_t> v = seg;
+            v[i] -= unit; v[j] += unit;
+            if (v[i] == 0) v.erase(v.begin() + long(i));
+            out.push_back(std::move(v));
+        }
+        if (seg[i] > unit) {                                   // one unit split off into a new last segment
+            std::vector<int64_t> v = seg;
+            v[i] -= unit; v.push_back(unit);
+            out.push_back(std::move(v));
+        }
+    }
+}
+
+int search_segmentation(int p, size_t msg_bytes, size_t unit, const Ticks &c, std::vector<int64_t> &best, int64_t *bestTicks)
+{
+    if (unit == 0 || (unit & 3u) || msg_bytes == 0 || msg_bytes % unit) return RD_ERR_INVALID_ARG;
+    const size_t units = msg_bytes / unit;
+    if (units > 4096) return RD_ERR_INVALID_ARG;
+    Schedule tmp;
+    auto timeOf = [&](const std::vector<int64_t> &seg) { gen_uni_greedy(p, seg, c, tmp, false); return tmp.completion; };
+    // every equi-segmentation (k units per segment) that reaches the best equi time is a starting point
+    std::vector<std::vector<int64_t>> starts;
+    int64_t equiT = -1;
+    for (size_t k = 1; k <= units; k++) {
+        std::vector<int64_t> seg = equal_segments(msg_bytes, k * unit);
+        const int64_t t = timeOf(seg);
+        if (equiT < 0 || t < equiT) { equiT = t; starts.clear(); }
+        if (t == equiT) starts.push_back(std::move(seg));
+    }
+    int64_t bestT = equiT;
+    best = starts.front();
+    std::vector<std::vector<int64_t>> near, far;
+    for (const std::vector<int64_t> &start : starts) {
+        std::vector<int64_t> cur = start;
+        int64_t curT = equiT;
+        for (bool improved = true; improved;) {
+            improved = false;
+            near.clear();
+            neighbours(cur, int64_t(unit), near);
+            std::vector<int64_t> pick;
+            int64_t pickT = curT;
+            for (const std::vector<int64_t> &v : near) {
+                const int64_t t = timeOf(v);
+                if (t < pickT) { pickT = t; pick = v; }
+            }
+            if (pickT == curT && near.size() * near.size() <= 40000) {     // nothing one move away: look two moves away
+                for (const std::vector<int64_t> &v : near) {
+                    far.clear();
+                    neighbours(v, int64_t(unit), far);
+                    for (const std::vector<int64_t> &w : far) {
+                        const int64_t t = timeOf(w);
+                        if (t < pickT) { pickT = t; pick = w; }
+                    }
+                }
+            }
+            if (pickT < curT) { curT = pickT; cur = pick; improved = true; }
+        }
+        if (curT < bestT) { bestT = curT; best = cur; }
+    }
+    *bestTicks = bestT;
+    return RD_OK;
+}
+
 }  // namespace rd

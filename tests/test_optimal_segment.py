@@ -82,3 +82,25 @@ def test_seg_bytes_zero_uses_the_optimum():
         h = rd.rd_schedule_create(algo, port, 64, m, 0, *M1)
         assert rd.rd_schedule_info(h)["q"] == -(-m // s)
         rd.rd_destroy(h)
+
+
+def test_unequal_segmentation_search_on_table4():
+    """Section VIII: the local search (one unit moved at a time, starting from the best equi-segmentation)
+    never ends worse than the best equi-segmentation, and on the table's experiments it reaches the true
+    optimum in most cases, as the paper observes for one or two unit moves."""
+    from test_oracle_schedules import TABLE4, COMPS
+    rows = [r for r in TABLE4 if r[0] <= 128]
+    reached = improved = 0
+    for p, a, g, ratio, equi, opts in rows:
+        # one paper unit = 4 bytes; beta = gamma_paper... per byte 1 tick, so every time is 4x the paper's
+        sizes, t = rd.rd_search_segmentation(p, 40, 4, 4 * a * 1e-15, 1e-15, g * 1e-15)
+        times = O.unequal_times(p, a, g)
+        best = int(times.min())
+        best_equi = min(int(times[COMPS.index(tuple(O.equal_sizes(10, s)))]) for s in range(1, 11))
+        assert sum(sizes) == 40 and all(s % 4 == 0 and s > 0 for s in sizes)
+        found = int(times[COMPS.index(tuple(s // 4 for s in sizes))])
+        assert t == 4 * found                   # the library's own prediction for what it returns
+        assert best <= found <= best_equi
+        improved += found < best_equi           # these are the experiments an unequal segmentation wins
+        reached += found == best
+    assert improved >= 0.9 * len(rows) and reached >= 0.8 * len(rows), (improved, reached, len(rows))
