@@ -204,39 +204,33 @@ int tiles_for(rd_schedule *s, int vec, const TileDesc **tiles, uint32_t *count)
         const std::vector<uint64_t> &off = s->sched.seg_off;
         std::vector<TileDesc> host;
         if (vec == 4) {
-            // Streaming path.  The message is cut into one contiguous range per CTA, all of the same
-            // length up to one granule of 128 elements, so that every CTA moves the same number of
-            // bytes; a range is then cut at segment boundaries and at the stage capacity.
+            // Streaming path.  Every segment is cut into equal tiles of at most one stage (whole 128-bit
+            // vectors of the buffers: where a segment starts or ends inside a vector the tile is padded to the
+            // vector and remembers how many elements are not its own).  CTAs get contiguous runs of tiles,
+            // the same NUMBER of tiles up to one: a tile costs a CTA about the same time however full it
+            // is (one ring hand-off per operation), so for small messages the number of tiles per CTA,
+            // not the number of elements, sets the kernel's duration; for large ones the two coincide.
             const uint64_t n = off.empty() ? 0 : off.back();
             d.stage_elems = stream_stage_elems(n / (uint64_t(d.sm_count) * 2) + 1);
             int ctasPerSm = 1;
             stream_shape(s->progs.stack_depth, d.smem_per_sm, d.stage_elems, &ctasPerSm, &d.stages);
-            const uint64_t granule = 128, granules = (n + granule - 1) / granule;
-            const uint64_t ctas = std::min<uint64_t>(uint64_t(d.sm_count) * uint64_t(ctasPerSm), std::max<uint64_t>(granules, 1));
             const uint32_t cap = uint32_t(d.stage_elems);
-            std::vector<uint32_t> first(size_t(ctas) + 1, 0);
-            size_t seg = 0;
-            for (uint64_t c = 0; c < ctas; c++) {
-                const uint64_t lo = std::min(n, granules * c / ctas * granule), hi = std::min(n, granules * (c + 1) / ctas * granule);
-                first[size_t(c)] = uint32_t(host.size());
-                uint64_t e = lo;
-                while (e < hi) {
-                    while (seg + 1 < off.size() && off[seg + 1] <= e) seg++;
-                    // The part of the range inside this segment, in equal tiles of at most one stage.  Tiles are
-                    // whole 128-bit vectors of the buffers: where the segment starts or ends inside a vector
-                    // the tile is padded to the vector and remembers how many elements are not its own.
-                    const uint64_t pieceEnd = std::min<uint64_t>(hi, off[seg + 1]);
-                    const uint64_t ps = e & ~uint64_t(3), pe = (pieceEnd + 3) & ~uint64_t(3);
-                    const uint64_t parts = (pe - ps + cap - 1) / cap;
-                    const uint64_t each = std::min<uint64_t>(cap, ((pe - ps + parts - 1) / parts + 31) / 32 * 32);
-                    for (uint64_t ts = ps; ts < pe; ts += each) {
-                        const uint64_t te = std::min<uint64_t>(pe, ts + each);
-                        const uint32_t head = ts < e ? uint32_t(e - ts) : 0u, tail = te > pieceEnd ? uint32_t(te - pieceEnd) : 0u;
-                        host.push_back(TileDesc{ts, uint32_t(te - ts) | (head << 16) | (tail << 18), s->progs.seg_prog[seg]});
-                    }
-                    e = pieceEnd;
+            for (size_t seg = 0; seg + 1 < off.size(); seg++) {
+                const uint64_t b = off[seg], e = off[seg + 1];
+                if (e == b) continue;
+                const uint64_t ps = b & ~uint64_t(3), pe = (e + 3) & ~uint64_t(3);
+                const uint64_t parts = (pe - ps + cap - 1) / cap;
+                const uint64_t each = std::min<uint64_t>(cap, ((pe - ps + parts - 1) / parts + 31) / 32 * 32);
+                for (uint64_t ts = ps; ts < pe; ts += each) {
+                    const uint64_t te = std::min<uint64_t>(pe, ts + each);
+                    const uint32_t head = ts < b ? uint32_t(b - ts) : 0u, tail = te > e ? uint32_t(te - e) : 0u;
+                    host.push_back(TileDesc{ts, uint32_t(te - ts) | (head << 16) | (tail << 18), s->progs.seg_prog[seg]});
                 }
             }
+            const uint64_t nTiles = host.size();
+            const uint64_t ctas = std::min<uint64_t>(uint64_t(d.sm_count) * uint64_t(ctasPerSm), std::max<uint64_t>(nTiles, 1));
+            std::vector<uint32_t> first(size_t(ctas) + 1, 0);
+            for (uint64_t c = 0; c < ctas; c++) first[size_t(c)] = uint32_t(nTiles * c / ctas);
             first[size_t(ctas)] = uint32_t(host.size());
             if (cudaMalloc(reinterpret_cast<void **>(&d.cta_first), first.size() * sizeof(uint32_t)) != cudaSuccess) return RD_ERR_NOMEM;
             if (cudaMemcpy(d.cta_first, first.data(), first.size() * sizeof(uint32_t), cudaMemcpyHostToDevice) != cudaSuccess)
