@@ -40,8 +40,8 @@ WORKLOAD_OPS = {"config1": ["sum"], "config2": ["sum"], "config3": ["sum"], "con
 # DRAM bytes per launch of the tree kernel from one ncu capture (profiles/rd_tree_stream_kernel_config2.md):
 # dram__bytes_read.sum + dram__bytes_write.sum, mean of three launches.  Reported only while the kernel
 # source is the one that was profiled.
-NCU_TRAFFIC = {"workload": "config2", "bytes_per_launch": 274.4e6,
-               "kernel_sha256": "edf7693b791db6f6b010ed9ae97d4bfe6accefad333ddcb98011795718e0eac8"}
+NCU_TRAFFIC = {"workload": "config2", "bytes_per_launch": 274.6e6,
+               "kernel_sha256": "c88f427fe66cc6ce4f4d773132d5467b12fcf02d7785385344c4b5abae21a174"}
 
 
 def profiled_traffic(wname):
