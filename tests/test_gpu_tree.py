@@ -207,3 +207,56 @@ def test_unequal_segmentation_end_to_end(mode):
             ev, off, _ = oracle_schedule(algo, port, p, 4 * n, 0, *M1, sizes=sizes)
             want = O.reduce(ev, x.cpu().numpy(), off, "sum")
             assert out.cpu().numpy().tobytes() == want.tobytes(), (parts, algo)
+
+
+def _sampled_parity(wname, schedules, ops, n_samples=5):
+    """Full-size workload in the launch configuration the benchmark uses; the oracle checks whole sampled
+    segments bit for bit and slabs of the message against the fp64 reference."""
+    w = WORKLOADS[wname]
+    model = (w["alpha"], w["beta"], w["gamma"])
+    p, n = w["p"], w["n"]
+    x = make_inputs(p, n, w["dist"], w["seed"], device="cuda")
+    tab = rd.PointerTable(x)
+    out = torch.empty(n, device="cuda")
+    for algo, port in schedules:
+        h = rd.rd_schedule_create(algo, port, p, 4 * n, w["seg_bytes"], *model)
+        ev = rd.rd_schedule_events(h)
+        off = rd.rd_schedule_segments(h).astype(np.int64)
+        oev = np.zeros(len(ev), dtype=O.EVENT_DTYPE)
+        for f in ("t_start", "seg", "src", "dst", "kind"):
+            oev[f] = ev[f]                       # identical to the oracle's own list (tests/test_scheduler_vs_oracle.py)
+        q = len(off) - 1
+        picks = sorted({0, 1, q // 3, q // 2, q - 2, q - 1})[:n_samples + 1]
+        for op in ops:
+            rd.rd_reduce(h, tab, out, OPS[op])
+            torch.cuda.synchronize()
+            for j in picks:
+                lo, hi = int(off[j]), int(off[j + 1])
+                if hi == lo:
+                    continue
+                xs = x[:, lo:hi].cpu().numpy()
+                sel = oev[oev["seg"] == j].copy()
+                sel["seg"] = 0
+                want = O.reduce(sel, xs, [0, hi - lo], op)
+                got = out[lo:hi].cpu().numpy()
+                assert got.tobytes() == want.tobytes(), (wname, algo, op, j)
+                if op == "sum":
+                    ref, mag = O.reference_f64(xs, "sum")
+                    assert (np.abs(got.astype(np.float64) - ref) <= 1e-5 * mag).all()
+        rd.rd_destroy(h)
+
+
+def test_config3_full_size_sampled():
+    """p = 256, n = 2^22 fp32 uniform [-1, 1), 64 KiB segments, two ports: bi-greedy, butterfly and the trees."""
+    _sampled_parity("config3", [(rd.RD_BI_GREEDY, rd.RD_PORT_BI), (rd.RD_BUTTERFLY, rd.RD_PORT_BI),
+                                (rd.RD_BINOMIAL, rd.RD_PORT_BI), (rd.RD_PIPELINE, rd.RD_PORT_BI),
+                                (rd.RD_BINARY, rd.RD_PORT_BI)], ["sum"], n_samples=3)
+
+
+def test_config4_full_size_sampled():
+    """p = 32, n = 2^28 fp32 N(0,1) (32 GiB), 1 MiB segments: uni- and bi-greedy, sum and max."""
+    free_b, _ = torch.cuda.mem_get_info()
+    if free_b < (40 << 30):
+        pytest.skip("needs 33 GiB of device memory")
+    _sampled_parity("config4", [(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI), (rd.RD_BI_GREEDY, rd.RD_PORT_BI)], ["sum", "max"],
+                    n_samples=3)
