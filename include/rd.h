@@ -195,7 +195,9 @@ RD_API int rd_schedule_program(const rd_schedule_t *s, size_t seg, uint32_t *ops
  *   stats     host, or NULL.
  * The first call on a schedule uploads its tables to the current device
  * (allocates device memory, synchronises); rd_schedule_upload does the same
- * ahead of time.  Buffers must be 4-byte aligned; 16-byte aligned buffers of a
+ * ahead of time.  After one such call per schedule, element type and operation, a
+ * tree-mode call with at most 256 processes is a single kernel launch and may be
+ * recorded into a CUDA graph.  Buffers must be 4-byte aligned; 16-byte aligned buffers of a
  * multiple of 4 elements take the 128-bit streaming path (segments may start
  * and end anywhere), anything else a slower element-wise path.
  */

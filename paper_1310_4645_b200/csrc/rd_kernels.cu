@@ -1,12 +1,17 @@
-// sm_100a kernels of the schedule-exact reduction.
+// sm_100a kernels of the schedule-exact reduction, tree mode.
 //
-// Tree kernel: every thread owns U vectors of V elements of the message and evaluates, for them,
-// the segment's combine program: a one-accumulator stack machine whose operands are the p
-// processes' elements at the same index.  The path is bound by HBM (4(p+1) bytes per output
-// element, p-1 combines), so the kernel is built around keeping many independent 128-bit loads in
-// flight per thread: operands are fetched K operations ahead, in program order, into a register
-// ring that is statically indexed by unrolling the interpreter K times.  Partial results that have
-// to wait (at most log2 p of them) live in a per-thread column of shared memory.
+// Every thread owns a few 128-bit vectors of the message and evaluates, for them, the segment's
+// combine program: a one-accumulator stack machine whose operands are the p processes' elements at
+// the same index.  The path is bound by HBM (4(p+1) bytes per output element, p-1 combines), so the
+// kernels are built around keeping many bytes in flight:
+//   rd_tree_stream_kernel  the throughput path (128-bit aligned buffers): operand tiles are streamed
+//                          into a shared-memory ring by bulk asynchronous copies issued by producer
+//                          threads, consumers execute the program on them;
+//   rd_tree_kernel         the element path (any 4-byte aligned buffers): operands are fetched K
+//                          operations ahead, in program order, into a register ring that is
+//                          statically indexed by unrolling the interpreter K times.
+// Partial results that have to wait (at most log2 p of them) live in a per-thread column of shared
+// memory in both.
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -435,9 +440,7 @@ cudaError_t launch_one(const TreeLaunch &l)
 template <int DT, int OPR>
 cudaError_t launch_dtop(const TreeLaunch &l)
 {
-    const bool packed = l.p <= kPackedPtrs;
-    if (l.vec == 4) return packed ? launch_one<DT, OPR, 4, true>(l) : launch_one<DT, OPR, 4, false>(l);
-    return packed ? launch_one<DT, OPR, 1, true>(l) : launch_one<DT, OPR, 1, false>(l);
+    return l.p <= kPackedPtrs ? launch_one<DT, OPR, 1, true>(l) : launch_one<DT, OPR, 1, false>(l);
 }
 
 template <int DT, int OPR, bool PACKED>

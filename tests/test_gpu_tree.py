@@ -260,3 +260,35 @@ def test_config4_full_size_sampled():
         pytest.skip("needs 33 GiB of device memory")
     _sampled_parity("config4", [(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI), (rd.RD_BI_GREEDY, rd.RD_PORT_BI)], ["sum", "max"],
                     n_samples=3)
+
+
+def test_tree_mode_launches_can_be_replayed_from_a_cuda_graph():
+    """Small messages are launch bound; after one ordinary call per schedule (which uploads its tables and
+    configures the kernel) a tree-mode rd_reduce with at most 256 processes is a single kernel launch and
+    can be recorded into a CUDA graph and replayed."""
+    p, n = 8, 4096
+    xs = [make_inputs(p, n, "normal", seed=s, device="cuda") for s in range(3)]
+    outs = [torch.zeros(n, device="cuda") for _ in range(3)]
+    tabs = [rd.PointerTable(x) for x in xs]
+    hs = [rd.rd_schedule_create(a, pt, p, 4 * n, 2048, *M1) for a, pt in
+          ((rd.RD_UNI_GREEDY, rd.RD_PORT_UNI), (rd.RD_BINOMIAL, rd.RD_PORT_UNI), (rd.RD_BI_GREEDY, rd.RD_PORT_BI))]
+    want = []
+    for h, t, o in zip(hs, tabs, outs):
+        rd.rd_reduce(h, t, o, rd.RD_SUM)                 # ordinary call first
+    torch.cuda.synchronize()
+    want = [o.clone() for o in outs]
+    for o in outs:
+        o.zero_()
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            for _ in range(4):
+                for h, t, o in zip(hs, tabs, outs):
+                    rd.rd_reduce(h, t, o, rd.RD_SUM, stream=stream)
+    graph.replay()
+    torch.cuda.synchronize()
+    for o, w in zip(outs, want):
+        assert torch.equal(o, w)
+    for h in hs:
+        rd.rd_destroy(h)
