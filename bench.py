@@ -214,7 +214,8 @@ def run_reference(args, wname, w):
     sample = "each step: every schedule x op of the workload on the first %d of %d elements per process" % (n, w["n"])
     line = {"impl": "reference", "metric": "reduction_throughput", "value": value, "unit": "GB/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "i32" if w["dist"].startswith("int") else "f32", "data": "synthetic",
             "config": {"workload": wname, "p": w["p"], "n_elems": w["n"], "segment_bytes": w["seg_bytes"],
                        "schedules": [s[0] for s in WORKLOAD_SCHEDULES[wname]], "ops": WORKLOAD_OPS[wname]},
             "cpu_baseline": {"value": value, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
@@ -276,7 +277,7 @@ def main():
     # arenas: the kernel never reads the arena the previous launch read, and two arenas together exceed L2
     n_arenas = 3 if p * n * 4 <= (1 << 30) else 1
     arenas = [make_inputs(p, n, w["dist"], w["seed"] + 1000 * a, device=str(dev)) for a in range(n_arenas)]
-    out = torch.empty(n, dtype=torch.float32, device=dev)
+    out = torch.empty(n, dtype=arenas[0].dtype, device=dev)
     tables = [rd.PointerTable(a) for a in arenas]
 
     t0 = time.perf_counter()
@@ -342,8 +343,8 @@ def main():
         host_bytes = p * n * 4
         if host_bytes <= (8 << 30):
             hx = arenas[0].cpu().pin_memory()
-            hout = torch.empty(n, dtype=torch.float32).pin_memory()
-            staging = torch.empty((p + 1) * n, dtype=torch.float32, device=dev)
+            hout = torch.empty(n, dtype=arenas[0].dtype).pin_memory()
+            staging = torch.empty((p + 1) * n, dtype=arenas[0].dtype, device=dev)
             e_steps = max(3, min(args.steps, int(2.0 / (launches_per_step * host_bytes / 40e9)) or 1))
             for _, h in e2e_n_plans:
                 rd.rd_reduce_host(h, hx, hout, staging, ops[0])
@@ -435,7 +436,7 @@ def main():
         line = {
             "metric": "reduction_throughput", "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "vs_baseline": None, "dtype": "i32" if w["dist"].startswith("int") else "f32", "data": "synthetic",
             "config": {"workload": wname, "p": p, "n_elems": n, "segment_bytes": w["seg_bytes"],
                        "schedules": [s[0] for s in WORKLOAD_SCHEDULES[wname]], "ops": WORKLOAD_OPS[wname],
                        "bytes_counted": "p*m + m per reduction",

@@ -31,11 +31,6 @@ enum { OPR_SUM = 0, OPR_MAX = 1 };
 template <int V> struct Vec { uint32_t w[V]; };
 
 template <int V> __device__ __forceinline__ Vec<V> load_stream(const uint32_t *p);
-template <> __device__ __forceinline__ Vec<4> load_stream<4>(const uint32_t *p)
-{
-    const uint4 v = __ldcs(reinterpret_cast<const uint4 *>(p));
-    Vec<4> r; r.w[0] = v.x; r.w[1] = v.y; r.w[2] = v.z; r.w[3] = v.w; return r;
-}
 template <> __device__ __forceinline__ Vec<1> load_stream<1>(const uint32_t *p)
 {
     Vec<1> r; r.w[0] = __ldcs(p); return r;
