@@ -318,6 +318,15 @@ RD_API int rd_reduce_faithful_static(rd_schedule_t *s, const void *const *d_inpu
 RD_API int rd_search_segmentation(int p, size_t msg_bytes, size_t unit_bytes, const rd_model_t *model,
                                   size_t *seg_bytes, size_t cap, size_t *q_out, int64_t *predicted_ticks);
 
+/*
+ * rd_schedule_status -- tree-mode calls are asynchronous, so a kernel that had to give up a bounded
+ * wait (see rd_schedule_set_wait_budget; it should never happen) cannot report it through rd_reduce's
+ * return value.  This waits for the schedule's device to be idle and returns the status word its
+ * kernels share: 0, or RD_ERR_TIMEOUT if some launch since the last query gave up (its output is then
+ * not valid); the word is cleared.  The paper has no counterpart.
+ */
+RD_API int rd_schedule_status(rd_schedule_t *s, int *device_status);
+
 /* rd_destroy -- frees the schedule and its device tables.  NULL is allowed. */
 RD_API void rd_destroy(rd_schedule_t *s);
 

@@ -29,7 +29,7 @@ ALGOS = {"uni_greedy": RD_UNI_GREEDY, "bi_greedy": RD_BI_GREEDY, "binomial": RD_
 EXPORTS = ("rd_schedule_create", "rd_schedule_create_segments", "rd_optimal_segment", "rd_schedule_info",
            "rd_schedule_events", "rd_schedule_segments", "rd_schedule_program", "rd_reduce",
            "rd_schedule_upload", "rd_reduce_host", "rd_destroy", "rd_strerror", "rd_schedule_set_wait_budget",
-           "rd_schedule_trace", "rd_schedule_faithful_shape", "rd_schedule_actions", "rd_reduce_faithful_static", "rd_search_segmentation")
+           "rd_schedule_trace", "rd_schedule_faithful_shape", "rd_schedule_actions", "rd_reduce_faithful_static", "rd_search_segmentation", "rd_schedule_status")
 
 
 class rd_model_t(C.Structure):
@@ -86,6 +86,7 @@ def lib():
         L.rd_reduce_faithful_static.argtypes = [vp, C.POINTER(vp), vp, sz, i32, i32, vp, C.POINTER(rd_stats_t)]
         L.rd_search_segmentation.argtypes = [i32, sz, sz, C.POINTER(rd_model_t), C.POINTER(sz), sz, C.POINTER(sz),
                                              C.POINTER(C.c_int64)]
+        L.rd_schedule_status.argtypes = [vp, C.POINTER(i32)]
         L.rd_destroy.argtypes = [vp]
         L.rd_destroy.restype = None
         L.rd_strerror.argtypes = [i32]
@@ -309,6 +310,13 @@ def rd_search_segmentation(p, msg_bytes, unit_bytes, alpha, beta, gamma, tick=0.
     _check(lib().rd_search_segmentation(int(p), int(msg_bytes), int(unit_bytes), C.byref(m), arr, cap, C.byref(q),
                                         C.byref(ticks)), "rd_search_segmentation")
     return [int(arr[j]) for j in range(q.value)], ticks.value
+
+
+def rd_schedule_status(h) -> int:
+    """Waits for the device and returns (and clears) the status word of the schedule's kernels."""
+    st = C.c_int(0)
+    _check(lib().rd_schedule_status(h, C.byref(st)), "rd_schedule_status")
+    return st.value
 
 
 def rd_destroy(h) -> None:

@@ -420,6 +420,18 @@ int reduce_faithful(rd_schedule *s, const void *const *d_inputs, void *d_out, si
     return RD_OK;
 }
 
+// Nothing may be thrown across the C boundary: host containers can run out of memory.
+template <typename F> int guarded(F &&body)
+{
+    try {
+        return body();
+    } catch (const std::bad_alloc &) {
+        return RD_ERR_NOMEM;
+    } catch (...) {
+        return RD_ERR_INTERNAL;
+    }
+}
+
 }  // namespace
 
 extern "C" {
@@ -528,7 +540,7 @@ int rd_schedule_program(const rd_schedule_t *s, size_t seg, uint32_t *ops, size_
 int rd_schedule_upload(rd_schedule_t *s)
 {
     if (!s) return RD_ERR_INVALID_ARG;
-    return upload(s);
+    return guarded([&] { return upload(s); });
 }
 
 int rd_reduce(rd_schedule_t *s, const void *const *d_inputs, void *d_out, size_t n_elems, rd_dtype_t dtype, rd_op_t op,
@@ -541,10 +553,12 @@ int rd_reduce(rd_schedule_t *s, const void *const *d_inputs, void *d_out, size_t
     for (int i = 0; i < s->p; i++)
         if ((n_elems > 0 && !d_inputs[i]) || (reinterpret_cast<uintptr_t>(d_inputs[i]) & 3u)) return RD_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(d_out) & 3u) return RD_ERR_INVALID_ARG;
-    if (int rc = upload(s)) return rc;
-    if (exec == RD_EXEC_FAITHFUL)
-        return reduce_faithful(s, d_inputs, d_out, n_elems, dtype, op, static_cast<cudaStream_t>(cuda_stream), stats);
-    return reduce_tree(s, d_inputs, d_out, n_elems, dtype, op, static_cast<cudaStream_t>(cuda_stream), stats);
+    return guarded([&] {
+        if (int rc = upload(s)) return rc;
+        if (exec == RD_EXEC_FAITHFUL)
+            return reduce_faithful(s, d_inputs, d_out, n_elems, dtype, op, static_cast<cudaStream_t>(cuda_stream), stats);
+        return reduce_tree(s, d_inputs, d_out, n_elems, dtype, op, static_cast<cudaStream_t>(cuda_stream), stats);
+    });
 }
 
 int rd_reduce_host(rd_schedule_t *s, const void *const *h_inputs, void *h_out, void *d_staging, size_t n_elems,
@@ -596,11 +610,28 @@ int rd_schedule_faithful_shape(rd_schedule_t *s, int *blocks_per_process, int *s
         if (scratch_bytes) *scratch_bytes = 0;
         return RD_OK;
     }
-    if (int rc = upload(s)) return rc;
-    if (int rc = prepare_faithful(s)) return rc;
-    if (blocks_per_process) *blocks_per_process = s->dev.f_lanes;
-    if (slots_per_process) *slots_per_process = s->dev.f_slots;
-    if (scratch_bytes) *scratch_bytes = size_t(s->p) * size_t(s->dev.f_slots) * size_t(s->dev.f_slot_elems) * 4;
+    return guarded([&] {
+        if (int rc = upload(s)) return rc;
+        if (int rc = prepare_faithful(s)) return rc;
+        if (blocks_per_process) *blocks_per_process = s->dev.f_lanes;
+        if (slots_per_process) *slots_per_process = s->dev.f_slots;
+        if (scratch_bytes) *scratch_bytes = size_t(s->p) * size_t(s->dev.f_slots) * size_t(s->dev.f_slot_elems) * 4;
+        return int(RD_OK);
+    });
+}
+
+int rd_schedule_status(rd_schedule_t *s, int *device_status)
+{
+    if (!s || !device_status) return RD_ERR_INVALID_ARG;
+    if (s->dev.device < 0) { *device_status = 0; return RD_OK; }     // nothing has run on a device yet
+    int prev = -1, st = 0;
+    if (cudaGetDevice(&prev) != cudaSuccess || cudaSetDevice(s->dev.device) != cudaSuccess) return RD_ERR_CUDA;
+    bool ok = cudaDeviceSynchronize() == cudaSuccess;
+    ok = ok && cudaMemcpy(&st, s->dev.status, sizeof(int), cudaMemcpyDeviceToHost) == cudaSuccess;
+    if (ok && st != 0) ok = cudaMemset(s->dev.status, 0, sizeof(int)) == cudaSuccess;
+    cudaSetDevice(prev);
+    if (!ok) return RD_ERR_CUDA;
+    *device_status = st;
     return RD_OK;
 }
 

@@ -143,7 +143,9 @@ def test_empty_message_and_stats():
     x = make_inputs(8, 1 << 16, "normal", seed=1, device="cuda")
     out = torch.empty(1 << 16, device="cuda")
     h = rd.rd_schedule_create(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, 8, 4 << 16, 4096, *M1)
+    assert rd.rd_schedule_status(h) == 0                         # nothing has run yet
     st = rd.rd_reduce(h, x, out, rd.RD_SUM, want_stats=True)
+    assert rd.rd_schedule_status(h) == 0
     assert st.kernel_ms > 0 and st.bytes_moved == 9 * (4 << 16) and st.n_launches == 1
     assert abs(st.predicted_s - rd.rd_schedule_info(h)["predicted_seconds"]) < 1e-12
     with pytest.raises(rd.RdError) as e:
