@@ -294,3 +294,19 @@ def test_tree_mode_launches_can_be_replayed_from_a_cuda_graph():
         assert torch.equal(o, w)
     for h in hs:
         rd.rd_destroy(h)
+
+
+def test_largest_process_count():
+    """p = 4096, the boundary's maximum: the tree kernel runs it (deepest stacks, pointer table); the
+    schedule-faithful kernel cannot keep that many processes resident and says so."""
+    p, n = 4096, 512
+    x = make_inputs(p, n, "int_pm2p20", seed=8, device="cuda")
+    for algo, port, seg in ((rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, 1024), (rd.RD_BINOMIAL, rd.RD_PORT_BI, 0),
+                            (rd.RD_BINARY, rd.RD_PORT_UNI, 512)):
+        check(algo, port, x, seg, "sum")
+    h = rd.rd_schedule_create(rd.RD_BINOMIAL, rd.RD_PORT_UNI, p, 4 * n, 0, *M1)
+    out = torch.empty(n, dtype=torch.int32, device="cuda")
+    with pytest.raises(rd.RdError) as e:
+        rd.rd_reduce(h, x, out, rd.RD_SUM, exec_mode=rd.RD_EXEC_FAITHFUL)
+    assert e.value.status == rd.RD_ERR_UNSUPPORTED
+    rd.rd_destroy(h)
