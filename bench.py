@@ -41,7 +41,7 @@ WORKLOAD_OPS = {"config1": ["sum"], "config2": ["sum"], "config3": ["sum"], "con
 # dram__bytes_read.sum + dram__bytes_write.sum, mean of three launches.  Reported only while the kernel
 # source is the one that was profiled.
 NCU_TRAFFIC = {"workload": "config2", "bytes_per_launch": 274.6e6,
-               "kernel_sha256": "c88f427fe66cc6ce4f4d773132d5467b12fcf02d7785385344c4b5abae21a174"}
+               "kernel_sha256": "989893266a8018cea509f69a36eb51d09c3b3e9fb05008e085cc0cca8b38e2bf"}
 
 
 def profiled_traffic(wname):

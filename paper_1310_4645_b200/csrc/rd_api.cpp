@@ -310,6 +310,11 @@ int prepare_faithful(rd_schedule *s)
 {
     DeviceTables &d = s->dev;
     if (d.faithful_ready) return RD_OK;
+    // an earlier attempt may have failed half-way (out of memory): start clean
+    cudaFree(d.f_actions); cudaFree(d.f_first); cudaFree(d.f_seg_off); cudaFree(d.f_flags); cudaFree(d.f_trace);
+    cudaFree(d.f_block_times); cudaFree(d.f_scratch); cudaFree(d.f_inputs); cudaFree(d.f_abort);
+    d.f_actions = nullptr; d.f_first = nullptr; d.f_seg_off = nullptr; d.f_flags = nullptr; d.f_trace = nullptr;
+    d.f_block_times = nullptr; d.f_scratch = nullptr; d.f_inputs = nullptr; d.f_abort = nullptr;
     ActionLists lists;
     const size_t q = s->sched.seg_off.size() - 1;
     if (int rc = build_actions(s->p, q, s->sched.events, lists)) return rc;
