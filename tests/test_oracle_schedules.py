@@ -377,3 +377,33 @@ def test_validator_catches_planted_mistakes():
     first0 = int(np.flatnonzero(bad["seg"] == 0)[0]); first1 = int(np.flatnonzero(bad["seg"] == 1)[0])
     bad["t_start"][first0], bad["t_start"][first1] = bad["t_start"][first1], bad["t_start"][first0]
     assert O.validate(bad, p, sizes, A, B, G, False, True, True)[0] != 0
+
+
+# --------------------------------------------------------------------------- Section V-B text (soft pins)
+def _best_times_p64(m, A=10, B=1, G=0, p=64):
+    """Best completion time of each algorithm over all integer segment sizes (the figures of Section V-B
+    use each algorithm's optimal segment size; alpha = 10, beta = 1, gamma = 0, p = 64)."""
+    greedy = min(O.uni_greedy(p, O.equal_sizes(m, s), A, B, G, want_events=False)[1] for s in range(1, m + 1))
+    unit = lambda s: A + (B + G) * s
+    N = clog2(p + 1)
+    binom = clog2(p) * unit(m)
+    pipe = min((p - 1 + 2 * (-(-m // s) - 1)) * unit(s) for s in range(1, m + 1))
+    binary = min((2 * (N - 1) + 4 * (-(-m // s) - 1)) * unit(s) for s in range(1, m + 1))
+    return greedy, binom, pipe, binary
+
+
+def test_section5_small_mid_and_large_message_regimes():
+    """Small messages: uni-greedy with one segment IS binomial; mid-size: about 50 % faster than the best
+    standard algorithm; large: pipeline approaches it."""
+    ratios = {}
+    for m in (4, 8, 16, 64, 128, 256, 512, 1024, 2048, 4096):
+        g, binom, pipe, binary = _best_times_p64(m)
+        assert g <= min(binom, pipe, binary)                       # Theorem 5: never worse than an in-order schedule
+        ratios[m] = min(binom, pipe, binary) / g
+        if m <= 16:
+            assert g == binom                                      # same time as binomial
+    assert 1.4 <= max(ratios.values()) <= 1.7                      # "approximately 50 % faster" in the middle
+    assert max(ratios, key=ratios.get) in (256, 512, 1024)
+    assert ratios[4096] < ratios[1024] < ratios[512]               # and the advantage fades for large messages
+    g, binom, pipe, binary = _best_times_p64(16384)
+    assert pipe == min(binom, pipe, binary) and pipe / g < 1.12    # pipeline approaches uni-greedy
