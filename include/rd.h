@@ -197,9 +197,10 @@ RD_API int rd_schedule_program(const rd_schedule_t *s, size_t seg, uint32_t *ops
  * (allocates device memory, synchronises); rd_schedule_upload does the same
  * ahead of time.  After one such call per schedule, element type and operation, a
  * tree-mode call with at most 256 processes is a single kernel launch and may be
- * recorded into a CUDA graph.  Buffers must be 4-byte aligned; 16-byte aligned buffers of a
- * multiple of 4 elements take the 128-bit streaming path (segments may start
- * and end anywhere), anything else a slower element-wise path.
+ * recorded into a CUDA graph.  Buffers must be 4-byte aligned; 16-byte aligned buffers take
+ * the 128-bit streaming path (segments may start and end anywhere; when n_elems is
+ * not a multiple of 4 the last elements are done by a second, tiny launch), other
+ * buffers a slower element-wise path.
  */
 RD_API int rd_reduce(rd_schedule_t *s, const void *const *d_inputs, void *d_out, size_t n_elems,
               rd_dtype_t dtype, rd_op_t op, rd_exec_t exec, void *cuda_stream, rd_stats_t *stats);

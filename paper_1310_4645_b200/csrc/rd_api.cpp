@@ -17,6 +17,7 @@ using namespace rd;
 namespace {
 
 constexpr int kPtrRing = 8;   // pointer tables in flight for p > kPackedPtrs
+constexpr int kTailTiles = 5; // key of the tile table for the elements the 128-bit path leaves over
 
 struct DeviceTables {
     int device = -1;
@@ -215,8 +216,9 @@ int tiles_for(rd_schedule *s, int vec, const TileDesc **tiles, uint32_t *count)
             int ctasPerSm = 1;
             stream_shape(s->progs.stack_depth, d.smem_per_sm, d.stage_elems, &ctasPerSm, &d.stages);
             const uint32_t cap = uint32_t(d.stage_elems);
+            const uint64_t n4 = n & ~uint64_t(3);          // the last n mod 4 elements go to the element kernel
             for (size_t seg = 0; seg + 1 < off.size(); seg++) {
-                const uint64_t b = off[seg], e = off[seg + 1];
+                const uint64_t b = std::min(off[seg], n4), e = std::min(off[seg + 1], n4);
                 if (e == b) continue;
                 const uint64_t ps = b & ~uint64_t(3), pe = (e + 3) & ~uint64_t(3);
                 const uint64_t parts = (pe - ps + cap - 1) / cap;
@@ -237,9 +239,12 @@ int tiles_for(rd_schedule *s, int vec, const TileDesc **tiles, uint32_t *count)
                 return RD_ERR_CUDA;
             d.n_ctas = uint32_t(ctas);
         } else {
-            const uint32_t cap = tree_tile_elems(vec);
+            // element path: the whole message (vec == 1), or only what the 128-bit path leaves over (kTailTiles)
+            const uint64_t n = off.empty() ? 0 : off.back();
+            const uint64_t from = vec == kTailTiles ? (n & ~uint64_t(3)) : 0;
+            const uint32_t cap = tree_tile_elems(1);
             for (size_t j = 0; j + 1 < off.size(); j++)
-                for (uint64_t e = off[j]; e < off[j + 1]; e += cap)
+                for (uint64_t e = std::max(off[j], from); e < off[j + 1]; e += cap)
                     host.push_back(TileDesc{e, uint32_t(std::min<uint64_t>(cap, off[j + 1] - e)), s->progs.seg_prog[j]});
         }
         if (int rc = upload_tiles(d, vec, host)) return rc;
@@ -254,12 +259,17 @@ int reduce_tree(rd_schedule *s, const void *const *d_inputs, void *d_out, size_t
                 cudaStream_t stream, rd_stats_t *stats)
 {
     DeviceTables &d = s->dev;
-    // 128-bit path: every buffer 16-byte aligned and a whole number of vectors (segments may start anywhere)
-    bool wide = (reinterpret_cast<uintptr_t>(d_out) & 15u) == 0 && (n & 3u) == 0;
+    // 128-bit path: every buffer 16-byte aligned (segments may start anywhere); the last n mod 4 elements
+    // of the message, if any, are left to a second, tiny launch of the element kernel
+    bool wide = (reinterpret_cast<uintptr_t>(d_out) & 15u) == 0;
     for (int i = 0; i < s->p && wide; i++) wide = (reinterpret_cast<uintptr_t>(d_inputs[i]) & 15u) == 0;
     TreeLaunch l{};
     l.vec = wide ? 4 : 1;
     if (int rc = tiles_for(s, l.vec, &l.tiles, &l.n_tiles)) return rc;
+    const TileDesc *tailTiles = nullptr;
+    uint32_t nTail = 0;
+    if (wide && (n & 3u) != 0)
+        if (int rc = tiles_for(s, kTailTiles, &tailTiles, &nTail)) return rc;
     l.host_ptrs = d_inputs;
     l.dev_ptr_table = nullptr;
     if (s->p > kPackedPtrs) {
@@ -276,6 +286,11 @@ int reduce_tree(rd_schedule *s, const void *const *d_inputs, void *d_out, size_t
     l.cta_first = d.cta_first; l.n_ctas = d.n_ctas; l.stages = d.stages; l.stage_elems = d.stage_elems; l.status = d.status; l.device = d.device;
     if (stats && cudaEventRecord(d.ev_start, stream) != cudaSuccess) return RD_ERR_CUDA;
     if ((wide ? launch_tree_stream(l) : launch_tree(l)) != 0) return RD_ERR_CUDA;
+    if (nTail > 0) {
+        TreeLaunch t = l;
+        t.vec = 1; t.tiles = tailTiles; t.n_tiles = nTail;
+        if (launch_tree(t) != 0) return RD_ERR_CUDA;
+    }
     if (s->p > kPackedPtrs) {
         const int slot = (d.ring_next + kPtrRing - 1) % kPtrRing;
         if (cudaEventRecord(d.ring_done[slot], stream) != cudaSuccess) return RD_ERR_CUDA;
@@ -290,7 +305,7 @@ int reduce_tree(rd_schedule *s, const void *const *d_inputs, void *d_out, size_t
         stats->bytes_moved = uint64_t(s->p + 1) * uint64_t(n) * 4u;
         stats->gbytes_per_s = ms > 0 ? double(stats->bytes_moved) / (double(ms) * 1e6) : 0.0;
         stats->predicted_s = double(s->sched.completion) * s->ticks.tick;
-        stats->n_launches = l.n_tiles ? 1 : 0;
+        stats->n_launches = (l.n_tiles ? 1 : 0) + (nTail ? 1 : 0);
         int st = 0;
         if (cudaMemcpy(&st, d.status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return RD_ERR_CUDA;
         stats->device_status = st;

@@ -44,7 +44,9 @@ def check(algo, port, x_dev, seg_bytes, op, model=M1):
 SHAPES = [(8, 4096, 512), (5, 10000, 2500), (13, 3 * 2048 + 36, 2048 + 520), (64, 8192, 1024), (2, 4100, 4100),
           (33, 6000, 1000), (16, 128, 8), (1, 5000, 1000),
           # segments that start and end inside a 128-bit vector (the message itself is whole vectors)
-          (8, 3000, 333), (16, 4100, 4100), (13, 6180, 999), (4, 64, 3), (8, 4096, 6), (32, 8192, 2049)]
+          (8, 3000, 333), (16, 4100, 4100), (13, 6180, 999), (4, 64, 3), (8, 4096, 6), (32, 8192, 2049),
+          # message lengths that are not whole vectors: the last elements go through the element kernel
+          (8, 4099, 1000), (16, 2050, 2050), (5, 7, 2), (3, 3, 1), (8, 6151, 333)]
 
 
 @pytest.mark.parametrize("name,algo,port", SCHEDULES)
