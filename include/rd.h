@@ -62,7 +62,7 @@ typedef enum {
     RD_BINOMIAL = 2,   /* Section IV; either port model                                          */
     RD_PIPELINE = 3,   /* Section IV; either port model                                          */
     RD_BINARY = 4,     /* Section IV; either port model                                          */
-    RD_BUTTERFLY = 5   /* Section III (reduce-scatter/gather); bidirectional, p a power of two   */
+    RD_BUTTERFLY = 5   /* Section III (reduce-scatter/gather); bidirectional ports only           */
 } rd_algo_t;
 
 typedef enum { RD_PORT_UNI = 0, RD_PORT_BI = 1 } rd_port_t;   /* Section II */
@@ -103,7 +103,10 @@ typedef struct {
  *   out        host; receives the new schedule; release with rd_destroy.
  *   algo/port  legal pairs: uni-greedy + UNI; bi-greedy + BI; butterfly + BI;
  *              binomial, pipeline, binary + either.  Others: RD_ERR_UNSUPPORTED.
- *   p          1..4096.  Butterfly: a power of two, else RD_ERR_UNSUPPORTED.
+ *   p          1..4096.  Butterfly: when p is not a power of two the processes beyond
+ *              the largest power of two P first send their whole message to a
+ *              partner below P (one extra round), then the butterfly runs on P
+ *              processes; the schedule then has P chunks ("segments").
  *   msg_bytes  multiple of 4; may be 0.
  *   seg_bytes  multiple of 4, 0 < seg_bytes; values above msg_bytes mean one
  *              segment.  0 selects the segment size rd_optimal_segment gives.

@@ -355,7 +355,13 @@ int orc_binary(int p, int q, const int64_t *sizes, int64_t A, int64_t B, int64_t
 
 /* ------------------------------------------------------------------------- */
 /* Butterfly (Section III): reduce-scatter by recursive halving, then gather */
-/* by recursive doubling; p a power of two, bidirectional ports.  Distance   */
+/* by recursive doubling, bidirectional ports, for p a power of two.  For    */
+/* other p (the paper only points to an improved algorithm it does not       */
+/* describe) the processes beyond the largest power of two first send their  */
+/* whole message to a partner below it, which combines it; the power-of-two  */
+/* algorithm then runs on the rest.  PARITY UNPINNED for that extension: the */
+/* paper fixes nothing about it; only validity and the contribution          */
+/* invariant are checked.  Distance                                          */
 /* p/2 first; of an exchanging pair the process with the distance bit clear  */
 /* keeps the lower half [lo, mid), mid = lo + floor((hi-lo)/2).  A "segment" */
 /* in the event list is a final chunk c (the range process c owns after the  */
@@ -364,12 +370,16 @@ int orc_binary(int p, int q, const int64_t *sizes, int64_t A, int64_t B, int64_t
 /* starts together; a round lasts as long as its largest message.            */
 /* n = message length in elements, esize = size units per element.           */
 /* chunk_off[p+1] receives the chunk boundaries in elements.                 */
-/* Event count: p(p-1) + (p/2) log2 p.                                       */
+/* Event count: P(P-1) + (P/2) log2 P + (p-P) P, P the power of two used.     */
 /* ------------------------------------------------------------------------- */
-int orc_butterfly(int p, int64_t n, int64_t esize, int64_t A, int64_t B, int64_t G,
+int orc_butterfly(int p_all, int64_t n, int64_t esize, int64_t A, int64_t B, int64_t G,
                   orc_event_t *events, int64_t *chunk_off, int64_t *completion)
 {
-    if (p < 1 || n < 0 || (p & (p - 1)) != 0) return ORC_BAD_ARG;
+    if (p_all < 1 || n < 0) return ORC_BAD_ARG;
+    /* p = largest power of two not above p_all; the r = p_all - p processes beyond it are folded in first */
+    int p = 1;
+    while (2 * p <= p_all) p *= 2;
+    int r_extra = p_all - p;
     int L = orc_ceil_log2(p);
     int64_t *lo = malloc(8 * (size_t)p), *hi = malloc(8 * (size_t)p);
     int64_t *clo = malloc(8 * (size_t)p), *chi = malloc(8 * (size_t)p);
@@ -388,6 +398,18 @@ int orc_butterfly(int p, int64_t n, int64_t esize, int64_t A, int64_t B, int64_t
     if (chunk_off) { for (int c = 0; c < p; c++) chunk_off[c] = clo[c]; chunk_off[p] = n; }
     size_t ne = 0;
     int64_t t = 0;
+    if (r_extra > 0) {                               /* fold: process p + i sends its whole message to i */
+        for (int i = 0; i < r_extra; i++) {
+            for (int c = 0; c < p; c++) {
+                if (events) {
+                    events[ne].seg = c; events[ne].src = p + i; events[ne].dst = i;
+                    events[ne].kind = 0; events[ne].t_start = 0;
+                }
+                ne++;
+            }
+        }
+        t = t_comm(A, B, n * esize) + t_comp(G, n * esize);
+    }
     for (int r = 0; r < L; r++) {
         int d = p >> (r + 1);
         int64_t longest = 0;

@@ -107,15 +107,20 @@ def binary(p, sizes, A, B, G, bidir):
 
 
 def butterfly(p, n, esize, A, B, G):
-    """Reduce-scatter/gather.  Returns (events, chunk_off[p+1] in elements, completion)."""
-    L = ceil_log2(p)
-    ev = np.zeros(max(p * (p - 1) + (p // 2) * L, 1), dtype=EVENT_DTYPE)
-    off = np.zeros(p + 1, dtype=np.int64)
+    """Reduce-scatter/gather.  Returns (events, chunk_off[P+1] in elements, completion); P = the largest
+    power of two not above p (the other p - P processes are folded in first)."""
+    P = 1
+    while 2 * P <= p:
+        P *= 2
+    L = ceil_log2(P)
+    count = P * (P - 1) + (P // 2) * L + (p - P) * P
+    ev = np.zeros(max(count, 1), dtype=EVENT_DTYPE)
+    off = np.zeros(P + 1, dtype=np.int64)
     comp = C.c_int64(0)
     rc = lib().orc_butterfly(C.c_int(p), C.c_int64(n), C.c_int64(esize), C.c_int64(A), C.c_int64(B),
                              C.c_int64(G), C.c_void_p(ev.ctypes.data), _p(off, C.c_int64), C.byref(comp))
     _check(rc, "butterfly")
-    return ev[: p * (p - 1) + (p // 2) * L], off, comp.value
+    return ev[:count], off, comp.value
 
 
 def validate(events, p, sizes, A, B, G, bidir, tree_rules=True, in_order=False):

@@ -463,7 +463,6 @@ int rd_schedule_create(rd_schedule_t **out, rd_algo_t algo, rd_port_t port, int 
     if (p < 1 || p > kMaxProcs) return RD_ERR_INVALID_ARG;
     if (int(algo) < 0 || int(algo) > RD_BUTTERFLY || (port != RD_PORT_UNI && port != RD_PORT_BI)) return RD_ERR_INVALID_ARG;
     if (!legal_pair(algo, port)) return RD_ERR_UNSUPPORTED;
-    if (algo == RD_BUTTERFLY && (p & (p - 1)) != 0) return RD_ERR_UNSUPPORTED;
     if (seg_bytes == 0) {
         Ticks t;
         if (int rc = make_ticks(model, t)) return rc;

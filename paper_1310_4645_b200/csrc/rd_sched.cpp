@@ -227,17 +227,27 @@ int gen_binary(int p, const std::vector<int64_t> &seg_bytes, const Ticks &c, boo
 
 // ---------------------------------------------------------------------------------------------
 // Section III butterfly: recursive halving (distance p/2 first, the process with the distance bit
-// clear keeps the lower half), then a binomial gather of the p reduced chunks to process 0.
+// clear keeps the lower half), then a binomial gather of the p reduced chunks to process 0.  When the
+// number of processes is not a power of two, those beyond the largest power of two are folded into
+// partners below it first (the improved algorithm the paper cites for that case is not described there).
 // ---------------------------------------------------------------------------------------------
-int gen_butterfly(int p, uint64_t n, const Ticks &c, Schedule &out)
+int gen_butterfly(int pAll, uint64_t n, const Ticks &c, Schedule &out)
 {
-    if (p < 1 || (p & (p - 1)) != 0) return RD_ERR_UNSUPPORTED;
+    if (pAll < 1) return RD_ERR_INVALID_ARG;
+    int p = 1;                                    // the largest power of two not above pAll
+    while (2 * p <= pAll) p *= 2;
     const int L = ceil_log2(uint64_t(p));
     const size_t P = size_t(p);
     // chunk boundaries: follow each process's range through the halvings
     std::vector<uint64_t> lo(P, 0), hi(P, n);
     out.events.clear();
     int64_t t = 0;
+    if (pAll > p) {
+        // fold: every process beyond the power of two hands its whole message to a partner below it
+        for (int i = 0; i < pAll - p; i++)
+            for (int ch = 0; ch < p; ch++) out.events.push_back(rd_event_t{ch, p + i, i, 0, 0});
+        t = c.comm(int64_t(n) * 4) + c.comp(int64_t(n) * 4);
+    }
     for (int r = 0; r < L; r++) {
         const int d = p >> (r + 1);
         int64_t longest = 0;

@@ -59,7 +59,6 @@ def test_create_rejects_bad_arguments():
     assert status_of(f, rd.RD_UNI_GREEDY, rd.RD_PORT_BI, 4, 64, 16, *MODEL) == rd.RD_ERR_UNSUPPORTED
     assert status_of(f, rd.RD_BI_GREEDY, rd.RD_PORT_UNI, 4, 64, 16, *MODEL) == rd.RD_ERR_UNSUPPORTED
     assert status_of(f, rd.RD_BUTTERFLY, rd.RD_PORT_UNI, 4, 64, 16, *MODEL) == rd.RD_ERR_UNSUPPORTED
-    assert status_of(f, rd.RD_BUTTERFLY, rd.RD_PORT_BI, 6, 64, 16, *MODEL) == rd.RD_ERR_UNSUPPORTED
     assert status_of(rd.rd_schedule_create_segments, rd.RD_BUTTERFLY, rd.RD_PORT_BI, 4, [32, 32], *MODEL) \
         == rd.RD_ERR_UNSUPPORTED
     assert status_of(rd.rd_schedule_create_segments, rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, 4, [32, 0], *MODEL) \

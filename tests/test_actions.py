@@ -183,7 +183,7 @@ def emulate_lanes(h, x, op, blocking_send, rng, lanes):
 @pytest.mark.parametrize("algo,port", CASES)
 def test_lanes_that_drift_apart_never_meet_in_a_slot(algo, port):
     """Unequal segments (a short last one), several blocks per process running at very different speeds."""
-    p, n, seg = 13 if algo != rd.RD_BUTTERFLY else 8, 618, 257
+    p, n, seg = 13, 618, 257
     rng = np.random.default_rng(algo)
     x = (rng.standard_normal((p, n)) * 10.0 ** rng.integers(-4, 5, size=(p, n))).astype(np.float32)
     h = rd.rd_schedule_create(algo, port, p, 4 * n, 4 * 256 if algo != rd.RD_BUTTERFLY else 0, *M1)
@@ -200,8 +200,6 @@ def test_lanes_that_drift_apart_never_meet_in_a_slot(algo, port):
 @pytest.mark.parametrize("algo,port", CASES)
 @pytest.mark.parametrize("p", [2, 3, 8, 13, 32])
 def test_action_lists_reproduce_the_oracle(algo, port, p):
-    if algo == rd.RD_BUTTERFLY and p & (p - 1):
-        pytest.skip("butterfly needs a power of two")
     n, seg = 96, 16
     rng = np.random.default_rng(7 * p + algo)
     xf = (rng.standard_normal((p, n)) * 10.0 ** rng.integers(-6, 7, size=(p, n))).astype(np.float32)

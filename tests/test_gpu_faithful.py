@@ -43,8 +43,6 @@ SHAPES = [(8, 4096, 512), (5, 10000, 2500), (13, 3 * 2048 + 36, 2048 + 520), (64
 @pytest.mark.parametrize("dist,op", [("int_pm2p20", "sum"), ("normal", "sum"), ("normal", "max")])
 def test_parity_small_shapes(name, algo, port, dist, op):
     for p, n, seg in SHAPES:
-        if algo == rd.RD_BUTTERFLY and p & (p - 1):
-            continue
         x = make_inputs(p, n, dist, seed=p * 1000 + n, device="cuda")
         if dist == "normal":
             x *= 10.0 ** torch.randint(-4, 5, x.shape, device="cuda", generator=torch.Generator("cuda").manual_seed(1))

@@ -145,9 +145,23 @@ def test_butterfly_ragged_and_short_messages():
         assert comp * p >= 2 * L * 7 * p + 2 * (p - 1) * 1 * 4 * n + (p - 1) * 1 * 4 * n
 
 
-def test_butterfly_rejects_non_power_of_two():
-    with pytest.raises(RuntimeError):
-        O.butterfly(6, 64, 1, 1, 1, 1)
+@pytest.mark.parametrize("p", [3, 5, 6, 7, 12, 24, 100])
+def test_butterfly_folds_extra_processes_in_first(p):
+    """Not a power of two (an extension: the paper only cites an improved algorithm): the processes beyond
+    the largest power of two P send their message to a partner first, one round of alpha + (beta+gamma) m,
+    then the P-process butterfly of Table III follows.  Valid, and every contribution arrives once."""
+    A, B, G = 7, 2, 1
+    P = 1 << (p.bit_length() - 1)
+    n = 4 * P
+    ev, off, comp = O.butterfly(p, n, 1, A, B, G)
+    L = clog2(P)
+    assert comp == (A + (B + G) * n) + 2 * L * A + 2 * (P - 1) * B * n // P + (P - 1) * G * n // P
+    assert len(off) == P + 1 and (np.diff(off) == n // P).all()
+    rc, last = O.validate(ev, p, np.diff(off), A, B, G, True, tree_rules=False)
+    assert rc == 0 and last == comp
+    assert O.contributions(ev, p, P) == 0
+    x = np.random.default_rng(p).integers(-2**31, 2**31, size=(p, n), dtype=np.int64).astype(np.int32)
+    assert (O.reduce(ev, x, off, "max") == x.max(axis=0)).all()
 
 
 # --------------------------------------------------------------------------- worked examples

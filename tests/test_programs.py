@@ -20,8 +20,6 @@ def wide_floats(rng, shape):
 @pytest.mark.parametrize("algo,port", CASES)
 @pytest.mark.parametrize("p", [1, 2, 3, 8, 21, 64])
 def test_programs_reproduce_the_oracle(algo, port, p):
-    if algo == rd.RD_BUTTERFLY and p & (p - 1):
-        pytest.skip("butterfly needs a power of two")
     msg, seg = 4 * 96, 4 * 16
     n = msg // 4
     rng = np.random.default_rng(1000 * algo + p)

@@ -39,8 +39,6 @@ def compare(algo, port, p, msg, seg, model, sizes=None):
 def test_grid_of_small_cases(algo):
     for port in PORTS[algo]:
         for p in (1, 2, 3, 4, 5, 7, 8, 13, 16, 31, 32, 33, 64):
-            if algo == rd.RD_BUTTERFLY and p & (p - 1):
-                continue
             for msg, seg in ((64, 64), (64, 16), (4096, 512), (1000, 96), (36, 4), (4, 4)):
                 compare(algo, port, p, msg, seg, M1)
             compare(algo, port, p, 2048, 256, (0.0, 1e-10, 0.0))          # ties everywhere
