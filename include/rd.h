@@ -14,7 +14,12 @@
  *     aborts, nothing throws across this boundary, and output arguments are
  *     left untouched on failure.
  *   - Processes are numbered 0..p-1 and the root is process 0 (the paper's
- *     implementation makes the same restriction, Fig. 2 caption).
+ *     implementation makes the same restriction, Fig. 2 caption).  The system
+ *     is homogeneous and fully connected (Section II), so a schedule does not
+ *     care which buffer plays which process: to reduce towards another root,
+ *     pass the pointer array permuted so that the root's buffer comes first.
+ *     On one GPU every process can read the result buffer, so an all-reduce
+ *     (Section III) needs no broadcast after the reduce.
  *   - Sizes called "bytes" are bytes; "elems" are 4-byte elements.
  *   - "host" / "device" in a comment says where a pointer must point.
  *   - Times of the linear model (Section II): a message of b bytes costs
