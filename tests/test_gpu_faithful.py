@@ -141,3 +141,26 @@ def test_calibration_tool_fits_positive_parameters(capsys):
     assert set(d["schedules"]) == {"uni_greedy", "binomial", "pipeline", "binary"}
     assert d["rank_by_model"][0] == "uni_greedy"          # Theorem 5: optimal among in-order one-port schedules
     assert all(v["measured_us"] > 0 for v in d["schedules"].values())
+
+
+def test_randomized_shapes_order_free_results():
+    """120 seeded random shapes through the schedule-faithful kernel: int32 sum and max are order free, so
+    torch's reductions are an exact reference; lengths and segment sizes ignore every alignment."""
+    rng = np.random.default_rng(54321)
+    for case in range(120):
+        name, algo, port = SCHEDULES[case % len(SCHEDULES)]
+        p = int(rng.choice([2, 3, 5, 8, 17, 40, 64, 100, 257]))
+        n = int(rng.integers(1, 20000))
+        seg = int(rng.integers(1, n + 1)) if rng.random() < 0.5 else int(rng.integers(1, 600))
+        x = make_inputs(p, n, "int_pm2p20", seed=case, device="cuda") * int(rng.integers(1, 5000))
+        h = rd.rd_schedule_create(algo, port, p, 4 * n, 4 * seg, *M1)
+        out = torch.empty(n, dtype=torch.int32, device="cuda")
+        try:
+            for op, want in ((rd.RD_SUM, x.sum(dim=0, dtype=torch.int64)), (rd.RD_MAX, x.amax(dim=0))):
+                out.fill_(-7)
+                rd.rd_reduce(h, x, out, op, exec_mode=rd.RD_EXEC_FAITHFUL)
+                if op == rd.RD_SUM:
+                    want = ((want + (1 << 31)) % (1 << 32) - (1 << 31)).to(torch.int32)
+                assert torch.equal(out, want), (case, name, p, n, seg, op)
+        finally:
+            rd.rd_destroy(h)

@@ -310,3 +310,28 @@ def test_largest_process_count():
         rd.rd_reduce(h, x, out, rd.RD_SUM, exec_mode=rd.RD_EXEC_FAITHFUL)
     assert e.value.status == rd.RD_ERR_UNSUPPORTED
     rd.rd_destroy(h)
+
+
+def test_randomized_shapes_order_free_results():
+    """200 seeded random shapes (process counts, message lengths and segment sizes with no regard for vector
+    or tile boundaries, every schedule): int32 sum and max do not depend on the combine order, so torch's own
+    reductions are an exact reference at any size."""
+    rng = np.random.default_rng(12345)
+    for case in range(200):
+        name, algo, port = SCHEDULES[case % len(SCHEDULES)]
+        p = int(rng.choice([2, 3, 5, 8, 17, 40, 64, 100, 257, 300]))
+        n = int(rng.integers(1, 30000))
+        seg = int(rng.integers(1, n + 1)) if rng.random() < 0.5 else int(rng.integers(1, 600))
+        x = make_inputs(p, n, "int_pm2p20", seed=case, device="cuda")
+        x = x * int(rng.integers(1, 5000))                        # let sums wrap now and then
+        h = rd.rd_schedule_create(algo, port, p, 4 * n, 4 * seg, *M1)
+        out = torch.empty(n, dtype=torch.int32, device="cuda")
+        try:
+            for op, want in ((rd.RD_SUM, x.sum(dim=0, dtype=torch.int64)), (rd.RD_MAX, x.amax(dim=0))):
+                out.fill_(-7)
+                rd.rd_reduce(h, x, out, op)
+                if op == rd.RD_SUM:
+                    want = ((want + (1 << 31)) % (1 << 32) - (1 << 31)).to(torch.int32)
+                assert torch.equal(out, want), (case, name, p, n, seg, op)
+        finally:
+            rd.rd_destroy(h)
