@@ -73,6 +73,8 @@ def main(argv=None):
     ap.add_argument("--p", type=int, nargs="*", default=[2 ** k for k in range(1, 11)])
     ap.add_argument("--min-log2-bytes", type=int, default=3)
     ap.add_argument("--max-log2-bytes", type=int, default=26)
+    ap.add_argument("--faithful", action="store_true",
+                    help="also run every schedule in schedule-faithful mode (fp32 sum) and record its makespan")
     args = ap.parse_args(argv)
     dev = torch.device("cuda", torch.cuda.current_device())
     sink = sys.stdout if args.out == "-" else open(args.out, "w")
@@ -97,6 +99,27 @@ def main(argv=None):
                 info = rd.rd_schedule_info(h)
                 rd.rd_schedule_upload(h)
                 try:
+                    if args.faithful and p > 1:
+                        x = arenas["fp32"][: p * n].view(p, n)
+                        out = out_buf["fp32"][:n]
+                        tab = rd.PointerTable(x)
+                        rec = {"faithful": True, "p": p, "msg_bytes": m, "schedule": name, "seg_bytes": seg, "q": info["q"],
+                               "predicted_us": info["predicted_seconds"] * 1e6}
+                        try:
+                            spans = []
+                            for rep in range(4):
+                                st = rd.rd_reduce(h, tab, out, rd.RD_SUM, exec_mode=rd.RD_EXEC_FAITHFUL, want_stats=True)
+                                if rep:
+                                    spans.append(st.makespan_ns)
+                            spans.sort()
+                            rec.update(makespan_us=spans[len(spans) // 2] / 1e3, ok=check(x, out, "sum"))
+                            n_bad += 0 if rec["ok"] else 1
+                        except rd.RdError as e:            # scratch does not fit beside the arenas, or too many processes
+                            if e.status not in (rd.RD_ERR_NOMEM, rd.RD_ERR_UNSUPPORTED):
+                                raise
+                            rec.update(skipped=rd.rd_strerror(e.status))
+                        sink.write(json.dumps(rec) + "\n")
+                        n_cases += 1
                     for dt in ("int32", "fp32"):
                         x = arenas[dt][: p * n].view(p, n)
                         out = out_buf[dt][:n]
