@@ -41,7 +41,7 @@ WORKLOAD_OPS = {"config1": ["sum"], "config2": ["sum"], "config3": ["sum"], "con
 # dram__bytes_read.sum + dram__bytes_write.sum, mean of three launches.  Reported only while the kernel
 # source is the one that was profiled.
 NCU_TRAFFIC = {"workload": "config2", "bytes_per_launch": 274.6e6,
-               "kernel_sha256": "989893266a8018cea509f69a36eb51d09c3b3e9fb05008e085cc0cca8b38e2bf"}
+               "kernel_sha256": "75e1c1467e519a89465b496ee09acc5feb139ee208448823ce86de9cd8342848"}
 
 
 def profiled_traffic(wname):

@@ -71,7 +71,10 @@ typedef enum {
 } rd_algo_t;
 
 typedef enum { RD_PORT_UNI = 0, RD_PORT_BI = 1 } rd_port_t;   /* Section II */
-typedef enum { RD_SUM = 0, RD_MAX = 1 } rd_op_t;
+/* Entry-wise operation (associative and commutative, as the method requires).  Integer sum and product
+ * wrap modulo 2^32; max / min keep the held value on ties (incoming > held ? incoming : held), which
+ * settles the sign of a zero result; fp32 sum and product are one IEEE operation per combine. */
+typedef enum { RD_SUM = 0, RD_MAX = 1, RD_MIN = 2, RD_PROD = 3 } rd_op_t;
 typedef enum { RD_INT32 = 0, RD_FP32 = 1 } rd_dtype_t;
 typedef enum { RD_EXEC_TREE = 0, RD_EXEC_FAITHFUL = 1 } rd_exec_t;
 
@@ -179,7 +182,8 @@ RD_API int rd_schedule_segments(const rd_schedule_t *s, uint64_t *off, size_t ca
  *   bits 14-17  npop: number of pops that follow
  *   bits 18-29  bit k = role of the k-th pop: 1: top = combine(held = popped, incoming = top)
  *                                              0: top = combine(held = top, incoming = popped)
- * combine(held, incoming) = held + incoming, or incoming > held ? incoming : held.
+ * combine(held, incoming) = held + incoming, held * incoming, or incoming > held ? incoming : held
+ * (min: <).
  * After the last operation top is the root's value (Section IV: the receiver
  * combines its segment with the one received).
  */

@@ -675,17 +675,23 @@ int orc_contributions(const orc_event_t *ev_in, int64_t n_ev, int p, int q)
 /* the end is the result.                                                    */
 /*   op 0: sum   (int32: wrap-around; fp32: one IEEE round-to-nearest add)   */
 /*   op 1: max   (incoming > held ? incoming : held)                         */
+/*   op 2: min   (incoming < held ? incoming : held)                         */
+/*   op 3: product (int32: wrap-around; fp32: one IEEE multiply)             */
 /* ------------------------------------------------------------------------- */
 static uint32_t comb_i32(uint32_t held, uint32_t in, int op)
 {
     if (op == 0) return held + in;
-    return ((int32_t)in > (int32_t)held) ? in : held;
+    if (op == 3) return held * in;
+    if (op == 1) return ((int32_t)in > (int32_t)held) ? in : held;
+    return ((int32_t)in < (int32_t)held) ? in : held;
 }
 
 static float comb_f32(float held, float in, int op)
 {
     if (op == 0) return held + in;
-    return (in > held) ? in : held;
+    if (op == 3) return held * in;
+    if (op == 1) return (in > held) ? in : held;
+    return (in < held) ? in : held;
 }
 
 static int cmp_seg_time(const void *x, const void *y)

@@ -152,7 +152,7 @@ def reduce(events, x, seg_off, op):
     assert seg_off[0] == 0 and seg_off[-1] == n
     out = np.empty(n, dtype=x.dtype)
     ptrs = (C.c_void_p * p)(*[x[i].ctypes.data for i in range(p)])
-    opc = {"sum": 0, "max": 1}[op]
+    opc = {"sum": 0, "max": 1, "min": 2, "prod": 3}[op]
     if x.dtype == np.int32:
         fn = lib().orc_reduce_i32
     elif x.dtype == np.float32:

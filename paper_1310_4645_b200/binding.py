@@ -19,7 +19,7 @@ RD_ERR_TIMEOUT, RD_ERR_SIZE_MISMATCH, RD_ERR_INTERNAL, RD_ERR_TOO_SMALL = -5, -6
 RD_ERR_TOO_LARGE = -9
 RD_UNI_GREEDY, RD_BI_GREEDY, RD_BINOMIAL, RD_PIPELINE, RD_BINARY, RD_BUTTERFLY = range(6)
 RD_PORT_UNI, RD_PORT_BI = 0, 1
-RD_SUM, RD_MAX = 0, 1
+RD_SUM, RD_MAX, RD_MIN, RD_PROD = 0, 1, 2, 3
 RD_INT32, RD_FP32 = 0, 1
 RD_EXEC_TREE, RD_EXEC_FAITHFUL = 0, 1
 

@@ -336,7 +336,7 @@ int prepare_faithful(rd_schedule *s)
     // all blocks have to be resident together: lanes per process from the least occupant variant
     int perSm = 1 << 30;
     for (int dt = 0; dt < 2; dt++)
-        for (int op = 0; op < 2; op++)
+        for (int op = 0; op < 4; op++)
             for (int wide = 0; wide < 2; wide++) {
                 int b = 0;
                 if (faithful_blocks_per_sm(dt, op, wide != 0, &b) != 0) return RD_ERR_CUDA;
@@ -565,7 +565,7 @@ int rd_schedule_upload(rd_schedule_t *s)
 int rd_reduce(rd_schedule_t *s, const void *const *d_inputs, void *d_out, size_t n_elems, rd_dtype_t dtype, rd_op_t op,
               rd_exec_t exec, void *cuda_stream, rd_stats_t *stats)
 {
-    if (!s || !d_inputs || (dtype != RD_INT32 && dtype != RD_FP32) || (op != RD_SUM && op != RD_MAX)) return RD_ERR_INVALID_ARG;
+    if (!s || !d_inputs || (dtype != RD_INT32 && dtype != RD_FP32) || (int(op) < RD_SUM || int(op) > RD_PROD)) return RD_ERR_INVALID_ARG;
     if (exec != RD_EXEC_TREE && exec != RD_EXEC_FAITHFUL) return RD_ERR_INVALID_ARG;
     if (n_elems * 4 != s->msg_bytes) return RD_ERR_SIZE_MISMATCH;
     if (n_elems > 0 && !d_out) return RD_ERR_INVALID_ARG;
@@ -678,7 +678,7 @@ int rd_schedule_actions(const rd_schedule_t *s, int process, int32_t *buf, size_
 int rd_reduce_faithful_static(rd_schedule_t *s, const void *const *d_inputs, void *d_out, size_t n_elems, rd_dtype_t dtype,
                               rd_op_t op, void *cuda_stream, rd_stats_t *stats)
 {
-    if (!s || !d_inputs || (dtype != RD_INT32 && dtype != RD_FP32) || (op != RD_SUM && op != RD_MAX)) return RD_ERR_INVALID_ARG;
+    if (!s || !d_inputs || (dtype != RD_INT32 && dtype != RD_FP32) || (int(op) < RD_SUM || int(op) > RD_PROD)) return RD_ERR_INVALID_ARG;
     if (n_elems * 4 != s->msg_bytes) return RD_ERR_SIZE_MISMATCH;
     if (n_elems > 0 && !d_out) return RD_ERR_INVALID_ARG;
     for (int i = 0; i < s->p; i++)

@@ -26,17 +26,21 @@ namespace rd {
 namespace {
 
 enum { DT_INT32 = 0, DT_FP32 = 1 };
-enum { OPR_SUM = 0, OPR_MAX = 1 };
+enum { OPR_SUM = 0, OPR_MAX = 1, OPR_MIN = 2, OPR_PROD = 3 };
 
 template <int DT, int OPR> __device__ __forceinline__ uint32_t combine(uint32_t held, uint32_t in)
 {
     if (DT == DT_INT32) {
         if (OPR == OPR_SUM) return held + in;
-        return (int32_t(in) > int32_t(held)) ? in : held;
+        if (OPR == OPR_PROD) return held * in;
+        if (OPR == OPR_MAX) return (int32_t(in) > int32_t(held)) ? in : held;
+        return (int32_t(in) < int32_t(held)) ? in : held;
     } else {
         const float h = __uint_as_float(held), i = __uint_as_float(in);
         if (OPR == OPR_SUM) return __float_as_uint(__fadd_rn(h, i));
-        return (i > h) ? in : held;
+        if (OPR == OPR_PROD) return __float_as_uint(__fmul_rn(h, i));
+        if (OPR == OPR_MAX) return (i > h) ? in : held;
+        return (i < h) ? in : held;
     }
 }
 
@@ -182,10 +186,15 @@ cudaError_t launch_dtop(const FaithfulParams &prm, bool wide, cudaStream_t strea
 
 cudaError_t dispatch(const FaithfulParams &prm, int dtype, int op, bool wide, cudaStream_t stream, bool occ, int *bps)
 {
-    if (dtype == DT_INT32) return op == OPR_SUM ? launch_dtop<DT_INT32, OPR_SUM>(prm, wide, stream, occ, bps)
-                                                 : launch_dtop<DT_INT32, OPR_MAX>(prm, wide, stream, occ, bps);
+    if (dtype == DT_INT32)
+        return op == OPR_SUM ? launch_dtop<DT_INT32, OPR_SUM>(prm, wide, stream, occ, bps)
+               : op == OPR_MAX ? launch_dtop<DT_INT32, OPR_MAX>(prm, wide, stream, occ, bps)
+               : op == OPR_MIN ? launch_dtop<DT_INT32, OPR_MIN>(prm, wide, stream, occ, bps)
+                               : launch_dtop<DT_INT32, OPR_PROD>(prm, wide, stream, occ, bps);
     return op == OPR_SUM ? launch_dtop<DT_FP32, OPR_SUM>(prm, wide, stream, occ, bps)
-                         : launch_dtop<DT_FP32, OPR_MAX>(prm, wide, stream, occ, bps);
+           : op == OPR_MAX ? launch_dtop<DT_FP32, OPR_MAX>(prm, wide, stream, occ, bps)
+           : op == OPR_MIN ? launch_dtop<DT_FP32, OPR_MIN>(prm, wide, stream, occ, bps)
+                           : launch_dtop<DT_FP32, OPR_PROD>(prm, wide, stream, occ, bps);
 }
 
 }  // namespace

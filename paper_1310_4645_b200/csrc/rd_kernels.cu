@@ -26,7 +26,7 @@ constexpr int kIdxBits = 12;
 constexpr uint32_t kIdxMask = (1u << kIdxBits) - 1;
 
 enum { DT_INT32 = 0, DT_FP32 = 1 };
-enum { OPR_SUM = 0, OPR_MAX = 1 };
+enum { OPR_SUM = 0, OPR_MAX = 1, OPR_MIN = 2, OPR_PROD = 3 };
 
 template <int V> struct Vec { uint32_t w[V]; };
 
@@ -47,13 +47,20 @@ template <int DT, int OPR> __device__ __forceinline__ uint32_t combine(uint32_t 
 {
     if (DT == DT_INT32) {
         if (OPR == OPR_SUM) return held + in;                       // wraps modulo 2^32
-        return (int32_t(in) > int32_t(held)) ? in : held;
+        if (OPR == OPR_PROD) return held * in;                      // wraps modulo 2^32
+        if (OPR == OPR_MAX) return (int32_t(in) > int32_t(held)) ? in : held;
+        return (int32_t(in) < int32_t(held)) ? in : held;
     } else {
         const float h = __uint_as_float(held), i = __uint_as_float(in);
         if (OPR == OPR_SUM) return __float_as_uint(__fadd_rn(h, i));   // one IEEE add, never contracted
-        return (i > h) ? in : held;
+        if (OPR == OPR_PROD) return __float_as_uint(__fmul_rn(h, i));  // one IEEE multiply
+        if (OPR == OPR_MAX) return (i > h) ? in : held;
+        return (i < h) ? in : held;
     }
 }
+
+// Sum and product give the same bits whichever operand was held (IEEE add and multiply commute).
+template <int OPR> struct Commutes { static constexpr bool value = OPR == OPR_SUM || OPR == OPR_PROD; };
 
 struct PtrPack { const uint32_t *ptr[kPackedPtrs]; };
 struct PtrRef { const uint32_t *const *table; };
@@ -130,7 +137,7 @@ rd_tree_kernel(const __grid_constant__ TreeParams<PACKED> a)
                     if (kind <= 1u) {                      // LOAD / PUSH_LOAD
 #pragma unroll
                         for (int u = 0; u < U; u++) top[u] = x[u];
-                    } else if (kind == 2u || OPR == OPR_SUM) {   // ACC_IN (a sum does not care who held what)
+                    } else if (kind == 2u || Commutes<OPR>::value) {   // ACC_IN (a sum does not care who held what)
 #pragma unroll
                         for (int u = 0; u < U; u++)
 #pragma unroll
@@ -152,7 +159,7 @@ rd_tree_kernel(const __grid_constant__ TreeParams<PACKED> a)
                             const Vec<V> y = stack[(sp * U + u) * kTreeThreads + tid];
 #pragma unroll
                             for (int v = 0; v < V; v++)
-                                top[u].w[v] = (poppedHeld || OPR == OPR_SUM) ? combine<DT, OPR>(y.w[v], top[u].w[v])
+                                top[u].w[v] = (poppedHeld || Commutes<OPR>::value) ? combine<DT, OPR>(y.w[v], top[u].w[v])
                                                                             : combine<DT, OPR>(top[u].w[v], y.w[v]);
                         }
                     }
@@ -355,7 +362,7 @@ rd_tree_stream_kernel(const __grid_constant__ StreamParams<PACKED> a)
             }
             if (kind <= 1u) {
                 top0 = x0; top1 = x1;
-            } else if (kind == 2u || OPR == OPR_SUM) {
+            } else if (kind == 2u || Commutes<OPR>::value) {
 #pragma unroll
                 for (int v = 0; v < 4; v++) {
                     top0.w[v] = combine<DT, OPR>(top0.w[v], x0.w[v]);
@@ -383,7 +390,7 @@ rd_tree_stream_kernel(const __grid_constant__ StreamParams<PACKED> a)
                 const uint32_t ya[4] = {y0.x, y0.y, y0.z, y0.w}, yb[4] = {y1.x, y1.y, y1.z, y1.w};
 #pragma unroll
                 for (int v = 0; v < 4; v++) {
-                    if (poppedHeld || OPR == OPR_SUM) {
+                    if (poppedHeld || Commutes<OPR>::value) {
                         top0.w[v] = combine<DT, OPR>(ya[v], top0.w[v]);
                         top1.w[v] = combine<DT, OPR>(yb[v], top1.w[v]);
                     } else {
@@ -514,8 +521,10 @@ int launch_tree_stream(const TreeLaunch &l)
 {
     if (l.n_tiles == 0 || l.n_ctas == 0) return 0;
     cudaError_t e;
-    if (l.dtype == DT_INT32) e = l.op == OPR_SUM ? launch_stream_dtop<DT_INT32, OPR_SUM>(l) : launch_stream_dtop<DT_INT32, OPR_MAX>(l);
-    else e = l.op == OPR_SUM ? launch_stream_dtop<DT_FP32, OPR_SUM>(l) : launch_stream_dtop<DT_FP32, OPR_MAX>(l);
+    if (l.dtype == DT_INT32) e = l.op == OPR_SUM ? launch_stream_dtop<DT_INT32, OPR_SUM>(l) : l.op == OPR_MAX ? launch_stream_dtop<DT_INT32, OPR_MAX>(l)
+                               : l.op == OPR_MIN ? launch_stream_dtop<DT_INT32, OPR_MIN>(l) : launch_stream_dtop<DT_INT32, OPR_PROD>(l);
+    else e = l.op == OPR_SUM ? launch_stream_dtop<DT_FP32, OPR_SUM>(l) : l.op == OPR_MAX ? launch_stream_dtop<DT_FP32, OPR_MAX>(l)
+             : l.op == OPR_MIN ? launch_stream_dtop<DT_FP32, OPR_MIN>(l) : launch_stream_dtop<DT_FP32, OPR_PROD>(l);
     return int(e);
 }
 
@@ -523,8 +532,10 @@ int launch_tree(const TreeLaunch &l)
 {
     if (l.n_tiles == 0) return 0;
     cudaError_t e;
-    if (l.dtype == DT_INT32) e = l.op == OPR_SUM ? launch_dtop<DT_INT32, OPR_SUM>(l) : launch_dtop<DT_INT32, OPR_MAX>(l);
-    else e = l.op == OPR_SUM ? launch_dtop<DT_FP32, OPR_SUM>(l) : launch_dtop<DT_FP32, OPR_MAX>(l);
+    if (l.dtype == DT_INT32) e = l.op == OPR_SUM ? launch_dtop<DT_INT32, OPR_SUM>(l) : l.op == OPR_MAX ? launch_dtop<DT_INT32, OPR_MAX>(l)
+                               : l.op == OPR_MIN ? launch_dtop<DT_INT32, OPR_MIN>(l) : launch_dtop<DT_INT32, OPR_PROD>(l);
+    else e = l.op == OPR_SUM ? launch_dtop<DT_FP32, OPR_SUM>(l) : l.op == OPR_MAX ? launch_dtop<DT_FP32, OPR_MAX>(l)
+             : l.op == OPR_MIN ? launch_dtop<DT_FP32, OPR_MIN>(l) : launch_dtop<DT_FP32, OPR_PROD>(l);
     return int(e);
 }
 

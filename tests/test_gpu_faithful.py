@@ -15,7 +15,7 @@ SCHEDULES = [("uni_greedy", rd.RD_UNI_GREEDY, rd.RD_PORT_UNI), ("bi_greedy", rd.
              ("binomial", rd.RD_BINOMIAL, rd.RD_PORT_UNI), ("pipeline_uni", rd.RD_PIPELINE, rd.RD_PORT_UNI),
              ("pipeline_bi", rd.RD_PIPELINE, rd.RD_PORT_BI), ("binary_uni", rd.RD_BINARY, rd.RD_PORT_UNI),
              ("binary_bi", rd.RD_BINARY, rd.RD_PORT_BI), ("butterfly", rd.RD_BUTTERFLY, rd.RD_PORT_BI)]
-OPS = {"sum": rd.RD_SUM, "max": rd.RD_MAX}
+OPS = {"sum": rd.RD_SUM, "max": rd.RD_MAX, "min": rd.RD_MIN, "prod": rd.RD_PROD}
 
 
 def run(algo, port, x, seg_bytes, op, rows=None, out=None):
@@ -40,7 +40,8 @@ SHAPES = [(8, 4096, 512), (5, 10000, 2500), (13, 3 * 2048 + 36, 2048 + 520), (64
 
 
 @pytest.mark.parametrize("name,algo,port", SCHEDULES)
-@pytest.mark.parametrize("dist,op", [("int_pm2p20", "sum"), ("normal", "sum"), ("normal", "max")])
+@pytest.mark.parametrize("dist,op", [("int_pm2p20", "sum"), ("normal", "sum"), ("normal", "max"), ("normal", "min"),
+                                     ("int_pm2p20", "prod"), ("uniform_pm1", "prod")])
 def test_parity_small_shapes(name, algo, port, dist, op):
     for p, n, seg in SHAPES:
         x = make_inputs(p, n, dist, seed=p * 1000 + n, device="cuda")

@@ -14,7 +14,7 @@ M1 = (2e-6, 1e-10, 5e-11)
 SCHEDULES = [("uni_greedy", rd.RD_UNI_GREEDY, rd.RD_PORT_UNI), ("bi_greedy", rd.RD_BI_GREEDY, rd.RD_PORT_BI),
              ("binomial", rd.RD_BINOMIAL, rd.RD_PORT_UNI), ("pipeline", rd.RD_PIPELINE, rd.RD_PORT_UNI),
              ("binary", rd.RD_BINARY, rd.RD_PORT_BI), ("butterfly", rd.RD_BUTTERFLY, rd.RD_PORT_BI)]
-OPS = {"sum": rd.RD_SUM, "max": rd.RD_MAX}
+OPS = {"sum": rd.RD_SUM, "max": rd.RD_MAX, "min": rd.RD_MIN, "prod": rd.RD_PROD}
 
 
 def gpu_reduce(algo, port, x_dev, seg_bytes, op, model=M1, out=None, rows=None):
@@ -57,6 +57,26 @@ def test_parity_small_shapes(name, algo, port, dist, op):
         if dist == "normal":
             x *= 10.0 ** torch.randint(-4, 5, x.shape, device="cuda", generator=torch.Generator("cuda").manual_seed(1))
         check(algo, port, x, 4 * seg, op)
+
+
+@pytest.mark.parametrize("name,algo,port", SCHEDULES)
+@pytest.mark.parametrize("dist,op", [("int_pm2p20", "min"), ("int_pm2p20", "prod"), ("normal", "min"), ("near_one", "prod")])
+def test_parity_min_and_product(name, algo, port, dist, op):
+    """Integer results are also checked against the order-free value; fp32 products use factors with
+    magnitude in [0.5, 2) so that no partial product overflows to a NaN-producing inf * 0."""
+    for p, n, seg in SHAPES:
+        if dist == "near_one":
+            g = torch.Generator("cuda").manual_seed(p * 1000 + n)
+            x = torch.empty((p, n), device="cuda").uniform_(0.5, 2.0, generator=g)
+            x *= torch.randint(0, 2, x.shape, device="cuda", generator=g) * 2.0 - 1.0
+        else:
+            x = make_inputs(p, n, dist, seed=p * 1000 + n, device="cuda")
+        got, xh = check(algo, port, x, 4 * seg, op)
+        if op == "min":
+            assert (got == xh.min(axis=0)).all()
+        elif dist == "int_pm2p20":
+            want = np.multiply.reduce(xh.view(np.uint32), axis=0, dtype=np.uint32).view(np.int32)
+            assert (got == want).all()
 
 
 def test_config1_bit_exact_and_order_free():

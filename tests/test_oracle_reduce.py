@@ -40,6 +40,60 @@ def test_integer_results_do_not_depend_on_the_order(p):
         assert (O.reduce(ev, x, off, "max") == want_max).all()
 
 
+@pytest.mark.parametrize("p", [2, 3, 8, 13, 64])
+def test_integer_min_and_wrapping_product_do_not_depend_on_the_order(p):
+    """min is the plain minimum; the product is the product of the residues modulo 2^32."""
+    rng = np.random.default_rng(50 + p)
+    sizes = [5, 5, 5, 2]
+    n = sum(sizes)
+    x = rng.integers(-2**31, 2**31, size=(p, n), dtype=np.int64).astype(np.int32)
+    x[:, :6] = rng.integers(-3, 4, size=(p, 6)) * 2 + 1            # small odd factors: the product stays non-zero
+    want_prod = np.array([int(np.prod([int(v) for v in x[:, e]], dtype=object)) & 0xFFFFFFFF for e in range(n)],
+                         dtype=np.uint64).astype(np.uint32).view(np.int32)
+    assert (want_prod[:6] != 0).all()
+    for name, ev in schedules(p, sizes):
+        assert (O.reduce(ev, x, seg_off(sizes), "min") == x.min(axis=0)).all(), name
+        assert (O.reduce(ev, x, seg_off(sizes), "prod") == want_prod).all(), name
+    ev, off, _ = O.butterfly(p, n, 4, 3, 1, 1)
+    assert (O.reduce(ev, x, off, "min") == x.min(axis=0)).all()
+    assert (O.reduce(ev, x, off, "prod") == want_prod).all()
+
+
+@pytest.mark.parametrize("p", [2, 5, 16, 33])
+def test_fp32_min_is_the_minimum_and_powers_of_two_multiply_exactly(p):
+    rng = np.random.default_rng(150 + p)
+    sizes = [7, 7, 3]
+    x = rng.standard_normal((p, 17)).astype(f32)
+    e = rng.integers(-3, 4, size=(p, 17))
+    pw = (np.ldexp(1.0, e) * rng.choice([-1.0, 1.0], size=(p, 17))).astype(f32)      # products are exact in any order
+    want = np.ldexp(1.0, e.sum(axis=0)) * np.prod(np.sign(pw), axis=0)
+    for name, ev in schedules(p, sizes):
+        assert (O.reduce(ev, x, seg_off(sizes), "min") == x.min(axis=0)).all(), name
+        assert (O.reduce(ev, pw, seg_off(sizes), "prod") == want.astype(f32)).all(), name
+
+
+def test_fp32_product_two_processes_is_one_multiply_and_min_keeps_the_held_zero():
+    rng = np.random.default_rng(8)
+    x = (rng.standard_normal((2, 1000)) * 10.0 ** rng.integers(-8, 8, size=(2, 1000))).astype(f32)
+    ev, _ = O.uni_greedy(2, [600, 400], 1, 1, 1)
+    assert (O.reduce(ev, x, [0, 600, 1000], "prod") == x[0] * x[1]).all()
+    z = np.array([[0.0], [-0.0]], dtype=f32)                          # incoming -0 is not less than held +0
+    ev, _ = O.uni_greedy(2, [1], 1, 1, 1)
+    assert np.signbit(O.reduce(ev, z, [0, 1], "min"))[0] == False
+    assert np.signbit(O.reduce(ev, z[::-1].copy(), [0, 1], "min"))[0] == True
+
+
+def test_fp32_product_pipeline_is_a_running_product_from_the_far_end():
+    p = 9
+    rng = np.random.default_rng(p)
+    x = rng.uniform(0.5, 2.0, size=(p, 64)).astype(f32)
+    want = x[p - 1].copy()
+    for k in range(p - 2, -1, -1):
+        want = (x[k] * want).astype(f32)
+    ev, _ = O.pipeline(p, [32, 32], 3, 1, 1, False)
+    assert O.reduce(ev, x, [0, 32, 64], "prod").tobytes() == want.tobytes()
+
+
 @pytest.mark.parametrize("p", [2, 5, 16, 33])
 def test_fp32_max_is_the_maximum(p):
     rng = np.random.default_rng(100 + p)

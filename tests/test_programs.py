@@ -32,8 +32,9 @@ def test_programs_reproduce_the_oracle(algo, port, p):
         off = rd.rd_schedule_segments(h).astype(np.int64)
         oev, ooff, _ = oracle_schedule(algo, port, p, msg, seg, *M1)
         assert info["stack_depth"] <= max(1, int(np.ceil(np.log2(max(p, 2)))))
-        for x in (xf, xi):
-            for op in ("sum", "max"):
+        xp = (rng.uniform(0.5, 2.0, size=(p, n)) * rng.choice([-1.0, 1.0], size=(p, n))).astype(np.float32)
+        for x, ops_ in ((xf, ("sum", "max", "min")), (xi, ("sum", "max", "min", "prod")), (xp, ("prod",))):
+            for op in ops_:
                 want = O.reduce(oev, x, ooff, op)
                 got = np.empty_like(want)
                 for j in range(info["q"]):
