@@ -41,7 +41,7 @@ WORKLOAD_OPS = {"config1": ["sum"], "config2": ["sum"], "config3": ["sum"], "con
 # dram__bytes_read.sum + dram__bytes_write.sum, mean of three launches.  Reported only while the kernel
 # source is the one that was profiled.
 NCU_TRAFFIC = {"workload": "config2", "bytes_per_launch": 274.6e6,
-               "kernel_sha256": "75e1c1467e519a89465b496ee09acc5feb139ee208448823ce86de9cd8342848"}
+               "kernel_sha256": "865a1a7ce78c3d93b799005d02865c719cdfc7ea647f5cc499c8878a8889de1c"}
 
 
 def profiled_traffic(wname):

@@ -1,8 +1,8 @@
 /*
  * rd.h -- C ABI of the schedule-exact pipelined reduction library (librd.so).
  *
- * The library reduces the messages of p "processes" (p buffers of n 4-byte
- * elements in the memory of ONE GPU) into a root buffer, combining entry-wise
+ * The library reduces the messages of p "processes" (p buffers of n 4- or
+ * 8-byte elements in the memory of ONE GPU) into a root buffer, combining entry-wise
  * in exactly the order a reduction schedule fixes.  Schedules follow
  * Lowery & Langou, "A Greedy Algorithm for Optimally Pipelining a Reduction":
  * uni-greedy (Algorithm 1), bi-greedy (Algorithm 2), and the algorithms the
@@ -20,7 +20,9 @@
  *     pass the pointer array permuted so that the root's buffer comes first.
  *     On one GPU every process can read the result buffer, so an all-reduce
  *     (Section III) needs no broadcast after the reduce.
- *   - Sizes called "bytes" are bytes; "elems" are 4-byte elements.
+ *   - Sizes called "bytes" are bytes.  A schedule knows sizes in bytes only and reports segment
+ *     boundaries in 4-byte words; n_elems of the reducing calls counts elements of the call's
+ *     rd_dtype_t (4 or 8 bytes each).
  *   - "host" / "device" in a comment says where a pointer must point.
  *   - Times of the linear model (Section II): a message of b bytes costs
  *     alpha + beta*b, combining it costs gamma*b.  Internally time is an exact
@@ -55,7 +57,7 @@ typedef enum {
     RD_ERR_NOMEM = -3,         /* host or device allocation failed                                      */
     RD_ERR_CUDA = -4,          /* a CUDA runtime call failed (including: no device, no driver)          */
     RD_ERR_TIMEOUT = -5,       /* a bounded wait inside the schedule-faithful kernel gave up            */
-    RD_ERR_SIZE_MISMATCH = -6, /* n_elems * 4 differs from the schedule's message size                  */
+    RD_ERR_SIZE_MISMATCH = -6, /* n_elems * element size differs from the schedule's message size       */
     RD_ERR_INTERNAL = -7,      /* a generated schedule failed the library's own consistency check       */
     RD_ERR_TOO_SMALL = -8,     /* an output array passed by the caller is too short                     */
     RD_ERR_TOO_LARGE = -9      /* rd_reduce_faithful_static: more scratch needed than its fixed array has */
@@ -72,10 +74,17 @@ typedef enum {
 
 typedef enum { RD_PORT_UNI = 0, RD_PORT_BI = 1 } rd_port_t;   /* Section II */
 /* Entry-wise operation (associative and commutative, as the method requires).  Integer sum and product
- * wrap modulo 2^32; max / min keep the held value on ties (incoming > held ? incoming : held), which
- * settles the sign of a zero result; fp32 sum and product are one IEEE operation per combine. */
+ * wrap modulo 2^32 (2^64 for RD_INT64); max / min keep the held value on ties (incoming > held ? incoming : held), which
+ * settles the sign of a zero result; fp32 and fp64 sum and product are one IEEE
+ * round-to-nearest operation per combine. */
 typedef enum { RD_SUM = 0, RD_MAX = 1, RD_MIN = 2, RD_PROD = 3 } rd_op_t;
-typedef enum { RD_INT32 = 0, RD_FP32 = 1 } rd_dtype_t;
+/* Element type.  The paper's implementation is restricted to int and notes that the restriction is
+ * not a consequence of the algorithm (Fig. 2 caption).  With an 8-byte type no segment may begin
+ * inside an element: msg_bytes and every segment size multiples of 8 (for the butterfly, whose
+ * chunks come from halving the message: n_elems a multiple of the largest power of two <= p);
+ * rd_optimal_segment returns multiples of 4, round them up.  Otherwise the reducing calls return
+ * RD_ERR_INVALID_ARG. */
+typedef enum { RD_INT32 = 0, RD_FP32 = 1, RD_INT64 = 2, RD_FP64 = 3 } rd_dtype_t;
 typedef enum { RD_EXEC_TREE = 0, RD_EXEC_FAITHFUL = 1 } rd_exec_t;
 
 /* Linear model of Section II.  alpha in seconds, beta and gamma in seconds per
@@ -195,7 +204,7 @@ RD_API int rd_schedule_program(const rd_schedule_t *s, size_t seg, uint32_t *ops
  *             message of n_elems elements.  Never written.
  *   d_out     DEVICE; n_elems elements; receives what the root holds at the
  *             end.  May alias d_inputs[0] in tree mode only.
- *   n_elems   must equal the schedule's msg_bytes / 4 (RD_ERR_SIZE_MISMATCH).
+ *   n_elems   must equal the schedule's msg_bytes / element size (RD_ERR_SIZE_MISMATCH).
  *   exec      RD_EXEC_TREE: one kernel evaluates, per element, the segment's
  *             combine program in registers; asynchronous on cuda_stream.
  *             RD_EXEC_FAITHFUL: a persistent kernel in which groups of thread
@@ -209,9 +218,9 @@ RD_API int rd_schedule_program(const rd_schedule_t *s, size_t seg, uint32_t *ops
  * (allocates device memory, synchronises); rd_schedule_upload does the same
  * ahead of time.  After one such call per schedule, element type and operation, a
  * tree-mode call with at most 256 processes is a single kernel launch and may be
- * recorded into a CUDA graph.  Buffers must be 4-byte aligned; 16-byte aligned buffers take
- * the 128-bit streaming path (segments may start and end anywhere; when n_elems is
- * not a multiple of 4 the last elements are done by a second, tiny launch), other
+ * recorded into a CUDA graph.  Buffers must be aligned to the element; 16-byte aligned buffers take
+ * the 128-bit streaming path (segments may start and end anywhere; when the message is
+ * not a multiple of 16 bytes the last elements are done by a second, tiny launch), other
  * buffers a slower element-wise path.
  */
 RD_API int rd_reduce(rd_schedule_t *s, const void *const *d_inputs, void *d_out, size_t n_elems,

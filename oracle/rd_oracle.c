@@ -760,6 +760,74 @@ int orc_reduce_f32(const orc_event_t *ev_in, int64_t n_ev, int p, int q, const i
     return ORC_OK;
 }
 
+/* The same for the 8-byte element types: int64 wraps modulo 2^64, fp64 is one
+ * IEEE round-to-nearest operation per combine.  seg_off counts elements.     */
+static uint64_t comb_i64(uint64_t held, uint64_t in, int op)
+{
+    if (op == 0) return held + in;
+    if (op == 3) return held * in;
+    if (op == 1) return ((int64_t)in > (int64_t)held) ? in : held;
+    return ((int64_t)in < (int64_t)held) ? in : held;
+}
+
+static double comb_f64(double held, double in, int op)
+{
+    if (op == 0) return held + in;
+    if (op == 3) return held * in;
+    if (op == 1) return (in > held) ? in : held;
+    return (in < held) ? in : held;
+}
+
+int orc_reduce_i64(const orc_event_t *ev_in, int64_t n_ev, int p, int q, const int64_t *seg_off,
+                   const int64_t *const *x, int64_t *out, int op)
+{
+    orc_event_t *ev = sorted_by_segment(ev_in, n_ev);
+    if (!ev) return ORC_NOMEM;
+    int64_t longest = 0;
+    for (int j = 0; j < q; j++) if (seg_off[j + 1] - seg_off[j] > longest) longest = seg_off[j + 1] - seg_off[j];
+    uint64_t *acc = malloc(sizeof(uint64_t) * (size_t)p * (size_t)(longest ? longest : 1));
+    if (!acc) { free(ev); return ORC_NOMEM; }
+    int64_t e = 0;
+    for (int j = 0; j < q; j++) {
+        int64_t len = seg_off[j + 1] - seg_off[j];
+        for (int i = 0; i < p; i++)
+            for (int64_t k = 0; k < len; k++) acc[(size_t)i * longest + k] = (uint64_t)x[i][seg_off[j] + k];
+        for (; e < n_ev && ev[e].seg == j; e++) {
+            uint64_t *held = acc + (size_t)ev[e].dst * longest, *in = acc + (size_t)ev[e].src * longest;
+            if (ev[e].kind == 0) for (int64_t k = 0; k < len; k++) held[k] = comb_i64(held[k], in[k], op);
+            else for (int64_t k = 0; k < len; k++) held[k] = in[k];
+        }
+        for (int64_t k = 0; k < len; k++) out[seg_off[j] + k] = (int64_t)acc[k];
+    }
+    free(acc); free(ev);
+    return ORC_OK;
+}
+
+int orc_reduce_f64(const orc_event_t *ev_in, int64_t n_ev, int p, int q, const int64_t *seg_off,
+                   const double *const *x, double *out, int op)
+{
+    orc_event_t *ev = sorted_by_segment(ev_in, n_ev);
+    if (!ev) return ORC_NOMEM;
+    int64_t longest = 0;
+    for (int j = 0; j < q; j++) if (seg_off[j + 1] - seg_off[j] > longest) longest = seg_off[j + 1] - seg_off[j];
+    double *acc = malloc(sizeof(double) * (size_t)p * (size_t)(longest ? longest : 1));
+    if (!acc) { free(ev); return ORC_NOMEM; }
+    int64_t e = 0;
+    for (int j = 0; j < q; j++) {
+        int64_t len = seg_off[j + 1] - seg_off[j];
+        for (int i = 0; i < p; i++)
+            for (int64_t k = 0; k < len; k++) acc[(size_t)i * longest + k] = x[i][seg_off[j] + k];
+        for (; e < n_ev && ev[e].seg == j; e++) {
+            double *held = acc + (size_t)ev[e].dst * longest, *in = acc + (size_t)ev[e].src * longest;
+            if (ev[e].kind == 0) for (int64_t k = 0; k < len; k++) held[k] = comb_f64(held[k], in[k], op);
+            else for (int64_t k = 0; k < len; k++) held[k] = in[k];
+        }
+        for (int64_t k = 0; k < len; k++) out[seg_off[j] + k] = acc[k];
+    }
+    free(acc); free(ev);
+    return ORC_OK;
+}
+
 /* Order-free fp64 reference: sum_i (double)x_i[e], and sum_i |x_i[e]| for the
  * error bound; for max the exact maximum as a double.                        */
 int orc_reference_f64(int p, int64_t n, const float *const *x, double *ref, double *abs_sum, int op)

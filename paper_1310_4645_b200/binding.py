@@ -20,7 +20,7 @@ RD_ERR_TOO_LARGE = -9
 RD_UNI_GREEDY, RD_BI_GREEDY, RD_BINOMIAL, RD_PIPELINE, RD_BINARY, RD_BUTTERFLY = range(6)
 RD_PORT_UNI, RD_PORT_BI = 0, 1
 RD_SUM, RD_MAX, RD_MIN, RD_PROD = 0, 1, 2, 3
-RD_INT32, RD_FP32 = 0, 1
+RD_INT32, RD_FP32, RD_INT64, RD_FP64 = 0, 1, 2, 3
 RD_EXEC_TREE, RD_EXEC_FAITHFUL = 0, 1
 
 ALGOS = {"uni_greedy": RD_UNI_GREEDY, "bi_greedy": RD_BI_GREEDY, "binomial": RD_BINOMIAL,
@@ -176,7 +176,11 @@ def _dtype_code(t):
         return RD_INT32
     if t.dtype == torch.float32:
         return RD_FP32
-    raise TypeError("int32 or float32 expected, got %s" % t.dtype)
+    if t.dtype == torch.int64:
+        return RD_INT64
+    if t.dtype == torch.float64:
+        return RD_FP64
+    raise TypeError("int32, float32, int64 or float64 expected, got %s" % t.dtype)
 
 
 class PointerTable:

@@ -255,6 +255,28 @@ int tiles_for(rd_schedule *s, int vec, const TileDesc **tiles, uint32_t *count)
     return RD_OK;
 }
 
+// Argument checks common to the reducing entry points.  On success *n_words is the message length
+// in 32-bit words, the unit in which the schedule's segment boundaries and the kernels count.
+size_t elem_bytes(rd_dtype_t dtype) { return (dtype == RD_INT64 || dtype == RD_FP64) ? 8 : 4; }
+
+int check_reduce_args(const rd_schedule *s, const void *const *d_inputs, const void *d_out, size_t n_elems, rd_dtype_t dtype,
+                      rd_op_t op, size_t *n_words)
+{
+    if (!s || !d_inputs || int(dtype) < RD_INT32 || int(dtype) > RD_FP64 || int(op) < RD_SUM || int(op) > RD_PROD)
+        return RD_ERR_INVALID_ARG;
+    const size_t esize = elem_bytes(dtype);
+    if (n_elems > s->msg_bytes / esize || n_elems * esize != s->msg_bytes) return RD_ERR_SIZE_MISMATCH;
+    if (n_elems > 0 && !d_out) return RD_ERR_INVALID_ARG;
+    for (int i = 0; i < s->p; i++)
+        if ((n_elems > 0 && !d_inputs[i]) || (reinterpret_cast<uintptr_t>(d_inputs[i]) & (esize - 1))) return RD_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(d_out) & (esize - 1)) return RD_ERR_INVALID_ARG;
+    if (esize == 8)                    // no segment may begin inside an element
+        for (uint64_t off : s->sched.seg_off)
+            if (off & 1u) return RD_ERR_INVALID_ARG;
+    *n_words = s->msg_bytes / 4;
+    return RD_OK;
+}
+
 int reduce_tree(rd_schedule *s, const void *const *d_inputs, void *d_out, size_t n, rd_dtype_t dtype, rd_op_t op,
                 cudaStream_t stream, rd_stats_t *stats)
 {
@@ -335,7 +357,7 @@ int prepare_faithful(rd_schedule *s)
     if (int rc = build_actions(s->p, q, s->sched.events, lists)) return rc;
     // all blocks have to be resident together: lanes per process from the least occupant variant
     int perSm = 1 << 30;
-    for (int dt = 0; dt < 2; dt++)
+    for (int dt = 0; dt < 4; dt++)
         for (int op = 0; op < 4; op++)
             for (int wide = 0; wide < 2; wide++) {
                 int b = 0;
@@ -565,18 +587,14 @@ int rd_schedule_upload(rd_schedule_t *s)
 int rd_reduce(rd_schedule_t *s, const void *const *d_inputs, void *d_out, size_t n_elems, rd_dtype_t dtype, rd_op_t op,
               rd_exec_t exec, void *cuda_stream, rd_stats_t *stats)
 {
-    if (!s || !d_inputs || (dtype != RD_INT32 && dtype != RD_FP32) || (int(op) < RD_SUM || int(op) > RD_PROD)) return RD_ERR_INVALID_ARG;
     if (exec != RD_EXEC_TREE && exec != RD_EXEC_FAITHFUL) return RD_ERR_INVALID_ARG;
-    if (n_elems * 4 != s->msg_bytes) return RD_ERR_SIZE_MISMATCH;
-    if (n_elems > 0 && !d_out) return RD_ERR_INVALID_ARG;
-    for (int i = 0; i < s->p; i++)
-        if ((n_elems > 0 && !d_inputs[i]) || (reinterpret_cast<uintptr_t>(d_inputs[i]) & 3u)) return RD_ERR_INVALID_ARG;
-    if (reinterpret_cast<uintptr_t>(d_out) & 3u) return RD_ERR_INVALID_ARG;
+    size_t n_words = 0;
+    if (int rc = check_reduce_args(s, d_inputs, d_out, n_elems, dtype, op, &n_words)) return rc;
     return guarded([&] {
         if (int rc = upload(s)) return rc;
         if (exec == RD_EXEC_FAITHFUL)
-            return reduce_faithful(s, d_inputs, d_out, n_elems, dtype, op, static_cast<cudaStream_t>(cuda_stream), stats);
-        return reduce_tree(s, d_inputs, d_out, n_elems, dtype, op, static_cast<cudaStream_t>(cuda_stream), stats);
+            return reduce_faithful(s, d_inputs, d_out, n_words, dtype, op, static_cast<cudaStream_t>(cuda_stream), stats);
+        return reduce_tree(s, d_inputs, d_out, n_words, dtype, op, static_cast<cudaStream_t>(cuda_stream), stats);
     });
 }
 
@@ -584,21 +602,22 @@ int rd_reduce_host(rd_schedule_t *s, const void *const *h_inputs, void *h_out, v
                    rd_dtype_t dtype, rd_op_t op, void *cuda_stream)
 {
     if (!s || !h_inputs || (n_elems > 0 && (!h_out || !d_staging))) return RD_ERR_INVALID_ARG;
-    if (n_elems * 4 != s->msg_bytes) return RD_ERR_SIZE_MISMATCH;
+    if (int(dtype) < RD_INT32 || int(dtype) > RD_FP64) return RD_ERR_INVALID_ARG;
+    if (n_elems > s->msg_bytes / elem_bytes(dtype) || n_elems * elem_bytes(dtype) != s->msg_bytes) return RD_ERR_SIZE_MISMATCH;
+    const size_t row = s->msg_bytes;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     std::vector<const void *> dptr;
     try { dptr.resize(size_t(s->p)); } catch (const std::bad_alloc &) { return RD_ERR_NOMEM; }
     char *base = static_cast<char *>(d_staging);
     for (int i = 0; i < s->p; i++) {
         if (n_elems > 0 && !h_inputs[i]) return RD_ERR_INVALID_ARG;
-        dptr[size_t(i)] = base + size_t(i) * n_elems * 4;
-        if (n_elems > 0 &&
-            cudaMemcpyAsync(base + size_t(i) * n_elems * 4, h_inputs[i], n_elems * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        dptr[size_t(i)] = base + size_t(i) * row;
+        if (n_elems > 0 && cudaMemcpyAsync(base + size_t(i) * row, h_inputs[i], row, cudaMemcpyHostToDevice, stream) != cudaSuccess)
             return RD_ERR_CUDA;
     }
-    void *d_out = base + size_t(s->p) * n_elems * 4;
+    void *d_out = base + size_t(s->p) * row;
     if (int rc = rd_reduce(s, dptr.data(), d_out, n_elems, dtype, op, RD_EXEC_TREE, cuda_stream, nullptr)) return rc;
-    if (n_elems > 0 && cudaMemcpyAsync(h_out, d_out, n_elems * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return RD_ERR_CUDA;
+    if (n_elems > 0 && cudaMemcpyAsync(h_out, d_out, row, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return RD_ERR_CUDA;
     if (cudaStreamSynchronize(stream) != cudaSuccess) return RD_ERR_CUDA;
     return RD_OK;
 }
@@ -678,20 +697,16 @@ int rd_schedule_actions(const rd_schedule_t *s, int process, int32_t *buf, size_
 int rd_reduce_faithful_static(rd_schedule_t *s, const void *const *d_inputs, void *d_out, size_t n_elems, rd_dtype_t dtype,
                               rd_op_t op, void *cuda_stream, rd_stats_t *stats)
 {
-    if (!s || !d_inputs || (dtype != RD_INT32 && dtype != RD_FP32) || (int(op) < RD_SUM || int(op) > RD_PROD)) return RD_ERR_INVALID_ARG;
-    if (n_elems * 4 != s->msg_bytes) return RD_ERR_SIZE_MISMATCH;
-    if (n_elems > 0 && !d_out) return RD_ERR_INVALID_ARG;
-    for (int i = 0; i < s->p; i++)
-        if ((n_elems > 0 && !d_inputs[i]) || (reinterpret_cast<uintptr_t>(d_inputs[i]) & 3u)) return RD_ERR_INVALID_ARG;
-    if (reinterpret_cast<uintptr_t>(d_out) & 3u) return RD_ERR_INVALID_ARG;
+    size_t n_words = 0;
+    if (int rc = check_reduce_args(s, d_inputs, d_out, n_elems, dtype, op, &n_words)) return rc;
     rd_stats_t st;
     std::memset(&st, 0, sizeof(st));
-    st.bytes_moved = uint64_t(s->p + 1) * uint64_t(n_elems) * 4u;
+    st.bytes_moved = uint64_t(s->p + 1) * uint64_t(n_words) * 4u;
     st.predicted_s = double(s->sched.completion) * s->ticks.tick;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (n_elems == 0) { if (stats) *stats = st; return RD_OK; }
     if (s->p == 1) {
-        if (d_out != d_inputs[0] && cudaMemcpyAsync(d_out, d_inputs[0], n_elems * 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+        if (d_out != d_inputs[0] && cudaMemcpyAsync(d_out, d_inputs[0], n_words * 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
             return RD_ERR_CUDA;
         if (cudaStreamSynchronize(stream) != cudaSuccess) return RD_ERR_CUDA;
         if (stats) *stats = st;

@@ -25,7 +25,10 @@ namespace rd {
 
 namespace {
 
-enum { DT_INT32 = 0, DT_FP32 = 1 };
+enum { DT_INT32 = 0, DT_FP32 = 1, DT_INT64 = 2, DT_FP64 = 3 };
+
+// Buffers are indexed in 32-bit words; an element is one word or two.
+template <int DT> struct ElemWords { static constexpr int value = DT >= DT_INT64 ? 2 : 1; };
 enum { OPR_SUM = 0, OPR_MAX = 1, OPR_MIN = 2, OPR_PROD = 3 };
 
 template <int DT, int OPR> __device__ __forceinline__ uint32_t combine(uint32_t held, uint32_t in)
@@ -42,6 +45,57 @@ template <int DT, int OPR> __device__ __forceinline__ uint32_t combine(uint32_t 
         if (OPR == OPR_MAX) return (i > h) ? in : held;
         return (i < h) ? in : held;
     }
+}
+
+template <int DT, int OPR> __device__ __forceinline__ unsigned long long combine64(unsigned long long held, unsigned long long in)
+{
+    if (DT == DT_INT64) {
+        if (OPR == OPR_SUM) return held + in;
+        if (OPR == OPR_PROD) return held * in;
+        if (OPR == OPR_MAX) return ((long long)in > (long long)held) ? in : held;
+        return ((long long)in < (long long)held) ? in : held;
+    } else {
+        const double h = __longlong_as_double((long long)held), i = __longlong_as_double((long long)in);
+        if (OPR == OPR_SUM) return (unsigned long long)__double_as_longlong(__dadd_rn(h, i));
+        if (OPR == OPR_PROD) return (unsigned long long)__double_as_longlong(__dmul_rn(h, i));
+        if (OPR == OPR_MAX) return (i > h) ? in : held;
+        return (i < h) ? in : held;
+    }
+}
+
+// V words as one access (V = 1, 2 or 4) through L2, where the other blocks' stores are visible.
+template <int V> struct Words { uint32_t w[V]; };
+template <int V> __device__ __forceinline__ Words<V> load_words(const uint32_t *p)
+{
+    Words<V> r;
+    if constexpr (V == 4) { const uint4 t = __ldcg(reinterpret_cast<const uint4 *>(p)); r.w[0] = t.x; r.w[1] = t.y; r.w[2] = t.z; r.w[3] = t.w; }
+    else if constexpr (V == 2) { const uint2 t = __ldcg(reinterpret_cast<const uint2 *>(p)); r.w[0] = t.x; r.w[1] = t.y; }
+    else r.w[0] = __ldcg(p);
+    return r;
+}
+template <int V> __device__ __forceinline__ void store_words(uint32_t *p, const Words<V> &v)
+{
+    if constexpr (V == 4) __stcg(reinterpret_cast<uint4 *>(p), make_uint4(v.w[0], v.w[1], v.w[2], v.w[3]));
+    else if constexpr (V == 2) __stcg(reinterpret_cast<uint2 *>(p), make_uint2(v.w[0], v.w[1]));
+    else __stcg(p, v.w[0]);
+}
+template <int DT, int OPR, int V> __device__ __forceinline__ Words<V> combine_words(const Words<V> &held, const Words<V> &in)
+{
+    Words<V> r;
+    if constexpr (ElemWords<DT>::value == 1) {
+#pragma unroll
+        for (int v = 0; v < V; v++) r.w[v] = combine<DT, OPR>(held.w[v], in.w[v]);
+    } else {
+        static_assert(V % 2 == 0, "an 8-byte element is never split between two accesses");
+#pragma unroll
+        for (int v = 0; v < V; v += 2) {
+            const unsigned long long h = (unsigned long long)held.w[v] | ((unsigned long long)held.w[v + 1] << 32);
+            const unsigned long long i = (unsigned long long)in.w[v] | ((unsigned long long)in.w[v + 1] << 32);
+            const unsigned long long c = combine64<DT, OPR>(h, i);
+            r.w[v] = uint32_t(c); r.w[v + 1] = uint32_t(c >> 32);
+        }
+    }
+    return r;
 }
 
 __device__ __forceinline__ unsigned long long now_ns()
@@ -135,20 +189,8 @@ rd_faithful_kernel(const FaithfulParams a)
         const uint32_t *held = act.first ? mine + seg_lo : dst;
         const bool store_only = act.kind == 1;
         for (uint64_t e = lo + uint64_t(threadIdx.x) * V; e < hi; e += uint64_t(kFaithfulThreads) * V) {
-            if (V == 4) {
-                const uint4 in = __ldcg(reinterpret_cast<const uint4 *>(src + e));
-                uint4 r = in;
-                if (!store_only) {
-                    const uint4 h = __ldcg(reinterpret_cast<const uint4 *>(held + e));
-                    r.x = combine<DT, OPR>(h.x, in.x); r.y = combine<DT, OPR>(h.y, in.y);
-                    r.z = combine<DT, OPR>(h.z, in.z); r.w = combine<DT, OPR>(h.w, in.w);
-                }
-                __stcg(reinterpret_cast<uint4 *>(dst + e), r);
-            } else {
-                const uint32_t in = __ldcg(src + e);
-                const uint32_t r = store_only ? in : combine<DT, OPR>(__ldcg(held + e), in);
-                __stcg(dst + e, r);
-            }
+            const Words<V> in = load_words<V>(src + e);
+            store_words<V>(dst + e, store_only ? in : combine_words<DT, OPR, V>(load_words<V>(held + e), in));
         }
         // the sender's value has been read: tell it
         __syncthreads();
@@ -173,28 +215,33 @@ rd_faithful_kernel(const FaithfulParams a)
 template <int DT, int OPR>
 cudaError_t launch_dtop(const FaithfulParams &prm, bool wide, cudaStream_t stream, bool occupancy_only, int *blocks_per_sm)
 {
+    constexpr int N = ElemWords<DT>::value;      // narrow variant: one element per access
     const void *fn = wide ? reinterpret_cast<const void *>(rd_faithful_kernel<DT, OPR, 4>)
-                          : reinterpret_cast<const void *>(rd_faithful_kernel<DT, OPR, 1>);
+                          : reinterpret_cast<const void *>(rd_faithful_kernel<DT, OPR, N>);
     if (occupancy_only) {
         return wide ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, rd_faithful_kernel<DT, OPR, 4>, kFaithfulThreads, 0)
-                    : cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, rd_faithful_kernel<DT, OPR, 1>, kFaithfulThreads, 0);
+                    : cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, rd_faithful_kernel<DT, OPR, N>, kFaithfulThreads, 0);
     }
     FaithfulParams copy = prm;
     void *args[] = {&copy};
     return cudaLaunchCooperativeKernel(fn, dim3(unsigned(prm.n_procs * prm.lanes)), dim3(kFaithfulThreads), args, 0, stream);
 }
 
+template <int DT>
+cudaError_t dispatch_op(const FaithfulParams &prm, int op, bool wide, cudaStream_t stream, bool occ, int *bps)
+{
+    return op == OPR_SUM ? launch_dtop<DT, OPR_SUM>(prm, wide, stream, occ, bps)
+           : op == OPR_MAX ? launch_dtop<DT, OPR_MAX>(prm, wide, stream, occ, bps)
+           : op == OPR_MIN ? launch_dtop<DT, OPR_MIN>(prm, wide, stream, occ, bps)
+                           : launch_dtop<DT, OPR_PROD>(prm, wide, stream, occ, bps);
+}
+
 cudaError_t dispatch(const FaithfulParams &prm, int dtype, int op, bool wide, cudaStream_t stream, bool occ, int *bps)
 {
-    if (dtype == DT_INT32)
-        return op == OPR_SUM ? launch_dtop<DT_INT32, OPR_SUM>(prm, wide, stream, occ, bps)
-               : op == OPR_MAX ? launch_dtop<DT_INT32, OPR_MAX>(prm, wide, stream, occ, bps)
-               : op == OPR_MIN ? launch_dtop<DT_INT32, OPR_MIN>(prm, wide, stream, occ, bps)
-                               : launch_dtop<DT_INT32, OPR_PROD>(prm, wide, stream, occ, bps);
-    return op == OPR_SUM ? launch_dtop<DT_FP32, OPR_SUM>(prm, wide, stream, occ, bps)
-           : op == OPR_MAX ? launch_dtop<DT_FP32, OPR_MAX>(prm, wide, stream, occ, bps)
-           : op == OPR_MIN ? launch_dtop<DT_FP32, OPR_MIN>(prm, wide, stream, occ, bps)
-                           : launch_dtop<DT_FP32, OPR_PROD>(prm, wide, stream, occ, bps);
+    return dtype == DT_INT32 ? dispatch_op<DT_INT32>(prm, op, wide, stream, occ, bps)
+           : dtype == DT_FP32 ? dispatch_op<DT_FP32>(prm, op, wide, stream, occ, bps)
+           : dtype == DT_INT64 ? dispatch_op<DT_INT64>(prm, op, wide, stream, occ, bps)
+                               : dispatch_op<DT_FP64>(prm, op, wide, stream, occ, bps);
 }
 
 }  // namespace

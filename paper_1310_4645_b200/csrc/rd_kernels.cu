@@ -7,7 +7,7 @@
 //   rd_tree_stream_kernel  the throughput path (128-bit aligned buffers): operand tiles are streamed
 //                          into a shared-memory ring by bulk asynchronous copies issued by producer
 //                          threads, consumers execute the program on them;
-//   rd_tree_kernel         the element path (any 4-byte aligned buffers): operands are fetched K
+//   rd_tree_kernel         the element path (buffers aligned to the element only): operands are fetched K
 //                          operations ahead, in program order, into a register ring that is
 //                          statically indexed by unrolling the interpreter K times.
 // Partial results that have to wait (at most log2 p of them) live in a per-thread column of shared
@@ -25,7 +25,10 @@ namespace {
 constexpr int kIdxBits = 12;
 constexpr uint32_t kIdxMask = (1u << kIdxBits) - 1;
 
-enum { DT_INT32 = 0, DT_FP32 = 1 };
+enum { DT_INT32 = 0, DT_FP32 = 1, DT_INT64 = 2, DT_FP64 = 3 };
+
+// The kernels move and index the message in 32-bit words; an element is one word or two.
+template <int DT> struct ElemWords { static constexpr int value = DT >= DT_INT64 ? 2 : 1; };
 enum { OPR_SUM = 0, OPR_MAX = 1, OPR_MIN = 2, OPR_PROD = 3 };
 
 template <int V> struct Vec { uint32_t w[V]; };
@@ -35,7 +38,16 @@ template <> __device__ __forceinline__ Vec<1> load_stream<1>(const uint32_t *p)
 {
     Vec<1> r; r.w[0] = __ldcs(p); return r;
 }
+template <> __device__ __forceinline__ Vec<2> load_stream<2>(const uint32_t *p)
+{
+    const uint2 t = __ldcs(reinterpret_cast<const uint2 *>(p));
+    Vec<2> r; r.w[0] = t.x; r.w[1] = t.y; return r;
+}
 template <int V> __device__ __forceinline__ void store_stream(uint32_t *p, const Vec<V> &v);
+template <> __device__ __forceinline__ void store_stream<2>(uint32_t *p, const Vec<2> &v)
+{
+    __stcs(reinterpret_cast<uint2 *>(p), make_uint2(v.w[0], v.w[1]));
+}
 template <> __device__ __forceinline__ void store_stream<4>(uint32_t *p, const Vec<4> &v)
 {
     __stcs(reinterpret_cast<uint4 *>(p), make_uint4(v.w[0], v.w[1], v.w[2], v.w[3]));
@@ -56,6 +68,41 @@ template <int DT, int OPR> __device__ __forceinline__ uint32_t combine(uint32_t 
         if (OPR == OPR_PROD) return __float_as_uint(__fmul_rn(h, i));  // one IEEE multiply
         if (OPR == OPR_MAX) return (i > h) ? in : held;
         return (i < h) ? in : held;
+    }
+}
+
+// The same for the 8-byte element types (low word first in memory).
+template <int DT, int OPR> __device__ __forceinline__ unsigned long long combine64(unsigned long long held, unsigned long long in)
+{
+    if (DT == DT_INT64) {
+        if (OPR == OPR_SUM) return held + in;                       // wraps modulo 2^64
+        if (OPR == OPR_PROD) return held * in;                      // wraps modulo 2^64
+        if (OPR == OPR_MAX) return ((long long)in > (long long)held) ? in : held;
+        return ((long long)in < (long long)held) ? in : held;
+    } else {
+        const double h = __longlong_as_double((long long)held), i = __longlong_as_double((long long)in);
+        if (OPR == OPR_SUM) return (unsigned long long)__double_as_longlong(__dadd_rn(h, i));
+        if (OPR == OPR_PROD) return (unsigned long long)__double_as_longlong(__dmul_rn(h, i));
+        if (OPR == OPR_MAX) return (i > h) ? in : held;
+        return (i < h) ? in : held;
+    }
+}
+
+// A vector of V words: V elements of a 4-byte type, V / 2 of an 8-byte type.  r may be held or in.
+template <int DT, int OPR, int V> __device__ __forceinline__ void combine_vec(Vec<V> &r, const Vec<V> &held, const Vec<V> &in)
+{
+    if constexpr (ElemWords<DT>::value == 1) {
+#pragma unroll
+        for (int v = 0; v < V; v++) r.w[v] = combine<DT, OPR>(held.w[v], in.w[v]);
+    } else {
+        static_assert(V % 2 == 0, "an 8-byte element never straddles two vectors");
+#pragma unroll
+        for (int v = 0; v < V; v += 2) {
+            const unsigned long long h = (unsigned long long)held.w[v] | ((unsigned long long)held.w[v + 1] << 32);
+            const unsigned long long i = (unsigned long long)in.w[v] | ((unsigned long long)in.w[v + 1] << 32);
+            const unsigned long long c = combine64<DT, OPR>(h, i);
+            r.w[v] = uint32_t(c); r.w[v + 1] = uint32_t(c >> 32);
+        }
     }
 }
 
@@ -139,14 +186,10 @@ rd_tree_kernel(const __grid_constant__ TreeParams<PACKED> a)
                         for (int u = 0; u < U; u++) top[u] = x[u];
                     } else if (kind == 2u || Commutes<OPR>::value) {   // ACC_IN (a sum does not care who held what)
 #pragma unroll
-                        for (int u = 0; u < U; u++)
-#pragma unroll
-                            for (int v = 0; v < V; v++) top[u].w[v] = combine<DT, OPR>(top[u].w[v], x[u].w[v]);
+                        for (int u = 0; u < U; u++) combine_vec<DT, OPR, V>(top[u], top[u], x[u]);
                     } else {                               // ACC_HELD
 #pragma unroll
-                        for (int u = 0; u < U; u++)
-#pragma unroll
-                            for (int v = 0; v < V; v++) top[u].w[v] = combine<DT, OPR>(x[u].w[v], top[u].w[v]);
+                        for (int u = 0; u < U; u++) combine_vec<DT, OPR, V>(top[u], x[u], top[u]);
                     }
                     uint32_t npop = (w >> (kIdxBits + 2)) & 0xFu;
                     uint32_t roles = w >> (kIdxBits + 6);
@@ -157,10 +200,8 @@ rd_tree_kernel(const __grid_constant__ TreeParams<PACKED> a)
 #pragma unroll
                         for (int u = 0; u < U; u++) {
                             const Vec<V> y = stack[(sp * U + u) * kTreeThreads + tid];
-#pragma unroll
-                            for (int v = 0; v < V; v++)
-                                top[u].w[v] = (poppedHeld || Commutes<OPR>::value) ? combine<DT, OPR>(y.w[v], top[u].w[v])
-                                                                            : combine<DT, OPR>(top[u].w[v], y.w[v]);
+                            if (poppedHeld || Commutes<OPR>::value) combine_vec<DT, OPR, V>(top[u], y, top[u]);
+                            else combine_vec<DT, OPR, V>(top[u], top[u], y);
                         }
                     }
                 }
@@ -363,17 +404,11 @@ rd_tree_stream_kernel(const __grid_constant__ StreamParams<PACKED> a)
             if (kind <= 1u) {
                 top0 = x0; top1 = x1;
             } else if (kind == 2u || Commutes<OPR>::value) {
-#pragma unroll
-                for (int v = 0; v < 4; v++) {
-                    top0.w[v] = combine<DT, OPR>(top0.w[v], x0.w[v]);
-                    top1.w[v] = combine<DT, OPR>(top1.w[v], x1.w[v]);
-                }
+                combine_vec<DT, OPR, 4>(top0, top0, x0);
+                combine_vec<DT, OPR, 4>(top1, top1, x1);
             } else {
-#pragma unroll
-                for (int v = 0; v < 4; v++) {
-                    top0.w[v] = combine<DT, OPR>(x0.w[v], top0.w[v]);
-                    top1.w[v] = combine<DT, OPR>(x1.w[v], top1.w[v]);
-                }
+                combine_vec<DT, OPR, 4>(top0, x0, top0);
+                combine_vec<DT, OPR, 4>(top1, x1, top1);
             }
             // the stage's data is in registers: hand the stage back to the producer
             __syncwarp();
@@ -387,16 +422,13 @@ rd_tree_stream_kernel(const __grid_constant__ StreamParams<PACKED> a)
                 roles >>= 1;
                 const uint4 y0 = stack[sp * levelVecs + tid];
                 const uint4 y1 = two ? stack[sp * levelVecs + kConsumers + tid] : make_uint4(0, 0, 0, 0);
-                const uint32_t ya[4] = {y0.x, y0.y, y0.z, y0.w}, yb[4] = {y1.x, y1.y, y1.z, y1.w};
-#pragma unroll
-                for (int v = 0; v < 4; v++) {
-                    if (poppedHeld || Commutes<OPR>::value) {
-                        top0.w[v] = combine<DT, OPR>(ya[v], top0.w[v]);
-                        top1.w[v] = combine<DT, OPR>(yb[v], top1.w[v]);
-                    } else {
-                        top0.w[v] = combine<DT, OPR>(top0.w[v], ya[v]);
-                        top1.w[v] = combine<DT, OPR>(top1.w[v], yb[v]);
-                    }
+                const Vec<4> ya = {{y0.x, y0.y, y0.z, y0.w}}, yb = {{y1.x, y1.y, y1.z, y1.w}};
+                if (poppedHeld || Commutes<OPR>::value) {
+                    combine_vec<DT, OPR, 4>(top0, ya, top0);
+                    combine_vec<DT, OPR, 4>(top1, yb, top1);
+                } else {
+                    combine_vec<DT, OPR, 4>(top0, top0, ya);
+                    combine_vec<DT, OPR, 4>(top1, top1, yb);
                 }
             }
             w = wn;
@@ -442,7 +474,8 @@ cudaError_t launch_one(const TreeLaunch &l)
 template <int DT, int OPR>
 cudaError_t launch_dtop(const TreeLaunch &l)
 {
-    return l.p <= kPackedPtrs ? launch_one<DT, OPR, 1, true>(l) : launch_one<DT, OPR, 1, false>(l);
+    constexpr int V = ElemWords<DT>::value;              // one element per thread and load
+    return l.p <= kPackedPtrs ? launch_one<DT, OPR, V, true>(l) : launch_one<DT, OPR, V, false>(l);
 }
 
 template <int DT, int OPR, bool PACKED>
@@ -517,26 +550,48 @@ void stream_shape(int stack_depth, int smem_per_sm, int stage_elems, int *ctas_p
     }
 }
 
+namespace {
+
+// Calls f.template operator()<DT, OPR>() for the run-time pair (dtype, op).
+template <int DT, typename F> cudaError_t with_op(int op, F &&f)
+{
+    switch (op) {
+    case OPR_SUM: return f.template operator()<DT, OPR_SUM>();
+    case OPR_MAX: return f.template operator()<DT, OPR_MAX>();
+    case OPR_MIN: return f.template operator()<DT, OPR_MIN>();
+    default: return f.template operator()<DT, OPR_PROD>();
+    }
+}
+template <typename F> cudaError_t with_type_and_op(int dtype, int op, F &&f)
+{
+    switch (dtype) {
+    case DT_INT32: return with_op<DT_INT32>(op, f);
+    case DT_FP32: return with_op<DT_FP32>(op, f);
+    case DT_INT64: return with_op<DT_INT64>(op, f);
+    default: return with_op<DT_FP64>(op, f);
+    }
+}
+struct StreamLauncher {
+    const TreeLaunch &l;
+    template <int DT, int OPR> cudaError_t operator()() const { return launch_stream_dtop<DT, OPR>(l); }
+};
+struct ElementLauncher {
+    const TreeLaunch &l;
+    template <int DT, int OPR> cudaError_t operator()() const { return launch_dtop<DT, OPR>(l); }
+};
+
+}  // namespace
+
 int launch_tree_stream(const TreeLaunch &l)
 {
     if (l.n_tiles == 0 || l.n_ctas == 0) return 0;
-    cudaError_t e;
-    if (l.dtype == DT_INT32) e = l.op == OPR_SUM ? launch_stream_dtop<DT_INT32, OPR_SUM>(l) : l.op == OPR_MAX ? launch_stream_dtop<DT_INT32, OPR_MAX>(l)
-                               : l.op == OPR_MIN ? launch_stream_dtop<DT_INT32, OPR_MIN>(l) : launch_stream_dtop<DT_INT32, OPR_PROD>(l);
-    else e = l.op == OPR_SUM ? launch_stream_dtop<DT_FP32, OPR_SUM>(l) : l.op == OPR_MAX ? launch_stream_dtop<DT_FP32, OPR_MAX>(l)
-             : l.op == OPR_MIN ? launch_stream_dtop<DT_FP32, OPR_MIN>(l) : launch_stream_dtop<DT_FP32, OPR_PROD>(l);
-    return int(e);
+    return int(with_type_and_op(l.dtype, l.op, StreamLauncher{l}));
 }
 
 int launch_tree(const TreeLaunch &l)
 {
     if (l.n_tiles == 0) return 0;
-    cudaError_t e;
-    if (l.dtype == DT_INT32) e = l.op == OPR_SUM ? launch_dtop<DT_INT32, OPR_SUM>(l) : l.op == OPR_MAX ? launch_dtop<DT_INT32, OPR_MAX>(l)
-                               : l.op == OPR_MIN ? launch_dtop<DT_INT32, OPR_MIN>(l) : launch_dtop<DT_INT32, OPR_PROD>(l);
-    else e = l.op == OPR_SUM ? launch_dtop<DT_FP32, OPR_SUM>(l) : l.op == OPR_MAX ? launch_dtop<DT_FP32, OPR_MAX>(l)
-             : l.op == OPR_MIN ? launch_dtop<DT_FP32, OPR_MIN>(l) : launch_dtop<DT_FP32, OPR_PROD>(l);
-    return int(e);
+    return int(with_type_and_op(l.dtype, l.op, ElementLauncher{l}));
 }
 
 }  // namespace rd

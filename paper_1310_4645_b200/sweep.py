@@ -6,10 +6,11 @@ size before comparing, Sections V-B and VII).
 
 For every case one JSON line: shape, segment size chosen, the schedule's predicted completion time
 under the linear model, measured microseconds and GB/s ((p+1)*m bytes per reduction), and whether the
-result passed its check (int32 and fp32 max: exact against torch's order-free result; fp32 sum:
-|r - r64| <= 1e-5 * sum|x| against an fp64 sum, on the whole message or on sampled slices of it).
-Inputs: uniform random numbers from seed 4 (int32 in [-2^20, 2^20], fp32 in [-1, 1)), one arena per
-element type, every case a view of its first p*n elements.
+result passed its check (integers, max and min: exact against torch's order-free result; fp32 sum:
+|r - r64| <= 1e-5 * sum|x| against an fp64 sum, fp64 sum: the same with 1e-14; on the whole message or
+on sampled slices of it).
+Inputs: uniform random numbers from seed 4 (integers in [-2^20, 2^20], floating point in [-1, 1)), one
+arena per element type (--dtypes), every case a view of its first p*n elements.
 """
 from __future__ import annotations
 
@@ -23,6 +24,8 @@ import torch
 from . import binding as rd
 
 ALPHA, BETA, GAMMA = 2e-6, 1e-10, 5e-11
+TORCH_DTYPES = {"int32": torch.int32, "fp32": torch.float32, "int64": torch.int64, "fp64": torch.float64}
+ELEM_BYTES = {"int32": 4, "fp32": 4, "int64": 8, "fp64": 8}
 SCHEDULES = [("uni_greedy", rd.RD_UNI_GREEDY, rd.RD_PORT_UNI), ("bi_greedy", rd.RD_BI_GREEDY, rd.RD_PORT_BI),
              ("binomial", rd.RD_BINOMIAL, rd.RD_PORT_UNI), ("pipeline", rd.RD_PIPELINE, rd.RD_PORT_UNI),
              ("binary", rd.RD_BINARY, rd.RD_PORT_UNI), ("butterfly", rd.RD_BUTTERFLY, rd.RD_PORT_BI)]
@@ -35,7 +38,7 @@ def fill_arena(n_elems, dtype, dev):
     step = 1 << 28
     for lo in range(0, n_elems, step):
         part = arena[lo:lo + step]
-        if dtype == torch.int32:
+        if dtype in (torch.int32, torch.int64):
             part.random_(-(1 << 20), (1 << 20) + 1, generator=gen)
         else:
             part.uniform_(-1.0, 1.0, generator=gen)
@@ -49,8 +52,11 @@ def check(x, out, op, max_check_elems=1 << 22):
     spans = [(0, n)] if n <= 3 * per else [(0, per), ((n - per) // 2, (n - per) // 2 + per), (n - per, n)]
     for lo, hi in spans:
         xs, o = x[:, lo:hi], out[lo:hi]
-        if op == "max":
-            if not torch.equal(o, xs.amax(dim=0)):
+        if op in ("max", "min"):
+            if not torch.equal(o, xs.amax(dim=0) if op == "max" else xs.amin(dim=0)):
+                return False
+        elif x.dtype == torch.int64:
+            if not torch.equal(o, xs.sum(dim=0)):
                 return False
         elif x.dtype == torch.int32:
             want = xs.to(torch.int64).sum(dim=0)
@@ -60,7 +66,7 @@ def check(x, out, op, max_check_elems=1 << 22):
         else:
             ref = xs.to(torch.float64).sum(dim=0)
             mag = xs.to(torch.float64).abs().sum(dim=0)
-            if not bool(((o.to(torch.float64) - ref).abs() <= 1e-5 * mag).all()):
+            if not bool(((o.to(torch.float64) - ref).abs() <= (1e-5 if x.dtype == torch.float32 else 1e-14) * mag).all()):
                 return False
     return True
 
@@ -75,15 +81,18 @@ def main(argv=None):
     ap.add_argument("--max-log2-bytes", type=int, default=26)
     ap.add_argument("--faithful", action="store_true",
                     help="also run every schedule in schedule-faithful mode (fp32 sum) and record its makespan")
+    ap.add_argument("--dtypes", nargs="*", default=["int32", "fp32"], choices=list(TORCH_DTYPES))
+    ap.add_argument("--ops", nargs="*", default=["sum", "max"], choices=["sum", "max", "min"])
     args = ap.parse_args(argv)
     dev = torch.device("cuda", torch.cuda.current_device())
     sink = sys.stdout if args.out == "-" else open(args.out, "w")
     sizes = [1 << k for k in range(args.min_log2_bytes, args.max_log2_bytes + 1)]
     limit = int(args.max_total_gib * (1 << 30))
     biggest = max(p * m for p in args.p for m in sizes if p * m <= limit)
-    arenas = {"int32": fill_arena(biggest // 4, torch.int32, dev), "fp32": fill_arena(biggest // 4, torch.float32, dev)}
-    out_buf = {"int32": torch.empty(max(sizes) // 4, dtype=torch.int32, device=dev),
-               "fp32": torch.empty(max(sizes) // 4, dtype=torch.float32, device=dev)}
+    want = list(args.dtypes) + (["fp32"] if args.faithful and "fp32" not in args.dtypes else [])
+    arenas = {dt: fill_arena(biggest // ELEM_BYTES[dt], TORCH_DTYPES[dt], dev) for dt in want}
+    out_buf = {dt: torch.empty(max(sizes) // ELEM_BYTES[dt], dtype=TORCH_DTYPES[dt], device=dev) for dt in want}
+    opcodes = {"sum": rd.RD_SUM, "max": rd.RD_MAX, "min": rd.RD_MIN}
     n_cases = n_bad = 0
     t_start = time.time()
     for p in args.p:
@@ -94,6 +103,8 @@ def main(argv=None):
             for name, algo, port in SCHEDULES:
                 t0 = time.perf_counter()
                 seg = rd.rd_optimal_segment(algo, port, p, m, ALPHA, BETA, GAMMA)
+                if any(ELEM_BYTES[dt] == 8 for dt in args.dtypes):
+                    seg = min(m, (seg + 7) // 8 * 8)       # whole elements of every type
                 h = rd.rd_schedule_create(algo, port, p, m, seg, ALPHA, BETA, GAMMA)
                 create_ms = (time.perf_counter() - t0) * 1e3
                 info = rd.rd_schedule_info(h)
@@ -120,11 +131,14 @@ def main(argv=None):
                             rec.update(skipped=rd.rd_strerror(e.status))
                         sink.write(json.dumps(rec) + "\n")
                         n_cases += 1
-                    for dt in ("int32", "fp32"):
-                        x = arenas[dt][: p * n].view(p, n)
-                        out = out_buf[dt][:n]
+                    for dt in args.dtypes:
+                        ne = m // ELEM_BYTES[dt]
+                        x = arenas[dt][: p * ne].view(p, ne)
+                        out = out_buf[dt][:ne]
                         tab = rd.PointerTable(x)
-                        for op, opc in (("sum", rd.RD_SUM), ("max", rd.RD_MAX)):
+                        if ELEM_BYTES[dt] == 8 and name == "butterfly" and ne % (1 << (p.bit_length() - 1)):
+                            continue                       # halving would cut through an element
+                        for op, opc in ((o, opcodes[o]) for o in args.ops):
                             rd.rd_reduce(h, tab, out, opc)
                             ok = check(x, out, op)
                             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

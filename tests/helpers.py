@@ -77,3 +77,42 @@ def run_program(ops, x, op):
             top = combine(y, top) if (roles >> k) & 1 else combine(top, y)
     assert not stack and loads == x.shape[0]
     return top
+
+
+M1_64 = (2e-6, 1e-10, 5e-11)
+OPS64 = {"sum": rd.RD_SUM, "max": rd.RD_MAX, "min": rd.RD_MIN, "prod": rd.RD_PROD}
+
+
+def check64(algo, port, x_dev, seg_bytes, op, exec_mode=0, rows=None, out=None):
+    """8-byte elements: the schedule counts in 4-byte words, the oracle in elements."""
+    import torch
+    p, n = x_dev.shape
+    h = rd.rd_schedule_create(algo, port, p, 8 * n, seg_bytes, *M1_64)
+    try:
+        out = torch.full((n,), 77, dtype=x_dev.dtype, device=x_dev.device) if out is None else out
+        rd.rd_reduce(h, rows if rows is not None else x_dev, out, OPS64[op], exec_mode=exec_mode, want_stats=exec_mode != rd.RD_EXEC_TREE)
+        torch.cuda.synchronize()
+    finally:
+        rd.rd_destroy(h)
+    ev, off, _ = oracle_schedule(algo, port, p, 8 * n, seg_bytes if seg_bytes else 8 * n, *M1_64)
+    assert (off % 2 == 0).all()
+    x = x_dev.cpu().numpy()
+    want = O.reduce(ev, x, off // 2, op)
+    got = out.cpu().numpy()
+    assert got.tobytes() == want.tobytes()
+    return got, x
+
+
+def inputs64(p, n, kind, seed):
+    import torch
+    g = torch.Generator("cuda").manual_seed(seed)
+    if kind == "int64":
+        return torch.randint(-2**62, 2**62, (p, n), dtype=torch.int64, device="cuda", generator=g)
+    if kind == "int64_small":
+        return torch.randint(-3, 4, (p, n), dtype=torch.int64, device="cuda", generator=g) * 2 + 1
+    x = torch.empty((p, n), dtype=torch.float64, device="cuda")
+    if kind == "near_one":
+        x.uniform_(0.5, 2.0, generator=g)
+        return x * (torch.randint(0, 2, x.shape, device="cuda", generator=g) * 2.0 - 1.0)
+    x.normal_(generator=g)
+    return x * 10.0 ** torch.randint(-12, 13, x.shape, device="cuda", generator=g)

@@ -97,6 +97,23 @@ def test_info_events_segments_program_capacity_checks():
         ptrs[3] = 0x1002                 # misaligned input
         assert L.rd_reduce(h, ptrs, 0x2000, 4096, rd.RD_INT32, rd.RD_SUM, rd.RD_EXEC_TREE, None, None) \
             == rd.RD_ERR_INVALID_ARG
+        # 8-byte element types: half as many elements, buffers aligned to 8 bytes
+        ptrs = (C.c_void_p * 8)(*([0x1000] * 8))
+        assert L.rd_reduce(h, ptrs, 0x2000, 4096, rd.RD_FP64, rd.RD_SUM, rd.RD_EXEC_TREE, None, None) \
+            == rd.RD_ERR_SIZE_MISMATCH
+        ptrs[5] = 0x1004
+        assert L.rd_reduce(h, ptrs, 0x2000, 2048, rd.RD_INT64, rd.RD_SUM, rd.RD_EXEC_TREE, None, None) \
+            == rd.RD_ERR_INVALID_ARG
+    finally:
+        rd.rd_destroy(h)
+    # a segment boundary inside an 8-byte element is refused before any CUDA call
+    h = rd.rd_schedule_create(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, 4, 64, 12, *MODEL)
+    try:
+        ptrs = (C.c_void_p * 4)(*([0x1000] * 4))
+        assert rd.lib().rd_reduce(h, ptrs, 0x2000, 8, rd.RD_FP64, rd.RD_SUM, rd.RD_EXEC_TREE, None, None) \
+            == rd.RD_ERR_INVALID_ARG
+        assert rd.lib().rd_reduce_faithful_static(h, ptrs, 0x2000, 8, rd.RD_INT64, rd.RD_MAX, None, None) \
+            == rd.RD_ERR_INVALID_ARG
     finally:
         rd.rd_destroy(h)
 

@@ -165,3 +165,17 @@ def test_randomized_shapes_order_free_results():
                 assert torch.equal(out, want), (case, name, p, n, seg, op)
         finally:
             rd.rd_destroy(h)
+
+
+def test_eight_byte_elements_in_schedule_faithful_mode():
+    """fp64 and int64 through the action lists: whole-vector segments (128-bit accesses) and segments
+    that begin 8 bytes into a vector (one element per access)."""
+    from helpers import check64, inputs64
+    for name, algo, port in SCHEDULES:
+        if name == "butterfly":
+            continue
+        for p, n, seg in ((8, 4096, 512), (13, 3090, 515), (33, 3000, 501), (2, 2050, 2050)):
+            check64(algo, port, inputs64(p, n, "normal64", seed=p + n), 8 * seg, "sum", exec_mode=rd.RD_EXEC_FAITHFUL)
+            check64(algo, port, inputs64(p, n, "int64", seed=p + n), 8 * seg, "max", exec_mode=rd.RD_EXEC_FAITHFUL)
+            check64(algo, port, inputs64(p, n, "near_one", seed=p + n), 8 * seg, "prod", exec_mode=rd.RD_EXEC_FAITHFUL)
+    check64(rd.RD_BUTTERFLY, rd.RD_PORT_BI, inputs64(16, 4096, "normal64", seed=3), 0, "sum", exec_mode=rd.RD_EXEC_FAITHFUL)

@@ -6,7 +6,7 @@ import torch
 import paper_1310_4645_b200 as rd
 from paper_1310_4645_b200.inputs import make_inputs, WORKLOADS
 from oracle import rd_oracle as O
-from helpers import oracle_schedule
+from helpers import oracle_schedule, check64, inputs64
 
 pytestmark = pytest.mark.gpu
 
@@ -77,6 +77,59 @@ def test_parity_min_and_product(name, algo, port, dist, op):
         elif dist == "int_pm2p20":
             want = np.multiply.reduce(xh.view(np.uint32), axis=0, dtype=np.uint32).view(np.int32)
             assert (got == want).all()
+
+
+# (p, n, segment elements) for 8-byte elements: tiles hold 1024 of them; segments that begin 8 bytes
+# into a 128-bit vector; message lengths that are not whole vectors
+SHAPES64 = [(8, 4096, 512), (5, 10000, 2500), (13, 3 * 1024 + 18, 1024 + 261), (64, 4096, 512), (2, 2050, 2050),
+            (33, 3000, 501), (16, 64, 4), (1, 2500, 500), (8, 1501, 333), (3, 3, 1), (8, 3077, 167)]
+
+
+@pytest.mark.parametrize("name,algo,port", [s for s in SCHEDULES if s[0] != "butterfly"])
+@pytest.mark.parametrize("kind,op", [("int64", "sum"), ("int64", "max"), ("int64", "min"), ("int64_small", "prod"),
+                                     ("normal64", "sum"), ("normal64", "max"), ("normal64", "min"), ("near_one", "prod")])
+def test_parity_eight_byte_elements(name, algo, port, kind, op):
+    for p, n, seg in SHAPES64:
+        x = inputs64(p, n, kind, seed=p * 1000 + n)
+        got, xh = check64(algo, port, x, 8 * seg, op)
+        if kind.startswith("int64") and op in ("sum", "max", "min"):
+            want = {"sum": lambda: x.sum(dim=0), "max": lambda: x.amax(dim=0), "min": lambda: x.amin(dim=0)}[op]()
+            assert (got == want.cpu().numpy()).all()                   # torch's int64 sum wraps as well
+
+
+def test_eight_byte_elements_butterfly_and_odd_boundaries():
+    """Halving keeps chunk boundaries on elements when n is a multiple of the power of two below p;
+    otherwise a boundary would fall inside an element and the call is refused."""
+    for p, n in ((8, 4096), (13, 1024 + 8), (32, 2048 + 32)):
+        check64(rd.RD_BUTTERFLY, rd.RD_PORT_BI, inputs64(p, n, "normal64", seed=p), 0, "sum")
+        check64(rd.RD_BUTTERFLY, rd.RD_PORT_BI, inputs64(p, n, "int64", seed=p), 0, "max")
+    x = inputs64(8, 4099, "normal64", seed=1)
+    with pytest.raises(rd.RdError) as e:
+        check64(rd.RD_BUTTERFLY, rd.RD_PORT_BI, x, 0, "sum")
+    assert e.value.status == rd.RD_ERR_INVALID_ARG
+    with pytest.raises(rd.RdError) as e:
+        check64(rd.RD_PIPELINE, rd.RD_PORT_UNI, x, 12, "sum")           # 12-byte segments split elements
+    assert e.value.status == rd.RD_ERR_INVALID_ARG
+
+
+def test_eight_byte_elements_off_the_vector_boundary():
+    """Buffers that start 8 bytes into a 128-bit vector take the element path (one element per thread)."""
+    p, n = 8, 3003
+    big = inputs64(p, n + 1, "normal64", seed=6)
+    rows = [big[i, 1:] for i in range(p)]
+    assert rows[0].data_ptr() % 16 == 8
+    out_big = torch.zeros(n + 1, dtype=torch.float64, device="cuda")
+    check64(rd.RD_BI_GREEDY, rd.RD_PORT_BI, big[:, 1:], 8 * 512, "sum", rows=rows, out=out_big[1:])
+    assert out_big[0].item() == 0.0
+
+
+def test_fp64_keeps_what_fp32_would_lose():
+    """2^30 + 1 + ... : exact in fp64 for any order, and different from an fp32 evaluation."""
+    p, n = 16, 4096
+    x = torch.ones((p, n), dtype=torch.float64, device="cuda")
+    x[0] = 2.0 ** 40
+    got, _ = check64(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, x, 8 * 512, "sum")
+    assert (got == 2.0 ** 40 + 15).all()
 
 
 def test_config1_bit_exact_and_order_free():

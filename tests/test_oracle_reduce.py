@@ -217,3 +217,60 @@ def test_empty_segments_and_single_process():
     x = np.ones((4, 3), dtype=np.int32)
     ev, off, _ = O.butterfly(4, 3, 4, 1, 1, 1)          # fewer elements than processes: empty chunks
     assert (O.reduce(ev, x, off, "sum") == 4).all()
+
+
+# ---- 8-byte element types ---------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("p", [2, 3, 8, 13, 64])
+def test_int64_results_do_not_depend_on_the_order(p):
+    """Sum and product modulo 2^64 (computed here with Python integers), max and min exactly."""
+    rng = np.random.default_rng(300 + p)
+    sizes = [5, 5, 5, 2]
+    n = sum(sizes)
+    x = rng.integers(-2**63, 2**63, size=(p, n), dtype=np.int64)
+    x[:, :6] = rng.integers(-3, 4, size=(p, 6)) * 2 + 1
+    cols = [[int(v) for v in x[:, e]] for e in range(n)]
+    wrap = lambda v: np.array([c & 0xFFFFFFFFFFFFFFFF for c in v], dtype=np.uint64).view(np.int64)
+    want_sum = wrap([sum(c) for c in cols])
+    want_prod = wrap([int(np.prod(np.array(c, dtype=object))) for c in cols])
+    assert (want_prod[:6] != 0).all()
+    for name, ev in schedules(p, sizes):
+        assert (O.reduce(ev, x, seg_off(sizes), "sum") == want_sum).all(), name
+        assert (O.reduce(ev, x, seg_off(sizes), "prod") == want_prod).all(), name
+        assert (O.reduce(ev, x, seg_off(sizes), "max") == x.max(axis=0)).all(), name
+        assert (O.reduce(ev, x, seg_off(sizes), "min") == x.min(axis=0)).all(), name
+    ev, off, _ = O.butterfly(p, n, 8, 3, 1, 1)
+    assert (O.reduce(ev, x, off, "sum") == want_sum).all()
+
+
+def test_fp64_two_processes_is_one_operation_and_the_pipeline_a_running_sum():
+    rng = np.random.default_rng(9)
+    x = rng.standard_normal((2, 1000)) * 10.0 ** rng.integers(-30, 30, size=(2, 1000))
+    ev, _ = O.uni_greedy(2, [600, 400], 1, 1, 1)
+    assert (O.reduce(ev, x, [0, 600, 1000], "sum") == x[0] + x[1]).all()
+    assert (O.reduce(ev, x, [0, 600, 1000], "prod") == x[0] * x[1]).all()
+    p = 9
+    x = rng.standard_normal((p, 64)) * 10.0 ** rng.integers(-8, 9, size=(p, 64))
+    want = x[p - 1].copy()
+    for k in range(p - 2, -1, -1):
+        want = x[k] + want
+    ev, _ = O.pipeline(p, [32, 32], 3, 1, 1, False)
+    assert O.reduce(ev, x, [0, 32, 64], "sum").tobytes() == want.tobytes()
+
+
+@pytest.mark.parametrize("p", [2, 5, 16, 33])
+def test_fp64_extrema_and_exact_sums(p):
+    """Integers below 2^40 add exactly in fp64 whatever the order; the same values do not in fp32, so a
+    reduction that went through fp32 anywhere would fail here."""
+    rng = np.random.default_rng(400 + p)
+    sizes = [7, 7, 3]
+    x = rng.standard_normal((p, 17))
+    k = rng.integers(-2**40, 2**40, size=(p, 17)).astype(np.float64)
+    for name, ev in schedules(p, sizes):
+        assert (O.reduce(ev, x, seg_off(sizes), "max") == x.max(axis=0)).all(), name
+        assert (O.reduce(ev, x, seg_off(sizes), "min") == x.min(axis=0)).all(), name
+        assert (O.reduce(ev, k, seg_off(sizes), "sum") == k.sum(axis=0)).all(), name
+    z = np.array([[0.0], [-0.0]])
+    ev, _ = O.uni_greedy(2, [1], 1, 1, 1)
+    assert np.signbit(O.reduce(ev, z, [0, 1], "max"))[0] == False
+    assert np.signbit(O.reduce(ev, z[::-1].copy(), [0, 1], "max"))[0] == True
