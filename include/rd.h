@@ -282,11 +282,13 @@ RD_API int rd_schedule_faithful_shape(rd_schedule_t *s, int *blocks_per_process,
  *   taken before the slot is overwritten, else -1).
  *   buf host, capacity cap_actions actions; n_actions / slots_per_process may be NULL.
  * RD_ERR_TOO_SMALL leaves buf untouched but still reports n_actions.
- * On the GPU a process is played by G thread blocks that never synchronise with each other; block
- * g works on offsets [U*g/G, U*(g+1)/G) * v of every segment, clipped to the segment's length,
- * with v = 4 elements on the 128-bit path (else 1) and U = ceil(L / v) for the largest segment
- * length L rounded up to a multiple of 4: the same offsets for every segment, so that blocks which
- * are at different points of the schedule never meet in a scratch slot.
+ * On the GPU a process is played by G thread blocks that never synchronise with each other.  A
+ * segment that begins at 4-byte word b of the message sits in its scratch slot from word b mod 4 on,
+ * so that slot and messages agree on where the 128-bit boundaries fall; a slot has W words, the
+ * largest (b mod 4) + length over the segments, rounded up to a multiple of 4.  Block g works on slot
+ * words [U*g/G, U*(g+1)/G) * v, clipped to the segment, with v = 4 words when all buffers are
+ * 16-byte aligned (else one element) and U = W / v: the same slot words for every segment, so that
+ * blocks which are at different points of the schedule never meet in a scratch slot.
  */
 RD_API int rd_schedule_actions(const rd_schedule_t *s, int process, int32_t *buf, size_t cap_actions,
                                size_t *n_actions, int *slots_per_process);

@@ -342,6 +342,15 @@ template <typename T> int dev_alloc(T **ptr, size_t count)
     return cudaMalloc(reinterpret_cast<void **>(ptr), std::max<size_t>(count, 1) * sizeof(T)) == cudaSuccess ? RD_OK : RD_ERR_NOMEM;
 }
 
+// Words of one scratch slot: a segment that begins at word b of the message sits b mod 4 words into
+// its slot (so that slot and messages agree on the 128-bit boundaries); whole vectors.
+uint64_t faithful_slot_words(const std::vector<uint64_t> &seg_off)
+{
+    uint64_t need = 0;
+    for (size_t j = 0; j + 1 < seg_off.size(); j++) need = std::max(need, (seg_off[j] & 3u) + (seg_off[j + 1] - seg_off[j]));
+    return (need + 3) / 4 * 4;
+}
+
 // Device tables and scratch of the schedule-faithful execution, built on its first use.
 int prepare_faithful(rd_schedule *s)
 {
@@ -368,9 +377,7 @@ int prepare_faithful(rd_schedule *s)
     if (capacity < s->p) return RD_ERR_UNSUPPORTED;
     d.f_lanes = int(std::min<long long>(16, capacity / s->p));
     d.f_slots = std::max(lists.slots_per_proc, 1);
-    uint64_t longest = 0;
-    for (size_t j = 0; j < q; j++) longest = std::max(longest, s->sched.seg_off[j + 1] - s->sched.seg_off[j]);
-    d.f_slot_elems = (longest + 3) / 4 * 4;
+    d.f_slot_elems = faithful_slot_words(s->sched.seg_off);
     const size_t nEvents = s->sched.events.size();
     std::vector<FaithfulAction> acts(lists.actions.size());
     for (size_t k = 0; k < acts.size(); k++) {
@@ -414,7 +421,6 @@ int reduce_faithful(rd_schedule *s, const void *const *d_inputs, void *d_out, si
         if (int rc = prepare_faithful(s)) return rc;
         bool wide = (reinterpret_cast<uintptr_t>(d_out) & 15u) == 0;
         for (int i = 0; i < s->p && wide; i++) wide = (reinterpret_cast<uintptr_t>(d_inputs[i]) & 15u) == 0;
-        for (size_t j = 0; j < s->sched.seg_off.size() && wide; j++) wide = (s->sched.seg_off[j] & 3u) == 0;
         if (cudaMemcpyAsync(d.f_inputs, d_inputs, size_t(s->p) * sizeof(void *), cudaMemcpyHostToDevice, stream) != cudaSuccess)
             return RD_ERR_CUDA;
         if (++d.f_epoch == 0) d.f_epoch = 1;
@@ -721,12 +727,9 @@ int rd_reduce_faithful_static(rd_schedule_t *s, const void *const *d_inputs, voi
             const Action &a = lists.actions[k];
             acts[k] = FaithfulAction{a.seg, a.peer, a.kind, a.slot, a.peer_slot, a.first, a.event, a.wait_event};
         }
-        uint64_t longest = 0;
-        for (size_t j = 0; j < q; j++) longest = std::max(longest, s->sched.seg_off[j + 1] - s->sched.seg_off[j]);
         std::vector<unsigned long long> times(2 * size_t(s->p) * 16);
         bool wide = (reinterpret_cast<uintptr_t>(d_out) & 15u) == 0;
         for (int i = 0; i < s->p && wide; i++) wide = (reinterpret_cast<uintptr_t>(d_inputs[i]) & 15u) == 0;
-        for (size_t j = 0; j < s->sched.seg_off.size() && wide; j++) wide = (s->sched.seg_off[j] & 3u) == 0;
         StaticRun r{};
         r.p = s->p;
         r.h_actions = acts.data(); r.n_actions = acts.size();
@@ -735,7 +738,7 @@ int rd_reduce_faithful_static(rd_schedule_t *s, const void *const *d_inputs, voi
         r.h_inputs = d_inputs; r.d_out = d_out;
         r.n_events = s->sched.events.size();
         r.slots = std::max(lists.slots_per_proc, 1);
-        r.slot_elems = (longest + 3) / 4 * 4;
+        r.slot_elems = faithful_slot_words(s->sched.seg_off);
         r.blocking_send = s->port == RD_PORT_UNI ? 1 : 0;
         r.dtype = int(dtype); r.op = int(op); r.wide = wide;
         r.wait_seconds = s->wait_budget_s;

@@ -1,7 +1,7 @@
 // Schedule-faithful execution on sm_100a: groups of thread blocks play the processes.
 //
-// Process i is played by G thread blocks ("lanes"); lane g owns the same range of offsets of every
-// segment (1/G of the largest segment, clipped), so the G lanes are G independent copies of the
+// Process i is played by G thread blocks ("lanes"); lane g owns the same range of words of every
+// scratch slot (1/G of it), so the G lanes are G independent copies of the
 // whole p-process system working on disjoint parts of the message and of the scratch slots, and
 // never synchronise with each other.  Each block walks its process's
 // action list in order:
@@ -173,24 +173,39 @@ rd_faithful_kernel(const FaithfulParams a)
         if (alive) alive = wait_flag(posted, a.epoch, a, &sh_ok);
         if (!alive) break;
         if (threadIdx.x == 0 && lane == 0) t_start = now_ns();
-        // This lane's share: the same offsets of EVERY segment (a fixed 1/G of the slot, clipped to the
-        // segment's length).  Lanes run independently of each other and share the slots, so a lane
-        // that is already re-using a slot for a later, shorter segment must never touch offsets that
+        // A segment that starts at word b of the message sits in its slot from word (b mod 4) on, so that
+        // slot, messages and output agree on where the 128-bit boundaries fall and whole vectors can be
+        // moved wherever a segment starts.  This lane's share is the same range of SLOT words for every
+        // segment (a fixed 1/G of the slot): lanes run independently of each other and share the slots,
+        // so a lane that is already re-using a slot for a later segment must never touch words that
         // belong to another lane's share of the segment still held there.
         const uint64_t seg_lo = a.seg_off[act.seg], seg_len = a.seg_off[act.seg + 1] - seg_lo;
-        const uint64_t units = (a.slot_elems + V - 1) / V;
+        const uint64_t phase = seg_lo & 3u, first = phase, last = phase + seg_len;      // the segment's slot words
+        const uint64_t units = a.slot_elems / V;
         uint64_t lo = units * uint64_t(lane) / uint64_t(a.lanes) * V;
         uint64_t hi = units * uint64_t(lane + 1) / uint64_t(a.lanes) * V;
-        if (lo > seg_len) lo = seg_len;
-        if (hi > seg_len) hi = seg_len;
+        if (hi > (last + V - 1) / V * V) hi = (last + V - 1) / V * V;
+        // all three pointers are indexed by slot word
         const uint32_t *src = act.peer_slot >= 0 ? a.scratch + (size_t(act.peer) * a.slots + size_t(act.peer_slot)) * a.slot_elems
-                              : act.peer_slot == -1 ? a.inputs[act.peer] + seg_lo : a.out + seg_lo;
-        uint32_t *dst = act.slot >= 0 ? a.scratch + (size_t(proc) * a.slots + size_t(act.slot)) * a.slot_elems : a.out + seg_lo;
-        const uint32_t *held = act.first ? mine + seg_lo : dst;
+                              : (act.peer_slot == -1 ? a.inputs[act.peer] : a.out) + (seg_lo - phase);
+        uint32_t *dst = act.slot >= 0 ? a.scratch + (size_t(proc) * a.slots + size_t(act.slot)) * a.slot_elems : a.out + (seg_lo - phase);
+        const uint32_t *held = act.first ? mine + (seg_lo - phase) : dst;
         const bool store_only = act.kind == 1;
-        for (uint64_t e = lo + uint64_t(threadIdx.x) * V; e < hi; e += uint64_t(kFaithfulThreads) * V) {
-            const Words<V> in = load_words<V>(src + e);
-            store_words<V>(dst + e, store_only ? in : combine_words<DT, OPR, V>(load_words<V>(held + e), in));
+        constexpr int E = ElemWords<DT>::value;
+        for (uint64_t w = lo + uint64_t(threadIdx.x) * V; w < hi; w += uint64_t(kFaithfulThreads) * V) {
+            if (w >= first && w + V <= last) {
+                const Words<V> in = load_words<V>(src + w);
+                store_words<V>(dst + w, store_only ? in : combine_words<DT, OPR, V>(load_words<V>(held + w), in));
+            } else {
+                // the vector holding the segment's first or last words: element by element
+#pragma unroll
+                for (int k = 0; k < V; k += E) {
+                    if (w + k >= first && w + k < last) {
+                        const Words<E> in = load_words<E>(src + w + k);
+                        store_words<E>(dst + w + k, store_only ? in : combine_words<DT, OPR, E>(load_words<E>(held + w + k), in));
+                    }
+                }
+            }
         }
         // the sender's value has been read: tell it
         __syncthreads();

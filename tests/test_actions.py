@@ -14,12 +14,18 @@ CASES = [(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI), (rd.RD_BI_GREEDY, rd.RD_PORT_BI), (
          (rd.RD_BINARY, rd.RD_PORT_BI), (rd.RD_BUTTERFLY, rd.RD_PORT_BI)]
 
 
-def lane_range(longest, lanes, g, seg_len, v=4):
-    """Offsets of a segment that block g of a process's G blocks works on (rule stated in include/rd.h)."""
-    slot_elems = (longest + 3) // 4 * 4
-    units = -(-slot_elems // v)
+def slot_words(off):
+    return (max(int(off[j]) % 4 + int(off[j + 1] - off[j]) for j in range(len(off) - 1)) + 3) // 4 * 4
+
+
+def lane_range(width, lanes, g, seg_start, seg_len, v=4):
+    """Slot words [lo, hi) of a segment that block g of a process's G blocks works on (rule stated in
+    include/rd.h): a fixed 1/G of the slot, clipped to where the segment sits in it."""
+    units = width // v
     lo, hi = units * g // lanes * v, units * (g + 1) // lanes * v
-    return min(lo, seg_len), min(hi, seg_len)
+    first, last = seg_start % 4, seg_start % 4 + seg_len
+    lo, hi = max(lo, first), min(hi, last)
+    return (lo, hi) if lo < hi else (first, first)
 
 
 def emulate(h, x, op, blocking_send, rng, lanes=1):
@@ -109,7 +115,8 @@ def emulate_lanes(h, x, op, blocking_send, rng, lanes):
     lists = [rd.rd_schedule_actions(h, i)[0] for i in range(p)]
     slots = rd.rd_schedule_actions(h, 0)[1]
     longest = int(np.diff(off).max())
-    scratch = np.zeros((p, max(slots, 1), (longest + 3) // 4 * 4), dtype=x.dtype)
+    width = slot_words(off)
+    scratch = np.zeros((p, max(slots, 1), width), dtype=x.dtype)
     owner = np.full(scratch.shape, -1, dtype=np.int64)      # segment whose value an offset of a slot holds
     out = np.zeros(n, dtype=x.dtype)
     n_events = rd.rd_schedule_info(h)["n_events"]
@@ -143,8 +150,9 @@ def emulate_lanes(h, x, op, blocking_send, rng, lanes):
             if pc[i, g] >= len(lists[i]):
                 continue
             seg, peer, kind, slot, peer_slot, first, ev, wait_ev = (int(v) for v in lists[i][pc[i, g]])
-            base, seg_len = off[seg], off[seg + 1] - off[seg]
-            lo, hi = lane_range(longest, lanes, g, seg_len)
+            seg_len = off[seg + 1] - off[seg]
+            lo, hi = lane_range(width, lanes, g, off[seg], seg_len)        # slot words
+            base = off[seg] - off[seg] % 4                                 # message word of slot word 0
             if kind == 2:
                 posted[ev, g] = True
                 if blocking_send:
@@ -181,14 +189,16 @@ def emulate_lanes(h, x, op, blocking_send, rng, lanes):
 
 
 @pytest.mark.parametrize("algo,port", CASES)
-def test_lanes_that_drift_apart_never_meet_in_a_slot(algo, port):
-    """Unequal segments (a short last one), several blocks per process running at very different speeds."""
-    p, n, seg = 13, 618, 257
+@pytest.mark.parametrize("seg", [256, 257, 101])
+def test_lanes_that_drift_apart_never_meet_in_a_slot(algo, port, seg):
+    """Unequal segments (a short last one; with 257 and 101 they also begin at every position inside a
+    128-bit vector), several blocks per process running at very different speeds."""
+    p, n = 13, 618
     rng = np.random.default_rng(algo)
     x = (rng.standard_normal((p, n)) * 10.0 ** rng.integers(-4, 5, size=(p, n))).astype(np.float32)
-    h = rd.rd_schedule_create(algo, port, p, 4 * n, 4 * 256 if algo != rd.RD_BUTTERFLY else 0, *M1)
+    h = rd.rd_schedule_create(algo, port, p, 4 * n, 4 * seg if algo != rd.RD_BUTTERFLY else 0, *M1)
     try:
-        ev, off, _ = oracle_schedule(algo, port, p, 4 * n, 4 * 256 if algo != rd.RD_BUTTERFLY else 4 * n, *M1)
+        ev, off, _ = oracle_schedule(algo, port, p, 4 * n, 4 * seg if algo != rd.RD_BUTTERFLY else 4 * n, *M1)
         want = O.reduce(ev, x, off, "sum")
         for trial in range(4):
             got, _ = emulate(h, x, "sum", port == rd.RD_PORT_UNI, np.random.default_rng(100 + trial), lanes=5)

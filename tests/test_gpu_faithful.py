@@ -36,7 +36,9 @@ def run(algo, port, x, seg_bytes, op, rows=None, out=None):
 
 
 SHAPES = [(8, 4096, 512), (5, 10000, 2500), (13, 3 * 2048 + 36, 2048 + 520), (64, 8192, 1024), (2, 4100, 4100),
-          (33, 6000, 1000), (16, 128, 8), (1, 5000, 1000)]
+          (33, 6000, 1000), (16, 128, 8), (1, 5000, 1000),
+          # segments that begin and end at every position inside a 128-bit vector
+          (8, 3000, 333), (13, 6180, 999), (4, 64, 3), (32, 8192, 2049), (8, 4099, 1000), (5, 7, 2)]
 
 
 @pytest.mark.parametrize("name,algo,port", SCHEDULES)
