@@ -152,19 +152,15 @@ void release_device(DeviceTables &d)
     d = DeviceTables();
 }
 
-int upload(rd_schedule *s)
+int upload_tables(rd_schedule *s, int cur)
 {
     DeviceTables &d = s->dev;
-    int cur = -1;
-    if (cudaGetDevice(&cur) != cudaSuccess) return RD_ERR_CUDA;
-    if (d.device == cur) return RD_OK;
-    if (d.device >= 0) release_device(d);
+    d.device = cur;                          // from here on release_device frees whatever exists
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, cur) != cudaSuccess) return RD_ERR_CUDA;
     d.sm_count = prop.multiProcessorCount;
     const size_t opBytes = std::max<size_t>(s->progs.ops.size(), 1) * sizeof(uint32_t);
     if (cudaMalloc(reinterpret_cast<void **>(&d.ops), opBytes) != cudaSuccess) return RD_ERR_NOMEM;
-    d.device = cur;
     if (!s->progs.ops.empty() &&
         cudaMemcpy(d.ops, s->progs.ops.data(), s->progs.ops.size() * sizeof(uint32_t), cudaMemcpyHostToDevice) != cudaSuccess)
         return RD_ERR_CUDA;
@@ -180,6 +176,20 @@ int upload(rd_schedule *s)
             if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return RD_ERR_CUDA;
     }
     return RD_OK;
+}
+
+// Copies the schedule's tables to the current device unless they are there already.  A failure
+// half-way leaves nothing behind, so that the next call starts again from the beginning.
+int upload(rd_schedule *s)
+{
+    DeviceTables &d = s->dev;
+    int cur = -1;
+    if (cudaGetDevice(&cur) != cudaSuccess) return RD_ERR_CUDA;
+    if (d.device == cur) return RD_OK;
+    if (d.device >= 0) release_device(d);
+    const int rc = upload_tables(s, cur);
+    if (rc != RD_OK) release_device(d);
+    return rc;
 }
 
 // Tiles of the element-path kernel: runs of at most `cap` elements inside a segment.
@@ -234,6 +244,8 @@ int tiles_for(rd_schedule *s, int vec, const TileDesc **tiles, uint32_t *count)
             std::vector<uint32_t> first(size_t(ctas) + 1, 0);
             for (uint64_t c = 0; c < ctas; c++) first[size_t(c)] = uint32_t(nTiles * c / ctas);
             first[size_t(ctas)] = uint32_t(host.size());
+            cudaFree(d.cta_first);                  // left by an attempt that failed after this point
+            d.cta_first = nullptr;
             if (cudaMalloc(reinterpret_cast<void **>(&d.cta_first), first.size() * sizeof(uint32_t)) != cudaSuccess) return RD_ERR_NOMEM;
             if (cudaMemcpy(d.cta_first, first.data(), first.size() * sizeof(uint32_t), cudaMemcpyHostToDevice) != cudaSuccess)
                 return RD_ERR_CUDA;
