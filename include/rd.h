@@ -226,6 +226,25 @@ RD_API int rd_schedule_program(const rd_schedule_t *s, size_t seg, uint32_t *ops
 RD_API int rd_reduce(rd_schedule_t *s, const void *const *d_inputs, void *d_out, size_t n_elems,
               rd_dtype_t dtype, rd_op_t op, rd_exec_t exec, void *cuda_stream, rd_stats_t *stats);
 
+/*
+ * rd_reduce_batch -- several independent tree-mode reductions issued together (the paper has no
+ * counterpart; Section VII runs the same messages under every schedule, and a library user reduces
+ * many buffers).  Job j reduces d_inputs[j][0..p_j) into d_outs[j] under schedules[j]; all jobs share
+ * dtype, op and stream.  Results are exactly those of n_jobs rd_reduce calls.  Because the jobs are
+ * independent, the library issues them alternately on two streams of its own, so that one job's
+ * thread blocks take the SM slots another job frees while its last blocks are still running; the
+ * batch as a whole is ordered after what precedes it on cuda_stream and before what follows it
+ * (event fork and join).  The two side streams and three events are created on a device's first
+ * batch and kept.
+ *   schedules, d_inputs, d_outs, n_elems   HOST arrays of n_jobs entries (d_inputs[j]: HOST array of
+ *             DEVICE pointers as in rd_reduce).  The same schedule may serve several jobs.
+ * RD_ERR_INVALID_ARG when a job's output overlaps another job's output or inputs (a job's output may
+ * alias its own root input); otherwise the errors of rd_reduce.  On an error jobs before the failing
+ * one have been launched.
+ */
+RD_API int rd_reduce_batch(size_t n_jobs, rd_schedule_t *const *schedules, const void *const *const *d_inputs,
+                    void *const *d_outs, const size_t *n_elems, rd_dtype_t dtype, rd_op_t op, void *cuda_stream);
+
 /* rd_schedule_upload -- copies the schedule's tables to the current device now. */
 RD_API int rd_schedule_upload(rd_schedule_t *s);
 

@@ -29,7 +29,8 @@ ALGOS = {"uni_greedy": RD_UNI_GREEDY, "bi_greedy": RD_BI_GREEDY, "binomial": RD_
 EXPORTS = ("rd_schedule_create", "rd_schedule_create_segments", "rd_optimal_segment", "rd_schedule_info",
            "rd_schedule_events", "rd_schedule_segments", "rd_schedule_program", "rd_reduce",
            "rd_schedule_upload", "rd_reduce_host", "rd_destroy", "rd_strerror", "rd_schedule_set_wait_budget",
-           "rd_schedule_trace", "rd_schedule_faithful_shape", "rd_schedule_actions", "rd_reduce_faithful_static", "rd_search_segmentation", "rd_schedule_status")
+           "rd_schedule_trace", "rd_schedule_faithful_shape", "rd_schedule_actions", "rd_reduce_faithful_static", "rd_search_segmentation", "rd_schedule_status",
+           "rd_reduce_batch")
 
 
 class rd_model_t(C.Structure):
@@ -87,6 +88,7 @@ def lib():
         L.rd_search_segmentation.argtypes = [i32, sz, sz, C.POINTER(rd_model_t), C.POINTER(sz), sz, C.POINTER(sz),
                                              C.POINTER(C.c_int64)]
         L.rd_schedule_status.argtypes = [vp, C.POINTER(i32)]
+        L.rd_reduce_batch.argtypes = [sz, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(sz), i32, i32, vp]
         L.rd_destroy.argtypes = [vp]
         L.rd_destroy.restype = None
         L.rd_strerror.argtypes = [i32]
@@ -234,6 +236,46 @@ def rd_reduce(h, inputs, out, op, exec_mode=RD_EXEC_TREE, stream=None, want_stat
         if out.device.index != prev:
             torch.cuda.set_device(prev)
     return stats
+
+
+class Batch:
+    """Marshalled arguments of rd_reduce_batch, built once and reused: jobs = [(schedule, inputs, out)], inputs
+    a PointerTable, a [p, n] CUDA tensor or a list of p CUDA tensors."""
+
+    def __init__(self, jobs):
+        self.tables = [t if isinstance(t, PointerTable) else PointerTable(t) for _, t, _ in jobs]
+        self.outs = [o for _, _, o in jobs]
+        k = len(jobs)
+        for tab, out in zip(self.tables, self.outs):
+            if not out.is_cuda or not out.is_contiguous() or not tab.is_cuda or tab.n != out.numel() or tab.dtype != out.dtype:
+                raise ValueError("every input must be a contiguous CUDA tensor with its output's dtype and length")
+            if out.dtype != self.outs[0].dtype or out.device != self.outs[0].device:
+                raise ValueError("all jobs of a batch share the element type and the device")
+        self.k = k
+        self.schedules = (C.c_void_p * k)(*[h for h, _, _ in jobs])
+        self.inputs = (C.c_void_p * k)(*[C.cast(t.array, C.c_void_p).value for t in self.tables])
+        self.out_ptrs = (C.c_void_p * k)(*[o.data_ptr() for o in self.outs])
+        self.n_elems = (C.c_size_t * k)(*[o.numel() for o in self.outs])
+        self.dtype = _dtype_code(self.outs[0]) if k else RD_FP32
+        self.device = self.outs[0].device if k else None
+
+
+def rd_reduce_batch(jobs, op, stream=None):
+    """jobs: a Batch, or a list of (schedule, inputs, out).  Independent reductions issued together."""
+    import torch
+    b = jobs if isinstance(jobs, Batch) else Batch(jobs)
+    if b.k == 0:
+        return
+    s = stream if stream is not None else torch.cuda.current_stream(b.device)
+    prev = torch.cuda.current_device()
+    if b.device.index != prev:
+        torch.cuda.set_device(b.device)
+    try:
+        _check(lib().rd_reduce_batch(b.k, b.schedules, b.inputs, b.out_ptrs, b.n_elems, b.dtype, int(op), s.cuda_stream),
+               "rd_reduce_batch")
+    finally:
+        if b.device.index != prev:
+            torch.cuda.set_device(prev)
 
 
 def rd_reduce_faithful_static(h, inputs, out, op, stream=None, want_stats=False):

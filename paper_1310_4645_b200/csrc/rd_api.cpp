@@ -5,6 +5,7 @@
 #include <cmath>
 #include <cstring>
 #include <map>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -17,6 +18,16 @@ using namespace rd;
 namespace {
 
 constexpr int kPtrRing = 8;   // pointer tables in flight for p > kPackedPtrs
+constexpr int kMaxDevices = 64;
+
+// Side streams of rd_reduce_batch, created on a device's first batch and kept for the process's life.
+struct BatchLanes {
+    bool ready = false;
+    cudaStream_t stream[2] = {nullptr, nullptr};
+    cudaEvent_t fork = nullptr, join[2] = {nullptr, nullptr};
+};
+BatchLanes g_lanes[kMaxDevices];
+std::mutex g_lanes_mutex;
 constexpr int kTailTiles = 5; // key of the tile table for the elements the 128-bit path leaves over
 
 struct DeviceTables {
@@ -613,6 +624,64 @@ int rd_reduce(rd_schedule_t *s, const void *const *d_inputs, void *d_out, size_t
         if (exec == RD_EXEC_FAITHFUL)
             return reduce_faithful(s, d_inputs, d_out, n_words, dtype, op, static_cast<cudaStream_t>(cuda_stream), stats);
         return reduce_tree(s, d_inputs, d_out, n_words, dtype, op, static_cast<cudaStream_t>(cuda_stream), stats);
+    });
+}
+
+int rd_reduce_batch(size_t n_jobs, rd_schedule_t *const *schedules, const void *const *const *d_inputs, void *const *d_outs,
+                    const size_t *n_elems, rd_dtype_t dtype, rd_op_t op, void *cuda_stream)
+{
+    if (n_jobs == 0) return RD_OK;
+    if (!schedules || !d_inputs || !d_outs || !n_elems) return RD_ERR_INVALID_ARG;
+    std::vector<size_t> words;
+    try { words.resize(n_jobs); } catch (const std::bad_alloc &) { return RD_ERR_NOMEM; }
+    for (size_t j = 0; j < n_jobs; j++) {
+        if (!schedules[j] || !d_inputs[j]) return RD_ERR_INVALID_ARG;
+        if (int rc = check_reduce_args(schedules[j], d_inputs[j], d_outs[j], n_elems[j], dtype, op, &words[j])) return rc;
+    }
+    // the jobs may run concurrently: no job's output may overlap another job's output or inputs
+    // (a job's own output may alias its own root input, as in rd_reduce)
+    auto overlap = [](const void *a, size_t na, const void *b, size_t nb) {
+        const uintptr_t x = reinterpret_cast<uintptr_t>(a), y = reinterpret_cast<uintptr_t>(b);
+        return na > 0 && nb > 0 && x < y + nb && y < x + na;
+    };
+    for (size_t j = 0; j < n_jobs; j++)
+        for (size_t k = 0; k < n_jobs; k++) {
+            if (k == j) continue;
+            if (k > j && overlap(d_outs[j], words[j] * 4, d_outs[k], words[k] * 4)) return RD_ERR_INVALID_ARG;
+            for (int i = 0; i < schedules[k]->p; i++)
+                if (overlap(d_outs[j], words[j] * 4, d_inputs[k][i], words[k] * 4)) return RD_ERR_INVALID_ARG;
+        }
+    cudaStream_t user = static_cast<cudaStream_t>(cuda_stream);
+    return guarded([&] {
+        for (size_t j = 0; j < n_jobs; j++)
+            if (int rc = upload(schedules[j])) return rc;
+        if (n_jobs == 1) return reduce_tree(schedules[0], d_inputs[0], d_outs[0], words[0], dtype, op, user, nullptr);
+        // Fork: two side streams wait for what precedes the batch on the caller's stream and take the
+        // jobs alternately, so that one job's thread blocks fill the SM slots the other job frees while
+        // its last blocks are still running.  Join: the caller's stream waits for both.
+        int device = -1;
+        if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kMaxDevices) return int(RD_ERR_CUDA);
+        std::lock_guard<std::mutex> hold(g_lanes_mutex);
+        BatchLanes &lanes = g_lanes[device];
+        if (!lanes.ready) {
+            bool ok = cudaEventCreateWithFlags(&lanes.fork, cudaEventDisableTiming) == cudaSuccess;
+            for (int l = 0; l < 2 && ok; l++)
+                ok = cudaStreamCreateWithFlags(&lanes.stream[l], cudaStreamNonBlocking) == cudaSuccess &&
+                     cudaEventCreateWithFlags(&lanes.join[l], cudaEventDisableTiming) == cudaSuccess;
+            if (!ok) return int(RD_ERR_CUDA);
+            lanes.ready = true;
+        }
+        if (cudaEventRecord(lanes.fork, user) != cudaSuccess) return int(RD_ERR_CUDA);
+        for (int l = 0; l < 2; l++)
+            if (cudaStreamWaitEvent(lanes.stream[l], lanes.fork, 0) != cudaSuccess) return int(RD_ERR_CUDA);
+        int rc = RD_OK;
+        for (size_t j = 0; j < n_jobs && rc == RD_OK; j++)
+            rc = reduce_tree(schedules[j], d_inputs[j], d_outs[j], words[j], dtype, op, lanes.stream[j & 1], nullptr);
+        // join also after a failure, so that what was launched stays ordered before the caller's next work
+        for (int l = 0; l < 2; l++)
+            if (cudaEventRecord(lanes.join[l], lanes.stream[l]) != cudaSuccess || cudaStreamWaitEvent(user, lanes.join[l], 0) != cudaSuccess)
+                rc = rc == RD_OK ? int(RD_ERR_CUDA) : rc;
+        return rc;
     });
 }
 

@@ -135,3 +135,26 @@ def test_empty_message_and_single_process():
     assert info["q"] == 4 and info["n_events"] == 0 and info["predicted_ticks"] == 0
     assert list(rd.rd_schedule_program(h, 2)) == [0]      # LOAD process 0
     rd.rd_destroy(h)
+
+
+def test_batch_argument_checks_come_before_any_cuda_call():
+    L = rd.lib()
+    h = rd.rd_schedule_create(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, 4, 4096, 1024, *MODEL)
+    try:
+        vp = C.c_void_p
+        def call(in_addrs, out_addrs, n=1024):
+            k = len(out_addrs)
+            tabs = [(vp * 4)(*a) for a in in_addrs]
+            return L.rd_reduce_batch(k, (vp * k)(*[h] * k), (vp * k)(*[C.cast(t, vp).value for t in tabs]),
+                                     (vp * k)(*out_addrs), (C.c_size_t * k)(*[n] * k), rd.RD_FP32, rd.RD_SUM, None)
+        rows = lambda base: [base + i * 4096 for i in range(4)]
+        assert L.rd_reduce_batch(0, None, None, None, None, rd.RD_FP32, rd.RD_SUM, None) == rd.RD_OK
+        assert L.rd_reduce_batch(1, None, None, None, None, rd.RD_FP32, rd.RD_SUM, None) == rd.RD_ERR_INVALID_ARG
+        # job 1 writes into job 0's second input
+        assert call([rows(0x100000), rows(0x200000)], [0x300000, 0x101000]) == rd.RD_ERR_INVALID_ARG
+        # the two outputs overlap
+        assert call([rows(0x100000), rows(0x200000)], [0x300000, 0x300800]) == rd.RD_ERR_INVALID_ARG
+        # wrong length
+        assert call([rows(0x100000)], [0x300000], n=1000) == rd.RD_ERR_SIZE_MISMATCH
+    finally:
+        rd.rd_destroy(h)

@@ -408,3 +408,109 @@ def test_randomized_shapes_order_free_results():
                 assert torch.equal(out, want), (case, name, p, n, seg, op)
         finally:
             rd.rd_destroy(h)
+
+
+def test_batch_equals_separate_calls_and_keeps_stream_order():
+    """Independent jobs issued together: bit-identical to one rd_reduce per job; what follows the batch on
+    the stream sees every result, what precedes it is seen by every job."""
+    p, n = 64, 1 << 18
+    specs = [(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, 16 << 10), (rd.RD_BINOMIAL, rd.RD_PORT_UNI, 16 << 10),
+             (rd.RD_PIPELINE, rd.RD_PORT_UNI, 16 << 10), (rd.RD_BINARY, rd.RD_PORT_UNI, 16 << 10),
+             (rd.RD_BI_GREEDY, rd.RD_PORT_BI, 64 << 10), (rd.RD_BUTTERFLY, rd.RD_PORT_BI, 0)]
+    hs = [rd.rd_schedule_create(a, pt, p, 4 * n, seg, *M1) for a, pt, seg in specs]
+    try:
+        x = torch.empty((p, n), device="cuda")
+        outs = [torch.empty(n, device="cuda") for _ in hs]
+        batch = rd.Batch([(h, x, o) for h, o in zip(hs, outs)])
+        for trial in range(5):
+            g = torch.Generator("cuda").manual_seed(trial)
+            x.normal_(generator=g)                                  # written on the stream just before the batch
+            x *= 10.0 ** torch.randint(-4, 5, x.shape, device="cuda", generator=g)
+            for o in outs:
+                o.fill_(-1.0)
+            rd.rd_reduce_batch(batch, rd.RD_SUM)
+            sums = torch.stack([o.double().sum() for o in outs])    # read on the stream just after it
+            ref = []
+            for h in hs:
+                r = torch.empty(n, device="cuda")
+                rd.rd_reduce(h, x, r, rd.RD_SUM)
+                ref.append(r)
+            torch.cuda.synchronize()
+            for o, r in zip(outs, ref):
+                assert torch.equal(o, r)
+            assert torch.equal(sums, torch.stack([r.double().sum() for r in ref]))
+        xh = x.cpu().numpy()
+        ev, off, _ = oracle_schedule(specs[0][0], specs[0][1], p, 4 * n, specs[0][2], *M1)
+        assert outs[0].cpu().numpy().tobytes() == O.reduce(ev, xh, off, "sum").tobytes()
+    finally:
+        for h in hs:
+            rd.rd_destroy(h)
+
+
+def test_batch_of_unlike_jobs():
+    """Jobs of different sizes and process counts, one with a ragged length (two launches), one with more
+    processes than travel as kernel parameters, and one whose output is its own root input."""
+    shapes = [(8, 4096, 2048), (13, 6151, 4 * 333), (300, 4096, 4096), (5, 10000, 4 * 2500), (2, 4100, 4 * 4100)]
+    hs, xs, outs = [], [], []
+    for k, (p, n, seg) in enumerate(shapes):
+        hs.append(rd.rd_schedule_create(rd.RD_BI_GREEDY, rd.RD_PORT_BI, p, 4 * n, seg, *M1))
+        xs.append(make_inputs(p, n, "int_pm2p20", seed=k, device="cuda"))
+        outs.append(torch.empty(n, dtype=torch.int32, device="cuda"))
+    keep = xs[0].clone()
+    outs[0] = xs[0][0]                                              # aliases its own root input
+    try:
+        rd.rd_reduce_batch([(h, x, o) for h, x, o in zip(hs, xs, outs)], rd.RD_SUM)
+        torch.cuda.synchronize()
+        xs[0] = keep
+        for x, o in zip(xs, outs):
+            want = ((x.sum(dim=0, dtype=torch.int64) + (1 << 31)) % (1 << 32) - (1 << 31)).to(torch.int32)
+            assert torch.equal(o, want)
+        with pytest.raises(rd.RdError) as e:                        # job 1 would write job 0's inputs
+            rd.rd_reduce_batch([(hs[1], xs[1], outs[1]), (hs[1], xs[1], xs[1][3])], rd.RD_SUM)
+        assert e.value.status == rd.RD_ERR_INVALID_ARG
+    finally:
+        for h in hs:
+            rd.rd_destroy(h)
+
+
+def test_config2_over_two_streams_as_the_benchmark_issues_it():
+    """The four schedules of config2 alternate over two CUDA streams (launches overlap each other's tail):
+    every output is bit-identical to the same reduction issued alone, and sampled segments of it to the oracle."""
+    w = WORKLOADS["config2"]
+    model = (w["alpha"], w["beta"], w["gamma"])
+    p, n = w["p"], w["n"]
+    arenas = [make_inputs(p, n, w["dist"], w["seed"] + 1000 * a, device="cuda") for a in range(3)]
+    tabs = [rd.PointerTable(a) for a in arenas]
+    algos = [rd.RD_UNI_GREEDY, rd.RD_BINOMIAL, rd.RD_PIPELINE, rd.RD_BINARY]
+    hs = [rd.rd_schedule_create(a, rd.RD_PORT_UNI, p, 4 * n, w["seg_bytes"], *model) for a in algos]
+    try:
+        outs = [torch.empty(n, device="cuda") for _ in hs]
+        streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+        torch.cuda.synchronize()
+        c = 0
+        for step in range(6):
+            for i, h in enumerate(hs):
+                rd.rd_reduce(h, tabs[c % 3], outs[i], rd.RD_SUM, stream=streams[i % 2])
+                c += 1
+        torch.cuda.synchronize()
+        # the last step read arenas (20, 21, 22, 23) mod 3
+        for i, h in enumerate(hs):
+            alone = torch.empty(n, device="cuda")
+            rd.rd_reduce(h, tabs[(20 + i) % 3], alone, rd.RD_SUM)
+            torch.cuda.synchronize()
+            assert torch.equal(outs[i], alone)
+            assert rd.rd_schedule_status(h) == 0
+        ev = rd.rd_schedule_events(hs[0])
+        off = rd.rd_schedule_segments(hs[0]).astype(np.int64)
+        oev = np.zeros(len(ev), dtype=O.EVENT_DTYPE)
+        for f in ("t_start", "seg", "src", "dst", "kind"):
+            oev[f] = ev[f]
+        for j in (0, 100, 255):
+            lo, hi = int(off[j]), int(off[j + 1])
+            sel = oev[oev["seg"] == j].copy()
+            sel["seg"] = 0
+            want = O.reduce(sel, arenas[20 % 3][:, lo:hi].cpu().numpy(), [0, hi - lo], "sum")
+            assert outs[0][lo:hi].cpu().numpy().tobytes() == want.tobytes()
+    finally:
+        for h in hs:
+            rd.rd_destroy(h)
