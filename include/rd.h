@@ -269,6 +269,19 @@ RD_API int rd_reduce_host(rd_schedule_t *s, const void *const *h_inputs, void *h
 RD_API int rd_schedule_set_wait_budget(rd_schedule_t *s, double seconds);
 
 /*
+ * rd_schedule_set_tree_variant -- which kernel serves tree-mode calls whose buffers are all 16-byte
+ * aligned (the paper has no counterpart; the result is the same bit for bit).
+ *   RD_TREE_AUTO    the library chooses (default): the direct kernel for one or two processes, else
+ *                   the streaming kernel.
+ *   RD_TREE_STREAM  operand tiles are streamed through a shared-memory ring by bulk asynchronous
+ *                   copies; any number of processes.
+ *   RD_TREE_DIRECT  every thread fetches all p operands of its elements into registers at once; at
+ *                   most 8 processes (RD_ERR_UNSUPPORTED beyond).
+ */
+typedef enum { RD_TREE_AUTO = 0, RD_TREE_STREAM = 1, RD_TREE_DIRECT = 2 } rd_tree_variant_t;
+RD_API int rd_schedule_set_tree_variant(rd_schedule_t *s, rd_tree_variant_t variant);
+
+/*
  * rd_schedule_trace -- measured times of the last schedule-faithful rd_reduce, to set against
  * the model's alpha + beta*s (+ gamma*s) per pair (Section V).  For every send/receive pair, in
  * the order of rd_schedule_events, three values in nanoseconds of the GPU's global timer, taken by

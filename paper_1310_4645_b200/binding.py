@@ -22,6 +22,7 @@ RD_PORT_UNI, RD_PORT_BI = 0, 1
 RD_SUM, RD_MAX, RD_MIN, RD_PROD = 0, 1, 2, 3
 RD_INT32, RD_FP32, RD_INT64, RD_FP64 = 0, 1, 2, 3
 RD_EXEC_TREE, RD_EXEC_FAITHFUL = 0, 1
+RD_TREE_AUTO, RD_TREE_STREAM, RD_TREE_DIRECT = 0, 1, 2
 
 ALGOS = {"uni_greedy": RD_UNI_GREEDY, "bi_greedy": RD_BI_GREEDY, "binomial": RD_BINOMIAL,
          "pipeline": RD_PIPELINE, "binary": RD_BINARY, "butterfly": RD_BUTTERFLY}
@@ -30,7 +31,7 @@ EXPORTS = ("rd_schedule_create", "rd_schedule_create_segments", "rd_optimal_segm
            "rd_schedule_events", "rd_schedule_segments", "rd_schedule_program", "rd_reduce",
            "rd_schedule_upload", "rd_reduce_host", "rd_destroy", "rd_strerror", "rd_schedule_set_wait_budget",
            "rd_schedule_trace", "rd_schedule_faithful_shape", "rd_schedule_actions", "rd_reduce_faithful_static", "rd_search_segmentation", "rd_schedule_status",
-           "rd_reduce_batch")
+           "rd_reduce_batch", "rd_schedule_set_tree_variant")
 
 
 class rd_model_t(C.Structure):
@@ -81,6 +82,7 @@ def lib():
         L.rd_schedule_upload.argtypes = [vp]
         L.rd_reduce_host.argtypes = [vp, C.POINTER(vp), vp, vp, sz, i32, i32, vp]
         L.rd_schedule_set_wait_budget.argtypes = [vp, C.c_double]
+        L.rd_schedule_set_tree_variant.argtypes = [vp, i32]
         L.rd_schedule_trace.argtypes = [vp, vp, sz]
         L.rd_schedule_faithful_shape.argtypes = [vp, C.POINTER(i32), C.POINTER(i32), C.POINTER(sz)]
         L.rd_schedule_actions.argtypes = [vp, i32, vp, sz, C.POINTER(sz), C.POINTER(i32)]
@@ -316,6 +318,10 @@ def rd_reduce_host(h, inputs, out, staging, op, stream=None):
 
 def rd_schedule_set_wait_budget(h, seconds) -> None:
     _check(lib().rd_schedule_set_wait_budget(h, float(seconds)), "rd_schedule_set_wait_budget")
+
+
+def rd_schedule_set_tree_variant(h, variant) -> None:
+    _check(lib().rd_schedule_set_tree_variant(h, int(variant)), "rd_schedule_set_tree_variant")
 
 
 def rd_schedule_trace(h) -> np.ndarray:

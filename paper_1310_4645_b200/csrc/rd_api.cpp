@@ -28,6 +28,7 @@ struct BatchLanes {
 };
 BatchLanes g_lanes[kMaxDevices];
 std::mutex g_lanes_mutex;
+constexpr int kDirectAutoProcs = 2;
 constexpr int kTailTiles = 5; // key of the tile table for the elements the 128-bit path leaves over
 
 struct DeviceTables {
@@ -77,6 +78,7 @@ struct rd_schedule {
     Schedule sched;
     Programs progs;
     double wait_budget_s = 2.0;             // bound of one wait inside the faithful kernel
+    int tree_variant = RD_TREE_AUTO;        // which tree-mode kernel serves 16-byte aligned buffers
     DeviceTables dev;
 };
 
@@ -234,8 +236,6 @@ int tiles_for(rd_schedule *s, int vec, const TileDesc **tiles, uint32_t *count)
             // not the number of elements, sets the kernel's duration; for large ones the two coincide.
             const uint64_t n = off.empty() ? 0 : off.back();
             d.stage_elems = stream_stage_elems(n / (uint64_t(d.sm_count) * 2) + 1);
-            int ctasPerSm = 1;
-            stream_shape(s->progs.stack_depth, d.smem_per_sm, d.stage_elems, &ctasPerSm, &d.stages);
             const uint32_t cap = uint32_t(d.stage_elems);
             const uint64_t n4 = n & ~uint64_t(3);          // the last n mod 4 elements go to the element kernel
             for (size_t seg = 0; seg + 1 < off.size(); seg++) {
@@ -251,6 +251,8 @@ int tiles_for(rd_schedule *s, int vec, const TileDesc **tiles, uint32_t *count)
                 }
             }
             const uint64_t nTiles = host.size();
+            int ctasPerSm = 1;
+            stream_shape(s->progs.stack_depth, d.smem_per_sm, d.stage_elems, nTiles, d.sm_count, &ctasPerSm, &d.stages);
             const uint64_t ctas = std::min<uint64_t>(uint64_t(d.sm_count) * uint64_t(ctasPerSm), std::max<uint64_t>(nTiles, 1));
             std::vector<uint32_t> first(size_t(ctas) + 1, 0);
             for (uint64_t c = 0; c < ctas; c++) first[size_t(c)] = uint32_t(nTiles * c / ctas);
@@ -329,8 +331,13 @@ int reduce_tree(rd_schedule *s, const void *const *d_inputs, void *d_out, size_t
     l.out = d_out; l.ops = d.ops; l.p = s->p; l.stack_depth = s->progs.stack_depth;
     l.dtype = int(dtype); l.op = int(op); l.sm_count = d.sm_count; l.stream = stream;
     l.cta_first = d.cta_first; l.n_ctas = d.n_ctas; l.stages = d.stages; l.stage_elems = d.stage_elems; l.status = d.status; l.device = d.device;
+    // Direct kernel: all operands of an element in registers at once.  Chosen by itself for one or two
+    // processes (measured on B200, p = 2: 6.8 TB/s against 6.1-6.2 of the streaming kernel for messages of
+    // 256 MiB and more; from three processes on the streaming kernel is level or ahead).
+    const bool direct = wide && direct_applies(s->p, s->progs.stack_depth) &&
+                        (s->tree_variant == RD_TREE_DIRECT || (s->tree_variant == RD_TREE_AUTO && s->p <= kDirectAutoProcs));
     if (stats && cudaEventRecord(d.ev_start, stream) != cudaSuccess) return RD_ERR_CUDA;
-    if ((wide ? launch_tree_stream(l) : launch_tree(l)) != 0) return RD_ERR_CUDA;
+    if ((direct ? launch_tree_direct(l) : wide ? launch_tree_stream(l) : launch_tree(l)) != 0) return RD_ERR_CUDA;
     if (nTail > 0) {
         TreeLaunch t = l;
         t.vec = 1; t.tiles = tailTiles; t.n_tiles = nTail;
@@ -713,6 +720,14 @@ int rd_schedule_set_wait_budget(rd_schedule_t *s, double seconds)
 {
     if (!s || !(seconds > 0) || !(seconds <= 60.0)) return RD_ERR_INVALID_ARG;
     s->wait_budget_s = seconds;
+    return RD_OK;
+}
+
+int rd_schedule_set_tree_variant(rd_schedule_t *s, rd_tree_variant_t variant)
+{
+    if (!s || int(variant) < RD_TREE_AUTO || int(variant) > RD_TREE_DIRECT) return RD_ERR_INVALID_ARG;
+    if (variant == RD_TREE_DIRECT && !direct_applies(s->p, s->progs.stack_depth)) return RD_ERR_UNSUPPORTED;
+    s->tree_variant = int(variant);
     return RD_OK;
 }
 

@@ -295,7 +295,7 @@ template <bool PACKED> struct StreamParams {
 };
 
 template <int DT, int OPR, bool PACKED>
-__global__ void __launch_bounds__(kStreamThreads, 2)
+__global__ void __launch_bounds__(kStreamThreads, 3)
 rd_tree_stream_kernel(const __grid_constant__ StreamParams<PACKED> a)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -442,6 +442,110 @@ rd_tree_stream_kernel(const __grid_constant__ StreamParams<PACKED> a)
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Direct variant (128-bit path, few processes).  With a handful of operands a tile is finished after a
+// handful of ring hand-offs and the ring's per-stage cost, not HBM, sets the pace.  Here a thread
+// fetches the vectors of all p operands of its elements at once, in program order, into registers
+// (P * U independent 128-bit loads in flight per thread) and then runs the program on them; the
+// partial results that have to wait (at most log2 P) sit in a register stack that is shifted on
+// push and pop, so that every register index is static.  Works on the streaming variant's tiles.
+// ---------------------------------------------------------------------------------------------
+constexpr int kDirectThreads = 256;
+
+template <int P> struct DirectShape;    // D = stack entries (log2 P), U = vectors per thread and pass, B = blocks per SM
+template <> struct DirectShape<2> { static constexpr int D = 1, U = 2, B = 4; };
+template <> struct DirectShape<4> { static constexpr int D = 2, U = 2, B = 3; };
+template <> struct DirectShape<8> { static constexpr int D = 3, U = 1, B = 4; };
+
+template <int DT, int OPR, int P>
+__global__ void __launch_bounds__(kDirectThreads, DirectShape<P>::B)
+rd_tree_direct_kernel(const __grid_constant__ TreeParams<true> a)
+{
+    constexpr int D = DirectShape<P>::D, U = DirectShape<P>::U;
+    const uint32_t tid = threadIdx.x;
+    const int p = a.p;
+    for (uint32_t tile = blockIdx.x; tile < a.n_tiles; tile += gridDim.x) {
+        const TileDesc td = a.tiles[tile];
+        const uint32_t *prog = a.ops + td.prog;
+        const uint32_t len = td.len & kLenMask;                       // padded to whole 128-bit vectors
+        const uint32_t head = (td.len >> 16) & 3u, tail = (td.len >> 18) & 3u, lastVec = len / 4u - 1u;
+        uint32_t w[P];
+#pragma unroll
+        for (int k = 0; k < P; k++) w[k] = k < p ? __ldg(prog + k) : 0u;
+        for (uint32_t v0 = 0; v0 * 4u < len; v0 += uint32_t(U) * kDirectThreads) {
+            uint32_t vec[U];
+            bool live[U];
+#pragma unroll
+            for (int u = 0; u < U; u++) { vec[u] = v0 + uint32_t(u) * kDirectThreads + tid; live[u] = vec[u] * 4u < len; }
+            Vec<4> x[P][U];
+#pragma unroll
+            for (int k = 0; k < P; k++) {
+                if (k < p) {
+                    const uint4 *src = reinterpret_cast<const uint4 *>(a.input(w[k] & kIdxMask) + td.elem_off);
+#pragma unroll
+                    for (int u = 0; u < U; u++) {
+                        uint4 r = make_uint4(0, 0, 0, 0);
+                        if (live[u]) r = __ldcs(src + vec[u]);
+                        x[k][u].w[0] = r.x; x[k][u].w[1] = r.y; x[k][u].w[2] = r.z; x[k][u].w[3] = r.w;
+                    }
+                }
+            }
+            Vec<4> top[U], st[D][U];
+#pragma unroll
+            for (int u = 0; u < U; u++) {
+#pragma unroll
+                for (int e = 0; e < 4; e++) {
+                    top[u].w[e] = 0;
+#pragma unroll
+                    for (int d = 0; d < D; d++) st[d][u].w[e] = 0;
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < P; k++) {
+                if (k < p) {
+                    const uint32_t kind = (w[k] >> kIdxBits) & 3u;
+                    if (kind == 1u) {                      // PUSH_LOAD: the stack moves down one entry
+#pragma unroll
+                        for (int u = 0; u < U; u++) {
+#pragma unroll
+                            for (int d = D - 1; d > 0; d--) st[d][u] = st[d - 1][u];
+                            st[0][u] = top[u];
+                        }
+                    }
+                    if (kind <= 1u) {
+#pragma unroll
+                        for (int u = 0; u < U; u++) top[u] = x[k][u];
+                    } else if (kind == 2u || Commutes<OPR>::value) {
+#pragma unroll
+                        for (int u = 0; u < U; u++) combine_vec<DT, OPR, 4>(top[u], top[u], x[k][u]);
+                    } else {
+#pragma unroll
+                        for (int u = 0; u < U; u++) combine_vec<DT, OPR, 4>(top[u], x[k][u], top[u]);
+                    }
+                    uint32_t npop = (w[k] >> (kIdxBits + 2)) & 0xFu;
+                    uint32_t roles = w[k] >> (kIdxBits + 6);
+                    while (npop--) {
+                        const bool poppedHeld = (roles & 1u) != 0;
+                        roles >>= 1;
+#pragma unroll
+                        for (int u = 0; u < U; u++) {
+                            const Vec<4> y = st[0][u];
+#pragma unroll
+                            for (int d = 0; d + 1 < D; d++) st[d][u] = st[d + 1][u];
+                            if (poppedHeld || Commutes<OPR>::value) combine_vec<DT, OPR, 4>(top[u], y, top[u]);
+                            else combine_vec<DT, OPR, 4>(top[u], top[u], y);
+                        }
+                    }
+                }
+            }
+            uint32_t *dst = a.out + td.elem_off;
+#pragma unroll
+            for (int u = 0; u < U; u++)
+                if (live[u]) store_part(dst + vec[u] * 4u, top[u], vec[u] == 0u ? head : 0u, vec[u] == lastVec ? tail : 0u);
+        }
+    }
+}
+
 constexpr int kU = 2;   // vectors per thread per operation
 constexpr int kK = 4;   // operations fetched ahead
 
@@ -516,6 +620,27 @@ cudaError_t launch_stream_dtop(const TreeLaunch &l)
     return l.p <= kPackedPtrs ? launch_stream<DT, OPR, true>(l) : launch_stream<DT, OPR, false>(l);
 }
 
+template <int DT, int OPR, int P>
+cudaError_t launch_direct(const TreeLaunch &l)
+{
+    TreeParams<true> prm;
+    for (int i = 0; i < kPackedPtrs; i++) prm.in.ptr[i] = i < l.p ? static_cast<const uint32_t *>(l.host_ptrs[i]) : nullptr;
+    prm.out = static_cast<uint32_t *>(l.out);
+    prm.tiles = l.tiles; prm.ops = l.ops; prm.n_tiles = l.n_tiles; prm.p = l.p;
+    uint32_t grid = uint32_t(l.sm_count) * uint32_t(DirectShape<P>::B);
+    if (grid > l.n_tiles) grid = l.n_tiles;
+    rd_tree_direct_kernel<DT, OPR, P><<<grid, kDirectThreads, 0, static_cast<cudaStream_t>(l.stream)>>>(prm);
+    return cudaGetLastError();
+}
+
+template <int DT, int OPR>
+cudaError_t launch_direct_dtop(const TreeLaunch &l)
+{
+    if (l.p <= 2) return launch_direct<DT, OPR, 2>(l);
+    if (l.p <= 4) return launch_direct<DT, OPR, 4>(l);
+    return launch_direct<DT, OPR, 8>(l);
+}
+
 }  // namespace
 
 uint32_t tree_tile_elems(int vec) { return uint32_t(kTreeThreads) * kU * uint32_t(vec); }
@@ -536,18 +661,34 @@ int stream_stage_elems(uint64_t elems_per_cta)
     return kMaxStageElems;
 }
 
-void stream_shape(int stack_depth, int smem_per_sm, int stage_elems, int *ctas_per_sm, int *stages)
+void stream_shape(int stack_depth, int smem_per_sm, int stage_elems, uint64_t n_tiles, int sm_count, int *ctas_per_sm, int *stages)
 {
     const int depth = stack_depth > 0 ? stack_depth : 1;
     const int stageBytes = stage_elems * 4;
-    // two CTAs per SM whenever each still gets three stages: measured on B200, two CTAs with 4-5 stages
-    // each (deep stacks, p = 512..1024) stream 6.6 TB/s where one CTA with 19 stages reaches 5.3
-    for (int ctas = 2; ctas >= 1; ctas--) {
-        const int budget = smem_per_sm / ctas - 2048;                 // leave room for the per-CTA reserve and statics
-        int s = (budget - depth * stack_level_bytes(stage_elems) - 512) / stageBytes;
-        if (s > kMaxStages) s = kMaxStages;
-        if (s >= 3 || ctas == 1) { *ctas_per_sm = ctas; *stages = s < 2 ? 2 : s; return; }
+    // Stages that fit when `ctas` CTAs share an SM (room left for the per-CTA reserve and statics).
+    auto fit = [&](int ctas) { return (smem_per_sm / ctas - 2048 - depth * stack_level_bytes(stage_elems) - 512) / stageBytes; };
+    // Measured on B200: with many tiles per CTA, three CTAs with 4 stages each stream 3-7 % more than two
+    // with 6 to 13 (6.8-7.0 TB/s for 3 to 256 processes); the bytes in flight are no more, the third set
+    // of consumers is what helps (three CTAs with 5 stages are behind 4, and 3 stages are too few to hide
+    // the hand-off).  With few tiles the count of tiles per CTA decides instead: every CTA of an SM gets
+    // 1 / ctas of its bandwidth, so a launch lasts about ceil(tiles / CTAs) * ctas tile times.  Three CTAs
+    // are chosen when their product is at most 8 % above that of two (512 tiles on 148 SMs: 2 * 3 against
+    // 2 * 2, two CTAs are 20 % faster; 768 tiles: 2 * 3 against 3 * 2, three are 4 % faster; 1024 tiles:
+    // 3 * 3 against 4 * 2, two are 3 % faster).  Two CTAs take all the stages that fit: a launch of one or
+    // two tiles per CTA is over sooner the more of it is in flight from the start.
+    const int s3 = fit(3), s2 = fit(2);
+    if (s3 >= 4 && s2 >= 3 && sm_count > 0) {
+        const uint64_t t = n_tiles > 0 ? n_tiles : 1;
+        const uint64_t cost3 = (t + 3u * uint64_t(sm_count) - 1) / (3u * uint64_t(sm_count)) * 3u;
+        const uint64_t cost2 = (t + 2u * uint64_t(sm_count) - 1) / (2u * uint64_t(sm_count)) * 2u;
+        if (cost3 * 100u <= cost2 * 108u) { *ctas_per_sm = 3; *stages = 4; return; }
     }
+    // Two CTAs per SM whenever each still gets three stages (deep stacks, p = 512..1024: two CTAs with
+    // 4-5 stages stream 6.6 TB/s where one CTA with 19 stages reaches 5.3).
+    if (s2 >= 3) { *ctas_per_sm = 2; *stages = s2 > kMaxStages ? kMaxStages : s2; return; }
+    const int s1 = fit(1);
+    *ctas_per_sm = 1;
+    *stages = s1 > kMaxStages ? kMaxStages : s1 < 2 ? 2 : s1;
 }
 
 namespace {
@@ -575,6 +716,10 @@ struct StreamLauncher {
     const TreeLaunch &l;
     template <int DT, int OPR> cudaError_t operator()() const { return launch_stream_dtop<DT, OPR>(l); }
 };
+struct DirectLauncher {
+    const TreeLaunch &l;
+    template <int DT, int OPR> cudaError_t operator()() const { return launch_direct_dtop<DT, OPR>(l); }
+};
 struct ElementLauncher {
     const TreeLaunch &l;
     template <int DT, int OPR> cudaError_t operator()() const { return launch_dtop<DT, OPR>(l); }
@@ -586,6 +731,18 @@ int launch_tree_stream(const TreeLaunch &l)
 {
     if (l.n_tiles == 0 || l.n_ctas == 0) return 0;
     return int(with_type_and_op(l.dtype, l.op, StreamLauncher{l}));
+}
+
+bool direct_applies(int p, int stack_depth)
+{
+    if (p > kDirectMaxProcs) return false;
+    return stack_depth <= (p <= 2 ? 1 : p <= 4 ? 2 : 3);   // DirectShape<P>::D of the instantiation that serves p
+}
+
+int launch_tree_direct(const TreeLaunch &l)
+{
+    if (l.n_tiles == 0) return 0;
+    return int(with_type_and_op(l.dtype, l.op, DirectLauncher{l}));
 }
 
 int launch_tree(const TreeLaunch &l)

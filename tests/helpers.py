@@ -83,12 +83,14 @@ M1_64 = (2e-6, 1e-10, 5e-11)
 OPS64 = {"sum": rd.RD_SUM, "max": rd.RD_MAX, "min": rd.RD_MIN, "prod": rd.RD_PROD}
 
 
-def check64(algo, port, x_dev, seg_bytes, op, exec_mode=0, rows=None, out=None):
+def check64(algo, port, x_dev, seg_bytes, op, exec_mode=0, rows=None, out=None, variant=None):
     """8-byte elements: the schedule counts in 4-byte words, the oracle in elements."""
     import torch
     p, n = x_dev.shape
     h = rd.rd_schedule_create(algo, port, p, 8 * n, seg_bytes, *M1_64)
     try:
+        if variant is not None:
+            rd.rd_schedule_set_tree_variant(h, variant)
         out = torch.full((n,), 77, dtype=x_dev.dtype, device=x_dev.device) if out is None else out
         rd.rd_reduce(h, rows if rows is not None else x_dev, out, OPS64[op], exec_mode=exec_mode, want_stats=exec_mode != rd.RD_EXEC_TREE)
         torch.cuda.synchronize()

@@ -17,10 +17,12 @@ SCHEDULES = [("uni_greedy", rd.RD_UNI_GREEDY, rd.RD_PORT_UNI), ("bi_greedy", rd.
 OPS = {"sum": rd.RD_SUM, "max": rd.RD_MAX, "min": rd.RD_MIN, "prod": rd.RD_PROD}
 
 
-def gpu_reduce(algo, port, x_dev, seg_bytes, op, model=M1, out=None, rows=None):
+def gpu_reduce(algo, port, x_dev, seg_bytes, op, model=M1, out=None, rows=None, variant=None):
     p, n = x_dev.shape
     h = rd.rd_schedule_create(algo, port, p, 4 * n, seg_bytes, *model)
     try:
+        if variant is not None:
+            rd.rd_schedule_set_tree_variant(h, variant)
         out = torch.full((n,), 77, dtype=x_dev.dtype, device=x_dev.device) if out is None else out
         rd.rd_reduce(h, rows if rows is not None else x_dev, out, OPS[op])
         torch.cuda.synchronize()
@@ -29,9 +31,9 @@ def gpu_reduce(algo, port, x_dev, seg_bytes, op, model=M1, out=None, rows=None):
     return out
 
 
-def check(algo, port, x_dev, seg_bytes, op, model=M1):
+def check(algo, port, x_dev, seg_bytes, op, model=M1, variant=None):
     p, n = x_dev.shape
-    got = gpu_reduce(algo, port, x_dev, seg_bytes, op, model).cpu().numpy()
+    got = gpu_reduce(algo, port, x_dev, seg_bytes, op, model, variant=variant).cpu().numpy()
     x = x_dev.cpu().numpy()
     ev, off, _ = oracle_schedule(algo, port, p, 4 * n, seg_bytes if seg_bytes else 4 * n, *model)
     want = O.reduce(ev, x, off, op)
@@ -46,7 +48,9 @@ SHAPES = [(8, 4096, 512), (5, 10000, 2500), (13, 3 * 2048 + 36, 2048 + 520), (64
           # segments that start and end inside a 128-bit vector (the message itself is whole vectors)
           (8, 3000, 333), (16, 4100, 4100), (13, 6180, 999), (4, 64, 3), (8, 4096, 6), (32, 8192, 2049),
           # message lengths that are not whole vectors: the last elements go through the element kernel
-          (8, 4099, 1000), (16, 2050, 2050), (5, 7, 2), (3, 3, 1), (8, 6151, 333)]
+          (8, 4099, 1000), (16, 2050, 2050), (5, 7, 2), (3, 3, 1), (8, 6151, 333),
+          # one and two processes (the direct kernel by default): ragged tiles, segments off the vector boundary
+          (2, 3 * 2048 + 36, 2048 + 520), (2, 6151, 333), (1, 4099, 1000), (2, 12288, 2048)]
 
 
 @pytest.mark.parametrize("name,algo,port", SCHEDULES)
@@ -57,6 +61,44 @@ def test_parity_small_shapes(name, algo, port, dist, op):
         if dist == "normal":
             x *= 10.0 ** torch.randint(-4, 5, x.shape, device="cuda", generator=torch.Generator("cuda").manual_seed(1))
         check(algo, port, x, 4 * seg, op)
+
+
+@pytest.mark.parametrize("name,algo,port", SCHEDULES)
+@pytest.mark.parametrize("dist,op", [("int_pm2p20", "sum"), ("normal", "sum"), ("normal", "max")])
+def test_parity_small_shapes_on_the_other_kernel(name, algo, port, dist, op):
+    """The library picks the direct kernel for one or two processes and the streaming kernel beyond (the test
+    above); here every shape goes through the kernel it would not get by itself: the streaming kernel
+    for p <= 2, the direct kernel for 3 <= p <= 8.  Same bits."""
+    for p, n, seg in SHAPES:
+        if p > 8:
+            continue
+        x = make_inputs(p, n, dist, seed=p * 1000 + n, device="cuda")
+        check(algo, port, x, 4 * seg, op, variant=rd.RD_TREE_STREAM if p <= 2 else rd.RD_TREE_DIRECT)
+
+
+def test_direct_kernel_limits():
+    """The direct kernel holds all operands of an element in registers: at most 8 processes."""
+    h = rd.rd_schedule_create(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, 9, 4096, 1024, *M1)
+    try:
+        with pytest.raises(rd.RdError) as e:
+            rd.rd_schedule_set_tree_variant(h, rd.RD_TREE_DIRECT)
+        assert e.value.status == rd.RD_ERR_UNSUPPORTED
+        with pytest.raises(rd.RdError) as e:
+            rd.rd_schedule_set_tree_variant(h, 7)
+        assert e.value.status == rd.RD_ERR_INVALID_ARG
+        rd.rd_schedule_set_tree_variant(h, rd.RD_TREE_STREAM)
+        rd.rd_schedule_set_tree_variant(h, rd.RD_TREE_AUTO)
+    finally:
+        rd.rd_destroy(h)
+    # every process count the direct kernel serves, every schedule, with both kernels on the same inputs
+    for p in range(1, 9):
+        n = 2048 * 3 + 4 * p
+        x = make_inputs(p, n, "normal", seed=p, device="cuda")
+        for name, algo, port in SCHEDULES:
+            a = gpu_reduce(algo, port, x, 4 * 1000, "sum", variant=rd.RD_TREE_DIRECT)
+            b = gpu_reduce(algo, port, x, 4 * 1000, "sum", variant=rd.RD_TREE_STREAM)
+            assert torch.equal(a.view(torch.int32), b.view(torch.int32)), (p, name)
+            check(algo, port, x, 4 * 1000, "max", variant=rd.RD_TREE_DIRECT)
 
 
 @pytest.mark.parametrize("name,algo,port", SCHEDULES)
@@ -95,6 +137,17 @@ def test_parity_eight_byte_elements(name, algo, port, kind, op):
         if kind.startswith("int64") and op in ("sum", "max", "min"):
             want = {"sum": lambda: x.sum(dim=0), "max": lambda: x.amax(dim=0), "min": lambda: x.amin(dim=0)}[op]()
             assert (got == want.cpu().numpy()).all()                   # torch's int64 sum wraps as well
+
+
+def test_eight_byte_elements_on_the_other_kernel():
+    for name, algo, port in SCHEDULES[:5]:
+        for p, n, seg in SHAPES64:
+            if p > 8:
+                continue
+            v = rd.RD_TREE_STREAM if p <= 2 else rd.RD_TREE_DIRECT
+            check64(algo, port, inputs64(p, n, "normal64", seed=p + n), 8 * seg, "sum", variant=v)
+            check64(algo, port, inputs64(p, n, "int64", seed=p + n), 8 * seg, "max", variant=v)
+            check64(algo, port, inputs64(p, n, "near_one", seed=p + n), 8 * seg, "prod", variant=v)
 
 
 def test_eight_byte_elements_butterfly_and_odd_boundaries():
