@@ -40,8 +40,8 @@ WORKLOAD_OPS = {"config1": ["sum"], "config2": ["sum"], "config3": ["sum"], "con
 # DRAM bytes per launch of the tree kernel from one ncu capture (profiles/rd_tree_stream_kernel_config2.md):
 # dram__bytes_read.sum + dram__bytes_write.sum, mean of three launches.  Reported only while the kernel
 # source is the one that was profiled.
-NCU_TRAFFIC = {"workload": "config2", "bytes_per_launch": 274.6e6,
-               "kernel_sha256": "865a1a7ce78c3d93b799005d02865c719cdfc7ea647f5cc499c8878a8889de1c"}
+NCU_TRAFFIC = {"workload": "config2", "bytes_per_launch": 274.4e6,
+               "kernel_sha256": "3c9ccb5876b0620a7fedb0db1b92334c4e5ecb8d8d94a82e4a5d52569c87360b"}
 
 
 def profiled_traffic(wname):

@@ -464,6 +464,11 @@ rd_tree_direct_kernel(const __grid_constant__ TreeParams<true> a)
     constexpr int D = DirectShape<P>::D, U = DirectShape<P>::U;
     const uint32_t tid = threadIdx.x;
     const int p = a.p;
+    // Programmatic dependent launch, as in the streaming variant: the next launch on the stream may start
+    // its blocks and read its tables while this grid runs; message data is touched only after the grid
+    // before this one has finished.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    bool waited = false;
     for (uint32_t tile = blockIdx.x; tile < a.n_tiles; tile += gridDim.x) {
         const TileDesc td = a.tiles[tile];
         const uint32_t *prog = a.ops + td.prog;
@@ -472,6 +477,7 @@ rd_tree_direct_kernel(const __grid_constant__ TreeParams<true> a)
         uint32_t w[P];
 #pragma unroll
         for (int k = 0; k < P; k++) w[k] = k < p ? __ldg(prog + k) : 0u;
+        if (!waited) { asm volatile("griddepcontrol.wait;" ::: "memory"); waited = true; }
         for (uint32_t v0 = 0; v0 * 4u < len; v0 += uint32_t(U) * kDirectThreads) {
             uint32_t vec[U];
             bool live[U];
@@ -629,8 +635,14 @@ cudaError_t launch_direct(const TreeLaunch &l)
     prm.tiles = l.tiles; prm.ops = l.ops; prm.n_tiles = l.n_tiles; prm.p = l.p;
     uint32_t grid = uint32_t(l.sm_count) * uint32_t(DirectShape<P>::B);
     if (grid > l.n_tiles) grid = l.n_tiles;
-    rd_tree_direct_kernel<DT, OPR, P><<<grid, kDirectThreads, 0, static_cast<cudaStream_t>(l.stream)>>>(prm);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kDirectThreads); cfg.dynamicSmemBytes = 0;
+    cfg.stream = static_cast<cudaStream_t>(l.stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, rd_tree_direct_kernel<DT, OPR, P>, prm);
 }
 
 template <int DT, int OPR>
