@@ -471,6 +471,7 @@ def main():
             cpu = {"value": v, "unit": "GB/s", "cores": 1, "kind": "oracle",
                    "sample": "%d passes over every schedule x op on %d of %d elements per process (%.1f s)"
                              % (passes, n_s, n, dt)}
+        shape0 = rd.rd_schedule_tree_shape(plans[0][1])
         line = {
             "metric": "reduction_throughput", "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
@@ -484,7 +485,10 @@ def main():
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": profiled_traffic(wname), "traffic_unit": "bytes per launch", "algorithmic_bytes": bytes_per_reduce,
-                         "peak_source": peak_src, "kernel": "rd_tree_stream_kernel",
+                         "peak_source": peak_src,
+                         "kernel": "rd_tree_direct_kernel" if shape0["variant"] == rd.RD_TREE_DIRECT else "rd_tree_stream_kernel",
+                         "launch_shape": {"blocks_per_sm": shape0["blocks_per_sm"], "ring_stages": shape0["ring_stages"],
+                                          "tiles": shape0["n_tiles"]},
                          "timed_over": "%d launches back to back on one stream, %.2f us each" % (k_steps * launches_per_step, kernel_ms_per_launch * 1e3),
                          "frac_of_nominal_8000": achieved / 8000.0},
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": args.steps * launches_per_step, "clocks": clocks,

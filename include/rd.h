@@ -282,6 +282,15 @@ typedef enum { RD_TREE_AUTO = 0, RD_TREE_STREAM = 1, RD_TREE_DIRECT = 2 } rd_tre
 RD_API int rd_schedule_set_tree_variant(rd_schedule_t *s, rd_tree_variant_t variant);
 
 /*
+ * rd_schedule_tree_shape -- how a tree-mode call with 16-byte aligned buffers will run this schedule on
+ * the current device (the paper has no counterpart): the kernel (RD_TREE_STREAM or RD_TREE_DIRECT), its
+ * thread blocks per SM, the stages of the streaming kernel's shared-memory ring (0 for the direct kernel)
+ * and the number of tiles the message is cut into (runs of at most 2048 4-byte words inside one segment).
+ * Uploads the schedule's tables if they are not on the device yet.  Any output pointer may be NULL.
+ */
+RD_API int rd_schedule_tree_shape(rd_schedule_t *s, int *variant, int *blocks_per_sm, int *ring_stages, size_t *n_tiles);
+
+/*
  * rd_schedule_trace -- measured times of the last schedule-faithful rd_reduce, to set against
  * the model's alpha + beta*s (+ gamma*s) per pair (Section V).  For every send/receive pair, in
  * the order of rd_schedule_events, three values in nanoseconds of the GPU's global timer, taken by

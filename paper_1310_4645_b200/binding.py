@@ -31,7 +31,7 @@ EXPORTS = ("rd_schedule_create", "rd_schedule_create_segments", "rd_optimal_segm
            "rd_schedule_events", "rd_schedule_segments", "rd_schedule_program", "rd_reduce",
            "rd_schedule_upload", "rd_reduce_host", "rd_destroy", "rd_strerror", "rd_schedule_set_wait_budget",
            "rd_schedule_trace", "rd_schedule_faithful_shape", "rd_schedule_actions", "rd_reduce_faithful_static", "rd_search_segmentation", "rd_schedule_status",
-           "rd_reduce_batch", "rd_schedule_set_tree_variant")
+           "rd_reduce_batch", "rd_schedule_set_tree_variant", "rd_schedule_tree_shape")
 
 
 class rd_model_t(C.Structure):
@@ -83,6 +83,7 @@ def lib():
         L.rd_reduce_host.argtypes = [vp, C.POINTER(vp), vp, vp, sz, i32, i32, vp]
         L.rd_schedule_set_wait_budget.argtypes = [vp, C.c_double]
         L.rd_schedule_set_tree_variant.argtypes = [vp, i32]
+        L.rd_schedule_tree_shape.argtypes = [vp, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32), C.POINTER(sz)]
         L.rd_schedule_trace.argtypes = [vp, vp, sz]
         L.rd_schedule_faithful_shape.argtypes = [vp, C.POINTER(i32), C.POINTER(i32), C.POINTER(sz)]
         L.rd_schedule_actions.argtypes = [vp, i32, vp, sz, C.POINTER(sz), C.POINTER(i32)]
@@ -322,6 +323,12 @@ def rd_schedule_set_wait_budget(h, seconds) -> None:
 
 def rd_schedule_set_tree_variant(h, variant) -> None:
     _check(lib().rd_schedule_set_tree_variant(h, int(variant)), "rd_schedule_set_tree_variant")
+
+
+def rd_schedule_tree_shape(h) -> dict:
+    v, b, r, t = C.c_int(), C.c_int(), C.c_int(), C.c_size_t()
+    _check(lib().rd_schedule_tree_shape(h, C.byref(v), C.byref(b), C.byref(r), C.byref(t)), "rd_schedule_tree_shape")
+    return dict(variant=v.value, blocks_per_sm=b.value, ring_stages=r.value, n_tiles=t.value)
 
 
 def rd_schedule_trace(h) -> np.ndarray:

@@ -40,6 +40,7 @@ struct DeviceTables {
     // streaming (128-bit) path: tiles grouped per CTA, every CTA the same number of elements
     uint32_t *cta_first = nullptr;
     uint32_t n_ctas = 0;
+    int ctas_per_sm = 0;
     int stages = 0;
     int stage_elems = 0;
     int *status = nullptr;                                  // device word written by a kernel that gave up a wait
@@ -263,6 +264,7 @@ int tiles_for(rd_schedule *s, int vec, const TileDesc **tiles, uint32_t *count)
             if (cudaMemcpy(d.cta_first, first.data(), first.size() * sizeof(uint32_t), cudaMemcpyHostToDevice) != cudaSuccess)
                 return RD_ERR_CUDA;
             d.n_ctas = uint32_t(ctas);
+            d.ctas_per_sm = ctasPerSm;
         } else {
             // element path: the whole message (vec == 1), or only what the 128-bit path leaves over (kTailTiles)
             const uint64_t n = off.empty() ? 0 : off.back();
@@ -756,6 +758,23 @@ int rd_schedule_faithful_shape(rd_schedule_t *s, int *blocks_per_process, int *s
         if (blocks_per_process) *blocks_per_process = s->dev.f_lanes;
         if (slots_per_process) *slots_per_process = s->dev.f_slots;
         if (scratch_bytes) *scratch_bytes = size_t(s->p) * size_t(s->dev.f_slots) * size_t(s->dev.f_slot_elems) * 4;
+        return int(RD_OK);
+    });
+}
+
+int rd_schedule_tree_shape(rd_schedule_t *s, int *variant, int *blocks_per_sm, int *ring_stages, size_t *n_tiles)
+{
+    if (!s) return RD_ERR_INVALID_ARG;
+    return guarded([&] {
+        if (int rc = upload(s)) return rc;
+        TreeLaunch l{};
+        if (int rc = tiles_for(s, 4, &l.tiles, &l.n_tiles)) return rc;
+        const bool direct = direct_applies(s->p, s->progs.stack_depth) &&
+                            (s->tree_variant == RD_TREE_DIRECT || (s->tree_variant == RD_TREE_AUTO && s->p <= kDirectAutoProcs));
+        if (variant) *variant = direct ? RD_TREE_DIRECT : RD_TREE_STREAM;
+        if (blocks_per_sm) *blocks_per_sm = direct ? direct_blocks_per_sm(s->p) : s->dev.ctas_per_sm;
+        if (ring_stages) *ring_stages = direct ? 0 : s->dev.stages;
+        if (n_tiles) *n_tiles = l.n_tiles;
         return int(RD_OK);
     });
 }

@@ -751,6 +751,8 @@ bool direct_applies(int p, int stack_depth)
     return stack_depth <= (p <= 2 ? 1 : p <= 4 ? 2 : 3);   // DirectShape<P>::D of the instantiation that serves p
 }
 
+int direct_blocks_per_sm(int p) { return p <= 2 ? DirectShape<2>::B : p <= 4 ? DirectShape<4>::B : DirectShape<8>::B; }
+
 int launch_tree_direct(const TreeLaunch &l)
 {
     if (l.n_tiles == 0) return 0;

@@ -53,6 +53,7 @@ int launch_tree_stream(const TreeLaunch &a);
 // are fetched into registers at once.  Uses the streaming variant's tiles.
 constexpr int kDirectMaxProcs = 8;
 bool direct_applies(int p, int stack_depth);
+int direct_blocks_per_sm(int p);
 int launch_tree_direct(const TreeLaunch &a);
 
 // ---- schedule-faithful execution (rd_faithful.cu)

@@ -158,3 +158,22 @@ def test_batch_argument_checks_come_before_any_cuda_call():
         assert call([rows(0x100000)], [0x300000], n=1000) == rd.RD_ERR_SIZE_MISMATCH
     finally:
         rd.rd_destroy(h)
+
+
+def test_tree_variant_is_checked_on_the_host():
+    """Choosing the tree-mode kernel is host work: the direct kernel exists for at most 8 processes."""
+    for p, direct_ok in ((1, True), (2, True), (8, True), (9, False), (64, False)):
+        h = rd.rd_schedule_create(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, p, 4096, 1024, *MODEL)
+        try:
+            rd.rd_schedule_set_tree_variant(h, rd.RD_TREE_STREAM)
+            rd.rd_schedule_set_tree_variant(h, rd.RD_TREE_AUTO)
+            if direct_ok:
+                rd.rd_schedule_set_tree_variant(h, rd.RD_TREE_DIRECT)
+            else:
+                assert status_of(rd.rd_schedule_set_tree_variant, h, rd.RD_TREE_DIRECT) == rd.RD_ERR_UNSUPPORTED
+            assert status_of(rd.rd_schedule_set_tree_variant, h, 3) == rd.RD_ERR_INVALID_ARG
+            assert status_of(rd.rd_schedule_set_tree_variant, h, -1) == rd.RD_ERR_INVALID_ARG
+        finally:
+            rd.rd_destroy(h)
+    assert rd.lib().rd_schedule_set_tree_variant(None, rd.RD_TREE_AUTO) == rd.RD_ERR_INVALID_ARG
+    assert rd.lib().rd_schedule_tree_shape(None, None, None, None, None) == rd.RD_ERR_INVALID_ARG

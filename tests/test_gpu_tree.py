@@ -76,6 +76,31 @@ def test_parity_small_shapes_on_the_other_kernel(name, algo, port, dist, op):
         check(algo, port, x, 4 * seg, op, variant=rd.RD_TREE_STREAM if p <= 2 else rd.RD_TREE_DIRECT)
 
 
+def test_launch_shapes_two_and_three_blocks_per_sm():
+    """The streaming kernel runs two or three thread blocks per SM depending on the number of tiles and on
+    the stack depth; the direct kernel serves one or two processes.  Every shape, element by element."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    seen = set()
+    # (p, n, segment elements, schedule): few tiles; between two and three blocks' worth of tiles; many tiles
+    # with ragged segments; a deep stack (binomial, p = 128) with many tiles; one or two processes
+    cases = [(5, 2048 * 40 + 36, 2048 + 520, SCHEDULES[0]), (5, 2048 * (2 * sms + 40) + 36, 4096, SCHEDULES[3]),
+             (9, 2048 * 7 * sms + 100, 3 * 2048 + 520, SCHEDULES[0]), (128, 2048 * 5 * sms, 4096, SCHEDULES[2]),
+             (2, 2048 * 9 * sms + 8, 2048 + 520, SCHEDULES[1]), (1, 2048 * 3 + 4, 1000, SCHEDULES[3])]
+    for p, n, seg, (name, algo, port) in cases:
+        x = make_inputs(p, n, "normal", seed=p + n, device="cuda")
+        h = rd.rd_schedule_create(algo, port, p, 4 * n, 4 * seg, *M1)
+        try:
+            shape = rd.rd_schedule_tree_shape(h)
+        finally:
+            rd.rd_destroy(h)
+        seen.add((shape["variant"], shape["blocks_per_sm"]))
+        assert shape["n_tiles"] >= n // 2048
+        assert (shape["variant"] == rd.RD_TREE_DIRECT) == (p <= 2)
+        assert shape["ring_stages"] >= 3 or shape["variant"] == rd.RD_TREE_DIRECT
+        check(algo, port, x, 4 * seg, "sum")
+    assert (rd.RD_TREE_STREAM, 2) in seen and (rd.RD_TREE_STREAM, 3) in seen and (rd.RD_TREE_DIRECT, 4) in seen
+
+
 def test_direct_kernel_limits():
     """The direct kernel holds all operands of an element in registers: at most 8 processes."""
     h = rd.rd_schedule_create(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, 9, 4096, 1024, *M1)
