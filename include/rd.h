@@ -230,17 +230,24 @@ RD_API int rd_reduce(rd_schedule_t *s, const void *const *d_inputs, void *d_out,
  * rd_reduce_batch -- several independent tree-mode reductions issued together (the paper has no
  * counterpart; Section VII runs the same messages under every schedule, and a library user reduces
  * many buffers).  Job j reduces d_inputs[j][0..p_j) into d_outs[j] under schedules[j]; all jobs share
- * dtype, op and stream.  Results are exactly those of n_jobs rd_reduce calls.  Because the jobs are
- * independent, the library issues them alternately on two streams of its own, so that one job's
- * thread blocks take the SM slots another job frees while its last blocks are still running; the
- * batch as a whole is ordered after what precedes it on cuda_stream and before what follows it
- * (event fork and join).  The two side streams and three events are created on a device's first
- * batch and kept.
+ * dtype, op and stream.  Results are exactly those of n_jobs rd_reduce calls, and the batch as a whole
+ * is ordered after what precedes it on cuda_stream and before what follows it.
+ *   When every buffer of every job is 16-byte aligned and every message a whole number of 128-bit
+ *   vectors, the batch is ONE launch of the streaming kernel: the tiles of all jobs are dealt to the
+ *   thread blocks as if they were one reduction, so the batch pays one launch, one ring fill and one
+ *   tail instead of n_jobs (16 jobs of p = 64 with 1 MiB messages: 6.3 TB/s against 3.5 TB/s for 16
+ *   calls; 32 jobs with 256 KiB messages: 5.4 against 1.1 TB/s).  Job descriptors, tile ranges and the
+ *   jobs' input pointers reach the device in one small copy from a pinned ring that a device's first
+ *   such batch allocates (it grows when a batch needs more); a bounded wait that gives up is reported
+ *   through rd_schedule_status of the first job's schedule.
+ *   Otherwise the jobs are issued alternately on two streams of the library's own, so that one job's
+ *   thread blocks take the SM slots another job frees while its last blocks are still running (event
+ *   fork and join around them; streams and events are created on a device's first such batch and kept).
  *   schedules, d_inputs, d_outs, n_elems   HOST arrays of n_jobs entries (d_inputs[j]: HOST array of
  *             DEVICE pointers as in rd_reduce).  The same schedule may serve several jobs.
  * RD_ERR_INVALID_ARG when a job's output overlaps another job's output or inputs (a job's output may
  * alias its own root input); otherwise the errors of rd_reduce.  On an error jobs before the failing
- * one have been launched.
+ * one may have been launched.
  */
 RD_API int rd_reduce_batch(size_t n_jobs, rd_schedule_t *const *schedules, const void *const *const *d_inputs,
                     void *const *d_outs, const size_t *n_elems, rd_dtype_t dtype, rd_op_t op, void *cuda_stream);

@@ -21,10 +21,18 @@ constexpr int kPtrRing = 8;   // pointer tables in flight for p > kPackedPtrs
 constexpr int kMaxDevices = 64;
 
 // Side streams of rd_reduce_batch, created on a device's first batch and kept for the process's life.
+constexpr int kBatchRing = 4; // per-call tables of fused batches in flight
 struct BatchLanes {
     bool ready = false;
     cudaStream_t stream[2] = {nullptr, nullptr};
     cudaEvent_t fork = nullptr, join[2] = {nullptr, nullptr};
+    // fused batches: a pinned host ring and a device ring for the per-call tables (job descriptors,
+    // per-CTA tile ranges, input pointer tables), one event per slot
+    unsigned char *h_tab = nullptr, *d_tab = nullptr;
+    size_t slot_bytes = 0;
+    cudaEvent_t tab_done[kBatchRing] = {};
+    bool tab_used[kBatchRing] = {};
+    int tab_next = 0;
 };
 BatchLanes g_lanes[kMaxDevices];
 std::mutex g_lanes_mutex;
@@ -500,6 +508,101 @@ int reduce_faithful(rd_schedule *s, const void *const *d_inputs, void *d_out, si
     return RD_OK;
 }
 
+// A batch as ONE launch of the streaming kernel: the tiles of all jobs are numbered through and dealt
+// to the thread blocks like the tiles of a single reduction, so the launch has one fill and one tail and
+// the ring shape is chosen for the batch's total number of tiles.  The job descriptors and the jobs' input
+// pointers travel as kernel parameters when they fit, else in one copy from a pinned ring.
+int reduce_batch_fused(size_t n_jobs, rd_schedule_t *const *schedules, const void *const *const *d_inputs, void *const *d_outs,
+                       rd_dtype_t dtype, rd_op_t op, cudaStream_t user)
+{
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kMaxDevices) return RD_ERR_CUDA;
+    std::vector<BatchJob> jobs(n_jobs);
+    uint64_t total = 0;
+    size_t nPtrs = 0;
+    int depth = 0;
+    for (size_t j = 0; j < n_jobs; j++) {
+        rd_schedule *s = schedules[j];
+        const TileDesc *tiles = nullptr;
+        uint32_t count = 0;
+        if (int rc = tiles_for(s, 4, &tiles, &count)) return rc;
+        BatchJob &b = jobs[j];
+        b.inputs = nullptr; b.out = static_cast<uint32_t *>(d_outs[j]); b.tiles = tiles; b.ops = s->dev.ops;
+        b.tile_begin = uint32_t(total); b.p = s->p; b.ptr_base = 0;
+        total += count;
+        if (total > 0xFFFFFFFFull) return RD_ERR_UNSUPPORTED;
+        b.tile_end = uint32_t(total);
+        nPtrs += size_t(s->p);
+        depth = std::max(depth, s->progs.stack_depth);
+    }
+    if (total == 0) return RD_OK;
+    DeviceTables &d0 = schedules[0]->dev;
+    const int stageElems = d0.stage_elems;
+    int ctasPerSm = 1, stages = 2;
+    stream_shape(depth, d0.smem_per_sm, stageElems, total, d0.sm_count, &ctasPerSm, &stages);
+    const uint64_t ctas = std::min<uint64_t>(uint64_t(d0.sm_count) * uint64_t(ctasPerSm), total);
+    BatchLaunch b{};
+    b.n_jobs = uint32_t(n_jobs); b.n_tiles = uint32_t(total); b.n_ctas = uint32_t(ctas);
+    b.stages = stages; b.stack_depth = depth; b.stage_elems = stageElems;
+    b.dtype = int(dtype); b.op = int(op); b.device = device; b.status = d0.status; b.stream = user;
+    if (n_jobs <= size_t(kBatchPackJobs) && nPtrs <= size_t(kBatchPackPtrs)) {
+        // small batch: descriptors and pointers travel as kernel parameters, nothing is copied ahead of the launch
+        std::vector<const void *> ptrs(nPtrs);
+        size_t at = 0;
+        for (size_t j = 0; j < n_jobs; j++) {
+            jobs[j].ptr_base = int(at);
+            for (int i = 0; i < schedules[j]->p; i++) ptrs[at++] = d_inputs[j][i];
+        }
+        b.host_jobs = jobs.data(); b.host_ptrs = ptrs.data(); b.n_ptrs = uint32_t(nPtrs);
+        return launch_tree_stream_batch(b) == 0 ? RD_OK : RD_ERR_CUDA;
+    }
+    // layout of a slot of the ring: job descriptors | input pointers of all jobs
+    const size_t oPtrs = (n_jobs * sizeof(BatchJob) + 15) & ~size_t(15);
+    const size_t need = oPtrs + nPtrs * sizeof(void *);
+
+    std::lock_guard<std::mutex> hold(g_lanes_mutex);
+    BatchLanes &lanes = g_lanes[device];
+    if (need > lanes.slot_bytes) {
+        // grow: wait for the launches that still read the old ring, then replace it
+        for (int k = 0; k < kBatchRing; k++)
+            if (lanes.tab_used[k] && cudaEventSynchronize(lanes.tab_done[k]) != cudaSuccess) return RD_ERR_CUDA;
+        if (lanes.h_tab) cudaFreeHost(lanes.h_tab);
+        cudaFree(lanes.d_tab);
+        lanes.h_tab = lanes.d_tab = nullptr;
+        lanes.slot_bytes = 0;
+        size_t slot = 64 << 10;
+        while (slot < need) slot *= 2;
+        if (cudaHostAlloc(reinterpret_cast<void **>(&lanes.h_tab), slot * kBatchRing, cudaHostAllocDefault) != cudaSuccess) return RD_ERR_NOMEM;
+        if (cudaMalloc(reinterpret_cast<void **>(&lanes.d_tab), slot * kBatchRing) != cudaSuccess) {
+            cudaFreeHost(lanes.h_tab);
+            lanes.h_tab = nullptr;
+            return RD_ERR_NOMEM;
+        }
+        for (int k = 0; k < kBatchRing; k++) {
+            if (!lanes.tab_done[k] && cudaEventCreateWithFlags(&lanes.tab_done[k], cudaEventDisableTiming) != cudaSuccess) return RD_ERR_CUDA;
+            lanes.tab_used[k] = false;
+        }
+        lanes.slot_bytes = slot;
+    }
+    const int slot = lanes.tab_next;
+    lanes.tab_next = (lanes.tab_next + 1) % kBatchRing;
+    if (lanes.tab_used[slot] && cudaEventSynchronize(lanes.tab_done[slot]) != cudaSuccess) return RD_ERR_CUDA;   // the slot's previous launch
+    unsigned char *h = lanes.h_tab + size_t(slot) * lanes.slot_bytes, *dv = lanes.d_tab + size_t(slot) * lanes.slot_bytes;
+    const void **hp = reinterpret_cast<const void **>(h + oPtrs);
+    size_t at = 0;
+    for (size_t j = 0; j < n_jobs; j++) {
+        jobs[j].inputs = reinterpret_cast<const uint32_t *const *>(dv + oPtrs) + at;
+        for (int i = 0; i < schedules[j]->p; i++) hp[at++] = d_inputs[j][i];
+    }
+    std::memcpy(h, jobs.data(), n_jobs * sizeof(BatchJob));
+    if (cudaMemcpyAsync(dv, h, need, cudaMemcpyHostToDevice, user) != cudaSuccess) return RD_ERR_CUDA;
+    b.jobs = reinterpret_cast<const BatchJob *>(dv);
+    const int launched = launch_tree_stream_batch(b);
+    lanes.tab_used[slot] = cudaEventRecord(lanes.tab_done[slot], user) == cudaSuccess;
+    if (launched != 0 || !lanes.tab_used[slot]) return RD_ERR_CUDA;
+    return RD_OK;
+}
+
 // Nothing may be thrown across the C boundary: host containers can run out of memory.
 template <typename F> int guarded(F &&body)
 {
@@ -665,6 +768,17 @@ int rd_reduce_batch(size_t n_jobs, rd_schedule_t *const *schedules, const void *
         for (size_t j = 0; j < n_jobs; j++)
             if (int rc = upload(schedules[j])) return rc;
         if (n_jobs == 1) return reduce_tree(schedules[0], d_inputs[0], d_outs[0], words[0], dtype, op, user, nullptr);
+        // One launch for the whole batch when every job can take the 128-bit streaming path by itself
+        // (all buffers 16-byte aligned, whole vectors).
+        bool fuse = true;
+        for (size_t j = 0; j < n_jobs && fuse; j++) {
+            fuse = (words[j] & 3u) == 0 && (reinterpret_cast<uintptr_t>(d_outs[j]) & 15u) == 0;
+            for (int i = 0; i < schedules[j]->p && fuse; i++) fuse = (reinterpret_cast<uintptr_t>(d_inputs[j][i]) & 15u) == 0;
+        }
+        if (fuse) {
+            const int rc = reduce_batch_fused(n_jobs, schedules, d_inputs, d_outs, dtype, op, user);
+            if (rc != RD_ERR_UNSUPPORTED) return rc;        // UNSUPPORTED: more tiles than one launch numbers
+        }
         // Fork: two side streams wait for what precedes the batch on the caller's stream and take the
         // jobs alternately, so that one job's thread blocks fill the SM slots the other job frees while
         // its last blocks are still running.  Join: the caller's stream waits for both.

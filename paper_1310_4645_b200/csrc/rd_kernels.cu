@@ -287,17 +287,100 @@ __device__ __forceinline__ void store_part(uint32_t *p, const Vec<4> &v, uint32_
         if (e >= skip_head && e < 4u - skip_tail) __stcs(p + e, v.w[e]);
 }
 
+// What a launch works on is reached through a "jobs" view: one reduction (the view is the kernel's
+// parameters and costs nothing), or several independent reductions fused into one launch (the tiles
+// of all jobs are numbered through; the view keeps the descriptor of the job its tile belongs to).
+template <bool PACKED> struct OneJob;
+template <bool PACKED> struct ManyJobs;
+
 template <bool PACKED> struct StreamParams {
+    using Jobs = OneJob<PACKED>;
     TreeParams<PACKED> t;
     const uint32_t *cta_first;   // per CTA: first tile; n_ctas + 1 entries
     int *status;                 // device word: 0, or the first error code
     int stages, depth, stage_elems;
+    __device__ __forceinline__ void tile_range(uint32_t cta, uint32_t &t0, uint32_t &t1) const { t0 = cta_first[cta]; t1 = cta_first[cta + 1]; }
 };
 
-template <int DT, int OPR, bool PACKED>
+// A batch: job descriptors and input pointers either inside the kernel's parameters (small batches: nothing
+// has to be copied to the device before the launch) or in device memory.  CTA c of n takes the tiles
+// [T c / n, T (c + 1) / n) of the batch's T tiles.
+template <bool PACKED> struct BatchStreamParams;
+template <> struct BatchStreamParams<true> {
+    using Jobs = ManyJobs<true>;
+    BatchJob jobs[kBatchPackJobs];
+    const uint32_t *ptrs[kBatchPackPtrs];
+    uint32_t n_jobs, n_tiles;
+    int *status;
+    int stages, depth, stage_elems;
+    __device__ __forceinline__ BatchJob job(uint32_t j) const { return jobs[j]; }
+    __device__ __forceinline__ uint32_t job_end(uint32_t j) const { return jobs[j].tile_end; }
+    __device__ __forceinline__ const uint32_t *input(const BatchJob &b, uint32_t i) const { return ptrs[uint32_t(b.ptr_base) + i]; }
+    __device__ __forceinline__ void tile_range(uint32_t cta, uint32_t &t0, uint32_t &t1) const
+    {
+        t0 = uint32_t(uint64_t(n_tiles) * cta / gridDim.x); t1 = uint32_t(uint64_t(n_tiles) * (cta + 1u) / gridDim.x);
+    }
+};
+template <> struct BatchStreamParams<false> {
+    using Jobs = ManyJobs<false>;
+    const BatchJob *jobs;        // device; n_jobs descriptors, tile ranges ascending
+    uint32_t n_jobs, n_tiles;
+    int *status;
+    int stages, depth, stage_elems;
+    __device__ __forceinline__ BatchJob job(uint32_t j) const { return jobs[j]; }
+    __device__ __forceinline__ uint32_t job_end(uint32_t j) const { return jobs[j].tile_end; }
+    __device__ __forceinline__ const uint32_t *input(const BatchJob &b, uint32_t i) const
+    {
+        return reinterpret_cast<const uint32_t *>(__ldg(reinterpret_cast<const unsigned long long *>(b.inputs) + i));
+    }
+    __device__ __forceinline__ void tile_range(uint32_t cta, uint32_t &t0, uint32_t &t1) const
+    {
+        t0 = uint32_t(uint64_t(n_tiles) * cta / gridDim.x); t1 = uint32_t(uint64_t(n_tiles) * (cta + 1u) / gridDim.x);
+    }
+};
+
+template <bool PACKED> struct OneJob {
+    const TreeParams<PACKED> &t;
+    __device__ __forceinline__ OneJob(const StreamParams<PACKED> &a, uint32_t, bool) : t(a.t) {}
+    __device__ __forceinline__ void seek(uint32_t) {}
+    __device__ __forceinline__ TileDesc tile(uint32_t g) const { return t.tiles[g]; }
+    __device__ __forceinline__ const uint32_t *ops() const { return t.ops; }
+    __device__ __forceinline__ const uint32_t *input(uint32_t i) const { return t.input(i); }
+    __device__ __forceinline__ uint32_t *out() const { return t.out; }
+    __device__ __forceinline__ int p() const { return t.p; }
+};
+
+template <bool PACKED> struct ManyJobs {
+    const BatchStreamParams<PACKED> &a;
+    BatchJob cur;
+    uint32_t j;
+    // Positioned on the job of tile g (the first job whose range ends after g) when `any` is set.
+    __device__ __forceinline__ ManyJobs(const BatchStreamParams<PACKED> &prm, uint32_t g, bool any) : a(prm), j(0)
+    {
+        cur = BatchJob{nullptr, nullptr, nullptr, nullptr, 0u, 0u, 1, 0};
+        if (!any) return;
+        uint32_t lo = 0, hi = a.n_jobs - 1u;
+        while (lo < hi) {
+            const uint32_t mid = (lo + hi) / 2u;
+            if (g >= a.job_end(mid)) lo = mid + 1u; else hi = mid;
+        }
+        j = lo;
+        cur = a.job(j);
+    }
+    // Tiles are visited in ascending order, so the job only ever moves forward.
+    __device__ __forceinline__ void seek(uint32_t g) { while (g >= cur.tile_end) cur = a.job(++j); }
+    __device__ __forceinline__ TileDesc tile(uint32_t g) const { return cur.tiles[g - cur.tile_begin]; }
+    __device__ __forceinline__ const uint32_t *ops() const { return cur.ops; }
+    __device__ __forceinline__ const uint32_t *input(uint32_t i) const { return a.input(cur, i); }
+    __device__ __forceinline__ uint32_t *out() const { return cur.out; }
+    __device__ __forceinline__ int p() const { return cur.p; }
+};
+
+template <int DT, int OPR, typename PRM>
 __global__ void __launch_bounds__(kStreamThreads, 3)
-rd_tree_stream_kernel(const __grid_constant__ StreamParams<PACKED> a)
+rd_tree_stream_kernel(const __grid_constant__ PRM a)
 {
+    using Jobs = typename PRM::Jobs;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int S = a.stages;
     const uint32_t stageVecs = uint32_t(a.stage_elems) / 4u;                                 // 128-bit vectors per stage
@@ -309,8 +392,8 @@ rd_tree_stream_kernel(const __grid_constant__ StreamParams<PACKED> a)
     uint64_t *empty = full + S;
     __shared__ int abort_flag;
     const uint32_t tid = threadIdx.x;
-    const int p = a.t.p;
-    const uint32_t tile0 = a.cta_first[blockIdx.x], tile1 = a.cta_first[blockIdx.x + 1];
+    uint32_t tile0, tile1;
+    a.tile_range(blockIdx.x, tile0, tile1);
 
     if (tid == 0) {
         abort_flag = 0;
@@ -335,9 +418,14 @@ rd_tree_stream_kernel(const __grid_constant__ StreamParams<PACKED> a)
         const int P = kProducers < S ? kProducers : S;
         const int j = int(tid - kConsumers) / 32;
         if (j >= P) return;
+        Jobs jobs(a, tile0, tile0 < tile1);
         uint32_t tile = tile0;
         int i = j;
-        while (i >= p && tile < tile1) { i -= p; tile++; }
+        int p = jobs.p();                       // of the job `tile` belongs to
+        while (tile < tile1 && i >= p) {
+            i -= p; tile++;
+            if (tile < tile1) { jobs.seek(tile); p = jobs.p(); }
+        }
         int stage = j % S;
         uint32_t laps = 0;                      // times this producer has gone round the ring
         uint32_t cur = 0xFFFFFFFFu;
@@ -346,14 +434,17 @@ rd_tree_stream_kernel(const __grid_constant__ StreamParams<PACKED> a)
         int lastStage = 0;
         uint32_t lastLap = 0;
         while (tile < tile1) {
-            if (tile != cur) { td = a.t.tiles[tile]; cur = tile; }
-            const uint32_t *src = a.t.input(__ldg(a.t.ops + td.prog + i) & kIdxMask) + td.elem_off;
+            if (tile != cur) { td = jobs.tile(tile); cur = tile; }
+            const uint32_t *src = jobs.input(__ldg(jobs.ops() + td.prog + i) & kIdxMask) + td.elem_off;
             if (laps >= 1u && !mbar_wait(empty + stage, (laps - 1u) & 1u, &abort_flag)) { ok = false; break; }
             mbar_expect_tx(full + stage, (td.len & kLenMask) * 4u);
             bulk_load(ring + size_t(stage) * stageVecs, src, (td.len & kLenMask) * 4u, full + stage);
             any = true; lastStage = stage; lastLap = laps;
             i += P;
-            while (i >= p && tile < tile1) { i -= p; tile++; }
+            while (tile < tile1 && i >= p) {
+                i -= p; tile++;
+                if (tile < tile1) { jobs.seek(tile); p = jobs.p(); }
+            }
             stage += P;
             if (stage >= S) { stage -= S; laps++; }
         }
@@ -372,9 +463,12 @@ rd_tree_stream_kernel(const __grid_constant__ StreamParams<PACKED> a)
     const uint32_t lane = tid & 31u;
     int stage = 0;
     uint32_t phase = 0;
+    Jobs jobs(a, tile0, tile0 < tile1);
     for (uint32_t tile = tile0; tile < tile1; tile++) {
-        const TileDesc td = a.t.tiles[tile];
-        const uint32_t *prog = a.t.ops + td.prog;
+        jobs.seek(tile);
+        const int p = jobs.p();
+        const TileDesc td = jobs.tile(tile);
+        const uint32_t *prog = jobs.ops() + td.prog;
         const uint32_t len = td.len & kLenMask;                       // padded to whole 128-bit vectors
         const bool live0 = tid * 4u < len, live1 = (kConsumers + tid) * 4u < len;
         Vec<4> top0, top1;
@@ -435,7 +529,7 @@ rd_tree_stream_kernel(const __grid_constant__ StreamParams<PACKED> a)
         }
         // A segment may begin or end inside a vector: the tile then starts / ends with a vector whose other
         // elements belong to the neighbouring segment (another tile writes those); only this tile's are stored.
-        uint32_t *dst = a.t.out + td.elem_off;
+        uint32_t *dst = jobs.out() + td.elem_off;
         const uint32_t head = (td.len >> 16) & 3u, tail = (td.len >> 18) & 3u, lastVec = len / 4u - 1u;
         if (live0) store_part(dst + tid * 4u, top0, tid == 0 ? head : 0u, tid == lastVec ? tail : 0u);
         if (live1) store_part(dst + (kConsumers + tid) * 4u, top1, 0u, kConsumers + tid == lastVec ? tail : 0u);
@@ -588,6 +682,30 @@ cudaError_t launch_dtop(const TreeLaunch &l)
     return l.p <= kPackedPtrs ? launch_one<DT, OPR, V, true>(l) : launch_one<DT, OPR, V, false>(l);
 }
 
+// Launches the streaming kernel for one parameter type (one job with packed pointers, one job with a
+// pointer table, or a batch); shared memory is opted into once per device and size.
+template <int DT, int OPR, typename PRM>
+cudaError_t launch_stream_kernel(const PRM &prm, uint32_t n_ctas, int device, void *stream)
+{
+    auto kernel = rd_tree_stream_kernel<DT, OPR, PRM>;
+    const size_t smem = stream_smem_bytes(prm.stages, prm.depth, prm.stage_elems);
+    static size_t configured[64] = {};     // per device: largest dynamic shared memory size opted into so far
+    const int dv = device & 63;
+    if (smem > configured[dv]) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+        if (e != cudaSuccess) return e;
+        configured[dv] = smem;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(n_ctas); cfg.blockDim = dim3(kStreamThreads); cfg.dynamicSmemBytes = smem;
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, prm);
+}
+
 template <int DT, int OPR, bool PACKED>
 cudaError_t launch_stream(const TreeLaunch &l)
 {
@@ -601,23 +719,27 @@ cudaError_t launch_stream(const TreeLaunch &l)
     prm.t.tiles = l.tiles; prm.t.ops = l.ops; prm.t.n_tiles = l.n_tiles; prm.t.p = l.p;
     prm.cta_first = l.cta_first; prm.status = l.status;
     prm.stages = l.stages; prm.depth = l.stack_depth > 0 ? l.stack_depth : 1; prm.stage_elems = l.stage_elems;
-    auto kernel = rd_tree_stream_kernel<DT, OPR, PACKED>;
-    const size_t smem = stream_smem_bytes(prm.stages, prm.depth, prm.stage_elems);
-    static size_t configured[64] = {};     // per device: largest dynamic shared memory size opted into so far
-    const int dv = l.device & 63;
-    if (smem > configured[dv]) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-        if (e != cudaSuccess) return e;
-        configured[dv] = smem;
+    return launch_stream_kernel<DT, OPR>(prm, l.n_ctas, l.device, l.stream);
+}
+
+template <int DT, int OPR>
+cudaError_t launch_stream_batch(const BatchLaunch &b)
+{
+    const int depth = b.stack_depth > 0 ? b.stack_depth : 1;
+    if (b.host_jobs) {
+        BatchStreamParams<true> prm;
+        for (uint32_t j = 0; j < uint32_t(kBatchPackJobs); j++)
+            prm.jobs[j] = j < b.n_jobs ? b.host_jobs[j] : BatchJob{nullptr, nullptr, nullptr, nullptr, b.n_tiles, b.n_tiles, 1, 0};
+        for (uint32_t i = 0; i < uint32_t(kBatchPackPtrs); i++)
+            prm.ptrs[i] = i < b.n_ptrs ? static_cast<const uint32_t *>(b.host_ptrs[i]) : nullptr;
+        prm.n_jobs = b.n_jobs; prm.n_tiles = b.n_tiles; prm.status = b.status;
+        prm.stages = b.stages; prm.depth = depth; prm.stage_elems = b.stage_elems;
+        return launch_stream_kernel<DT, OPR>(prm, b.n_ctas, b.device, b.stream);
     }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(l.n_ctas); cfg.blockDim = dim3(kStreamThreads); cfg.dynamicSmemBytes = smem;
-    cfg.stream = static_cast<cudaStream_t>(l.stream);
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kernel, prm);
+    BatchStreamParams<false> prm;
+    prm.jobs = b.jobs; prm.n_jobs = b.n_jobs; prm.n_tiles = b.n_tiles; prm.status = b.status;
+    prm.stages = b.stages; prm.depth = depth; prm.stage_elems = b.stage_elems;
+    return launch_stream_kernel<DT, OPR>(prm, b.n_ctas, b.device, b.stream);
 }
 
 template <int DT, int OPR>
@@ -728,6 +850,10 @@ struct StreamLauncher {
     const TreeLaunch &l;
     template <int DT, int OPR> cudaError_t operator()() const { return launch_stream_dtop<DT, OPR>(l); }
 };
+struct BatchLauncher {
+    const BatchLaunch &b;
+    template <int DT, int OPR> cudaError_t operator()() const { return launch_stream_batch<DT, OPR>(b); }
+};
 struct DirectLauncher {
     const TreeLaunch &l;
     template <int DT, int OPR> cudaError_t operator()() const { return launch_direct_dtop<DT, OPR>(l); }
@@ -743,6 +869,12 @@ int launch_tree_stream(const TreeLaunch &l)
 {
     if (l.n_tiles == 0 || l.n_ctas == 0) return 0;
     return int(with_type_and_op(l.dtype, l.op, StreamLauncher{l}));
+}
+
+int launch_tree_stream_batch(const BatchLaunch &b)
+{
+    if (b.n_jobs == 0 || b.n_ctas == 0) return 0;
+    return int(with_type_and_op(b.dtype, b.op, BatchLauncher{b}));
 }
 
 bool direct_applies(int p, int stack_depth)

@@ -39,6 +39,33 @@ struct TreeLaunch {
     int *status;                      // device word
 };
 
+// One reduction of a batch that runs as a single launch of the streaming kernel.
+struct BatchJob {
+    const uint32_t *const *inputs;    // device table of the job's p input pointers (batches that do not fit the parameters)
+    uint32_t *out;
+    const TileDesc *tiles;            // the tiles of the job's schedule (streaming path)
+    const uint32_t *ops;              // its operation table
+    uint32_t tile_begin, tile_end;    // the job's tiles are [tile_begin, tile_end) of the launch's tiles
+    int p;
+    int ptr_base;                     // first of the job's p pointers in the launch's pointer array (small batches)
+};
+constexpr int kBatchPackJobs = 16;    // a batch of at most this many jobs and kBatchPackPtrs input pointers
+constexpr int kBatchPackPtrs = 1024;  // travels inside the kernel's parameters
+
+struct BatchLaunch {
+    const BatchJob *host_jobs;        // host: small batch, descriptors and pointers go into the parameters ...
+    const void *const *host_ptrs;     //       ... n_ptrs device pointers, job after job
+    uint32_t n_ptrs;
+    const BatchJob *jobs;             // device, n_jobs entries (when host_jobs is null)
+    uint32_t n_jobs, n_tiles;
+    uint32_t n_ctas;
+    int stages, stack_depth, stage_elems;
+    int dtype, op, device;
+    int *status;                      // device word
+    void *stream;
+};
+int launch_tree_stream_batch(const BatchLaunch &b);
+
 // Elements one tile of the element-path kernel may hold for the given vector width.
 uint32_t tree_tile_elems(int vec);
 // Launches the tree kernel; returns a cudaError_t value (0 = success).

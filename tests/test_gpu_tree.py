@@ -551,6 +551,49 @@ def test_batch_of_unlike_jobs():
             rd.rd_destroy(h)
 
 
+def test_batch_as_one_launch_of_unlike_jobs():
+    """Whole-vector, 16-byte aligned jobs run as ONE launch of the streaming kernel whatever their shapes:
+    different process counts (one, two, more than travel as kernel parameters), lengths, segmentations with
+    boundaries inside a vector, stack depths, a schedule that serves two jobs, an output that aliases its own
+    root input.  Called more often than the library keeps per-call tables in flight; every call bit-identical
+    to separate rd_reduce calls, integer results also to the order-free value."""
+    shapes = [(8, 4096, 2048), (13, 6152, 4 * 333), (300, 4096, 4096), (5, 10000, 4 * 2500), (2, 4100, 4 * 4100),
+              (1, 2048 * 3 + 4, 4 * 1000), (64, 2048 * 40, 16 << 10), (33, 2048 * 7 + 12, 4 * 999)]
+    for dist, op, dt in (("int_pm2p20", rd.RD_SUM, torch.int32), ("normal", rd.RD_SUM, torch.float32), ("normal", rd.RD_MAX, torch.float32)):
+        hs, xs, outs = [], [], []
+        for k, (p, n, seg) in enumerate(shapes):
+            algo, port = [(rd.RD_BI_GREEDY, rd.RD_PORT_BI), (rd.RD_UNI_GREEDY, rd.RD_PORT_UNI), (rd.RD_BINOMIAL, rd.RD_PORT_UNI)][k % 3]
+            hs.append(rd.rd_schedule_create(algo, port, p, 4 * n, seg, *M1))
+            xs.append(make_inputs(p, n, dist, seed=k, device="cuda"))
+            outs.append(torch.empty(n, dtype=dt, device="cuda"))
+        hs.append(hs[1]); xs.append(make_inputs(13, 6152, dist, seed=99, device="cuda")); outs.append(torch.empty(6152, dtype=dt, device="cuda"))
+        keep = xs[0].clone()
+        outs[0] = xs[0][0]                                          # aliases its own root input
+        try:
+            for h in hs:                                            # the comparison below must see this kernel, not the direct one
+                rd.rd_schedule_set_tree_variant(h, rd.RD_TREE_STREAM)
+                assert rd.rd_schedule_tree_shape(h)["n_tiles"] >= 1
+            for call in range(7):
+                xs[0].copy_(keep)
+                for o in outs[1:]:
+                    o.zero_()
+                rd.rd_reduce_batch([(h, x, o) for h, x, o in zip(hs, xs, outs)], op)
+                got = [o.clone() for o in outs]
+                xs[0].copy_(keep)
+                for h, x, o, g in zip(hs, xs, outs, got):
+                    r = torch.empty_like(g)
+                    rd.rd_reduce(h, x, r, op)
+                    assert torch.equal(r.view(torch.int32), g.view(torch.int32))
+                    if dt == torch.int32:
+                        want = ((x.sum(dim=0, dtype=torch.int64) + (1 << 31)) % (1 << 32) - (1 << 31)).to(torch.int32)
+                        assert torch.equal(g, want)
+                    elif op == rd.RD_MAX:
+                        assert torch.equal(g, x.amax(dim=0))
+        finally:
+            for h in hs[:-1]:
+                rd.rd_destroy(h)
+
+
 def test_config2_over_two_streams_as_the_benchmark_issues_it():
     """The four schedules of config2 alternate over two CUDA streams (launches overlap each other's tail):
     every output is bit-identical to the same reduction issued alone, and sampled segments of it to the oracle."""
