@@ -37,21 +37,22 @@ WORKLOAD_SCHEDULES = {
 WORKLOAD_OPS = {"config1": ["sum"], "config2": ["sum"], "config3": ["sum"], "config4": ["sum", "max"]}
 
 
-# DRAM bytes per launch of the tree kernel from one ncu capture (profiles/rd_tree_stream_kernel_config2.md):
-# dram__bytes_read.sum + dram__bytes_write.sum, mean of three launches.  Reported only while the kernel
-# source is the one that was profiled.
-NCU_TRAFFIC = {"workload": "config2", "bytes_per_launch": 274.4e6,
-               "kernel_sha256": "3c9ccb5876b0620a7fedb0db1b92334c4e5ecb8d8d94a82e4a5d52569c87360b"}
+# DRAM bytes per launch of the streaming kernel from ncu captures (profiles/rd_tree_stream_kernel_config2.md):
+# dram__bytes_read.sum + dram__bytes_write.sum, mean of three launches, for the batch launch (four reductions)
+# and for a single reduction's launch.  Reported only while the kernel source is the one that was profiled.
+NCU_TRAFFIC = {"workload": "config2",
+               "bytes_per_launch": {"calls": 274.2e6, "batch": 1092.4e6},
+               "kernel_sha256": "50ddfd82fcd64aa230e2eb56ee39a492d5ad30d9084d2cd13199a073186c53eb"}
 
 
-def profiled_traffic(wname):
+def profiled_traffic(wname, issue):
     import hashlib
     try:
         with open(os.path.join(ROOT, "paper_1310_4645_b200", "csrc", "rd_kernels.cu"), "rb") as f:
             same = hashlib.sha256(f.read()).hexdigest() == NCU_TRAFFIC["kernel_sha256"]
     except OSError:
         same = False
-    return NCU_TRAFFIC["bytes_per_launch"] if same and wname == NCU_TRAFFIC["workload"] else None
+    return NCU_TRAFFIC["bytes_per_launch"][issue] if same and wname == NCU_TRAFFIC["workload"] else None
 
 
 def measured_peak():
@@ -235,6 +236,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-large", action="store_true", help="skip the extra large-message (config4) measurement")
     ap.add_argument("--no-faithful", action="store_true", help="skip the schedule-faithful makespan measurement")
+    ap.add_argument("--issue", default="batch", choices=["batch", "calls"],
+                    help="batch: a step is one rd_reduce_batch call per operation (one launch for all schedules); "
+                         "calls: one rd_reduce call per schedule and operation")
     ap.add_argument("--streams", type=int, default=2, choices=[1, 2],
                     help="CUDA streams the independent reductions of the timed region alternate over (default 2)")
     args = ap.parse_args()
@@ -276,8 +280,17 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     model = (w["alpha"], w["beta"], w["gamma"])
-    # arenas: the kernel never reads the arena the previous launch read, and two arenas together exceed L2
-    n_arenas = 3 if p * n * 4 <= (1 << 30) else 1
+    n_plans = len(WORKLOAD_SCHEDULES[wname])
+    # Batch issue: every job of a step reads its own messages (jobs of one launch that read the same bytes
+    # would meet in L2), and steps that may overlap on two streams read different sets of them.
+    batch_sets = max(2, args.streams)
+    if args.issue == "batch" and p * n * 4 * n_plans * batch_sets > (48 << 30):
+        args.issue = "calls"
+    # Call issue: the kernel never reads the arena the previous launch read, and two arenas together exceed L2.
+    if args.issue == "batch":
+        n_arenas = n_plans * batch_sets
+    else:
+        n_arenas = 3 if p * n * 4 <= (1 << 30) else 1
     arenas = [make_inputs(p, n, w["dist"], w["seed"] + 1000 * a, device=str(dev)) for a in range(n_arenas)]
     out = torch.empty(n, dtype=arenas[0].dtype, device=dev)
     tables = [rd.PointerTable(a) for a in arenas]
@@ -292,19 +305,32 @@ def main():
     for _, h in plans:
         rd.rd_schedule_upload(h)
     ops = [rd.RD_SUM if o == "sum" else rd.RD_MAX for o in WORKLOAD_OPS[wname]]
-    launches_per_step = len(plans) * len(ops)
+    reduces_per_step = len(plans) * len(ops)
+    launches_per_step = len(ops) if args.issue == "batch" else reduces_per_step
 
     counter = [0]
-    # A step reduces the same messages under every schedule (and operation) of the workload: independent
-    # reductions, each with its own output.  They are issued as plain rd_reduce calls that alternate over
-    # args.streams CUDA streams: with two streams one reduction's thread blocks take the SM slots the other
-    # frees while its last blocks are still running, which a single launch of this size (1.7 waves of tiles)
-    # cannot do for itself.  Launch i of the run reads arena i mod n_arenas.
-    outs = [torch.empty(n, dtype=arenas[0].dtype, device=dev) for _ in range(launches_per_step)]
+    # A step reduces messages under every schedule (and operation) of the workload: independent reductions,
+    # each with its own output.
+    #   batch issue: one rd_reduce_batch call per operation, i.e. ONE launch of the streaming kernel whose
+    #     tiles are those of all the schedules' reductions (each job on its own messages);
+    #   call issue: one rd_reduce call per schedule and operation; launch i of the run reads arena i mod n_arenas.
+    # Either way the calls alternate over args.streams CUDA streams: with two streams one launch's thread
+    # blocks take the SM slots the other frees while its last blocks are still running.
+    outs = [torch.empty(n, dtype=arenas[0].dtype, device=dev) for _ in range(reduces_per_step)]
     main_stream = torch.cuda.current_stream(dev)
     side = [torch.cuda.Stream(device=dev) for _ in range(args.streams)] if args.streams > 1 else [main_stream]
+    batches = None
+    if args.issue == "batch":
+        batches = [[rd.Batch([(h, tables[s_ * n_plans + j], outs[k * n_plans + j]) for j, (_, h) in enumerate(plans)])
+                    for k in range(len(ops))] for s_ in range(batch_sets)]
 
     def step(streams):
+        if batches is not None:
+            for k, op in enumerate(ops):
+                c = counter[0]
+                rd.rd_reduce_batch(batches[c % batch_sets][k], op, stream=streams[c % len(streams)])
+                counter[0] += 1
+            return
         i = 0
         for _, h in plans:
             for op in ops:
@@ -344,7 +370,7 @@ def main():
     barrier()
     clocks = sampler.stop()
     ms = max_over_ranks(e0.elapsed_time(e1), dev)
-    value = replica_throughput(args.steps * launches_per_step * bytes_per_reduce, ms, world)
+    value = replica_throughput(args.steps * reduces_per_step * bytes_per_reduce, ms, world)
 
     # the kernel by itself: the same launches back to back on ONE stream (what the roofline entry reports)
     if args.streams > 1:
@@ -384,7 +410,7 @@ def main():
             hx = arenas[0].cpu().pin_memory()
             hout = torch.empty(n, dtype=arenas[0].dtype).pin_memory()
             staging = torch.empty((p + 1) * n, dtype=arenas[0].dtype, device=dev)
-            e_steps = max(3, min(args.steps, int(2.0 / (launches_per_step * host_bytes / 40e9)) or 1))
+            e_steps = max(3, min(args.steps, int(2.0 / (reduces_per_step * host_bytes / 40e9)) or 1))
             for _, h in e2e_n_plans:
                 rd.rd_reduce_host(h, hx, hout, staging, ops[0])
             barrier()
@@ -397,8 +423,8 @@ def main():
             b.record()
             barrier()
             e_ms = max_over_ranks(a.elapsed_time(b), dev)
-            e2e = {"value": replica_throughput(e_steps * launches_per_step * bytes_per_reduce, e_ms, world), "unit": "GB/s",
-                   "h2d_bytes_per_step": launches_per_step * host_bytes, "d2h_bytes_per_step": launches_per_step * n * 4,
+            e2e = {"value": replica_throughput(e_steps * reduces_per_step * bytes_per_reduce, e_ms, world), "unit": "GB/s",
+                   "h2d_bytes_per_step": reduces_per_step * host_bytes, "d2h_bytes_per_step": reduces_per_step * n * 4,
                    "steps": e_steps}
             del hx, hout, staging
 
@@ -463,7 +489,8 @@ def main():
         if large:
             large["frac_of_measured_peak"] = large["value"] / peak
             large["frac_of_nominal_8000"] = large["value"] / 8000.0
-        achieved = bytes_per_reduce / (kernel_ms_per_launch * 1e-3) / 1e9
+        bytes_per_launch = bytes_per_reduce * reduces_per_step // launches_per_step
+        achieved = bytes_per_launch / (kernel_ms_per_launch * 1e-3) / 1e9
         cpu = None
         if not args.no_cpu_baseline and world == 1:
             x, n_s = host_slab(w, wname, 1 << 30)
@@ -472,6 +499,10 @@ def main():
                    "sample": "%d passes over every schedule x op on %d of %d elements per process (%.1f s)"
                              % (passes, n_s, n, dt)}
         shape0 = rd.rd_schedule_tree_shape(plans[0][1])
+        if args.issue == "batch":                   # the batch launch: all jobs' tiles, the deepest stack among them
+            tiles = sum(rd.rd_schedule_tree_shape(h)["n_tiles"] for _, h in plans)
+            shape0 = dict(variant=rd.RD_TREE_STREAM, n_tiles=tiles, blocks_per_sm="chosen for the batch's tiles and deepest stack",
+                          ring_stages="chosen for the batch's tiles and deepest stack")
         line = {
             "metric": "reduction_throughput", "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
@@ -479,12 +510,17 @@ def main():
             "config": {"workload": wname, "p": p, "n_elems": n, "segment_bytes": w["seg_bytes"],
                        "schedules": [s[0] for s in WORKLOAD_SCHEDULES[wname]], "ops": WORKLOAD_OPS[wname],
                        "bytes_counted": "p*m + m per reduction",
-                       "issue": "the step's independent reductions alternate over %d CUDA stream(s)" % args.streams,
-                       "l2": "inputs rotate over %d arenas of %.0f MiB each (> L2 between reuses)" % (n_arenas, p * n * 4 / 2**20)
+                       "issue": ("a step is one rd_reduce_batch call per operation: one launch for the step's %d independent "
+                                 "reductions, each on its own messages; steps alternate over %d CUDA stream(s) and %d sets of messages"
+                                 % (n_plans, args.streams, batch_sets)) if args.issue == "batch" else
+                                "the step's independent reductions are separate rd_reduce calls that alternate over %d CUDA stream(s)" % args.streams,
+                       "l2": "a launch reads %.0f MiB that no launch running beside it reads (%d arenas of %.0f MiB)"
+                             % (n_plans * p * n * 4 / 2**20, n_arenas, p * n * 4 / 2**20) if args.issue == "batch" else
+                             "inputs rotate over %d arenas of %.0f MiB each (> L2 between reuses)" % (n_arenas, p * n * 4 / 2**20)
                              if n_arenas > 1 else "inputs (%.1f GiB) exceed L2" % (p * n * 4 / 2**30),
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": profiled_traffic(wname), "traffic_unit": "bytes per launch", "algorithmic_bytes": bytes_per_reduce,
+                         "traffic": profiled_traffic(wname, args.issue), "traffic_unit": "bytes per launch", "algorithmic_bytes": bytes_per_launch,
                          "peak_source": peak_src,
                          "kernel": "rd_tree_direct_kernel" if shape0["variant"] == rd.RD_TREE_DIRECT else "rd_tree_stream_kernel",
                          "launch_shape": {"blocks_per_sm": shape0["blocks_per_sm"], "ring_stages": shape0["ring_stages"],
@@ -492,6 +528,7 @@ def main():
                          "timed_over": "%d launches back to back on one stream, %.2f us each" % (k_steps * launches_per_step, kernel_ms_per_launch * 1e3),
                          "frac_of_nominal_8000": achieved / 8000.0},
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": args.steps * launches_per_step, "clocks": clocks,
+            "reductions_per_step": reduces_per_step,
             "per_schedule_gbs": per_schedule, "schedule_create_ms": create_ms, "large_message": large, "faithful": faithful,
             "percent_of_peak": {"measured_copy": 100 * value / peak, "nominal_8TBs": 100 * value / 8000.0},
         }

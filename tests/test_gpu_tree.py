@@ -635,3 +635,41 @@ def test_config2_over_two_streams_as_the_benchmark_issues_it():
     finally:
         for h in hs:
             rd.rd_destroy(h)
+
+
+def test_config2_as_batches_over_two_streams_as_the_benchmark_issues_it():
+    """The benchmark's step: the four schedules of config2, each on its own messages, as ONE rd_reduce_batch
+    call (one launch); steps alternate over two CUDA streams and two sets of messages.  Every output is
+    bit-identical to the same reduction issued alone, and sampled segments of every job to the oracle run on
+    the oracle's own schedule."""
+    w = WORKLOADS["config2"]
+    model = (w["alpha"], w["beta"], w["gamma"])
+    p, n = w["p"], w["n"]
+    specs = [("uni_greedy", rd.RD_UNI_GREEDY), ("binomial", rd.RD_BINOMIAL), ("pipeline", rd.RD_PIPELINE), ("binary", rd.RD_BINARY)]
+    hs = [rd.rd_schedule_create(a, rd.RD_PORT_UNI, p, 4 * n, w["seg_bytes"], *model) for _, a in specs]
+    try:
+        arenas = [[make_inputs(p, n, w["dist"], w["seed"] + 1000 * (4 * s + j), device="cuda") for j in range(4)] for s in range(2)]
+        outs = [[torch.full((n,), -3.0, device="cuda") for _ in hs] for _ in range(2)]
+        batches = [rd.Batch([(h, x, o) for h, x, o in zip(hs, arenas[s], outs[s])]) for s in range(2)]
+        streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+        torch.cuda.synchronize()
+        for step in range(6):
+            rd.rd_reduce_batch(batches[step % 2], rd.RD_SUM, stream=streams[step % 2])
+        torch.cuda.synchronize()
+        assert rd.rd_schedule_status(hs[0]) == 0
+        for s in range(2):
+            for j, (h, (name, algo)) in enumerate(zip(hs, specs)):
+                alone = torch.empty(n, device="cuda")
+                rd.rd_reduce(h, arenas[s][j], alone, rd.RD_SUM)
+                torch.cuda.synchronize()
+                assert torch.equal(outs[s][j].view(torch.int32), alone.view(torch.int32)), (s, name)
+                ev, off, _ = oracle_schedule(algo, rd.RD_PORT_UNI, p, 4 * n, w["seg_bytes"], *model)
+                for seg in (0, 77 + j, 255):
+                    lo, hi = int(off[seg]), int(off[seg + 1])
+                    sel = ev[ev["seg"] == seg].copy()
+                    sel["seg"] = 0
+                    want = O.reduce(sel, arenas[s][j][:, lo:hi].cpu().numpy(), [0, hi - lo], "sum")
+                    assert outs[s][j][lo:hi].cpu().numpy().tobytes() == want.tobytes(), (s, name, seg)
+    finally:
+        for h in hs:
+            rd.rd_destroy(h)
