@@ -594,6 +594,47 @@ def test_batch_as_one_launch_of_unlike_jobs():
                 rd.rd_destroy(h)
 
 
+def test_batch_too_large_for_the_kernel_parameters():
+    """More than 16 jobs (or 1024 input pointers): descriptors and pointers reach the device through the
+    library's pinned ring, which has four slots and grows on demand: many calls in a row, then a larger batch."""
+    def make(k, p, n, seg):
+        hs = [rd.rd_schedule_create([rd.RD_UNI_GREEDY, rd.RD_PIPELINE, rd.RD_BINARY][j % 3], rd.RD_PORT_UNI, p, 4 * n, seg, *M1)
+              for j in range(k)]
+        xs = [make_inputs(p, n, "int_pm2p20", seed=100 * k + j, device="cuda") for j in range(k)]
+        outs = [torch.empty(n, dtype=torch.int32, device="cuda") for _ in range(k)]
+        return hs, xs, outs
+    def run(hs, xs, outs, calls):
+        batch = rd.Batch([(h, x, o) for h, x, o in zip(hs, xs, outs)])
+        for call in range(calls):
+            for o in outs:
+                o.fill_(call)
+            rd.rd_reduce_batch(batch, rd.RD_SUM)
+            for x, o in zip(xs, outs):
+                want = ((x.sum(dim=0, dtype=torch.int64) + (1 << 31)) % (1 << 32) - (1 << 31)).to(torch.int32)
+                assert torch.equal(o, want)
+    small = make(20, 7, 2048 * 3 + 8, 4 * 1000)          # 20 jobs
+    wide = make(3, 400, 4096, 4 * 1024)                    # 1200 pointers
+    big = make(40, 300, 2048 + 4, 4 * 512)                 # 12000 pointers: the ring has to grow
+    try:
+        run(*small, calls=9)
+        run(*wide, calls=2)
+        run(*big, calls=6)
+        run(*small, calls=2)
+        # fp32 in the order of each job's schedule
+        p, n, seg = 7, 2048 * 3 + 8, 4 * 1000
+        xs = [make_inputs(p, n, "normal", seed=j, device="cuda") for j in range(20)]
+        outs = [torch.empty(n, device="cuda") for _ in range(20)]
+        rd.rd_reduce_batch([(h, x, o) for h, x, o in zip(small[0], xs, outs)], rd.RD_SUM)
+        for j in (0, 1, 2, 19):
+            algo = [rd.RD_UNI_GREEDY, rd.RD_PIPELINE, rd.RD_BINARY][j % 3]
+            ev, off, _ = oracle_schedule(algo, rd.RD_PORT_UNI, p, 4 * n, seg, *M1)
+            assert outs[j].cpu().numpy().tobytes() == O.reduce(ev, xs[j].cpu().numpy(), off, "sum").tobytes()
+    finally:
+        for hs in (small[0], wide[0], big[0]):
+            for h in hs:
+                rd.rd_destroy(h)
+
+
 def test_config2_over_two_streams_as_the_benchmark_issues_it():
     """The four schedules of config2 alternate over two CUDA streams (launches overlap each other's tail):
     every output is bit-identical to the same reduction issued alone, and sampled segments of it to the oracle."""
