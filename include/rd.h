@@ -218,7 +218,8 @@ RD_API int rd_schedule_program(const rd_schedule_t *s, size_t seg, uint32_t *ops
  * (allocates device memory, synchronises); rd_schedule_upload does the same
  * ahead of time.  After one such call per schedule, element type and operation, a
  * tree-mode call with at most 256 processes is a single kernel launch and may be
- * recorded into a CUDA graph.  Buffers must be aligned to the element; 16-byte aligned buffers take
+ * recorded into a CUDA graph (so may an rd_reduce_batch call of at most 16 aligned jobs with at most
+ * 1024 input pointers in all, after one ordinary call of it).  Buffers must be aligned to the element; 16-byte aligned buffers take
  * the 128-bit streaming path (segments may start and end anywhere; when the message is
  * not a multiple of 16 bytes the last elements are done by a second, tiny launch), other
  * buffers a slower element-wise path.

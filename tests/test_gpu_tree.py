@@ -443,7 +443,30 @@ def test_tree_mode_launches_can_be_replayed_from_a_cuda_graph():
     torch.cuda.synchronize()
     for o, w in zip(outs, want):
         assert torch.equal(o, w)
-    for h in hs:
+    # the same for a batch that fits the kernel's parameters (one launch, nothing copied ahead of it) and for
+    # the direct kernel (two processes)
+    h2 = rd.rd_schedule_create(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, 2, 4 * n, 2048, *M1)
+    o2, w2 = torch.zeros(n, device="cuda"), torch.zeros(n, device="cuda")
+    batch = rd.Batch([(h, t, o) for h, t, o in zip(hs, tabs, outs)])
+    rd.rd_reduce_batch(batch, rd.RD_SUM)                 # ordinary calls first
+    rd.rd_reduce(h2, xs[0][:2], w2, rd.RD_SUM)
+    torch.cuda.synchronize()
+    assert rd.rd_schedule_tree_shape(h2)["variant"] == rd.RD_TREE_DIRECT
+    for o, w in zip(outs, want):
+        assert torch.equal(o, w)
+        o.zero_()
+    graph2 = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph2, stream=stream):
+            for _ in range(3):
+                rd.rd_reduce_batch(batch, rd.RD_SUM, stream=stream)
+                rd.rd_reduce(h2, xs[0][:2], o2, rd.RD_SUM, stream=stream)
+    graph2.replay()
+    torch.cuda.synchronize()
+    for o, w in zip(outs, want):
+        assert torch.equal(o, w)
+    assert torch.equal(o2, w2)
+    for h in hs + [h2]:
         rd.rd_destroy(h)
 
 
