@@ -760,6 +760,57 @@ int orc_reduce_f32(const orc_event_t *ev_in, int64_t n_ev, int p, int q, const i
     return ORC_OK;
 }
 
+/* bf16 elements combined in fp32 (the paper leaves the element type open, Fig. 2
+ * caption; this is the usual meaning of "16-bit storage, 32-bit accumulation"):
+ * every input is widened exactly (a bf16 is the upper half of an fp32), the
+ * replay above runs on fp32 values, one IEEE fp32 operation per combine, and only
+ * what process 0 holds at the end is rounded to bf16, once, to nearest with
+ * ties to even.  NaN inputs are outside the parity tests.  seg_off counts
+ * elements.                                                                   */
+static float bf16_to_f32(uint16_t h)
+{
+    uint32_t u = (uint32_t)h << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return f;
+}
+
+static uint16_t f32_to_bf16(float f)
+{
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    if ((u & 0x7FFFFFFFu) > 0x7F800000u) return (uint16_t)((u >> 16) | 0x0040u);   /* NaN stays NaN */
+    /* the 16 bits that are dropped: above half -> up, below -> down, exactly half -> to the even neighbour */
+    uint32_t lower = u & 0xFFFFu, keep = u >> 16;
+    if (lower > 0x8000u || (lower == 0x8000u && (keep & 1u))) keep++;
+    return (uint16_t)keep;
+}
+
+int orc_reduce_bf16(const orc_event_t *ev_in, int64_t n_ev, int p, int q, const int64_t *seg_off,
+                    const uint16_t *const *x, uint16_t *out, int op)
+{
+    orc_event_t *ev = sorted_by_segment(ev_in, n_ev);
+    if (!ev) return ORC_NOMEM;
+    int64_t longest = 0;
+    for (int j = 0; j < q; j++) if (seg_off[j + 1] - seg_off[j] > longest) longest = seg_off[j + 1] - seg_off[j];
+    float *acc = malloc(sizeof(float) * (size_t)p * (size_t)(longest ? longest : 1));
+    if (!acc) { free(ev); return ORC_NOMEM; }
+    int64_t e = 0;
+    for (int j = 0; j < q; j++) {
+        int64_t len = seg_off[j + 1] - seg_off[j];
+        for (int i = 0; i < p; i++)
+            for (int64_t k = 0; k < len; k++) acc[(size_t)i * longest + k] = bf16_to_f32(x[i][seg_off[j] + k]);
+        for (; e < n_ev && ev[e].seg == j; e++) {
+            float *held = acc + (size_t)ev[e].dst * longest, *in = acc + (size_t)ev[e].src * longest;
+            if (ev[e].kind == 0) for (int64_t k = 0; k < len; k++) held[k] = comb_f32(held[k], in[k], op);
+            else for (int64_t k = 0; k < len; k++) held[k] = in[k];
+        }
+        for (int64_t k = 0; k < len; k++) out[seg_off[j] + k] = f32_to_bf16(acc[k]);
+    }
+    free(acc); free(ev);
+    return ORC_OK;
+}
+
 /* The same for the 8-byte element types: int64 wraps modulo 2^64, fp64 is one
  * IEEE round-to-nearest operation per combine.  seg_off counts elements.     */
 static uint64_t comb_i64(uint64_t held, uint64_t in, int op)

@@ -274,3 +274,82 @@ def test_fp64_extrema_and_exact_sums(p):
     ev, _ = O.uni_greedy(2, [1], 1, 1, 1)
     assert np.signbit(O.reduce(ev, z, [0, 1], "max"))[0] == False
     assert np.signbit(O.reduce(ev, z[::-1].copy(), [0, 1], "max"))[0] == True
+
+
+# ---------------------------------------------------------------------------------------------
+# bf16 elements combined in fp32: inputs widened exactly, fp32 partial results in the schedule's
+# order, one rounding to bf16 (nearest, ties to even) of what the root holds at the end.
+# The pins use torch's CPU conversion as the independent statement of "round an fp32 to bf16".
+# ---------------------------------------------------------------------------------------------
+def bf16_bits(a):
+    """fp32 array -> uint16 bf16 bit patterns, rounded by torch (library routine, not the oracle's)."""
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=f32)).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+
+
+def bf16_value(bits):
+    return (bits.astype(np.uint32) << 16).view(f32)
+
+
+def test_bf16_two_processes_is_one_fp32_add_rounded_once():
+    rng = np.random.default_rng(11)
+    x = bf16_bits(rng.standard_normal((2, 4000)) * 10.0 ** rng.integers(-6, 7, size=(2, 4000)))
+    ev, _ = O.uni_greedy(2, [2400, 1600], 1, 1, 1)
+    got = O.reduce(ev, x, [0, 2400, 4000], "sum")
+    assert got.dtype == np.uint16
+    assert (got == bf16_bits(bf16_value(x[0]) + bf16_value(x[1]))).all()
+    prod = O.reduce(ev, x, [0, 2400, 4000], "prod")
+    assert (prod == bf16_bits(bf16_value(x[0]) * bf16_value(x[1]))).all()
+
+
+def test_bf16_rounding_ties_go_to_the_even_neighbour_and_the_rest_to_the_nearest():
+    """1 + k * 2^-9 for k = 0..8 around the bf16 neighbours 1, 1 + 2^-7, 1 + 2^-6 (spacing 2^-7): a single
+    process pair adds 1 and k * 2^-9 exactly in fp32."""
+    ks = np.arange(0, 9)
+    x = np.stack([bf16_bits(np.ones(9)), bf16_bits(ks * 2.0 ** -9)])
+    ev, _ = O.uni_greedy(2, [9], 1, 1, 1)
+    got = bf16_value(O.reduce(ev, x, [0, 9], "sum"))
+    # k: 0 1 -> 1; 2 is the tie between 1 (even mantissa) and 1 + 2^-7 -> 1; 3 4 5 -> 1 + 2^-7;
+    # 6 is the tie between 1 + 2^-7 (odd) and 1 + 2^-6 (even) -> 1 + 2^-6; 7 8 -> 1 + 2^-6
+    want = 1 + np.array([0, 0, 0, 1, 1, 1, 2, 2, 2]) * 2.0 ** -7
+    assert (got == want.astype(f32)).all()
+
+
+def test_bf16_partial_results_stay_in_fp32():
+    """Pipeline of 4: 1 + 2^-9 + 2^-9 + 2^-9.  Kept in fp32 the sum is 1 + 3 * 2^-9, above the half-way point,
+    and rounds to 1 + 2^-7; rounding every partial result to bf16 would give 1."""
+    x = np.stack([bf16_bits(np.full(8, v)) for v in (2.0 ** -9, 2.0 ** -9, 2.0 ** -9, 1.0)])
+    ev, _ = O.pipeline(4, [8], 1, 1, 1, False)
+    got = bf16_value(O.reduce(ev, x, [0, 8], "sum"))
+    assert (got == f32(1 + 2.0 ** -7)).all()
+
+
+@pytest.mark.parametrize("p", [2, 5, 16, 64])
+def test_bf16_small_integers_sum_exactly_and_extrema_are_order_free(p):
+    """Integers up to 256 in magnitude are bf16 values, so sums that stay there are exact for any order; max and
+    min pick one of the inputs, which is a bf16 value already."""
+    rng = np.random.default_rng(p)
+    n, sizes = 96, [40, 40, 16]
+    xi = rng.integers(-3, 4, size=(p, n))
+    x = bf16_bits(xi.astype(f32))
+    y = bf16_bits(rng.standard_normal((p, n)) * 10.0 ** rng.integers(-5, 6, size=(p, n)))
+    for name, ev in schedules(p, sizes):
+        assert (bf16_value(O.reduce(ev, x, seg_off(sizes), "sum")) == xi.sum(axis=0)).all(), name
+        assert (bf16_value(O.reduce(ev, y, seg_off(sizes), "max")) == bf16_value(y).max(axis=0)).all(), name
+        assert (bf16_value(O.reduce(ev, y, seg_off(sizes), "min")) == bf16_value(y).min(axis=0)).all(), name
+
+
+@pytest.mark.parametrize("p", [3, 9, 32])
+def test_bf16_sum_is_the_fp32_schedule_sum_rounded(p):
+    """The same events on the widened inputs through the fp32 evaluator (pinned above), then one rounding."""
+    rng = np.random.default_rng(100 + p)
+    n, sizes = 200, [64, 64, 72]
+    x = bf16_bits(rng.standard_normal((p, n)) * 10.0 ** rng.integers(-3, 4, size=(p, n)))
+    for name, ev in schedules(p, sizes):
+        wide = O.reduce(ev, bf16_value(x), seg_off(sizes), "sum")
+        assert (O.reduce(ev, x, seg_off(sizes), "sum") == bf16_bits(wide)).all(), name
+        # and close to the order-free fp64 sum: one bf16 rounding (8 significant bits: 2^-8 relative) on top of the fp32 bound
+        ref = bf16_value(x).astype(np.float64).sum(axis=0)
+        mag = np.abs(bf16_value(x).astype(np.float64)).sum(axis=0)
+        got = bf16_value(O.reduce(ev, x, seg_off(sizes), "sum")).astype(np.float64)
+        assert (np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + p * 2.0 ** -23 * mag + 1e-30).all(), name
