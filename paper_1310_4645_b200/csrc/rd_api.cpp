@@ -47,10 +47,13 @@ struct DeviceTables {
     uint32_t *ops = nullptr;
     std::map<int, std::pair<TileDesc *, uint32_t>> tiles;   // vector width -> (device table, count)
     // streaming (128-bit) path: tiles grouped per CTA, every CTA the same number of elements
-    uint32_t *cta_first = nullptr;
-    uint32_t n_ctas = 0;
-    int ctas_per_sm = 0;
-    int stages = 0;
+    struct StreamPlan {                     // per-CTA tile ranges and ring shape of a single reduction's launch
+        uint32_t *cta_first = nullptr;
+        uint32_t n_ctas = 0;
+        int ctas_per_sm = 0;
+        int stages = 0;
+    };
+    std::map<int, StreamPlan> plans;        // key: words of partial result per message word (1; 2 for bf16)
     int stage_elems = 0;
     int *status = nullptr;                                  // device word written by a kernel that gave up a wait
     // pointer tables for large p: pinned host ring + device ring, one event per slot
@@ -161,7 +164,7 @@ void release_device(DeviceTables &d)
     cudaGetDevice(&prev);
     cudaSetDevice(d.device);
     cudaFree(d.ops);
-    cudaFree(d.cta_first);
+    for (auto &kv : d.plans) cudaFree(kv.second.cta_first);
     cudaFree(d.status);
     for (auto &kv : d.tiles) cudaFree(kv.second.first);
     if (d.h_ring) cudaFreeHost(d.h_ring);
@@ -240,10 +243,7 @@ int tiles_for(rd_schedule *s, int vec, const TileDesc **tiles, uint32_t *count)
         if (vec == 4) {
             // Streaming path.  Every segment is cut into equal tiles of at most one stage (whole 128-bit
             // vectors of the buffers: where a segment starts or ends inside a vector the tile is padded to the
-            // vector and remembers how many elements are not its own).  CTAs get contiguous runs of tiles,
-            // the same NUMBER of tiles up to one: a tile costs a CTA about the same time however full it
-            // is (one ring hand-off per operation), so for small messages the number of tiles per CTA,
-            // not the number of elements, sets the kernel's duration; for large ones the two coincide.
+            // vector and remembers how many elements are not its own).
             const uint64_t n = off.empty() ? 0 : off.back();
             d.stage_elems = stream_stage_elems(n / (uint64_t(d.sm_count) * 2) + 1);
             const uint32_t cap = uint32_t(d.stage_elems);
@@ -260,20 +260,6 @@ int tiles_for(rd_schedule *s, int vec, const TileDesc **tiles, uint32_t *count)
                     host.push_back(TileDesc{ts, uint32_t(te - ts) | (head << 16) | (tail << 18), s->progs.seg_prog[seg]});
                 }
             }
-            const uint64_t nTiles = host.size();
-            int ctasPerSm = 1;
-            stream_shape(s->progs.stack_depth, d.smem_per_sm, d.stage_elems, nTiles, d.sm_count, &ctasPerSm, &d.stages);
-            const uint64_t ctas = std::min<uint64_t>(uint64_t(d.sm_count) * uint64_t(ctasPerSm), std::max<uint64_t>(nTiles, 1));
-            std::vector<uint32_t> first(size_t(ctas) + 1, 0);
-            for (uint64_t c = 0; c < ctas; c++) first[size_t(c)] = uint32_t(nTiles * c / ctas);
-            first[size_t(ctas)] = uint32_t(host.size());
-            cudaFree(d.cta_first);                  // left by an attempt that failed after this point
-            d.cta_first = nullptr;
-            if (cudaMalloc(reinterpret_cast<void **>(&d.cta_first), first.size() * sizeof(uint32_t)) != cudaSuccess) return RD_ERR_NOMEM;
-            if (cudaMemcpy(d.cta_first, first.data(), first.size() * sizeof(uint32_t), cudaMemcpyHostToDevice) != cudaSuccess)
-                return RD_ERR_CUDA;
-            d.n_ctas = uint32_t(ctas);
-            d.ctas_per_sm = ctasPerSm;
         } else {
             // element path: the whole message (vec == 1), or only what the 128-bit path leaves over (kTailTiles)
             const uint64_t n = off.empty() ? 0 : off.back();
@@ -291,21 +277,52 @@ int tiles_for(rd_schedule *s, int vec, const TileDesc **tiles, uint32_t *count)
     return RD_OK;
 }
 
+// Launch shape of a single reduction on the streaming path: CTAs get contiguous runs of tiles, the same
+// NUMBER of tiles up to one (a tile costs a CTA about the same time however full it is, one ring hand-off
+// per operation, so for small messages the number of tiles per CTA, not the number of elements, sets the
+// kernel's duration; for large ones the two coincide).  acc_words: 2 for bf16, whose partial results are fp32.
+int stream_plan(rd_schedule *s, int acc_words, const DeviceTables::StreamPlan **out)
+{
+    DeviceTables &d = s->dev;
+    auto it = d.plans.find(acc_words);
+    if (it == d.plans.end()) {
+        const TileDesc *tiles = nullptr;
+        uint32_t nTiles = 0;
+        if (int rc = tiles_for(s, 4, &tiles, &nTiles)) return rc;
+        DeviceTables::StreamPlan plan;
+        stream_shape(s->progs.stack_depth, acc_words, d.smem_per_sm, d.stage_elems, nTiles, d.sm_count, &plan.ctas_per_sm, &plan.stages);
+        const uint64_t ctas = std::min<uint64_t>(uint64_t(d.sm_count) * uint64_t(plan.ctas_per_sm), std::max<uint64_t>(nTiles, 1));
+        std::vector<uint32_t> first(size_t(ctas) + 1, 0);
+        for (uint64_t c = 0; c < ctas; c++) first[size_t(c)] = uint32_t(uint64_t(nTiles) * c / ctas);
+        first[size_t(ctas)] = nTiles;
+        if (cudaMalloc(reinterpret_cast<void **>(&plan.cta_first), first.size() * sizeof(uint32_t)) != cudaSuccess) return RD_ERR_NOMEM;
+        if (cudaMemcpy(plan.cta_first, first.data(), first.size() * sizeof(uint32_t), cudaMemcpyHostToDevice) != cudaSuccess) {
+            cudaFree(plan.cta_first);
+            return RD_ERR_CUDA;
+        }
+        plan.n_ctas = uint32_t(ctas);
+        it = d.plans.emplace(acc_words, plan).first;
+    }
+    *out = &it->second;
+    return RD_OK;
+}
+
 // Argument checks common to the reducing entry points.  On success *n_words is the message length
 // in 32-bit words, the unit in which the schedule's segment boundaries and the kernels count.
-size_t elem_bytes(rd_dtype_t dtype) { return (dtype == RD_INT64 || dtype == RD_FP64) ? 8 : 4; }
+size_t elem_bytes(rd_dtype_t dtype) { return (dtype == RD_INT64 || dtype == RD_FP64) ? 8 : dtype == RD_BF16 ? 2 : 4; }
 
 int check_reduce_args(const rd_schedule *s, const void *const *d_inputs, const void *d_out, size_t n_elems, rd_dtype_t dtype,
                       rd_op_t op, size_t *n_words)
 {
-    if (!s || !d_inputs || int(dtype) < RD_INT32 || int(dtype) > RD_FP64 || int(op) < RD_SUM || int(op) > RD_PROD)
+    if (!s || !d_inputs || int(dtype) < RD_INT32 || int(dtype) > RD_BF16 || int(op) < RD_SUM || int(op) > RD_PROD)
         return RD_ERR_INVALID_ARG;
     const size_t esize = elem_bytes(dtype);
+    const size_t align = esize < 4 ? 4 : esize;          // the kernels move whole 32-bit words
     if (n_elems > s->msg_bytes / esize || n_elems * esize != s->msg_bytes) return RD_ERR_SIZE_MISMATCH;
     if (n_elems > 0 && !d_out) return RD_ERR_INVALID_ARG;
     for (int i = 0; i < s->p; i++)
-        if ((n_elems > 0 && !d_inputs[i]) || (reinterpret_cast<uintptr_t>(d_inputs[i]) & (esize - 1))) return RD_ERR_INVALID_ARG;
-    if (reinterpret_cast<uintptr_t>(d_out) & (esize - 1)) return RD_ERR_INVALID_ARG;
+        if ((n_elems > 0 && !d_inputs[i]) || (reinterpret_cast<uintptr_t>(d_inputs[i]) & (align - 1))) return RD_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(d_out) & (align - 1)) return RD_ERR_INVALID_ARG;
     if (esize == 8)                    // no segment may begin inside an element
         for (uint64_t off : s->sched.seg_off)
             if (off & 1u) return RD_ERR_INVALID_ARG;
@@ -324,6 +341,9 @@ int reduce_tree(rd_schedule *s, const void *const *d_inputs, void *d_out, size_t
     TreeLaunch l{};
     l.vec = wide ? 4 : 1;
     if (int rc = tiles_for(s, l.vec, &l.tiles, &l.n_tiles)) return rc;
+    const DeviceTables::StreamPlan *plan = nullptr;
+    if (wide)
+        if (int rc = stream_plan(s, dtype == RD_BF16 ? 2 : 1, &plan)) return rc;
     const TileDesc *tailTiles = nullptr;
     uint32_t nTail = 0;
     if (wide && (n & 3u) != 0)
@@ -341,11 +361,12 @@ int reduce_tree(rd_schedule *s, const void *const *d_inputs, void *d_out, size_t
     }
     l.out = d_out; l.ops = d.ops; l.p = s->p; l.stack_depth = s->progs.stack_depth;
     l.dtype = int(dtype); l.op = int(op); l.sm_count = d.sm_count; l.stream = stream;
-    l.cta_first = d.cta_first; l.n_ctas = d.n_ctas; l.stages = d.stages; l.stage_elems = d.stage_elems; l.status = d.status; l.device = d.device;
+    if (plan) { l.cta_first = plan->cta_first; l.n_ctas = plan->n_ctas; l.stages = plan->stages; }
+    l.stage_elems = d.stage_elems; l.status = d.status; l.device = d.device;
     // Direct kernel: all operands of an element in registers at once.  Chosen by itself for one or two
     // processes (measured on B200, p = 2: 6.8 TB/s against 6.1-6.2 of the streaming kernel for messages of
     // 256 MiB and more; from three processes on the streaming kernel is level or ahead).
-    const bool direct = wide && direct_applies(s->p, s->progs.stack_depth) &&
+    const bool direct = wide && dtype != RD_BF16 && direct_applies(s->p, s->progs.stack_depth) &&
                         (s->tree_variant == RD_TREE_DIRECT || (s->tree_variant == RD_TREE_AUTO && s->p <= kDirectAutoProcs));
     if (stats && cudaEventRecord(d.ev_start, stream) != cudaSuccess) return RD_ERR_CUDA;
     if ((direct ? launch_tree_direct(l) : wide ? launch_tree_stream(l) : launch_tree(l)) != 0) return RD_ERR_CUDA;
@@ -543,7 +564,7 @@ int reduce_batch_fused(size_t n_jobs, rd_schedule_t *const *schedules, const voi
     DeviceTables &d0 = schedules[0]->dev;
     const int stageElems = d0.stage_elems;
     int ctasPerSm = 1, stages = 2;
-    stream_shape(depth, d0.smem_per_sm, stageElems, total, d0.sm_count, &ctasPerSm, &stages);
+    stream_shape(depth, dtype == RD_BF16 ? 2 : 1, d0.smem_per_sm, stageElems, total, d0.sm_count, &ctasPerSm, &stages);
     const uint64_t ctas = std::min<uint64_t>(uint64_t(d0.sm_count) * uint64_t(ctasPerSm), total);
     BatchLaunch b{};
     b.n_jobs = uint32_t(n_jobs); b.n_tiles = uint32_t(total); b.n_ctas = uint32_t(ctas);
@@ -735,6 +756,7 @@ int rd_reduce(rd_schedule_t *s, const void *const *d_inputs, void *d_out, size_t
     if (exec != RD_EXEC_TREE && exec != RD_EXEC_FAITHFUL) return RD_ERR_INVALID_ARG;
     size_t n_words = 0;
     if (int rc = check_reduce_args(s, d_inputs, d_out, n_elems, dtype, op, &n_words)) return rc;
+    if (exec == RD_EXEC_FAITHFUL && dtype == RD_BF16) return RD_ERR_UNSUPPORTED;   // partial segments would be fp32
     return guarded([&] {
         if (int rc = upload(s)) return rc;
         if (exec == RD_EXEC_FAITHFUL)
@@ -816,7 +838,7 @@ int rd_reduce_host(rd_schedule_t *s, const void *const *h_inputs, void *h_out, v
                    rd_dtype_t dtype, rd_op_t op, void *cuda_stream)
 {
     if (!s || !h_inputs || (n_elems > 0 && (!h_out || !d_staging))) return RD_ERR_INVALID_ARG;
-    if (int(dtype) < RD_INT32 || int(dtype) > RD_FP64) return RD_ERR_INVALID_ARG;
+    if (int(dtype) < RD_INT32 || int(dtype) > RD_BF16) return RD_ERR_INVALID_ARG;
     if (n_elems > s->msg_bytes / elem_bytes(dtype) || n_elems * elem_bytes(dtype) != s->msg_bytes) return RD_ERR_SIZE_MISMATCH;
     const size_t row = s->msg_bytes;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -890,8 +912,10 @@ int rd_schedule_tree_shape(rd_schedule_t *s, int *variant, int *blocks_per_sm, i
         const bool direct = direct_applies(s->p, s->progs.stack_depth) &&
                             (s->tree_variant == RD_TREE_DIRECT || (s->tree_variant == RD_TREE_AUTO && s->p <= kDirectAutoProcs));
         if (variant) *variant = direct ? RD_TREE_DIRECT : RD_TREE_STREAM;
-        if (blocks_per_sm) *blocks_per_sm = direct ? direct_blocks_per_sm(s->p) : s->dev.ctas_per_sm;
-        if (ring_stages) *ring_stages = direct ? 0 : s->dev.stages;
+        const DeviceTables::StreamPlan *plan = nullptr;
+        if (int rc = stream_plan(s, 1, &plan)) return rc;
+        if (blocks_per_sm) *blocks_per_sm = direct ? direct_blocks_per_sm(s->p) : plan->ctas_per_sm;
+        if (ring_stages) *ring_stages = direct ? 0 : plan->stages;
         if (n_tiles) *n_tiles = l.n_tiles;
         return int(RD_OK);
     });
@@ -938,6 +962,7 @@ int rd_reduce_faithful_static(rd_schedule_t *s, const void *const *d_inputs, voi
 {
     size_t n_words = 0;
     if (int rc = check_reduce_args(s, d_inputs, d_out, n_elems, dtype, op, &n_words)) return rc;
+    if (dtype == RD_BF16) return RD_ERR_UNSUPPORTED;
     rd_stats_t st;
     std::memset(&st, 0, sizeof(st));
     st.bytes_moved = uint64_t(s->p + 1) * uint64_t(n_words) * 4u;

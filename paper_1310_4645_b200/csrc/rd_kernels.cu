@@ -12,6 +12,7 @@
 //                          statically indexed by unrolling the interpreter K times.
 // Partial results that have to wait (at most log2 p of them) live in a per-thread column of shared
 // memory in both.
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -25,10 +26,17 @@ namespace {
 constexpr int kIdxBits = 12;
 constexpr uint32_t kIdxMask = (1u << kIdxBits) - 1;
 
-enum { DT_INT32 = 0, DT_FP32 = 1, DT_INT64 = 2, DT_FP64 = 3 };
+enum { DT_INT32 = 0, DT_FP32 = 1, DT_INT64 = 2, DT_FP64 = 3, DT_BF16 = 4 };
 
-// The kernels move and index the message in 32-bit words; an element is one word or two.
-template <int DT> struct ElemWords { static constexpr int value = DT >= DT_INT64 ? 2 : 1; };
+// The kernels move and index the message in 32-bit words; an element is one word or two, or (bf16) half
+// a word: a word then holds two elements, the lower-addressed one in its low half.
+template <int DT> struct ElemWords { static constexpr int value = (DT == DT_INT64 || DT == DT_FP64) ? 2 : 1; };
+// bf16 elements are combined in fp32: a word of the message becomes W = 2 words of partial result (two
+// fp32 values), the arithmetic is that of fp32, and only the root's value is rounded back to bf16.
+template <int DT> struct Wide {
+    static constexpr int W = DT == DT_BF16 ? 2 : 1;
+    static constexpr int ADT = DT == DT_BF16 ? DT_FP32 : DT;
+};
 enum { OPR_SUM = 0, OPR_MAX = 1, OPR_MIN = 2, OPR_PROD = 3 };
 
 template <int V> struct Vec { uint32_t w[V]; };
@@ -106,6 +114,37 @@ template <int DT, int OPR, int V> __device__ __forceinline__ void combine_vec(Ve
     }
 }
 
+// A vector of V message words as V * W words of partial result, and back (bf16: exact widening, one
+// rounding to nearest even on the way back; other types: the same words).
+template <int DT, int V> __device__ __forceinline__ Vec<V * Wide<DT>::W> widen(const Vec<V> &m)
+{
+    Vec<V * Wide<DT>::W> a;
+    if constexpr (Wide<DT>::W == 1) {
+#pragma unroll
+        for (int v = 0; v < V; v++) a.w[v] = m.w[v];
+    } else {
+#pragma unroll
+        for (int v = 0; v < V; v++) { a.w[2 * v] = m.w[v] << 16; a.w[2 * v + 1] = m.w[v] & 0xFFFF0000u; }
+    }
+    return a;
+}
+template <int DT, int V> __device__ __forceinline__ Vec<V> narrow(const Vec<V * Wide<DT>::W> &a)
+{
+    Vec<V> m;
+    if constexpr (Wide<DT>::W == 1) {
+#pragma unroll
+        for (int v = 0; v < V; v++) m.w[v] = a.w[v];
+    } else {
+#pragma unroll
+        for (int v = 0; v < V; v++) {
+            const uint32_t lo = __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(a.w[2 * v])));
+            const uint32_t hi = __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(a.w[2 * v + 1])));
+            m.w[v] = lo | (hi << 16);
+        }
+    }
+    return m;
+}
+
 // Sum and product give the same bits whichever operand was held (IEEE add and multiply commute).
 template <int OPR> struct Commutes { static constexpr bool value = OPR == OPR_SUM || OPR == OPR_PROD; };
 
@@ -129,8 +168,10 @@ template <int DT, int OPR, int V, int U, int K, bool PACKED>
 __global__ void __launch_bounds__(kTreeThreads, 2)
 rd_tree_kernel(const __grid_constant__ TreeParams<PACKED> a)
 {
+    constexpr int AV = V * Wide<DT>::W;                       // words of partial result per vector
+    constexpr int ADT = Wide<DT>::ADT;
     extern __shared__ uint4 stack_raw[];
-    Vec<V> *stack = reinterpret_cast<Vec<V> *>(stack_raw);   // [depth][U][threads]
+    Vec<AV> *stack = reinterpret_cast<Vec<AV> *>(stack_raw);  // [depth][U][threads]
     const uint32_t tid = threadIdx.x;
     const int p = a.p;
 
@@ -154,11 +195,11 @@ rd_tree_kernel(const __grid_constant__ TreeParams<PACKED> a)
                     if (live[u]) ring[k][u] = load_stream<V>(src + eoff[u]);
             }
         }
-        Vec<V> top[U];
+        Vec<AV> top[U];
 #pragma unroll
         for (int u = 0; u < U; u++)
 #pragma unroll
-            for (int v = 0; v < V; v++) top[u].w[v] = 0;
+            for (int v = 0; v < AV; v++) top[u].w[v] = 0;
         int sp = 0;
         for (int base = 0; base < p; base += K) {
 #pragma unroll
@@ -166,9 +207,9 @@ rd_tree_kernel(const __grid_constant__ TreeParams<PACKED> a)
                 const int i = base + k;
                 if (i < p) {
                     const uint32_t w = __ldg(prog + i);
-                    Vec<V> x[U];
+                    Vec<AV> x[U];
 #pragma unroll
-                    for (int u = 0; u < U; u++) x[u] = ring[k][u];
+                    for (int u = 0; u < U; u++) x[u] = widen<DT, V>(ring[k][u]);
                     if (i + K < p) {                       // refill this ring slot, K operations ahead
                         const uint32_t *src = a.input(__ldg(prog + i + K) & kIdxMask) + td.elem_off;
 #pragma unroll
@@ -186,10 +227,10 @@ rd_tree_kernel(const __grid_constant__ TreeParams<PACKED> a)
                         for (int u = 0; u < U; u++) top[u] = x[u];
                     } else if (kind == 2u || Commutes<OPR>::value) {   // ACC_IN (a sum does not care who held what)
 #pragma unroll
-                        for (int u = 0; u < U; u++) combine_vec<DT, OPR, V>(top[u], top[u], x[u]);
+                        for (int u = 0; u < U; u++) combine_vec<ADT, OPR, AV>(top[u], top[u], x[u]);
                     } else {                               // ACC_HELD
 #pragma unroll
-                        for (int u = 0; u < U; u++) combine_vec<DT, OPR, V>(top[u], x[u], top[u]);
+                        for (int u = 0; u < U; u++) combine_vec<ADT, OPR, AV>(top[u], x[u], top[u]);
                     }
                     uint32_t npop = (w >> (kIdxBits + 2)) & 0xFu;
                     uint32_t roles = w >> (kIdxBits + 6);
@@ -199,9 +240,9 @@ rd_tree_kernel(const __grid_constant__ TreeParams<PACKED> a)
                         roles >>= 1;
 #pragma unroll
                         for (int u = 0; u < U; u++) {
-                            const Vec<V> y = stack[(sp * U + u) * kTreeThreads + tid];
-                            if (poppedHeld || Commutes<OPR>::value) combine_vec<DT, OPR, V>(top[u], y, top[u]);
-                            else combine_vec<DT, OPR, V>(top[u], top[u], y);
+                            const Vec<AV> y = stack[(sp * U + u) * kTreeThreads + tid];
+                            if (poppedHeld || Commutes<OPR>::value) combine_vec<ADT, OPR, AV>(top[u], y, top[u]);
+                            else combine_vec<ADT, OPR, AV>(top[u], top[u], y);
                         }
                     }
                 }
@@ -209,7 +250,7 @@ rd_tree_kernel(const __grid_constant__ TreeParams<PACKED> a)
         }
 #pragma unroll
         for (int u = 0; u < U; u++)
-            if (live[u]) store_stream<V>(a.out + td.elem_off + eoff[u], top[u]);
+            if (live[u]) store_stream<V>(a.out + td.elem_off + eoff[u], narrow<DT, V>(top[u]));
     }
 }
 
@@ -376,6 +417,60 @@ template <bool PACKED> struct ManyJobs {
     __device__ __forceinline__ int p() const { return cur.p; }
 };
 
+// What a consumer thread carries for its (up to) two 128-bit vectors of a stage: the vectors themselves,
+// or (bf16) their elements widened to fp32, twice as many words.
+template <int DT> struct StageAcc {
+    static constexpr int W = Wide<DT>::W;
+    static constexpr int ADT = Wide<DT>::ADT;
+    Vec<4> v[2 * W];
+    __device__ __forceinline__ void clear()
+    {
+#pragma unroll
+        for (int k = 0; k < 2 * W; k++)
+#pragma unroll
+            for (int e = 0; e < 4; e++) v[k].w[e] = 0;
+    }
+    __device__ __forceinline__ void load(const uint4 &r0, const uint4 &r1)
+    {
+        const Vec<4> m0 = {{r0.x, r0.y, r0.z, r0.w}}, m1 = {{r1.x, r1.y, r1.z, r1.w}};
+        const Vec<4 * W> a0 = widen<DT, 4>(m0), a1 = widen<DT, 4>(m1);
+#pragma unroll
+        for (int k = 0; k < W; k++)
+#pragma unroll
+            for (int e = 0; e < 4; e++) { v[k].w[e] = a0.w[4 * k + e]; v[W + k].w[e] = a1.w[4 * k + e]; }
+    }
+    // *this = combine(held, in); *this may be either of them
+    template <int OPR> __device__ __forceinline__ void combine(const StageAcc &held, const StageAcc &in)
+    {
+#pragma unroll
+        for (int k = 0; k < 2 * W; k++) combine_vec<ADT, OPR, 4>(v[k], held.v[k], in.v[k]);
+    }
+    // one stack level: [vector][consumer thread], the first stage vector's words first
+    __device__ __forceinline__ void push(uint4 *level, uint32_t tid, bool two) const
+    {
+#pragma unroll
+        for (int k = 0; k < 2 * W; k++)
+            if (k < W || two) level[k * kConsumers + tid] = make_uint4(v[k].w[0], v[k].w[1], v[k].w[2], v[k].w[3]);
+    }
+    __device__ __forceinline__ void pop(const uint4 *level, uint32_t tid, bool two)
+    {
+#pragma unroll
+        for (int k = 0; k < 2 * W; k++) {
+            const uint4 y = (k < W || two) ? level[k * kConsumers + tid] : make_uint4(0, 0, 0, 0);
+            v[k].w[0] = y.x; v[k].w[1] = y.y; v[k].w[2] = y.z; v[k].w[3] = y.w;
+        }
+    }
+    __device__ __forceinline__ void result(Vec<4> &o0, Vec<4> &o1) const
+    {
+        Vec<4 * W> a0, a1;
+#pragma unroll
+        for (int k = 0; k < W; k++)
+#pragma unroll
+            for (int e = 0; e < 4; e++) { a0.w[4 * k + e] = v[k].w[e]; a1.w[4 * k + e] = v[W + k].w[e]; }
+        o0 = narrow<DT, 4>(a0); o1 = narrow<DT, 4>(a1);
+    }
+};
+
 template <int DT, int OPR, typename PRM>
 __global__ void __launch_bounds__(kStreamThreads, 3)
 rd_tree_stream_kernel(const __grid_constant__ PRM a)
@@ -386,8 +481,8 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
     const uint32_t stageVecs = uint32_t(a.stage_elems) / 4u;                                 // 128-bit vectors per stage
     uint4 *ring = reinterpret_cast<uint4 *>(smem_raw);                                       // [S][stageVecs]
     const bool two = a.stage_elems > 4 * kConsumers;                                         // a second vector per thread
-    const uint32_t levelVecs = two ? 2u * kConsumers : uint32_t(kConsumers);
-    uint4 *stack = ring + size_t(S) * stageVecs;                                              // [depth][1 or 2][256]
+    const uint32_t levelVecs = (two ? 2u : 1u) * uint32_t(Wide<DT>::W) * kConsumers;
+    uint4 *stack = ring + size_t(S) * stageVecs;                                              // [depth][(1 or 2) * W][256]
     uint64_t *full = reinterpret_cast<uint64_t *>(stack + size_t(a.depth) * levelVecs);
     uint64_t *empty = full + S;
     __shared__ int abort_flag;
@@ -471,9 +566,8 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
         const uint32_t *prog = jobs.ops() + td.prog;
         const uint32_t len = td.len & kLenMask;                       // padded to whole 128-bit vectors
         const bool live0 = tid * 4u < len, live1 = (kConsumers + tid) * 4u < len;
-        Vec<4> top0, top1;
-#pragma unroll
-        for (int v = 0; v < 4; v++) { top0.w[v] = 0; top1.w[v] = 0; }
+        StageAcc<DT> top;
+        top.clear();
         int sp = 0;
         uint32_t w = __ldg(prog);
         for (int i = 0; i < p; i++) {
@@ -486,23 +580,19 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
             uint4 r0 = make_uint4(0, 0, 0, 0), r1 = make_uint4(0, 0, 0, 0);
             if (live0) r0 = st[tid];
             if (live1) r1 = st[kConsumers + tid];
-            Vec<4> x0, x1;
-            x0.w[0] = r0.x; x0.w[1] = r0.y; x0.w[2] = r0.z; x0.w[3] = r0.w;
-            x1.w[0] = r1.x; x1.w[1] = r1.y; x1.w[2] = r1.z; x1.w[3] = r1.w;
+            StageAcc<DT> x;
+            x.load(r0, r1);
             const uint32_t kind = (w >> kIdxBits) & 3u;
             if (kind == 1u) {
-                stack[sp * levelVecs + tid] = make_uint4(top0.w[0], top0.w[1], top0.w[2], top0.w[3]);
-                if (two) stack[sp * levelVecs + kConsumers + tid] = make_uint4(top1.w[0], top1.w[1], top1.w[2], top1.w[3]);
+                top.push(stack + sp * levelVecs, tid, two);
                 sp++;
             }
             if (kind <= 1u) {
-                top0 = x0; top1 = x1;
+                top = x;
             } else if (kind == 2u || Commutes<OPR>::value) {
-                combine_vec<DT, OPR, 4>(top0, top0, x0);
-                combine_vec<DT, OPR, 4>(top1, top1, x1);
+                top.template combine<OPR>(top, x);
             } else {
-                combine_vec<DT, OPR, 4>(top0, x0, top0);
-                combine_vec<DT, OPR, 4>(top1, x1, top1);
+                top.template combine<OPR>(x, top);
             }
             // the stage's data is in registers: hand the stage back to the producer
             __syncwarp();
@@ -514,19 +604,15 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
                 sp--;
                 const bool poppedHeld = (roles & 1u) != 0;
                 roles >>= 1;
-                const uint4 y0 = stack[sp * levelVecs + tid];
-                const uint4 y1 = two ? stack[sp * levelVecs + kConsumers + tid] : make_uint4(0, 0, 0, 0);
-                const Vec<4> ya = {{y0.x, y0.y, y0.z, y0.w}}, yb = {{y1.x, y1.y, y1.z, y1.w}};
-                if (poppedHeld || Commutes<OPR>::value) {
-                    combine_vec<DT, OPR, 4>(top0, ya, top0);
-                    combine_vec<DT, OPR, 4>(top1, yb, top1);
-                } else {
-                    combine_vec<DT, OPR, 4>(top0, top0, ya);
-                    combine_vec<DT, OPR, 4>(top1, top1, yb);
-                }
+                StageAcc<DT> y;
+                y.pop(stack + sp * levelVecs, tid, two);
+                if (poppedHeld || Commutes<OPR>::value) top.template combine<OPR>(y, top);
+                else top.template combine<OPR>(top, y);
             }
             w = wn;
         }
+        Vec<4> top0, top1;
+        top.result(top0, top1);
         // A segment may begin or end inside a vector: the tile then starts / ends with a vector whose other
         // elements belong to the neighbouring segment (another tile writes those); only this tile's are stored.
         uint32_t *dst = jobs.out() + td.elem_off;
@@ -662,7 +748,7 @@ cudaError_t launch_one(const TreeLaunch &l)
     prm.tiles = l.tiles; prm.ops = l.ops; prm.n_tiles = l.n_tiles; prm.p = l.p;
     auto kernel = rd_tree_kernel<DT, OPR, V, kU, kK, PACKED>;
     const int depth = l.stack_depth > 0 ? l.stack_depth : 1;
-    const size_t smem = size_t(depth) * kU * kTreeThreads * sizeof(Vec<V>);
+    const size_t smem = size_t(depth) * kU * kTreeThreads * sizeof(Vec<V * Wide<DT>::W>);
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
     if (e != cudaSuccess) return e;
     int perSm = 0;
@@ -688,7 +774,7 @@ template <int DT, int OPR, typename PRM>
 cudaError_t launch_stream_kernel(const PRM &prm, uint32_t n_ctas, int device, void *stream)
 {
     auto kernel = rd_tree_stream_kernel<DT, OPR, PRM>;
-    const size_t smem = stream_smem_bytes(prm.stages, prm.depth, prm.stage_elems);
+    const size_t smem = stream_smem_bytes(prm.stages, prm.depth, prm.stage_elems, Wide<DT>::W);
     static size_t configured[64] = {};     // per device: largest dynamic shared memory size opted into so far
     const int dv = device & 63;
     if (smem > configured[dv]) {
@@ -780,11 +866,12 @@ cudaError_t launch_direct_dtop(const TreeLaunch &l)
 uint32_t tree_tile_elems(int vec) { return uint32_t(kTreeThreads) * kU * uint32_t(vec); }
 
 // One stack level holds one 128-bit vector per consumer thread, two when a stage has more than 1024 elements.
-static int stack_level_bytes(int stage_elems) { return (stage_elems > 4 * kConsumers ? 2 : 1) * kConsumers * 16; }
+// (acc_words: words of partial result per message word, 2 for bf16 whose elements are combined in fp32, else 1)
+static int stack_level_bytes(int stage_elems, int acc_words) { return (stage_elems > 4 * kConsumers ? 2 : 1) * acc_words * kConsumers * 16; }
 
-size_t stream_smem_bytes(int stages, int depth, int stage_elems)
+size_t stream_smem_bytes(int stages, int depth, int stage_elems, int acc_words)
 {
-    return size_t(stages) * size_t(stage_elems) * 4 + size_t(depth) * stack_level_bytes(stage_elems) + size_t(2 * stages) * sizeof(uint64_t);
+    return size_t(stages) * size_t(stage_elems) * 4 + size_t(depth) * stack_level_bytes(stage_elems, acc_words) + size_t(2 * stages) * sizeof(uint64_t);
 }
 
 int stream_stage_elems(uint64_t elems_per_cta)
@@ -795,12 +882,12 @@ int stream_stage_elems(uint64_t elems_per_cta)
     return kMaxStageElems;
 }
 
-void stream_shape(int stack_depth, int smem_per_sm, int stage_elems, uint64_t n_tiles, int sm_count, int *ctas_per_sm, int *stages)
+void stream_shape(int stack_depth, int acc_words, int smem_per_sm, int stage_elems, uint64_t n_tiles, int sm_count, int *ctas_per_sm, int *stages)
 {
     const int depth = stack_depth > 0 ? stack_depth : 1;
     const int stageBytes = stage_elems * 4;
     // Stages that fit when `ctas` CTAs share an SM (room left for the per-CTA reserve and statics).
-    auto fit = [&](int ctas) { return (smem_per_sm / ctas - 2048 - depth * stack_level_bytes(stage_elems) - 512) / stageBytes; };
+    auto fit = [&](int ctas) { return (smem_per_sm / ctas - 2048 - depth * stack_level_bytes(stage_elems, acc_words) - 512) / stageBytes; };
     // Measured on B200: with many tiles per CTA, three CTAs with 4 stages each stream 3-7 % more than two
     // with 6 to 13 (6.8-7.0 TB/s for 3 to 256 processes); the bytes in flight are no more, the third set
     // of consumers is what helps (three CTAs with 5 stages are behind 4, and 3 stages are too few to hide
@@ -843,6 +930,7 @@ template <typename F> cudaError_t with_type_and_op(int dtype, int op, F &&f)
     case DT_INT32: return with_op<DT_INT32>(op, f);
     case DT_FP32: return with_op<DT_FP32>(op, f);
     case DT_INT64: return with_op<DT_INT64>(op, f);
+    case DT_BF16: return with_op<DT_BF16>(op, f);
     default: return with_op<DT_FP64>(op, f);
     }
 }
@@ -856,7 +944,11 @@ struct BatchLauncher {
 };
 struct DirectLauncher {
     const TreeLaunch &l;
-    template <int DT, int OPR> cudaError_t operator()() const { return launch_direct_dtop<DT, OPR>(l); }
+    template <int DT, int OPR> cudaError_t operator()() const
+    {
+        if constexpr (DT == DT_BF16) return cudaErrorInvalidValue;      // bf16 goes through the streaming kernel
+        else return launch_direct_dtop<DT, OPR>(l);
+    }
 };
 struct ElementLauncher {
     const TreeLaunch &l;

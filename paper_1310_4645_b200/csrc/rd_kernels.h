@@ -73,8 +73,8 @@ int launch_tree(const TreeLaunch &a);
 // Streaming variant (128-bit path): stage size for a CTA's share of the message, ring shape for a
 // stack depth and the SM's shared memory, launch.
 int stream_stage_elems(uint64_t elems_per_cta);
-void stream_shape(int stack_depth, int smem_per_sm, int stage_elems, uint64_t n_tiles, int sm_count, int *ctas_per_sm, int *stages);
-size_t stream_smem_bytes(int stages, int depth, int stage_elems);
+void stream_shape(int stack_depth, int acc_words, int smem_per_sm, int stage_elems, uint64_t n_tiles, int sm_count, int *ctas_per_sm, int *stages);
+size_t stream_smem_bytes(int stages, int depth, int stage_elems, int acc_words);
 int launch_tree_stream(const TreeLaunch &a);
 // Direct variant (128-bit path, at most kDirectMaxProcs processes): all operands of a thread's elements
 // are fetched into registers at once.  Uses the streaming variant's tiles.

@@ -737,3 +737,102 @@ def test_config2_as_batches_over_two_streams_as_the_benchmark_issues_it():
     finally:
         for h in hs:
             rd.rd_destroy(h)
+
+
+# ---------------------------------------------------------------------------------------------
+# bf16 elements combined in fp32 (tree mode): every schedule and operation against the oracle's
+# bit patterns; the oracle widens, combines in fp32 in schedule order and rounds once at the root.
+# ---------------------------------------------------------------------------------------------
+def bf16_inputs(p, n, kind, seed):
+    g = torch.Generator("cuda").manual_seed(seed)
+    if kind == "small_int":
+        return torch.randint(-3, 4, (p, n), device="cuda", generator=g).to(torch.bfloat16)
+    x = torch.empty((p, n), device="cuda")
+    if kind == "near_one":
+        x.uniform_(0.5, 2.0, generator=g)
+        x *= torch.randint(0, 2, x.shape, device="cuda", generator=g) * 2.0 - 1.0
+    else:
+        x.normal_(generator=g)
+        x *= 10.0 ** torch.randint(-4, 5, x.shape, device="cuda", generator=g)
+    return x.to(torch.bfloat16)
+
+
+def bits(t):
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def check_bf16(algo, port, x, seg_bytes, op, rows=None, out=None):
+    p, n = x.shape                                                   # n bf16 elements = 2 n bytes
+    h = rd.rd_schedule_create(algo, port, p, 2 * n, seg_bytes, *M1)
+    try:
+        out = torch.full((n,), 7.0, dtype=torch.bfloat16, device="cuda") if out is None else out
+        rd.rd_reduce(h, rows if rows is not None else x, out, OPS[op])
+        torch.cuda.synchronize()
+    finally:
+        rd.rd_destroy(h)
+    ev, off, _ = oracle_schedule(algo, port, p, 2 * n, seg_bytes if seg_bytes else 2 * n, *M1)
+    want = O.reduce(ev, bits(x), off * 2, op)                        # the schedule counts 4-byte words
+    assert bits(out).tobytes() == want.tobytes()
+    return out
+
+
+# (p, n bf16 elements, segment in bf16 elements): tiles hold 4096 of them; ragged tails; segments that
+# begin inside a 128-bit vector (multiples of 2 elements); lengths that are not whole vectors
+SHAPES_BF16 = [(8, 8192, 1024), (5, 20000, 5000), (13, 3 * 4096 + 72, 4096 + 1040), (64, 16384, 2048), (2, 8200, 8200),
+               (33, 12000, 2000), (16, 256, 16), (1, 10000, 2000), (8, 6000, 666), (4, 128, 6), (32, 16384, 4098),
+               (8, 8198, 2000), (5, 14, 4), (3, 6, 2), (8, 12302, 666), (128, 8192, 1024), (300, 4096, 4096)]
+
+
+@pytest.mark.parametrize("name,algo,port", SCHEDULES)
+@pytest.mark.parametrize("kind,op", [("normal", "sum"), ("normal", "max"), ("normal", "min"), ("near_one", "prod"), ("small_int", "sum")])
+def test_bf16_parity(name, algo, port, kind, op):
+    for p, n, seg in SHAPES_BF16:
+        x = bf16_inputs(p, n, kind, seed=p * 1000 + n)
+        out = check_bf16(algo, port, x, 2 * seg, op)
+        if kind == "small_int":                                      # exact for any order
+            assert torch.equal(out.float(), x.float().sum(dim=0))
+        elif op in ("max", "min"):
+            assert torch.equal(out, x.amax(dim=0) if op == "max" else x.amin(dim=0))
+
+
+def test_bf16_partial_results_stay_in_fp32_and_ties_round_to_even():
+    """1 + 2^-9 + 2^-9 + 2^-9 through a pipeline: 1 + 2^-7 when the partial sums are fp32 (1 if they were
+    rounded to bf16 each time); 1 + 2 * 2^-9 is a tie and goes to the even neighbour 1."""
+    n = 4096 * 3
+    x = torch.full((4, n), 2.0 ** -9, dtype=torch.bfloat16, device="cuda")
+    x[3] = 1.0
+    out = check_bf16(rd.RD_PIPELINE, rd.RD_PORT_UNI, x, 2 * 4096, "sum")
+    assert (out.float() == 1 + 2.0 ** -7).all()
+    out = check_bf16(rd.RD_PIPELINE, rd.RD_PORT_UNI, x[1:].contiguous(), 2 * 4096, "sum")
+    assert (out.float() == 1.0).all()
+
+
+def test_bf16_buffers_off_the_vector_boundary_and_batches():
+    """Buffers 4 bytes into a 128-bit vector take the element path; a batch of bf16 jobs is one launch."""
+    p, n = 8, 6006
+    big = bf16_inputs(p, n + 2, "normal", seed=5)
+    rows = [big[i, 2:] for i in range(p)]
+    assert rows[0].data_ptr() % 16 == 4
+    out_big = torch.zeros(n + 2, dtype=torch.bfloat16, device="cuda")
+    check_bf16(rd.RD_BI_GREEDY, rd.RD_PORT_BI, big[:, 2:], 2 * 1024, "sum", rows=rows, out=out_big[2:])
+    assert out_big[0].item() == 0.0 and out_big[1].item() == 0.0
+    with pytest.raises(rd.RdError) as e:                             # 2 bytes off a word: refused
+        check_bf16(rd.RD_PIPELINE, rd.RD_PORT_UNI, big[:, 1:-1], 2 * 1024, "sum", rows=[big[i, 1:-1] for i in range(p)],
+                   out=out_big[1:-1])
+    assert e.value.status == rd.RD_ERR_INVALID_ARG
+    shapes = [(8, 8192, 1024), (13, 12304, 2 * 333), (64, 4096 * 5, 4096), (2, 8200, 8200)]
+    hs = [rd.rd_schedule_create(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, p, 2 * n, 2 * seg, *M1) for p, n, seg in shapes]
+    try:
+        xs = [bf16_inputs(p, n, "normal", seed=k) for k, (p, n, seg) in enumerate(shapes)]
+        outs = [torch.empty(n, dtype=torch.bfloat16, device="cuda") for p, n, seg in shapes]
+        rd.rd_reduce_batch([(h, x, o) for h, x, o in zip(hs, xs, outs)], rd.RD_SUM)
+        torch.cuda.synchronize()
+        for (p, n, seg), x, o in zip(shapes, xs, outs):
+            ev, off, _ = oracle_schedule(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, p, 2 * n, 2 * seg, *M1)
+            assert bits(o).tobytes() == O.reduce(ev, bits(x), off * 2, "sum").tobytes()
+        with pytest.raises(rd.RdError) as e:                         # no schedule-faithful execution for bf16
+            rd.rd_reduce(hs[0], xs[0], outs[0], rd.RD_SUM, exec_mode=rd.RD_EXEC_FAITHFUL)
+        assert e.value.status == rd.RD_ERR_UNSUPPORTED
+    finally:
+        for h in hs:
+            rd.rd_destroy(h)
