@@ -41,8 +41,8 @@ WORKLOAD_OPS = {"config1": ["sum"], "config2": ["sum"], "config3": ["sum"], "con
 # dram__bytes_read.sum + dram__bytes_write.sum, mean of three launches, for the batch launch (four reductions)
 # and for a single reduction's launch.  Reported only while the kernel source is the one that was profiled.
 NCU_TRAFFIC = {"workload": "config2",
-               "bytes_per_launch": {"calls": 274.2e6, "batch": 1092.4e6},
-               "kernel_sha256": "50ddfd82fcd64aa230e2eb56ee39a492d5ad30d9084d2cd13199a073186c53eb"}
+               "bytes_per_launch": {"calls": 274.3e6, "batch": 1092.4e6},
+               "kernel_sha256": "b18daf48dfc7b7c3a00f8fcd4fa9e99d3c4c1e6cf9eb4cf950ecf52a0bbdc824"}
 
 
 def profiled_traffic(wname, issue):

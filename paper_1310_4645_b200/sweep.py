@@ -7,8 +7,8 @@ size before comparing, Sections V-B and VII).
 For every case one JSON line: shape, segment size chosen, the schedule's predicted completion time
 under the linear model, measured microseconds and GB/s ((p+1)*m bytes per reduction), and whether the
 result passed its check (integers, max and min: exact against torch's order-free result; fp32 sum:
-|r - r64| <= 1e-5 * sum|x| against an fp64 sum, fp64 sum: the same with 1e-14; on the whole message or
-on sampled slices of it).
+|r - r64| <= 1e-5 * sum|x| against an fp64 sum, fp64 sum: the same with 1e-14, bf16 sum: the fp32 bound plus
+one rounding, 2^-8 |r64|; on the whole message or on sampled slices of it).
 Inputs: uniform random numbers from seed 4 (integers in [-2^20, 2^20], floating point in [-1, 1)), one
 arena per element type (--dtypes), every case a view of its first p*n elements.
 """
@@ -24,8 +24,9 @@ import torch
 from . import binding as rd
 
 ALPHA, BETA, GAMMA = 2e-6, 1e-10, 5e-11
-TORCH_DTYPES = {"int32": torch.int32, "fp32": torch.float32, "int64": torch.int64, "fp64": torch.float64}
-ELEM_BYTES = {"int32": 4, "fp32": 4, "int64": 8, "fp64": 8}
+TORCH_DTYPES = {"int32": torch.int32, "fp32": torch.float32, "int64": torch.int64, "fp64": torch.float64,
+                "bf16": torch.bfloat16}
+ELEM_BYTES = {"int32": 4, "fp32": 4, "int64": 8, "fp64": 8, "bf16": 2}
 SCHEDULES = [("uni_greedy", rd.RD_UNI_GREEDY, rd.RD_PORT_UNI), ("bi_greedy", rd.RD_BI_GREEDY, rd.RD_PORT_BI),
              ("binomial", rd.RD_BINOMIAL, rd.RD_PORT_UNI), ("pipeline", rd.RD_PIPELINE, rd.RD_PORT_UNI),
              ("binary", rd.RD_BINARY, rd.RD_PORT_UNI), ("butterfly", rd.RD_BUTTERFLY, rd.RD_PORT_BI)]
@@ -66,7 +67,10 @@ def check(x, out, op, max_check_elems=1 << 22):
         else:
             ref = xs.to(torch.float64).sum(dim=0)
             mag = xs.to(torch.float64).abs().sum(dim=0)
-            if not bool(((o.to(torch.float64) - ref).abs() <= (1e-5 if x.dtype == torch.float32 else 1e-14) * mag).all()):
+            tol = (1e-14 if x.dtype == torch.float64 else 1e-5) * mag
+            if x.dtype == torch.bfloat16:           # combined in fp32, then one rounding to 8 significant bits
+                tol = tol + 2.0 ** -8 * ref.abs()
+            if not bool(((o.to(torch.float64) - ref).abs() <= tol).all()):
                 return False
     return True
 
