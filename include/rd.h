@@ -287,8 +287,8 @@ RD_API int rd_schedule_set_wait_budget(rd_schedule_t *s, double seconds);
 /*
  * rd_schedule_set_tree_variant -- which kernel serves tree-mode calls whose buffers are all 16-byte
  * aligned (the paper has no counterpart; the result is the same bit for bit).
- *   RD_TREE_AUTO    the library chooses (default): the direct kernel for one or two processes, else
- *                   the streaming kernel.
+ *   RD_TREE_AUTO    the library chooses (default; at present always the streaming kernel, which is
+ *                   the faster one for every process count).
  *   RD_TREE_STREAM  operand tiles are streamed through a shared-memory ring by bulk asynchronous
  *                   copies; any number of processes.
  *   RD_TREE_DIRECT  every thread fetches all p operands of its elements into registers at once; at

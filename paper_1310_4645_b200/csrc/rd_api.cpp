@@ -3,6 +3,7 @@
 
 #include <algorithm>
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <mutex>
@@ -37,7 +38,54 @@ struct BatchLanes {
 };
 BatchLanes g_lanes[kMaxDevices];
 std::mutex g_lanes_mutex;
-constexpr int kDirectAutoProcs = 2;
+
+// Counters for handing tiles out on demand (streaming kernel): a pool of word pairs per device, all zero
+// between launches (the launch that used a pair zeroes it when its last CTA runs dry).  Launch k of the
+// process on a device takes pair k mod kTileCounters, so a pair is shared only by launches that are 65536
+// launches apart.  A launch that is being captured into a CUDA graph takes none (its CTAs work through fixed
+// ranges): a replayed launch would otherwise keep using one pair beside whatever else is running.
+constexpr uint32_t kTileCounters = 1u << 16;
+struct TileCounters {
+    uint32_t *pool = nullptr;
+    bool failed = false;
+    uint32_t next = 0;
+};
+TileCounters g_tile_counters[kMaxDevices];
+std::mutex g_tile_counters_mutex;
+
+uint32_t *next_tile_counter(int device, cudaStream_t stream)
+{
+    if (device < 0 || device >= kMaxDevices) return nullptr;
+    if (stream) {
+        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(stream, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone) return nullptr;
+    }
+    std::lock_guard<std::mutex> hold(g_tile_counters_mutex);
+    TileCounters &t = g_tile_counters[device];
+    if (!t.pool && !t.failed) {
+        const size_t bytes = size_t(kTileCounters) * 2 * sizeof(uint32_t);
+        if (cudaMalloc(reinterpret_cast<void **>(&t.pool), bytes) != cudaSuccess || cudaMemset(t.pool, 0, bytes) != cudaSuccess) {
+            cudaFree(t.pool);
+            t.pool = nullptr;
+            t.failed = true;
+            (void)cudaGetLastError();
+        }
+    }
+    if (!t.pool) return nullptr;
+    uint32_t *pair = t.pool + 2u * size_t(t.next);
+    t.next = (t.next + 1u) % kTileCounters;
+    return pair;
+}
+
+// After a launch gave up a wait its pair may have been left non-zero: start again from a clean pool.
+void reset_tile_counters(int device)
+{
+    if (device < 0 || device >= kMaxDevices) return;
+    std::lock_guard<std::mutex> hold(g_tile_counters_mutex);
+    TileCounters &t = g_tile_counters[device];
+    if (t.pool) cudaMemset(t.pool, 0, size_t(kTileCounters) * 2 * sizeof(uint32_t));
+}
+constexpr int kDirectAutoProcs = 0;     // the direct kernel is never chosen by the library itself
 constexpr int kTailTiles = 5; // key of the tile table for the elements the 128-bit path leaves over
 
 struct DeviceTables {
@@ -362,10 +410,11 @@ int reduce_tree(rd_schedule *s, const void *const *d_inputs, void *d_out, size_t
     l.out = d_out; l.ops = d.ops; l.p = s->p; l.stack_depth = s->progs.stack_depth;
     l.dtype = int(dtype); l.op = int(op); l.sm_count = d.sm_count; l.stream = stream;
     if (plan) { l.cta_first = plan->cta_first; l.n_ctas = plan->n_ctas; l.stages = plan->stages; }
+    l.tile_counter = wide ? next_tile_counter(d.device, stream) : nullptr;
     l.stage_elems = d.stage_elems; l.status = d.status; l.device = d.device;
-    // Direct kernel: all operands of an element in registers at once.  Chosen by itself for one or two
-    // processes (measured on B200, p = 2: 6.8 TB/s against 6.1-6.2 of the streaming kernel for messages of
-    // 256 MiB and more; from three processes on the streaming kernel is level or ahead).
+    // Direct kernel: all operands of an element in registers at once.  Only on request: since the streaming
+    // kernel hands its tiles out on demand it is ahead for every process count (measured on B200, p = 2,
+    // 1 GiB messages: 7.12 against 6.74 TB/s; p = 4: 7.24 against 6.94).
     const bool direct = wide && dtype != RD_BF16 && direct_applies(s->p, s->progs.stack_depth) &&
                         (s->tree_variant == RD_TREE_DIRECT || (s->tree_variant == RD_TREE_AUTO && s->p <= kDirectAutoProcs));
     if (stats && cudaEventRecord(d.ev_start, stream) != cudaSuccess) return RD_ERR_CUDA;
@@ -570,6 +619,7 @@ int reduce_batch_fused(size_t n_jobs, rd_schedule_t *const *schedules, const voi
     b.n_jobs = uint32_t(n_jobs); b.n_tiles = uint32_t(total); b.n_ctas = uint32_t(ctas);
     b.stages = stages; b.stack_depth = depth; b.stage_elems = stageElems;
     b.dtype = int(dtype); b.op = int(op); b.device = device; b.status = d0.status; b.stream = user;
+    b.tile_counter = next_tile_counter(device, user);
     if (n_jobs <= size_t(kBatchPackJobs) && nPtrs <= size_t(kBatchPackPtrs)) {
         // small batch: descriptors and pointers travel as kernel parameters, nothing is copied ahead of the launch
         std::vector<const void *> ptrs(nPtrs);
@@ -929,7 +979,10 @@ int rd_schedule_status(rd_schedule_t *s, int *device_status)
     if (cudaGetDevice(&prev) != cudaSuccess || cudaSetDevice(s->dev.device) != cudaSuccess) return RD_ERR_CUDA;
     bool ok = cudaDeviceSynchronize() == cudaSuccess;
     ok = ok && cudaMemcpy(&st, s->dev.status, sizeof(int), cudaMemcpyDeviceToHost) == cudaSuccess;
-    if (ok && st != 0) ok = cudaMemset(s->dev.status, 0, sizeof(int)) == cudaSuccess;
+    if (ok && st != 0) {
+        ok = cudaMemset(s->dev.status, 0, sizeof(int)) == cudaSuccess;
+        reset_tile_counters(s->dev.device);          // the device is idle here
+    }
     cudaSetDevice(prev);
     if (!ok) return RD_ERR_CUDA;
     *device_status = st;

@@ -339,8 +339,11 @@ template <bool PACKED> struct StreamParams {
     TreeParams<PACKED> t;
     const uint32_t *cta_first;   // per CTA: first tile; n_ctas + 1 entries
     int *status;                 // device word: 0, or the first error code
+    uint32_t *tile_counter;      // two device words (next tile, CTAs done), both 0 at launch: tiles are handed out
+                                 // on demand; null: every CTA works through its own range
     int stages, depth, stage_elems;
     __device__ __forceinline__ void tile_range(uint32_t cta, uint32_t &t0, uint32_t &t1) const { t0 = cta_first[cta]; t1 = cta_first[cta + 1]; }
+    __device__ __forceinline__ uint32_t total_tiles() const { return t.n_tiles; }
 };
 
 // A batch: job descriptors and input pointers either inside the kernel's parameters (small batches: nothing
@@ -353,7 +356,9 @@ template <> struct BatchStreamParams<true> {
     const uint32_t *ptrs[kBatchPackPtrs];
     uint32_t n_jobs, n_tiles;
     int *status;
+    uint32_t *tile_counter;
     int stages, depth, stage_elems;
+    __device__ __forceinline__ uint32_t total_tiles() const { return n_tiles; }
     __device__ __forceinline__ BatchJob job(uint32_t j) const { return jobs[j]; }
     __device__ __forceinline__ uint32_t job_end(uint32_t j) const { return jobs[j].tile_end; }
     __device__ __forceinline__ const uint32_t *input(const BatchJob &b, uint32_t i) const { return ptrs[uint32_t(b.ptr_base) + i]; }
@@ -367,7 +372,9 @@ template <> struct BatchStreamParams<false> {
     const BatchJob *jobs;        // device; n_jobs descriptors, tile ranges ascending
     uint32_t n_jobs, n_tiles;
     int *status;
+    uint32_t *tile_counter;
     int stages, depth, stage_elems;
+    __device__ __forceinline__ uint32_t total_tiles() const { return n_tiles; }
     __device__ __forceinline__ BatchJob job(uint32_t j) const { return jobs[j]; }
     __device__ __forceinline__ uint32_t job_end(uint32_t j) const { return jobs[j].tile_end; }
     __device__ __forceinline__ const uint32_t *input(const BatchJob &b, uint32_t i) const
@@ -415,6 +422,99 @@ template <bool PACKED> struct ManyJobs {
     __device__ __forceinline__ const uint32_t *input(uint32_t i) const { return a.input(cur, i); }
     __device__ __forceinline__ uint32_t *out() const { return cur.out; }
     __device__ __forceinline__ int p() const { return cur.p; }
+};
+
+// ---- which tiles a CTA works on.  One producer thread decides (from the CTA's own range, or by taking
+// the next tile from a counter all CTAs of the launch share, so that CTAs which get through their tiles
+// faster take more of them) and publishes the sequence through a small queue in shared memory; the other
+// producer and the consumers read it.  An entry is written long before it is needed and overwritten only
+// kTileQ tiles later, when every reader is past it (nobody is more than a ring of stages, i.e. at most
+// kMaxStages tiles, behind the writer).
+constexpr uint32_t kNoTile = 0xFFFFFFFFu;
+constexpr uint32_t kTileQ = 64;
+static_assert(kTileQ > uint32_t(kMaxStages) + 2u, "a queue entry must outlive the ring's look-ahead");
+
+struct TileQueue {
+    uint32_t slot[kTileQ];
+    uint32_t published;          // entries written so far
+};
+
+// Reader side: the k-th tile of this CTA, kNoTile after the last one.  Bounded wait; when it gives up (or
+// another thread of the CTA already did) the CTA winds down: kNoTile, with the error recorded.
+__device__ __forceinline__ uint32_t tile_at(TileQueue *q, uint32_t k, volatile int *abort_flag, int *status)
+{
+    volatile uint32_t *pub = &q->published;
+    if (*pub <= k) {
+        const long long start = clock64();
+        while (*pub <= k) {
+            if (*abort_flag) return kNoTile;
+            if (clock64() - start > kWaitCycles) {
+                atomicCAS(status, 0, -5);
+                *abort_flag = 1;
+                return kNoTile;
+            }
+        }
+    }
+    __threadfence_block();
+    return reinterpret_cast<volatile uint32_t *>(q->slot)[k % kTileQ];
+}
+
+// Writer side (one thread per CTA).  With a shared counter, CTA c starts with tile c and the counter hands
+// out the tiles from the number of CTAs on; the id of the next entry is fetched while the current tile is
+// being issued, so that the counter's round trip to L2 is over when the entry is published.
+struct TileSource {
+    TileQueue *q;
+    uint32_t *counter;           // null: the CTA's own range [next, end)
+    uint32_t next, end, total, base;
+    uint32_t pub;                // entries published
+    uint32_t ahead;              // id fetched for the next entry
+    bool drained;                // the source has returned kNoTile (it is asked no more after that)
+    __device__ __forceinline__ uint32_t fetch()
+    {
+        if (drained) return kNoTile;
+        uint32_t t;
+        if (counter) { t = atomicAdd(counter, 1u) + base; if (t >= total) t = kNoTile; }
+        else { t = next < end ? next++ : kNoTile; }
+        if (t == kNoTile) drained = true;
+        return t;
+    }
+    __device__ __forceinline__ void start(TileQueue *queue, uint32_t *ctr, uint32_t t0, uint32_t t1, uint32_t n)
+    {
+        q = queue; counter = ctr; next = t0; end = t1; total = n; base = gridDim.x; pub = 0; drained = false;
+        if (counter) ahead = blockIdx.x < total ? blockIdx.x : kNoTile;
+        else ahead = fetch();
+        if (ahead == kNoTile) drained = true;
+    }
+    __device__ __forceinline__ void publish_one()
+    {
+        reinterpret_cast<volatile uint32_t *>(q->slot)[pub % kTileQ] = ahead;
+        __threadfence_block();
+        *reinterpret_cast<volatile uint32_t *>(&q->published) = ++pub;
+        ahead = fetch();
+    }
+    // the k-th tile (publishing it if it is not out yet; the fetch for entry k + 1 is then under way)
+    __device__ __forceinline__ uint32_t get(uint32_t k)
+    {
+        while (pub <= k) publish_one();
+        return reinterpret_cast<volatile uint32_t *>(q->slot)[k % kTileQ];
+    }
+    // called after a step of tile k has been issued: entry k + 1 goes out ahead of need
+    __device__ __forceinline__ void poke(uint32_t k)
+    {
+        if (pub == k + 1u) publish_one();
+    }
+    // After the last tile: the CTA that is last to run dry puts the two words back to 0 for the next launch
+    // that is given them.
+    __device__ __forceinline__ void finish(uint32_t n_ctas)
+    {
+        if (!counter) return;
+        while (!drained) (void)fetch();          // (a CTA that stopped early still takes its end marker)
+        __threadfence();
+        if (atomicAdd(counter + 1, 1u) == n_ctas - 1u) {
+            counter[0] = 0u; counter[1] = 0u;
+            __threadfence();
+        }
+    }
 };
 
 // What a consumer thread carries for its (up to) two 128-bit vectors of a stage: the vectors themselves,
@@ -486,12 +586,12 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
     uint64_t *full = reinterpret_cast<uint64_t *>(stack + size_t(a.depth) * levelVecs);
     uint64_t *empty = full + S;
     __shared__ int abort_flag;
+    __shared__ TileQueue tileq;
     const uint32_t tid = threadIdx.x;
-    uint32_t tile0, tile1;
-    a.tile_range(blockIdx.x, tile0, tile1);
 
     if (tid == 0) {
         abort_flag = 0;
+        tileq.published = 0;
         for (int s = 0; s < S; s++) { mbar_init(full + s, 1); mbar_init(empty + s, kConsumers / 32); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -513,13 +613,21 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
         const int P = kProducers < S ? kProducers : S;
         const int j = int(tid - kConsumers) / 32;
         if (j >= P) return;
-        Jobs jobs(a, tile0, tile0 < tile1);
-        uint32_t tile = tile0;
+        TileSource source;                      // used by producer 0 only
+        if (j == 0) {
+            uint32_t tile0 = 0, tile1 = 0;
+            if (!a.tile_counter) a.tile_range(blockIdx.x, tile0, tile1);
+            source.start(&tileq, a.tile_counter, tile0, tile1, a.total_tiles());
+        }
+        uint32_t k = 0;                         // position in this CTA's sequence of tiles
+        uint32_t tile = j == 0 ? source.get(0) : tile_at(&tileq, 0, &abort_flag, a.status);
+        Jobs jobs(a, tile, tile != kNoTile);
         int i = j;
         int p = jobs.p();                       // of the job `tile` belongs to
-        while (tile < tile1 && i >= p) {
-            i -= p; tile++;
-            if (tile < tile1) { jobs.seek(tile); p = jobs.p(); }
+        while (tile != kNoTile && i >= p) {
+            i -= p; k++;
+            tile = j == 0 ? source.get(k) : tile_at(&tileq, k, &abort_flag, a.status);
+            if (tile != kNoTile) { jobs.seek(tile); p = jobs.p(); }
         }
         int stage = j % S;
         uint32_t laps = 0;                      // times this producer has gone round the ring
@@ -528,21 +636,24 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
         bool ok = true, any = false;
         int lastStage = 0;
         uint32_t lastLap = 0;
-        while (tile < tile1) {
+        while (tile != kNoTile) {
             if (tile != cur) { td = jobs.tile(tile); cur = tile; }
             const uint32_t *src = jobs.input(__ldg(jobs.ops() + td.prog + i) & kIdxMask) + td.elem_off;
             if (laps >= 1u && !mbar_wait(empty + stage, (laps - 1u) & 1u, &abort_flag)) { ok = false; break; }
             mbar_expect_tx(full + stage, (td.len & kLenMask) * 4u);
             bulk_load(ring + size_t(stage) * stageVecs, src, (td.len & kLenMask) * 4u, full + stage);
             any = true; lastStage = stage; lastLap = laps;
+            if (j == 0) source.poke(k);
             i += P;
-            while (tile < tile1 && i >= p) {
-                i -= p; tile++;
-                if (tile < tile1) { jobs.seek(tile); p = jobs.p(); }
+            while (tile != kNoTile && i >= p) {
+                i -= p; k++;
+                tile = j == 0 ? source.get(k) : tile_at(&tileq, k, &abort_flag, a.status);
+                if (tile != kNoTile) { jobs.seek(tile); p = jobs.p(); }
             }
             stage += P;
             if (stage >= S) { stage -= S; laps++; }
         }
+        if (j == 0) source.finish(gridDim.x);
         if (!ok) {
             if (!abort_flag) { atomicCAS(a.status, 0, -5); abort_flag = 1; }
             // leave only after this producer's last copy has landed (bounded); its earlier ones were consumed
@@ -558,8 +669,10 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
     const uint32_t lane = tid & 31u;
     int stage = 0;
     uint32_t phase = 0;
-    Jobs jobs(a, tile0, tile0 < tile1);
-    for (uint32_t tile = tile0; tile < tile1; tile++) {
+    uint32_t k = 0;
+    uint32_t tile = tile_at(&tileq, 0, &abort_flag, a.status);
+    Jobs jobs(a, tile, tile != kNoTile);
+    for (; tile != kNoTile; tile = tile_at(&tileq, ++k, &abort_flag, a.status)) {
         jobs.seek(tile);
         const int p = jobs.p();
         const TileDesc td = jobs.tile(tile);
@@ -803,7 +916,7 @@ cudaError_t launch_stream(const TreeLaunch &l)
     }
     prm.t.out = static_cast<uint32_t *>(l.out);
     prm.t.tiles = l.tiles; prm.t.ops = l.ops; prm.t.n_tiles = l.n_tiles; prm.t.p = l.p;
-    prm.cta_first = l.cta_first; prm.status = l.status;
+    prm.cta_first = l.cta_first; prm.status = l.status; prm.tile_counter = l.tile_counter;
     prm.stages = l.stages; prm.depth = l.stack_depth > 0 ? l.stack_depth : 1; prm.stage_elems = l.stage_elems;
     return launch_stream_kernel<DT, OPR>(prm, l.n_ctas, l.device, l.stream);
 }
@@ -818,12 +931,12 @@ cudaError_t launch_stream_batch(const BatchLaunch &b)
             prm.jobs[j] = j < b.n_jobs ? b.host_jobs[j] : BatchJob{nullptr, nullptr, nullptr, nullptr, b.n_tiles, b.n_tiles, 1, 0};
         for (uint32_t i = 0; i < uint32_t(kBatchPackPtrs); i++)
             prm.ptrs[i] = i < b.n_ptrs ? static_cast<const uint32_t *>(b.host_ptrs[i]) : nullptr;
-        prm.n_jobs = b.n_jobs; prm.n_tiles = b.n_tiles; prm.status = b.status;
+        prm.n_jobs = b.n_jobs; prm.n_tiles = b.n_tiles; prm.status = b.status; prm.tile_counter = b.tile_counter;
         prm.stages = b.stages; prm.depth = depth; prm.stage_elems = b.stage_elems;
         return launch_stream_kernel<DT, OPR>(prm, b.n_ctas, b.device, b.stream);
     }
     BatchStreamParams<false> prm;
-    prm.jobs = b.jobs; prm.n_jobs = b.n_jobs; prm.n_tiles = b.n_tiles; prm.status = b.status;
+    prm.jobs = b.jobs; prm.n_jobs = b.n_jobs; prm.n_tiles = b.n_tiles; prm.status = b.status; prm.tile_counter = b.tile_counter;
     prm.stages = b.stages; prm.depth = depth; prm.stage_elems = b.stage_elems;
     return launch_stream_kernel<DT, OPR>(prm, b.n_ctas, b.device, b.stream);
 }

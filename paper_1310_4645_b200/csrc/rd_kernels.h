@@ -37,6 +37,7 @@ struct TreeLaunch {
     int stages;
     int stage_elems;
     int *status;                      // device word
+    uint32_t *tile_counter;           // device: two words, both 0, for handing tiles out on demand; null: fixed ranges
 };
 
 // One reduction of a batch that runs as a single launch of the streaming kernel.
@@ -62,6 +63,7 @@ struct BatchLaunch {
     int stages, stack_depth, stage_elems;
     int dtype, op, device;
     int *status;                      // device word
+    uint32_t *tile_counter;           // as in TreeLaunch
     void *stream;
 };
 int launch_tree_stream_batch(const BatchLaunch &b);

@@ -65,20 +65,19 @@ def test_parity_small_shapes(name, algo, port, dist, op):
 
 @pytest.mark.parametrize("name,algo,port", SCHEDULES)
 @pytest.mark.parametrize("dist,op", [("int_pm2p20", "sum"), ("normal", "sum"), ("normal", "max")])
-def test_parity_small_shapes_on_the_other_kernel(name, algo, port, dist, op):
-    """The library picks the direct kernel for one or two processes and the streaming kernel beyond (the test
-    above); here every shape goes through the kernel it would not get by itself: the streaming kernel
-    for p <= 2, the direct kernel for 3 <= p <= 8.  Same bits."""
+def test_parity_small_shapes_on_the_direct_kernel(name, algo, port, dist, op):
+    """The library picks the streaming kernel by itself (the test above); here every shape with at most 8
+    processes goes through the direct kernel.  Same bits."""
     for p, n, seg in SHAPES:
         if p > 8:
             continue
         x = make_inputs(p, n, dist, seed=p * 1000 + n, device="cuda")
-        check(algo, port, x, 4 * seg, op, variant=rd.RD_TREE_STREAM if p <= 2 else rd.RD_TREE_DIRECT)
+        check(algo, port, x, 4 * seg, op, variant=rd.RD_TREE_DIRECT)
 
 
 def test_launch_shapes_two_and_three_blocks_per_sm():
     """The streaming kernel runs two or three thread blocks per SM depending on the number of tiles and on
-    the stack depth; the direct kernel serves one or two processes.  Every shape, element by element."""
+    the stack depth; the direct kernel runs when asked for.  Every shape, element by element."""
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     seen = set()
     # (p, n, segment elements, schedule): few tiles; between two and three blocks' worth of tiles; many tiles
@@ -88,8 +87,11 @@ def test_launch_shapes_two_and_three_blocks_per_sm():
              (2, 2048 * 9 * sms + 8, 2048 + 520, SCHEDULES[1]), (1, 2048 * 3 + 4, 1000, SCHEDULES[3])]
     for p, n, seg, (name, algo, port) in cases:
         x = make_inputs(p, n, "normal", seed=p + n, device="cuda")
+        variant = rd.RD_TREE_DIRECT if p <= 2 else None
         h = rd.rd_schedule_create(algo, port, p, 4 * n, 4 * seg, *M1)
         try:
+            if variant is not None:
+                rd.rd_schedule_set_tree_variant(h, variant)
             shape = rd.rd_schedule_tree_shape(h)
         finally:
             rd.rd_destroy(h)
@@ -97,7 +99,8 @@ def test_launch_shapes_two_and_three_blocks_per_sm():
         assert shape["n_tiles"] >= n // 2048
         assert (shape["variant"] == rd.RD_TREE_DIRECT) == (p <= 2)
         assert shape["ring_stages"] >= 3 or shape["variant"] == rd.RD_TREE_DIRECT
-        check(algo, port, x, 4 * seg, "sum")
+        check(algo, port, x, 4 * seg, "sum", variant=variant)
+        check(algo, port, x, 4 * seg, "sum")                          # and the library's own choice
     assert (rd.RD_TREE_STREAM, 2) in seen and (rd.RD_TREE_STREAM, 3) in seen and (rd.RD_TREE_DIRECT, 4) in seen
 
 
@@ -164,12 +167,12 @@ def test_parity_eight_byte_elements(name, algo, port, kind, op):
             assert (got == want.cpu().numpy()).all()                   # torch's int64 sum wraps as well
 
 
-def test_eight_byte_elements_on_the_other_kernel():
+def test_eight_byte_elements_on_the_direct_kernel():
     for name, algo, port in SCHEDULES[:5]:
         for p, n, seg in SHAPES64:
             if p > 8:
                 continue
-            v = rd.RD_TREE_STREAM if p <= 2 else rd.RD_TREE_DIRECT
+            v = rd.RD_TREE_DIRECT
             check64(algo, port, inputs64(p, n, "normal64", seed=p + n), 8 * seg, "sum", variant=v)
             check64(algo, port, inputs64(p, n, "int64", seed=p + n), 8 * seg, "max", variant=v)
             check64(algo, port, inputs64(p, n, "near_one", seed=p + n), 8 * seg, "prod", variant=v)
@@ -448,6 +451,7 @@ def test_tree_mode_launches_can_be_replayed_from_a_cuda_graph():
     h2 = rd.rd_schedule_create(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, 2, 4 * n, 2048, *M1)
     o2, w2 = torch.zeros(n, device="cuda"), torch.zeros(n, device="cuda")
     batch = rd.Batch([(h, t, o) for h, t, o in zip(hs, tabs, outs)])
+    rd.rd_schedule_set_tree_variant(h2, rd.RD_TREE_DIRECT)
     rd.rd_reduce_batch(batch, rd.RD_SUM)                 # ordinary calls first
     rd.rd_reduce(h2, xs[0][:2], w2, rd.RD_SUM)
     torch.cuda.synchronize()
