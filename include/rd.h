@@ -223,7 +223,10 @@ RD_API int rd_schedule_program(const rd_schedule_t *s, size_t seg, uint32_t *ops
  *   stats     host, or NULL.
  * The first call on a schedule uploads its tables to the current device
  * (allocates device memory, synchronises); rd_schedule_upload does the same
- * ahead of time.  After one such call per schedule, element type and operation, a
+ * ahead of time.  The first tree-mode call on a device also allocates 512 KiB of counters there,
+ * kept until the process ends: a launch of the streaming kernel hands its tiles to its thread
+ * blocks on demand through one of them (a launch recorded into a CUDA graph uses none and gives
+ * every thread block a fixed range of tiles instead).  After one such call per schedule, element type and operation, a
  * tree-mode call with at most 256 processes is a single kernel launch and may be
  * recorded into a CUDA graph (so may an rd_reduce_batch call of at most 16 aligned jobs with at most
  * 1024 input pointers in all, after one ordinary call of it).  Buffers must be aligned to the element; 16-byte aligned buffers take
