@@ -840,3 +840,42 @@ def test_bf16_buffers_off_the_vector_boundary_and_batches():
     finally:
         for h in hs:
             rd.rd_destroy(h)
+
+
+def test_tiles_on_demand_over_many_launches_and_streams():
+    """The streaming kernel's thread blocks take their tiles from a counter that the launch's last block puts
+    back to zero.  Hundreds of launches of unlike shapes (different numbers of thread blocks and tiles per
+    block, single reductions and batches), alternating over three streams, must all give the bits of a launch
+    issued alone, and no launch may report a wait that gave up."""
+    shapes = [(5, 2048 * 37 + 8, 4 * 3000), (64, 2048 * 300, 16 << 10), (9, 2048 * 1500 + 36, 4 * (2048 + 520)), (3, 2048 * 2, 4096)]
+    hs, xs, refs = [], [], []
+    for k, (p, n, seg) in enumerate(shapes):
+        algo, port = SCHEDULES[k % 4][1:]
+        hs.append(rd.rd_schedule_create(algo, port, p, 4 * n, seg, *M1))
+        xs.append(make_inputs(p, n, "normal", seed=50 + k, device="cuda"))
+        r = torch.empty(n, device="cuda")
+        rd.rd_reduce(hs[-1], xs[-1], r, rd.RD_SUM)
+        refs.append(r)
+    torch.cuda.synchronize()
+    try:
+        streams = [torch.cuda.Stream() for _ in range(3)]
+        outs = [[torch.zeros_like(r) for r in refs] for _ in streams]
+        batch = [rd.Batch([(hs[0], xs[0], o[0]), (hs[3], xs[3], o[3])]) for o in outs]
+        for it in range(120):
+            si = it % 3
+            with torch.cuda.stream(streams[si]):
+                for o in outs[si]:
+                    o.zero_()
+                rd.rd_reduce(hs[1], xs[1], outs[si][1], rd.RD_SUM, stream=streams[si])
+                rd.rd_reduce_batch(batch[si], rd.RD_SUM, stream=streams[si])
+                rd.rd_reduce(hs[2], xs[2], outs[si][2], rd.RD_SUM, stream=streams[si])
+            if it % 30 == 29:
+                torch.cuda.synchronize()
+                for o in outs:
+                    for got, want in zip(o, refs):
+                        assert torch.equal(got.view(torch.int32), want.view(torch.int32))
+        for h in hs:
+            assert rd.rd_schedule_status(h) == 0
+    finally:
+        for h in hs:
+            rd.rd_destroy(h)
