@@ -284,11 +284,8 @@ def main():
     # Batch issue: every job of a step reads its own messages (jobs of one launch that read the same bytes
     # would meet in L2), and steps that may overlap on two streams read different sets of them.
     batch_sets = max(2, args.streams)
-    # rd_reduce_batch does not fuse jobs that fill the GPU by themselves (12 tiles of 2048 words per SM or more):
-    # those workloads are timed as separate calls
-    sms = torch.cuda.get_device_properties(dev).multi_processor_count
-    if args.issue == "batch" and (p * n * 4 * n_plans * batch_sets > (48 << 30) or (n + 2047) // 2048 >= 12 * sms):
-        args.issue = "calls"
+    if args.issue == "batch" and p * n * 4 * n_plans * batch_sets > (48 << 30):
+        args.issue = "calls"                # too much memory for a set of messages per job and stream
     # Call issue: the kernel never reads the arena the previous launch read, and two arenas together exceed L2.
     if args.issue == "batch":
         n_arenas = n_plans * batch_sets

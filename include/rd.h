@@ -243,9 +243,8 @@ RD_API int rd_reduce(rd_schedule_t *s, const void *const *d_inputs, void *d_out,
  * many buffers).  Job j reduces d_inputs[j][0..p_j) into d_outs[j] under schedules[j]; all jobs share
  * dtype, op and stream.  Results are exactly those of n_jobs rd_reduce calls, and the batch as a whole
  * is ordered after what precedes it on cuda_stream and before what follows it.
- *   When every buffer of every job is 16-byte aligned, every message a whole number of 128-bit
- *   vectors and no job large enough to fill the GPU by itself (12 tiles of 2048 words per SM, i.e.
- *   messages of about 14 MiB on a B200), the batch is ONE launch of the streaming kernel: the tiles of all jobs are dealt to the
+ *   When every buffer of every job is 16-byte aligned and every message a whole number of 128-bit
+ *   vectors, the batch is ONE launch of the streaming kernel: the tiles of all jobs are dealt to the
  *   thread blocks as if they were one reduction, so the batch pays one launch, one ring fill and one
  *   tail instead of n_jobs (16 jobs of p = 64 with 1 MiB messages: 6.3 TB/s against 3.5 TB/s for 16
  *   calls; 32 jobs with 256 KiB messages: 5.4 against 1.1 TB/s).  Job descriptors, tile ranges and the

@@ -23,7 +23,6 @@ constexpr int kMaxDevices = 64;
 
 // Side streams of rd_reduce_batch, created on a device's first batch and kept for the process's life.
 constexpr int kBatchRing = 4; // per-call tables of fused batches in flight
-constexpr uint64_t kFuseMaxTilesPerSm = 12;   // a job with this many tiles per SM or more is launched by itself
 struct BatchLanes {
     bool ready = false;
     cudaStream_t stream[2] = {nullptr, nullptr};
@@ -601,10 +600,7 @@ int reduce_batch_fused(size_t n_jobs, rd_schedule_t *const *schedules, const voi
         b.inputs = nullptr; b.out = static_cast<uint32_t *>(d_outs[j]); b.tiles = tiles; b.ops = s->dev.ops;
         b.tile_begin = uint32_t(total); b.p = s->p; b.ptr_base = 0;
         total += count;
-        // Jobs that fill the GPU by themselves gain nothing from sharing a launch, and a shared launch takes
-        // the ring shape of its deepest program (config3's five schedules: 6.58 TB/s fused against 6.6-7.0
-        // one by one): such batches go to the two-stream path.
-        if (total > 0xFFFFFFFFull || uint64_t(count) >= kFuseMaxTilesPerSm * uint64_t(s->dev.sm_count)) return RD_ERR_UNSUPPORTED;
+        if (total > 0xFFFFFFFFull) return RD_ERR_UNSUPPORTED;
         b.tile_end = uint32_t(total);
         nPtrs += size_t(s->p);
         depth = std::max(depth, s->progs.stack_depth);
@@ -853,7 +849,7 @@ int rd_reduce_batch(size_t n_jobs, rd_schedule_t *const *schedules, const void *
         }
         if (fuse) {
             const int rc = reduce_batch_fused(n_jobs, schedules, d_inputs, d_outs, dtype, op, user);
-            if (rc != RD_ERR_UNSUPPORTED) return rc;        // UNSUPPORTED: a job large enough to be launched by itself
+            if (rc != RD_ERR_UNSUPPORTED) return rc;        // UNSUPPORTED: more tiles than one launch can number
         }
         // Fork: two side streams wait for what precedes the batch on the caller's stream and take the
         // jobs alternately, so that one job's thread blocks fill the SM slots the other job frees while
