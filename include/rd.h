@@ -269,7 +269,8 @@ RD_API int rd_schedule_upload(rd_schedule_t *s);
 /*
  * rd_reduce_host -- rd_reduce (tree mode) for messages that live in HOST memory.
  *   h_inputs  HOST array of p HOST pointers (pinned memory makes the copies
- *             asynchronous); h_out HOST, n_elems elements.
+ *             asynchronous; messages that follow each other in memory, such as
+ *             the rows of one array, travel in one copy); h_out HOST, n_elems elements.
  *   d_staging DEVICE; (p + 1) * n_elems elements of scratch owned by the
  *             caller: the p messages are copied there, reduced, and the
  *             result copied back.  The call returns after the result is in

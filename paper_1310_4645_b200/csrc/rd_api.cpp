@@ -894,8 +894,14 @@ int rd_reduce_host(rd_schedule_t *s, const void *const *h_inputs, void *h_out, v
     for (int i = 0; i < s->p; i++) {
         if (n_elems > 0 && !h_inputs[i]) return RD_ERR_INVALID_ARG;
         dptr[size_t(i)] = base + size_t(i) * row;
-        if (n_elems > 0 && cudaMemcpyAsync(base + size_t(i) * row, h_inputs[i], row, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+    }
+    // messages that follow each other in host memory (the rows of one array) travel in one copy
+    for (int i = 0; i < s->p && n_elems > 0;) {
+        int j = i + 1;
+        while (j < s->p && static_cast<const char *>(h_inputs[j]) == static_cast<const char *>(h_inputs[j - 1]) + row) j++;
+        if (cudaMemcpyAsync(base + size_t(i) * row, h_inputs[i], size_t(j - i) * row, cudaMemcpyHostToDevice, stream) != cudaSuccess)
             return RD_ERR_CUDA;
+        i = j;
     }
     void *d_out = base + size_t(s->p) * row;
     if (int rc = rd_reduce(s, dptr.data(), d_out, n_elems, dtype, op, RD_EXEC_TREE, cuda_stream, nullptr)) return rc;

@@ -315,9 +315,20 @@ def test_reduce_host_round_trip():
     staging = torch.empty((p + 1) * n, dtype=torch.float32, device="cuda")
     h = rd.rd_schedule_create(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, p, 4 * n, 4000, *M1)
     rd.rd_reduce_host(h, x, out, staging, rd.RD_SUM)
-    rd.rd_destroy(h)
     ev, off, _ = oracle_schedule(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, p, 4 * n, 4000, *M1)
-    assert out.numpy().tobytes() == O.reduce(ev, x.numpy(), off, "sum").tobytes()
+    want = O.reduce(ev, x.numpy(), off, "sum").tobytes()
+    assert out.numpy().tobytes() == want
+    # rows of one array travel in one copy; rows scattered over the host (here: in reverse order of address,
+    # and two of them in buffers of their own) are copied one by one
+    back = torch.empty((p, n), dtype=torch.float32).pin_memory()
+    rows = [back[p - 1 - i] for i in range(p)]
+    rows[2], rows[5] = torch.empty(n).pin_memory(), torch.empty(n, dtype=torch.float32)        # one of them pageable
+    for i in range(p):
+        rows[i].copy_(x[i])
+    out.zero_()
+    rd.rd_reduce_host(h, rows, out, staging, rd.RD_SUM)
+    rd.rd_destroy(h)
+    assert out.numpy().tobytes() == want
 
 
 @pytest.mark.parametrize("name,algo,port", SCHEDULES[:5])
