@@ -786,8 +786,27 @@ static uint16_t f32_to_bf16(float f)
     return (uint16_t)keep;
 }
 
-int orc_reduce_bf16(const orc_event_t *ev_in, int64_t n_ev, int p, int q, const int64_t *seg_off,
-                    const uint16_t *const *x, uint16_t *out, int op)
+/* fp16 (IEEE binary16) elements, treated the same way: widened exactly, combined in fp32, rounded once at
+ * the root to nearest with ties to even (overflow goes to infinity, small results become subnormal).  The
+ * conversions are the compiler's own for _Float16, which are the IEEE ones.                              */
+static float f16_to_f32(uint16_t h)
+{
+    _Float16 x;
+    memcpy(&x, &h, sizeof x);
+    return (float)x;
+}
+
+static uint16_t f32_to_f16(float f)
+{
+    _Float16 x = (_Float16)f;
+    uint16_t h;
+    memcpy(&h, &x, sizeof h);
+    return h;
+}
+
+static int reduce_half(const orc_event_t *ev_in, int64_t n_ev, int p, int q, const int64_t *seg_off,
+                       const uint16_t *const *x, uint16_t *out, int op,
+                       float (*widen)(uint16_t), uint16_t (*narrow)(float))
 {
     orc_event_t *ev = sorted_by_segment(ev_in, n_ev);
     if (!ev) return ORC_NOMEM;
@@ -799,16 +818,28 @@ int orc_reduce_bf16(const orc_event_t *ev_in, int64_t n_ev, int p, int q, const 
     for (int j = 0; j < q; j++) {
         int64_t len = seg_off[j + 1] - seg_off[j];
         for (int i = 0; i < p; i++)
-            for (int64_t k = 0; k < len; k++) acc[(size_t)i * longest + k] = bf16_to_f32(x[i][seg_off[j] + k]);
+            for (int64_t k = 0; k < len; k++) acc[(size_t)i * longest + k] = widen(x[i][seg_off[j] + k]);
         for (; e < n_ev && ev[e].seg == j; e++) {
             float *held = acc + (size_t)ev[e].dst * longest, *in = acc + (size_t)ev[e].src * longest;
             if (ev[e].kind == 0) for (int64_t k = 0; k < len; k++) held[k] = comb_f32(held[k], in[k], op);
             else for (int64_t k = 0; k < len; k++) held[k] = in[k];
         }
-        for (int64_t k = 0; k < len; k++) out[seg_off[j] + k] = f32_to_bf16(acc[k]);
+        for (int64_t k = 0; k < len; k++) out[seg_off[j] + k] = narrow(acc[k]);
     }
     free(acc); free(ev);
     return ORC_OK;
+}
+
+int orc_reduce_bf16(const orc_event_t *ev_in, int64_t n_ev, int p, int q, const int64_t *seg_off,
+                    const uint16_t *const *x, uint16_t *out, int op)
+{
+    return reduce_half(ev_in, n_ev, p, q, seg_off, x, out, op, bf16_to_f32, f32_to_bf16);
+}
+
+int orc_reduce_f16(const orc_event_t *ev_in, int64_t n_ev, int p, int q, const int64_t *seg_off,
+                   const uint16_t *const *x, uint16_t *out, int op)
+{
+    return reduce_half(ev_in, n_ev, p, q, seg_off, x, out, op, f16_to_f32, f32_to_f16);
 }
 
 /* The same for the 8-byte element types: int64 wraps modulo 2^64, fp64 is one

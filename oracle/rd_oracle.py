@@ -142,9 +142,9 @@ def contributions(events, p, q):
                                        C.c_int(q)))
 
 
-def reduce(events, x, seg_off, op):
-    """O2.  x: array [p, n] of int32, float32, int64, float64, or uint16 holding bf16 bit patterns
-    (C-contiguous); seg_off in elements of x; op 'sum', 'max', 'min' or 'prod'."""
+def reduce(events, x, seg_off, op, half="bf16"):
+    """O2.  x: array [p, n] of int32, float32, int64, float64, or uint16 holding bf16 (half="bf16") or IEEE
+    binary16 (half="fp16") bit patterns (C-contiguous); seg_off in elements of x; op 'sum', 'max', 'min' or 'prod'."""
     events = np.ascontiguousarray(events, dtype=EVENT_DTYPE)
     x = np.ascontiguousarray(x)
     p, n = x.shape
@@ -162,8 +162,8 @@ def reduce(events, x, seg_off, op):
         fn = lib().orc_reduce_i64
     elif x.dtype == np.float64:
         fn = lib().orc_reduce_f64
-    elif x.dtype == np.uint16:                 # bf16 bit patterns: combined in fp32, rounded to bf16 once at the end
-        fn = lib().orc_reduce_bf16
+    elif x.dtype == np.uint16:                 # 16-bit patterns: combined in fp32, rounded once at the end
+        fn = lib().orc_reduce_bf16 if half == "bf16" else lib().orc_reduce_f16
     else:
         raise TypeError(x.dtype)
     rc = fn(C.c_void_p(events.ctypes.data), C.c_int64(len(events)), C.c_int(p), C.c_int(q),

@@ -353,3 +353,56 @@ def test_bf16_sum_is_the_fp32_schedule_sum_rounded(p):
         mag = np.abs(bf16_value(x).astype(np.float64)).sum(axis=0)
         got = bf16_value(O.reduce(ev, x, seg_off(sizes), "sum")).astype(np.float64)
         assert (np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + p * 2.0 ** -23 * mag + 1e-30).all(), name
+
+
+# fp16 (IEEE binary16) elements, combined in fp32 like bf16.
+def f16_bits(a):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=f32)).to(torch.float16).view(torch.int16).numpy().view(np.uint16)
+
+
+def f16_value(bits):
+    return bits.view(np.float16).astype(f32)
+
+
+def test_fp16_two_processes_is_one_fp32_operation_rounded_once():
+    rng = np.random.default_rng(12)
+    x = f16_bits(rng.standard_normal((2, 4000)) * 10.0 ** rng.integers(-3, 3, size=(2, 4000)))
+    ev, _ = O.uni_greedy(2, [2400, 1600], 1, 1, 1)
+    got = O.reduce(ev, x, [0, 2400, 4000], "sum", half="fp16")
+    assert (got == f16_bits(f16_value(x[0]) + f16_value(x[1]))).all()
+    prod = O.reduce(ev, x, [0, 2400, 4000], "prod", half="fp16")
+    assert (prod == f16_bits(f16_value(x[0]) * f16_value(x[1]))).all()
+    # overflow goes to infinity, tiny products to subnormals and zero: whatever torch's conversion says
+    y = f16_bits(np.array([[60000.0, 6e-5, 6e-8, -60000.0], [60000.0, 6e-5, 0.5, 2.0]]))
+    ev, _ = O.uni_greedy(2, [4], 1, 1, 1)
+    assert (O.reduce(ev, y, [0, 4], "sum", half="fp16") == f16_bits(f16_value(y[0]) + f16_value(y[1]))).all()
+    assert (O.reduce(ev, y, [0, 4], "prod", half="fp16") == f16_bits(f16_value(y[0]) * f16_value(y[1]))).all()
+
+
+def test_fp16_ties_to_even_and_fp32_partial_results():
+    """Spacing of fp16 at 1 is 2^-10: 1 + k * 2^-12 for k = 0..8; and 1 + 3 * 2^-12 through a pipeline of four."""
+    ks = np.arange(0, 9)
+    x = np.stack([f16_bits(np.ones(9)), f16_bits(ks * 2.0 ** -12)])
+    ev, _ = O.uni_greedy(2, [9], 1, 1, 1)
+    got = f16_value(O.reduce(ev, x, [0, 9], "sum", half="fp16"))
+    want = 1 + np.array([0, 0, 0, 1, 1, 1, 2, 2, 2]) * 2.0 ** -10
+    assert (got == want.astype(f32)).all()
+    x = np.stack([f16_bits(np.full(8, v)) for v in (2.0 ** -12, 2.0 ** -12, 2.0 ** -12, 1.0)])
+    ev, _ = O.pipeline(4, [8], 1, 1, 1, False)
+    assert (f16_value(O.reduce(ev, x, [0, 8], "sum", half="fp16")) == f32(1 + 2.0 ** -10)).all()
+
+
+@pytest.mark.parametrize("p", [2, 5, 16, 64])
+def test_fp16_small_integers_sum_exactly_and_extrema_are_order_free(p):
+    rng = np.random.default_rng(p)
+    n, sizes = 96, [40, 40, 16]
+    xi = rng.integers(-3, 4, size=(p, n))
+    x = f16_bits(xi.astype(f32))
+    y = f16_bits(rng.standard_normal((p, n)) * 10.0 ** rng.integers(-3, 4, size=(p, n)))
+    for name, ev in schedules(p, sizes):
+        assert (f16_value(O.reduce(ev, x, seg_off(sizes), "sum", half="fp16")) == xi.sum(axis=0)).all(), name
+        assert (f16_value(O.reduce(ev, y, seg_off(sizes), "max", half="fp16")) == f16_value(y).max(axis=0)).all(), name
+        assert (f16_value(O.reduce(ev, y, seg_off(sizes), "min", half="fp16")) == f16_value(y).min(axis=0)).all(), name
+        wide = O.reduce(ev, f16_value(y), seg_off(sizes), "sum")
+        assert (O.reduce(ev, y, seg_off(sizes), "sum", half="fp16") == f16_bits(wide)).all(), name
