@@ -85,13 +85,14 @@ typedef enum { RD_SUM = 0, RD_MAX = 1, RD_MIN = 2, RD_PROD = 3 } rd_op_t;
  * rd_optimal_segment returns multiples of 4, round them up.  Otherwise the reducing calls return
  * RD_ERR_INVALID_ARG.
  *
- * RD_BF16: bf16 elements combined in fp32 (the usual "16-bit storage, 32-bit accumulation"; the paper fixes
- * nothing here).  Every input is widened exactly, partial results are fp32 values combined by one IEEE
- * fp32 operation per combine in the schedule's order, and only what the root holds at the end is rounded
- * to bf16, once, to nearest with ties to even.  n_elems counts bf16 elements (msg_bytes / 2, always
- * even); buffers must be aligned to 4 bytes.  Tree mode only: the schedule-faithful execution would have
- * to hand fp32 partial segments between processes and returns RD_ERR_UNSUPPORTED. */
-typedef enum { RD_INT32 = 0, RD_FP32 = 1, RD_INT64 = 2, RD_FP64 = 3, RD_BF16 = 4 } rd_dtype_t;
+ * RD_BF16, RD_FP16: bf16 / IEEE binary16 elements combined in fp32 (the usual "16-bit storage, 32-bit
+ * accumulation"; the paper fixes nothing here).  Every input is widened exactly, partial results are fp32
+ * values combined by one IEEE fp32 operation per combine in the schedule's order, and only what the root
+ * holds at the end is rounded to 16 bits, once, to nearest with ties to even (fp16: overflow to infinity,
+ * gradual underflow).  n_elems counts 16-bit elements (msg_bytes / 2, always even); buffers must be aligned
+ * to 4 bytes.  Tree mode only: the schedule-faithful execution would have to hand fp32 partial segments
+ * between processes and returns RD_ERR_UNSUPPORTED. */
+typedef enum { RD_INT32 = 0, RD_FP32 = 1, RD_INT64 = 2, RD_FP64 = 3, RD_BF16 = 4, RD_FP16 = 5 } rd_dtype_t;
 typedef enum { RD_EXEC_TREE = 0, RD_EXEC_FAITHFUL = 1 } rd_exec_t;
 
 /* Linear model of Section II.  alpha in seconds, beta and gamma in seconds per

@@ -20,7 +20,7 @@ RD_ERR_TOO_LARGE = -9
 RD_UNI_GREEDY, RD_BI_GREEDY, RD_BINOMIAL, RD_PIPELINE, RD_BINARY, RD_BUTTERFLY = range(6)
 RD_PORT_UNI, RD_PORT_BI = 0, 1
 RD_SUM, RD_MAX, RD_MIN, RD_PROD = 0, 1, 2, 3
-RD_INT32, RD_FP32, RD_INT64, RD_FP64, RD_BF16 = 0, 1, 2, 3, 4
+RD_INT32, RD_FP32, RD_INT64, RD_FP64, RD_BF16, RD_FP16 = 0, 1, 2, 3, 4, 5
 RD_EXEC_TREE, RD_EXEC_FAITHFUL = 0, 1
 RD_TREE_AUTO, RD_TREE_STREAM, RD_TREE_DIRECT = 0, 1, 2
 
@@ -187,7 +187,9 @@ def _dtype_code(t):
         return RD_FP64
     if t.dtype == torch.bfloat16:
         return RD_BF16
-    raise TypeError("int32, float32, int64, float64 or bfloat16 expected, got %s" % t.dtype)
+    if t.dtype == torch.float16:
+        return RD_FP16
+    raise TypeError("int32, float32, int64, float64, bfloat16 or float16 expected, got %s" % t.dtype)
 
 
 class PointerTable:

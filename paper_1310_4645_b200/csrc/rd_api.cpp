@@ -356,12 +356,13 @@ int stream_plan(rd_schedule *s, int acc_words, const DeviceTables::StreamPlan **
 
 // Argument checks common to the reducing entry points.  On success *n_words is the message length
 // in 32-bit words, the unit in which the schedule's segment boundaries and the kernels count.
-size_t elem_bytes(rd_dtype_t dtype) { return (dtype == RD_INT64 || dtype == RD_FP64) ? 8 : dtype == RD_BF16 ? 2 : 4; }
+bool is_half(rd_dtype_t dtype) { return dtype == RD_BF16 || dtype == RD_FP16; }
+size_t elem_bytes(rd_dtype_t dtype) { return (dtype == RD_INT64 || dtype == RD_FP64) ? 8 : is_half(dtype) ? 2 : 4; }
 
 int check_reduce_args(const rd_schedule *s, const void *const *d_inputs, const void *d_out, size_t n_elems, rd_dtype_t dtype,
                       rd_op_t op, size_t *n_words)
 {
-    if (!s || !d_inputs || int(dtype) < RD_INT32 || int(dtype) > RD_BF16 || int(op) < RD_SUM || int(op) > RD_PROD)
+    if (!s || !d_inputs || int(dtype) < RD_INT32 || int(dtype) > RD_FP16 || int(op) < RD_SUM || int(op) > RD_PROD)
         return RD_ERR_INVALID_ARG;
     const size_t esize = elem_bytes(dtype);
     const size_t align = esize < 4 ? 4 : esize;          // the kernels move whole 32-bit words
@@ -390,7 +391,7 @@ int reduce_tree(rd_schedule *s, const void *const *d_inputs, void *d_out, size_t
     if (int rc = tiles_for(s, l.vec, &l.tiles, &l.n_tiles)) return rc;
     const DeviceTables::StreamPlan *plan = nullptr;
     if (wide)
-        if (int rc = stream_plan(s, dtype == RD_BF16 ? 2 : 1, &plan)) return rc;
+        if (int rc = stream_plan(s, is_half(dtype) ? 2 : 1, &plan)) return rc;
     const TileDesc *tailTiles = nullptr;
     uint32_t nTail = 0;
     if (wide && (n & 3u) != 0)
@@ -414,7 +415,7 @@ int reduce_tree(rd_schedule *s, const void *const *d_inputs, void *d_out, size_t
     // Direct kernel: all operands of an element in registers at once.  Only on request: since the streaming
     // kernel hands its tiles out on demand it is ahead for every process count (measured on B200, p = 2,
     // 1 GiB messages: 7.12 against 6.74 TB/s; p = 4: 7.24 against 6.94).
-    const bool direct = wide && dtype != RD_BF16 && direct_applies(s->p, s->progs.stack_depth) &&
+    const bool direct = wide && !is_half(dtype) && direct_applies(s->p, s->progs.stack_depth) &&
                         (s->tree_variant == RD_TREE_DIRECT || (s->tree_variant == RD_TREE_AUTO && s->p <= kDirectAutoProcs));
     if (stats && cudaEventRecord(d.ev_start, stream) != cudaSuccess) return RD_ERR_CUDA;
     if ((direct ? launch_tree_direct(l) : wide ? launch_tree_stream(l) : launch_tree(l)) != 0) return RD_ERR_CUDA;
@@ -609,7 +610,7 @@ int reduce_batch_fused(size_t n_jobs, rd_schedule_t *const *schedules, const voi
     DeviceTables &d0 = schedules[0]->dev;
     const int stageElems = d0.stage_elems;
     int ctasPerSm = 1, stages = 2;
-    stream_shape(depth, dtype == RD_BF16 ? 2 : 1, d0.smem_per_sm, stageElems, total, d0.sm_count, &ctasPerSm, &stages);
+    stream_shape(depth, is_half(dtype) ? 2 : 1, d0.smem_per_sm, stageElems, total, d0.sm_count, &ctasPerSm, &stages);
     const uint64_t ctas = std::min<uint64_t>(uint64_t(d0.sm_count) * uint64_t(ctasPerSm), total);
     BatchLaunch b{};
     b.n_jobs = uint32_t(n_jobs); b.n_tiles = uint32_t(total); b.n_ctas = uint32_t(ctas);
@@ -802,7 +803,7 @@ int rd_reduce(rd_schedule_t *s, const void *const *d_inputs, void *d_out, size_t
     if (exec != RD_EXEC_TREE && exec != RD_EXEC_FAITHFUL) return RD_ERR_INVALID_ARG;
     size_t n_words = 0;
     if (int rc = check_reduce_args(s, d_inputs, d_out, n_elems, dtype, op, &n_words)) return rc;
-    if (exec == RD_EXEC_FAITHFUL && dtype == RD_BF16) return RD_ERR_UNSUPPORTED;   // partial segments would be fp32
+    if (exec == RD_EXEC_FAITHFUL && is_half(dtype)) return RD_ERR_UNSUPPORTED;   // partial segments would be fp32
     return guarded([&] {
         if (int rc = upload(s)) return rc;
         if (exec == RD_EXEC_FAITHFUL)
@@ -884,7 +885,7 @@ int rd_reduce_host(rd_schedule_t *s, const void *const *h_inputs, void *h_out, v
                    rd_dtype_t dtype, rd_op_t op, void *cuda_stream)
 {
     if (!s || !h_inputs || (n_elems > 0 && (!h_out || !d_staging))) return RD_ERR_INVALID_ARG;
-    if (int(dtype) < RD_INT32 || int(dtype) > RD_BF16) return RD_ERR_INVALID_ARG;
+    if (int(dtype) < RD_INT32 || int(dtype) > RD_FP16) return RD_ERR_INVALID_ARG;
     if (n_elems > s->msg_bytes / elem_bytes(dtype) || n_elems * elem_bytes(dtype) != s->msg_bytes) return RD_ERR_SIZE_MISMATCH;
     const size_t row = s->msg_bytes;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -1017,7 +1018,7 @@ int rd_reduce_faithful_static(rd_schedule_t *s, const void *const *d_inputs, voi
 {
     size_t n_words = 0;
     if (int rc = check_reduce_args(s, d_inputs, d_out, n_elems, dtype, op, &n_words)) return rc;
-    if (dtype == RD_BF16) return RD_ERR_UNSUPPORTED;
+    if (is_half(dtype)) return RD_ERR_UNSUPPORTED;
     rd_stats_t st;
     std::memset(&st, 0, sizeof(st));
     st.bytes_moved = uint64_t(s->p + 1) * uint64_t(n_words) * 4u;

@@ -13,6 +13,7 @@
 // Partial results that have to wait (at most log2 p of them) live in a per-thread column of shared
 // memory in both.
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -26,16 +27,17 @@ namespace {
 constexpr int kIdxBits = 12;
 constexpr uint32_t kIdxMask = (1u << kIdxBits) - 1;
 
-enum { DT_INT32 = 0, DT_FP32 = 1, DT_INT64 = 2, DT_FP64 = 3, DT_BF16 = 4 };
+enum { DT_INT32 = 0, DT_FP32 = 1, DT_INT64 = 2, DT_FP64 = 3, DT_BF16 = 4, DT_FP16 = 5 };
 
-// The kernels move and index the message in 32-bit words; an element is one word or two, or (bf16) half
-// a word: a word then holds two elements, the lower-addressed one in its low half.
+// The kernels move and index the message in 32-bit words; an element is one word or two, or (bf16, fp16)
+// half a word: a word then holds two elements, the lower-addressed one in its low half.
 template <int DT> struct ElemWords { static constexpr int value = (DT == DT_INT64 || DT == DT_FP64) ? 2 : 1; };
-// bf16 elements are combined in fp32: a word of the message becomes W = 2 words of partial result (two
-// fp32 values), the arithmetic is that of fp32, and only the root's value is rounded back to bf16.
+// 16-bit elements are combined in fp32: a word of the message becomes W = 2 words of partial result (two
+// fp32 values), the arithmetic is that of fp32, and only the root's value is rounded back to 16 bits.
 template <int DT> struct Wide {
-    static constexpr int W = DT == DT_BF16 ? 2 : 1;
-    static constexpr int ADT = DT == DT_BF16 ? DT_FP32 : DT;
+    static constexpr bool half = DT == DT_BF16 || DT == DT_FP16;
+    static constexpr int W = half ? 2 : 1;
+    static constexpr int ADT = half ? DT_FP32 : DT;
 };
 enum { OPR_SUM = 0, OPR_MAX = 1, OPR_MIN = 2, OPR_PROD = 3 };
 
@@ -114,7 +116,7 @@ template <int DT, int OPR, int V> __device__ __forceinline__ void combine_vec(Ve
     }
 }
 
-// A vector of V message words as V * W words of partial result, and back (bf16: exact widening, one
+// A vector of V message words as V * W words of partial result, and back (bf16, fp16: exact widening, one
 // rounding to nearest even on the way back; other types: the same words).
 template <int DT, int V> __device__ __forceinline__ Vec<V * Wide<DT>::W> widen(const Vec<V> &m)
 {
@@ -124,7 +126,14 @@ template <int DT, int V> __device__ __forceinline__ Vec<V * Wide<DT>::W> widen(c
         for (int v = 0; v < V; v++) a.w[v] = m.w[v];
     } else {
 #pragma unroll
-        for (int v = 0; v < V; v++) { a.w[2 * v] = m.w[v] << 16; a.w[2 * v + 1] = m.w[v] & 0xFFFF0000u; }
+        for (int v = 0; v < V; v++) {
+            if constexpr (DT == DT_BF16) {                      // a bf16 is the upper half of an fp32
+                a.w[2 * v] = m.w[v] << 16; a.w[2 * v + 1] = m.w[v] & 0xFFFF0000u;
+            } else {
+                a.w[2 * v] = __float_as_uint(__half2float(__ushort_as_half((unsigned short)(m.w[v] & 0xFFFFu))));
+                a.w[2 * v + 1] = __float_as_uint(__half2float(__ushort_as_half((unsigned short)(m.w[v] >> 16))));
+            }
+        }
     }
     return a;
 }
@@ -137,8 +146,14 @@ template <int DT, int V> __device__ __forceinline__ Vec<V> narrow(const Vec<V * 
     } else {
 #pragma unroll
         for (int v = 0; v < V; v++) {
-            const uint32_t lo = __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(a.w[2 * v])));
-            const uint32_t hi = __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(a.w[2 * v + 1])));
+            uint32_t lo, hi;
+            if constexpr (DT == DT_BF16) {
+                lo = __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(a.w[2 * v])));
+                hi = __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(a.w[2 * v + 1])));
+            } else {
+                lo = __half_as_ushort(__float2half_rn(__uint_as_float(a.w[2 * v])));
+                hi = __half_as_ushort(__float2half_rn(__uint_as_float(a.w[2 * v + 1])));
+            }
             m.w[v] = lo | (hi << 16);
         }
     }
@@ -518,7 +533,7 @@ struct TileSource {
 };
 
 // What a consumer thread carries for its (up to) two 128-bit vectors of a stage: the vectors themselves,
-// or (bf16) their elements widened to fp32, twice as many words.
+// or (bf16, fp16) their elements widened to fp32, twice as many words.
 template <int DT> struct StageAcc {
     static constexpr int W = Wide<DT>::W;
     static constexpr int ADT = Wide<DT>::ADT;
@@ -1044,6 +1059,7 @@ template <typename F> cudaError_t with_type_and_op(int dtype, int op, F &&f)
     case DT_FP32: return with_op<DT_FP32>(op, f);
     case DT_INT64: return with_op<DT_INT64>(op, f);
     case DT_BF16: return with_op<DT_BF16>(op, f);
+    case DT_FP16: return with_op<DT_FP16>(op, f);
     default: return with_op<DT_FP64>(op, f);
     }
 }
@@ -1059,7 +1075,7 @@ struct DirectLauncher {
     const TreeLaunch &l;
     template <int DT, int OPR> cudaError_t operator()() const
     {
-        if constexpr (DT == DT_BF16) return cudaErrorInvalidValue;      // bf16 goes through the streaming kernel
+        if constexpr (Wide<DT>::half) return cudaErrorInvalidValue;     // 16-bit types go through the streaming kernel
         else return launch_direct_dtop<DT, OPR>(l);
     }
 };

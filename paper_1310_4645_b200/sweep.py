@@ -25,8 +25,8 @@ from . import binding as rd
 
 ALPHA, BETA, GAMMA = 2e-6, 1e-10, 5e-11
 TORCH_DTYPES = {"int32": torch.int32, "fp32": torch.float32, "int64": torch.int64, "fp64": torch.float64,
-                "bf16": torch.bfloat16}
-ELEM_BYTES = {"int32": 4, "fp32": 4, "int64": 8, "fp64": 8, "bf16": 2}
+                "bf16": torch.bfloat16, "fp16": torch.float16}
+ELEM_BYTES = {"int32": 4, "fp32": 4, "int64": 8, "fp64": 8, "bf16": 2, "fp16": 2}
 SCHEDULES = [("uni_greedy", rd.RD_UNI_GREEDY, rd.RD_PORT_UNI), ("bi_greedy", rd.RD_BI_GREEDY, rd.RD_PORT_BI),
              ("binomial", rd.RD_BINOMIAL, rd.RD_PORT_UNI), ("pipeline", rd.RD_PIPELINE, rd.RD_PORT_UNI),
              ("binary", rd.RD_BINARY, rd.RD_PORT_UNI), ("butterfly", rd.RD_BUTTERFLY, rd.RD_PORT_BI)]
@@ -70,6 +70,8 @@ def check(x, out, op, max_check_elems=1 << 22):
             tol = (1e-14 if x.dtype == torch.float64 else 1e-5) * mag
             if x.dtype == torch.bfloat16:           # combined in fp32, then one rounding to 8 significant bits
                 tol = tol + 2.0 ** -8 * ref.abs()
+            if x.dtype == torch.float16:            # ... to 11 significant bits (inputs in [-1, 1): no overflow)
+                tol = tol + 2.0 ** -11 * ref.abs() + 2.0 ** -24
             if not bool(((o.to(torch.float64) - ref).abs() <= tol).all()):
                 return False
     return True

@@ -758,18 +758,19 @@ def test_config2_as_batches_over_two_streams_as_the_benchmark_issues_it():
 # bf16 elements combined in fp32 (tree mode): every schedule and operation against the oracle's
 # bit patterns; the oracle widens, combines in fp32 in schedule order and rounds once at the root.
 # ---------------------------------------------------------------------------------------------
-def bf16_inputs(p, n, kind, seed):
+def bf16_inputs(p, n, kind, seed, dtype=torch.bfloat16):
     g = torch.Generator("cuda").manual_seed(seed)
     if kind == "small_int":
-        return torch.randint(-3, 4, (p, n), device="cuda", generator=g).to(torch.bfloat16)
+        return torch.randint(-3, 4, (p, n), device="cuda", generator=g).to(dtype)
     x = torch.empty((p, n), device="cuda")
     if kind == "near_one":
         x.uniform_(0.5, 2.0, generator=g)
         x *= torch.randint(0, 2, x.shape, device="cuda", generator=g) * 2.0 - 1.0
     else:
         x.normal_(generator=g)
-        x *= 10.0 ** torch.randint(-4, 5, x.shape, device="cuda", generator=g)
-    return x.to(torch.bfloat16)
+        span = 4 if dtype == torch.bfloat16 else 2                    # fp16: sums of 300 such values stay finite
+        x *= 10.0 ** torch.randint(-span, span + 1, x.shape, device="cuda", generator=g)
+    return x.to(dtype)
 
 
 def bits(t):
@@ -777,16 +778,16 @@ def bits(t):
 
 
 def check_bf16(algo, port, x, seg_bytes, op, rows=None, out=None):
-    p, n = x.shape                                                   # n bf16 elements = 2 n bytes
+    p, n = x.shape                                                   # n 16-bit elements = 2 n bytes
     h = rd.rd_schedule_create(algo, port, p, 2 * n, seg_bytes, *M1)
     try:
-        out = torch.full((n,), 7.0, dtype=torch.bfloat16, device="cuda") if out is None else out
+        out = torch.full((n,), 7.0, dtype=x.dtype, device="cuda") if out is None else out
         rd.rd_reduce(h, rows if rows is not None else x, out, OPS[op])
         torch.cuda.synchronize()
     finally:
         rd.rd_destroy(h)
     ev, off, _ = oracle_schedule(algo, port, p, 2 * n, seg_bytes if seg_bytes else 2 * n, *M1)
-    want = O.reduce(ev, bits(x), off * 2, op)                        # the schedule counts 4-byte words
+    want = O.reduce(ev, bits(x), off * 2, op, half="bf16" if x.dtype == torch.bfloat16 else "fp16")   # the schedule counts 4-byte words
     assert bits(out).tobytes() == want.tobytes()
     return out
 
@@ -798,11 +799,14 @@ SHAPES_BF16 = [(8, 8192, 1024), (5, 20000, 5000), (13, 3 * 4096 + 72, 4096 + 104
                (8, 8198, 2000), (5, 14, 4), (3, 6, 2), (8, 12302, 666), (128, 8192, 1024), (300, 4096, 4096)]
 
 
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
 @pytest.mark.parametrize("name,algo,port", SCHEDULES)
 @pytest.mark.parametrize("kind,op", [("normal", "sum"), ("normal", "max"), ("normal", "min"), ("near_one", "prod"), ("small_int", "sum")])
-def test_bf16_parity(name, algo, port, kind, op):
+def test_bf16_parity(name, algo, port, kind, op, dtype):
     for p, n, seg in SHAPES_BF16:
-        x = bf16_inputs(p, n, kind, seed=p * 1000 + n)
+        if dtype == torch.float16 and op == "prod" and p > 16:
+            continue                                                 # products of many factors leave fp16's range
+        x = bf16_inputs(p, n, kind, seed=p * 1000 + n, dtype=dtype)
         out = check_bf16(algo, port, x, 2 * seg, op)
         if kind == "small_int":                                      # exact for any order
             assert torch.equal(out.float(), x.float().sum(dim=0))
@@ -820,6 +824,18 @@ def test_bf16_partial_results_stay_in_fp32_and_ties_round_to_even():
     assert (out.float() == 1 + 2.0 ** -7).all()
     out = check_bf16(rd.RD_PIPELINE, rd.RD_PORT_UNI, x[1:].contiguous(), 2 * 4096, "sum")
     assert (out.float() == 1.0).all()
+    # the same for fp16, whose spacing at 1 is 2^-10, and its overflow to infinity
+    y = torch.full((4, n), 2.0 ** -12, dtype=torch.float16, device="cuda")
+    y[3] = 1.0
+    out = check_bf16(rd.RD_PIPELINE, rd.RD_PORT_UNI, y, 2 * 4096, "sum")
+    assert (out.float() == 1 + 2.0 ** -10).all()
+    out = check_bf16(rd.RD_PIPELINE, rd.RD_PORT_UNI, y[1:].contiguous(), 2 * 4096, "sum")
+    assert (out.float() == 1.0).all()
+    z = torch.full((3, n), 30000.0, dtype=torch.float16, device="cuda")
+    out = check_bf16(rd.RD_BINOMIAL, rd.RD_PORT_UNI, z, 2 * 4096, "sum")
+    assert torch.isinf(out.float()).all()
+    out = check_bf16(rd.RD_BINOMIAL, rd.RD_PORT_UNI, z[:2].contiguous(), 2 * 4096, "sum")
+    assert (out.float() == 60000.0).all()                             # 60000 is below fp16's largest value 65504
 
 
 def test_bf16_buffers_off_the_vector_boundary_and_batches():
