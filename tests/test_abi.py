@@ -177,3 +177,25 @@ def test_tree_variant_is_checked_on_the_host():
             rd.rd_destroy(h)
     assert rd.lib().rd_schedule_set_tree_variant(None, rd.RD_TREE_AUTO) == rd.RD_ERR_INVALID_ARG
     assert rd.lib().rd_schedule_tree_shape(None, None, None, None, None) == rd.RD_ERR_INVALID_ARG
+
+
+def test_binding_constants_match_the_header():
+    """Every enumerator of include/rd.h has the same value in the binding."""
+    text = open(os.path.join(ROOT, "include", "rd.h")).read()
+    seen = 0
+    for body in re.findall(r"typedef enum\s*\{(.*?)\}", text, flags=re.S):
+        body = re.sub(r"/\*.*?\*/", "", body, flags=re.S)
+        value = -1
+        for item in body.split(","):
+            item = item.strip()
+            if not item:
+                continue
+            if "=" in item:
+                name, v = [t.strip() for t in item.split("=")]
+                value = int(v, 0)
+            else:
+                name, value = item, value + 1
+            assert hasattr(rd, name), name
+            assert getattr(rd, name) == value, name
+            seen += 1
+    assert seen >= 30
