@@ -29,6 +29,9 @@
  *     integer count of `tick` seconds, so that equal times are decided the
  *     same way everywhere: t_comm = round(alpha/tick) + round(beta/tick)*b,
  *     t_comp = round(gamma/tick)*b.
+ *   - A communication must take time: a model whose alpha and beta both round to zero ticks is
+ *     refused with RD_ERR_INVALID_ARG (every send would start and end at time 0 and the order of the
+ *     events, hence of the combines, would be undefined).  gamma may be zero.
  *   - Thread safety: distinct schedules may be used from distinct threads.
  *     One schedule may be used by one thread at a time.
  */
@@ -56,7 +59,7 @@ typedef enum {
     RD_ERR_UNSUPPORTED = -2,   /* a combination the method does not define (see rd_schedule_create)     */
     RD_ERR_NOMEM = -3,         /* host or device allocation failed                                      */
     RD_ERR_CUDA = -4,          /* a CUDA runtime call failed (including: no device, no driver)          */
-    RD_ERR_TIMEOUT = -5,       /* a bounded wait inside the schedule-faithful kernel gave up            */
+    RD_ERR_TIMEOUT = -5,       /* a bounded wait inside a kernel (tree mode or schedule-faithful) gave up */
     RD_ERR_SIZE_MISMATCH = -6, /* n_elems * element size differs from the schedule's message size       */
     RD_ERR_INTERNAL = -7,      /* a generated schedule failed the library's own consistency check       */
     RD_ERR_TOO_SMALL = -8,     /* an output array passed by the caller is too short                     */
@@ -247,11 +250,13 @@ RD_API int rd_reduce(rd_schedule_t *s, const void *const *d_inputs, void *d_out,
  *   When every buffer of every job is 16-byte aligned and every message a whole number of 128-bit
  *   vectors, the batch is ONE launch of the streaming kernel: the tiles of all jobs are dealt to the
  *   thread blocks as if they were one reduction, so the batch pays one launch, one ring fill and one
- *   tail instead of n_jobs (16 jobs of p = 64 with 1 MiB messages: 6.3 TB/s against 3.5 TB/s for 16
- *   calls; 32 jobs with 256 KiB messages: 5.4 against 1.1 TB/s).  Job descriptors, tile ranges and the
- *   jobs' input pointers reach the device in one small copy from a pinned ring that a device's first
- *   such batch allocates (it grows when a batch needs more); a bounded wait that gives up is reported
- *   through rd_schedule_status of the first job's schedule.
+ *   tail instead of n_jobs (measured on B200, 16 jobs of p = 64 with 1 MiB messages: about twice the
+ *   throughput of 16 calls; 32 jobs with 256 KiB messages: about five times).  A batch of at most 16
+ *   jobs with at most 1024 input pointers in all carries its job descriptors and pointers inside the
+ *   kernel's parameters and copies nothing ahead of the launch; a larger one sends them to the device in
+ *   one small copy from a pinned ring that a device's first such batch allocates (it grows when a batch
+ *   needs more).  A bounded wait that gives up is reported through rd_schedule_status of the first
+ *   job's schedule.
  *   Otherwise the jobs are issued alternately on two streams of the library's own, so that one job's
  *   thread blocks take the SM slots another job frees while its last blocks are still running (event
  *   fork and join around them; streams and events are created on a device's first such batch and kept).

@@ -152,6 +152,9 @@ int make_ticks(const rd_model_t *m, Ticks &t)
     const double a = m->alpha / tick, b = m->beta / tick, g = m->gamma / tick;
     if (!(a < 4e18) || !(b < 4e18) || !(g < 4e18)) return RD_ERR_INVALID_ARG;
     t.A = llround(a); t.B = llround(b); t.G = llround(g); t.tick = tick;
+    // A communication must take time: with alpha and beta both zero (in ticks) every send of every schedule
+    // starts and ends at time 0, the order of the events, and with it the combine order, is undefined.
+    if (t.A == 0 && t.B == 0) return RD_ERR_INVALID_ARG;
     return RD_OK;
 }
 
@@ -1032,7 +1035,7 @@ int rd_reduce_faithful_static(rd_schedule_t *s, const void *const *d_inputs, voi
         if (stats) *stats = st;
         return RD_OK;
     }
-    try {
+    return guarded([&]() -> int {
         ActionLists lists;
         const size_t q = s->sched.seg_off.size() - 1;
         if (int rc = build_actions(s->p, q, s->sched.events, lists)) return rc;
@@ -1069,9 +1072,7 @@ int rd_reduce_faithful_static(rd_schedule_t *s, const void *const *d_inputs, voi
         st.n_launches = 1;
         if (stats) *stats = st;
         return r.device_status != 0 ? RD_ERR_TIMEOUT : RD_OK;
-    } catch (const std::bad_alloc &) {
-        return RD_ERR_NOMEM;
-    }
+    });
 }
 
 int rd_search_segmentation(int p, size_t msg_bytes, size_t unit_bytes, const rd_model_t *model, size_t *seg_bytes, size_t cap,
@@ -1109,7 +1110,7 @@ const char *rd_strerror(int status)
     case RD_ERR_UNSUPPORTED: return "combination not supported";
     case RD_ERR_NOMEM: return "out of memory";
     case RD_ERR_CUDA: return "CUDA runtime call failed";
-    case RD_ERR_TIMEOUT: return "a bounded wait in the schedule-faithful kernel gave up";
+    case RD_ERR_TIMEOUT: return "a bounded wait inside a kernel gave up";
     case RD_ERR_SIZE_MISMATCH: return "n_elems does not match the schedule's message size";
     case RD_ERR_INTERNAL: return "generated schedule failed the consistency check";
     case RD_ERR_TOO_SMALL: return "output array too small";

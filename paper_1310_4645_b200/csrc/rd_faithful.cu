@@ -18,6 +18,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdint>
+#include <mutex>
 
 #include "rd_kernels.h"
 
@@ -286,6 +287,7 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBy
 namespace {
 
 unsigned char *g_static_base[64] = {};   // per device: address of g_static_scratch once looked up
+std::mutex g_static_base_lock;
 
 size_t carve(size_t &cursor, size_t bytes)
 {
@@ -302,12 +304,16 @@ int faithful_static_run(StaticRun &r)
 {
     int device = -1;
     if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return 1;
-    if (!g_static_base[device]) {
-        void *ptr = nullptr;
-        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return 1;
-        g_static_base[device] = static_cast<unsigned char *>(ptr);
+    unsigned char *base = nullptr;
+    {
+        std::lock_guard<std::mutex> hold(g_static_base_lock);
+        if (!g_static_base[device]) {
+            void *ptr = nullptr;
+            if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return 1;
+            g_static_base[device] = static_cast<unsigned char *>(ptr);
+        }
+        base = g_static_base[device];
     }
-    unsigned char *base = g_static_base[device];
     // blocks per process: everything must be resident at once
     int perSm = 0, sms = 0, khz = 0;
     if (dispatch(FaithfulParams{}, r.dtype, r.op, r.wide, nullptr, true, &perSm) != cudaSuccess) return 1;

@@ -17,12 +17,34 @@
 #include <cuda_runtime.h>
 
 #include <cstdint>
+#include <mutex>
 
 #include "rd_kernels.h"
 
 namespace rd {
 
 namespace {
+
+// Dynamic shared memory: every kernel instantiation that uses it is opted into the device's largest
+// per-block size exactly once per device, under a lock, before its first launch there.  The limit then
+// never moves again, so launches of different ring shapes from different threads cannot undercut each
+// other (setting it per launch to that launch's own size could leave it below what a concurrent launch
+// of a larger shape was about to ask for).
+template <typename K> cudaError_t opt_in_shared_memory(K kernel, int device)
+{
+    static std::mutex lock;
+    static bool done[64] = {};
+    if (device < 0 || device >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> hold(lock);
+    if (done[device]) return cudaSuccess;
+    int most = 0;
+    cudaError_t e = cudaDeviceGetAttribute(&most, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    if (e != cudaSuccess) return e;
+    done[device] = true;
+    return cudaSuccess;
+}
 
 constexpr int kIdxBits = 12;
 constexpr uint32_t kIdxMask = (1u << kIdxBits) - 1;
@@ -877,7 +899,7 @@ cudaError_t launch_one(const TreeLaunch &l)
     auto kernel = rd_tree_kernel<DT, OPR, V, kU, kK, PACKED>;
     const int depth = l.stack_depth > 0 ? l.stack_depth : 1;
     const size_t smem = size_t(depth) * kU * kTreeThreads * sizeof(Vec<V * Wide<DT>::W>);
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+    cudaError_t e = opt_in_shared_memory(kernel, l.device);
     if (e != cudaSuccess) return e;
     int perSm = 0;
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&perSm, kernel, kTreeThreads, smem);
@@ -897,19 +919,13 @@ cudaError_t launch_dtop(const TreeLaunch &l)
 }
 
 // Launches the streaming kernel for one parameter type (one job with packed pointers, one job with a
-// pointer table, or a batch); shared memory is opted into once per device and size.
+// pointer table, or a batch).
 template <int DT, int OPR, typename PRM>
 cudaError_t launch_stream_kernel(const PRM &prm, uint32_t n_ctas, int device, void *stream)
 {
     auto kernel = rd_tree_stream_kernel<DT, OPR, PRM>;
     const size_t smem = stream_smem_bytes(prm.stages, prm.depth, prm.stage_elems, Wide<DT>::W);
-    static size_t configured[64] = {};     // per device: largest dynamic shared memory size opted into so far
-    const int dv = device & 63;
-    if (smem > configured[dv]) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-        if (e != cudaSuccess) return e;
-        configured[dv] = smem;
-    }
+    if (cudaError_t e = opt_in_shared_memory(kernel, device)) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(n_ctas); cfg.blockDim = dim3(kStreamThreads); cfg.dynamicSmemBytes = smem;
     cfg.stream = static_cast<cudaStream_t>(stream);

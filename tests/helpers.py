@@ -45,8 +45,7 @@ def run_program(ops, x, op):
     def combine(held, incoming):
         if op == "sum":
             if x.dtype == np.int32:
-                return (held.astype(np.int64) + incoming.astype(np.int64)).astype(np.uint64).astype(np.uint32) \
-                    .view(np.int32) if False else ((held.view(np.uint32) + incoming.view(np.uint32)).view(np.int32))
+                return (held.view(np.uint32) + incoming.view(np.uint32)).view(np.int32)
             return (held + incoming).astype(np.float32)
         if op == "prod":
             if x.dtype == np.int32:

@@ -36,7 +36,7 @@ def test_only_the_abi_is_exported():
 
 def test_strerror():
     assert rd.rd_strerror(0) == "success"
-    for code in range(-8, 0):
+    for code in range(-9, 0):
         assert rd.rd_strerror(code) and rd.rd_strerror(code) != "unknown status"
     assert rd.rd_strerror(-99) == "unknown status"
 
@@ -199,3 +199,55 @@ def test_binding_constants_match_the_header():
             assert getattr(rd, name) == value, name
             seen += 1
     assert seen >= 30
+
+
+def test_a_model_whose_communications_take_no_time_is_refused():
+    """alpha = beta = 0 (in ticks): every send would start and end at time 0, the event order is undefined."""
+    for f, args in ((rd.rd_schedule_create, (rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, 8, 4096, 1024)),
+                    (rd.rd_schedule_create, (rd.RD_BI_GREEDY, rd.RD_PORT_BI, 8, 4096, 1024)),
+                    (rd.rd_schedule_create, (rd.RD_BUTTERFLY, rd.RD_PORT_BI, 8, 4096, 0)),
+                    (rd.rd_schedule_create_segments, (rd.RD_PIPELINE, rd.RD_PORT_UNI, 8, [1024, 512])),
+                    (rd.rd_optimal_segment, (rd.RD_BINARY, rd.RD_PORT_BI, 8, 4096)),
+                    (rd.rd_search_segmentation, (8, 4096, 4))):
+        assert status_of(f, *args, 0.0, 0.0, 0.0) == rd.RD_ERR_INVALID_ARG
+        assert status_of(f, *args, 0.0, 0.0, 5e-11) == rd.RD_ERR_INVALID_ARG
+        assert status_of(f, *args, 1e-17, 1e-17, 5e-11) == rd.RD_ERR_INVALID_ARG      # both round to 0 ticks of 1 fs
+    # either of the two alone is enough, and gamma may be zero
+    for model in ((2e-6, 0.0, 0.0), (0.0, 1e-10, 0.0), (0.0, 1.0, 1.0, 1.0)):
+        h = rd.rd_schedule_create(rd.RD_BI_GREEDY, rd.RD_PORT_BI, 8, 4096, 1024, *model)
+        assert rd.rd_schedule_info(h)["n_events"] == 7 * 4
+        rd.rd_destroy(h)
+
+
+def test_distinct_schedules_from_distinct_threads():
+    """The header's promise: threads that each own their schedules need no lock around the library."""
+    import threading
+    from helpers import oracle_schedule
+    cases = [(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, 37, 40000, 1000), (rd.RD_BI_GREEDY, rd.RD_PORT_BI, 24, 36000, 1200),
+             (rd.RD_BINARY, rd.RD_PORT_BI, 100, 8000, 400), (rd.RD_BUTTERFLY, rd.RD_PORT_BI, 16, 64000, 0)]
+    want = [oracle_schedule(a, pt, p, m, s if s else m, *MODEL) for a, pt, p, m, s in cases]
+    errors = []
+
+    def work(k):
+        try:
+            for rep in range(20):
+                a, pt, p, m, s = cases[(k + rep) % len(cases)]
+                ev, off, comp = want[(k + rep) % len(cases)]
+                h = rd.rd_schedule_create(a, pt, p, m, s, *MODEL)
+                try:
+                    got = rd.rd_schedule_events(h)
+                    assert rd.rd_schedule_info(h)["predicted_ticks"] == comp
+                    for f in ("seg", "src", "dst", "t_start"):
+                        assert (got[f] == ev[f]).all()
+                    assert (rd.rd_schedule_segments(h) == off).all()
+                finally:
+                    rd.rd_destroy(h)
+        except BaseException as e:      # noqa: BLE001 - reported by the main thread
+            errors.append(repr(e))
+
+    threads = [threading.Thread(target=work, args=(k,)) for k in range(4)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
