@@ -301,16 +301,21 @@ RD_API int rd_schedule_set_wait_budget(rd_schedule_t *s, double seconds);
  *   RD_TREE_STREAM  operand tiles are streamed through a shared-memory ring by bulk asynchronous
  *                   copies; any number of processes.
  *   RD_TREE_DIRECT  every thread fetches all p operands of its elements into registers at once; at
- *                   most 8 processes (RD_ERR_UNSUPPORTED beyond).
+ *                   most 8 processes (RD_ERR_UNSUPPORTED beyond); 4- and 8-byte element types.
+ *   RD_TREE_STREAM_PAIRED  the streaming kernel on tiles of half the length (1024 words), a ring stage
+ *                   holding the tiles of two consecutive operands: the partial results that wait in the
+ *                   stack take half the shared memory per tile, the bytes per stage hand-over stay the same.
+ *                   What RD_TREE_AUTO picks for the 16-bit element types, whose partial results are fp32.
  */
-typedef enum { RD_TREE_AUTO = 0, RD_TREE_STREAM = 1, RD_TREE_DIRECT = 2 } rd_tree_variant_t;
+typedef enum { RD_TREE_AUTO = 0, RD_TREE_STREAM = 1, RD_TREE_DIRECT = 2, RD_TREE_STREAM_PAIRED = 3 } rd_tree_variant_t;
 RD_API int rd_schedule_set_tree_variant(rd_schedule_t *s, rd_tree_variant_t variant);
 
 /*
  * rd_schedule_tree_shape -- how a tree-mode call with 16-byte aligned buffers will run this schedule on
- * the current device (the paper has no counterpart): the kernel (RD_TREE_STREAM or RD_TREE_DIRECT), its
- * thread blocks per SM, the stages of the streaming kernel's shared-memory ring (0 for the direct kernel)
- * and the number of tiles the message is cut into (runs of at most 2048 4-byte words inside one segment).
+ * the current device with a 4- or 8-byte element type (the paper has no counterpart): the kernel
+ * (RD_TREE_STREAM, RD_TREE_STREAM_PAIRED or RD_TREE_DIRECT), its thread blocks per SM, the stages of the
+ * streaming kernel's shared-memory ring (0 for the direct kernel) and the number of tiles the message is cut
+ * into (runs of at most 2048 4-byte words inside one segment; 1024 for RD_TREE_STREAM_PAIRED).
  * Uploads the schedule's tables if they are not on the device yet.  Any output pointer may be NULL.
  */
 RD_API int rd_schedule_tree_shape(rd_schedule_t *s, int *variant, int *blocks_per_sm, int *ring_stages, size_t *n_tiles);

@@ -33,11 +33,18 @@
  * uni-greedy process identities (only the makespan of the Fig. 3 example is
  * checkable).  The tie-break used is (time, process index) ascending.
  *
- * Build: gcc -O2 -ffp-contract=off -fno-fast-math -shared -fPIC.
+ * Build: gcc -O2 -ffp-contract=off -fno-fast-math -shared -fPIC.  A second build of the same file
+ * with -fopenmp added lets several threads share the int32 and fp32 evaluators: every thread replays
+ * all the events on its own range of the elements of each segment (an element's result depends on
+ * that element of the p inputs only), so the arithmetic per element is the same and so are the bits.
+ * It exists so that the benchmark can time the oracle on all host cores; parity tests use the plain build.
  */
 #include <stdint.h>
 #include <stdlib.h>
 #include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
 
 typedef struct {
     int32_t seg;     /* segment index, 0-based (butterfly: final chunk index)      */
@@ -694,6 +701,32 @@ static float comb_f32(float held, float in, int op)
     return (in < held) ? in : held;
 }
 
+/* Threads this build runs the evaluators on (1 without OpenMP). */
+int orc_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* The calling thread's share [lo, hi) of a segment's len elements (all of them without OpenMP): the
+ * same share of the `longest` places of the accumulators for every segment, clipped to the segment, so
+ * that a thread which is already on the next segment never touches a place another thread still uses. */
+static void my_share(int64_t len, int64_t longest, int64_t *lo, int64_t *hi)
+{
+#ifdef _OPENMP
+    const int64_t T = omp_get_num_threads(), t = omp_get_thread_num();
+#else
+    const int64_t T = 1, t = 0;
+#endif
+    *lo = longest * t / T;
+    *hi = longest * (t + 1) / T;
+    if (*hi > len) *hi = len;
+    if (*lo > len) *lo = len;
+}
+
 static int cmp_seg_time(const void *x, const void *y)
 {
     const orc_event_t *u = x, *v = y;
@@ -719,17 +752,21 @@ int orc_reduce_i32(const orc_event_t *ev_in, int64_t n_ev, int p, int q, const i
     for (int j = 0; j < q; j++) if (seg_off[j + 1] - seg_off[j] > longest) longest = seg_off[j + 1] - seg_off[j];
     uint32_t *acc = malloc(sizeof(uint32_t) * (size_t)p * (size_t)(longest ? longest : 1));
     if (!acc) { free(ev); return ORC_NOMEM; }
+#pragma omp parallel
+    {
     int64_t e = 0;
     for (int j = 0; j < q; j++) {
-        int64_t len = seg_off[j + 1] - seg_off[j];
+        int64_t len = seg_off[j + 1] - seg_off[j], lo, hi;
+        my_share(len, longest, &lo, &hi);
         for (int i = 0; i < p; i++)                    /* every process starts from its own segment */
-            for (int64_t k = 0; k < len; k++) acc[(size_t)i * longest + k] = (uint32_t)x[i][seg_off[j] + k];
+            for (int64_t k = lo; k < hi; k++) acc[(size_t)i * longest + k] = (uint32_t)x[i][seg_off[j] + k];
         for (; e < n_ev && ev[e].seg == j; e++) {
             uint32_t *held = acc + (size_t)ev[e].dst * longest, *in = acc + (size_t)ev[e].src * longest;
-            if (ev[e].kind == 0) for (int64_t k = 0; k < len; k++) held[k] = comb_i32(held[k], in[k], op);
-            else for (int64_t k = 0; k < len; k++) held[k] = in[k];
+            if (ev[e].kind == 0) for (int64_t k = lo; k < hi; k++) held[k] = comb_i32(held[k], in[k], op);
+            else for (int64_t k = lo; k < hi; k++) held[k] = in[k];
         }
-        for (int64_t k = 0; k < len; k++) out[seg_off[j] + k] = (int32_t)acc[k];
+        for (int64_t k = lo; k < hi; k++) out[seg_off[j] + k] = (int32_t)acc[k];
+    }
     }
     free(acc); free(ev);
     return ORC_OK;
@@ -744,17 +781,21 @@ int orc_reduce_f32(const orc_event_t *ev_in, int64_t n_ev, int p, int q, const i
     for (int j = 0; j < q; j++) if (seg_off[j + 1] - seg_off[j] > longest) longest = seg_off[j + 1] - seg_off[j];
     float *acc = malloc(sizeof(float) * (size_t)p * (size_t)(longest ? longest : 1));
     if (!acc) { free(ev); return ORC_NOMEM; }
+#pragma omp parallel
+    {
     int64_t e = 0;
     for (int j = 0; j < q; j++) {
-        int64_t len = seg_off[j + 1] - seg_off[j];
+        int64_t len = seg_off[j + 1] - seg_off[j], lo, hi;
+        my_share(len, longest, &lo, &hi);
         for (int i = 0; i < p; i++)
-            for (int64_t k = 0; k < len; k++) acc[(size_t)i * longest + k] = x[i][seg_off[j] + k];
+            for (int64_t k = lo; k < hi; k++) acc[(size_t)i * longest + k] = x[i][seg_off[j] + k];
         for (; e < n_ev && ev[e].seg == j; e++) {
             float *held = acc + (size_t)ev[e].dst * longest, *in = acc + (size_t)ev[e].src * longest;
-            if (ev[e].kind == 0) for (int64_t k = 0; k < len; k++) held[k] = comb_f32(held[k], in[k], op);
-            else for (int64_t k = 0; k < len; k++) held[k] = in[k];
+            if (ev[e].kind == 0) for (int64_t k = lo; k < hi; k++) held[k] = comb_f32(held[k], in[k], op);
+            else for (int64_t k = lo; k < hi; k++) held[k] = in[k];
         }
-        for (int64_t k = 0; k < len; k++) out[seg_off[j] + k] = acc[k];
+        for (int64_t k = lo; k < hi; k++) out[seg_off[j] + k] = acc[k];
+    }
     }
     free(acc); free(ev);
     return ORC_OK;

@@ -14,6 +14,7 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "rd_oracle.c")
 _LIB = os.path.join(_HERE, "librd_oracle.so")
+_LIB_OMP = os.path.join(_HERE, "librd_oracle_omp.so")       # the same source built with -fopenmp (benchmark only)
 CFLAGS = ["-O2", "-ffp-contract=off", "-fno-fast-math", "-shared", "-fPIC"]
 
 EVENT_DTYPE = np.dtype(
@@ -22,23 +23,35 @@ EVENT_DTYPE = np.dtype(
 assert EVENT_DTYPE.itemsize == 24
 
 
-def build(force: bool = False) -> str:
-    """Compile rd_oracle.c with gcc when the shared object is missing or stale."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
-        tmp = _LIB + ".%d.tmp" % os.getpid()
-        subprocess.check_call(["gcc", *CFLAGS, "-o", tmp, _SRC])
-        os.replace(tmp, _LIB)
-    return _LIB
+def build(force: bool = False, openmp: bool = False) -> str:
+    """Compile rd_oracle.c with gcc when the shared object is missing or stale.  openmp: the second build,
+    in which the threads of an OpenMP team share the elements of the int32 and fp32 evaluators."""
+    path = _LIB_OMP if openmp else _LIB
+    if force or not os.path.exists(path) or os.path.getmtime(path) < os.path.getmtime(_SRC):
+        tmp = path + ".%d.tmp" % os.getpid()
+        subprocess.check_call(["gcc", *CFLAGS, *(["-fopenmp"] if openmp else []), "-o", tmp, _SRC])
+        os.replace(tmp, path)
+    return path
 
 
 _lib = None
+_lib_omp = None
 
 
-def lib():
-    global _lib
+def lib(openmp: bool = False):
+    global _lib, _lib_omp
+    if openmp:
+        if _lib_omp is None:
+            _lib_omp = C.CDLL(build(openmp=True))
+        return _lib_omp
     if _lib is None:
         _lib = C.CDLL(build())
     return _lib
+
+
+def threads(openmp: bool = False) -> int:
+    """Threads the evaluators of the chosen build run on."""
+    return int(lib(openmp).orc_threads())
 
 
 def _i64(a):
@@ -142,9 +155,10 @@ def contributions(events, p, q):
                                        C.c_int(q)))
 
 
-def reduce(events, x, seg_off, op, half="bf16"):
+def reduce(events, x, seg_off, op, half="bf16", openmp=False):
     """O2.  x: array [p, n] of int32, float32, int64, float64, or uint16 holding bf16 (half="bf16") or IEEE
-    binary16 (half="fp16") bit patterns (C-contiguous); seg_off in elements of x; op 'sum', 'max', 'min' or 'prod'."""
+    binary16 (half="fp16") bit patterns (C-contiguous); seg_off in elements of x; op 'sum', 'max', 'min' or 'prod'.
+    openmp: run the OpenMP build (int32 and float32 only; same bits, used by the benchmark's all-cores leg)."""
     events = np.ascontiguousarray(events, dtype=EVENT_DTYPE)
     x = np.ascontiguousarray(x)
     p, n = x.shape
@@ -155,9 +169,11 @@ def reduce(events, x, seg_off, op, half="bf16"):
     ptrs = (C.c_void_p * p)(*[x[i].ctypes.data for i in range(p)])
     opc = {"sum": 0, "max": 1, "min": 2, "prod": 3}[op]
     if x.dtype == np.int32:
-        fn = lib().orc_reduce_i32
+        fn = lib(openmp).orc_reduce_i32
     elif x.dtype == np.float32:
-        fn = lib().orc_reduce_f32
+        fn = lib(openmp).orc_reduce_f32
+    elif openmp:
+        raise TypeError("the OpenMP build serves int32 and float32 only")
     elif x.dtype == np.int64:
         fn = lib().orc_reduce_i64
     elif x.dtype == np.float64:

@@ -22,7 +22,7 @@ RD_PORT_UNI, RD_PORT_BI = 0, 1
 RD_SUM, RD_MAX, RD_MIN, RD_PROD = 0, 1, 2, 3
 RD_INT32, RD_FP32, RD_INT64, RD_FP64, RD_BF16, RD_FP16 = 0, 1, 2, 3, 4, 5
 RD_EXEC_TREE, RD_EXEC_FAITHFUL = 0, 1
-RD_TREE_AUTO, RD_TREE_STREAM, RD_TREE_DIRECT = 0, 1, 2
+RD_TREE_AUTO, RD_TREE_STREAM, RD_TREE_DIRECT, RD_TREE_STREAM_PAIRED = 0, 1, 2, 3
 
 ALGOS = {"uni_greedy": RD_UNI_GREEDY, "bi_greedy": RD_BI_GREEDY, "binomial": RD_BINOMIAL,
          "pipeline": RD_PIPELINE, "binary": RD_BINARY, "butterfly": RD_BUTTERFLY}

@@ -86,6 +86,7 @@ void reset_tile_counters(int device)
 }
 constexpr int kDirectAutoProcs = 0;     // the direct kernel is never chosen by the library itself
 constexpr int kTailTiles = 5; // key of the tile table for the elements the 128-bit path leaves over
+constexpr int kPairTiles = 8; // key of the tile table of the 128-bit path with two operand tiles per ring stage
 
 struct DeviceTables {
     int device = -1;
@@ -100,7 +101,8 @@ struct DeviceTables {
         int ctas_per_sm = 0;
         int stages = 0;
     };
-    std::map<int, StreamPlan> plans;        // key: words of partial result per message word (1; 2 for bf16)
+    std::map<int, StreamPlan> plans;        // key: 4 * (words of partial result per message word: 1, or 2 for 16-bit
+                                            // elements) + operand tiles per ring stage (1 or 2)
     int stage_elems = 0;
     int *status = nullptr;                                  // device word written by a kernel that gave up a wait
     // pointer tables for large p: pinned host ring + device ring, one event per slot
@@ -290,13 +292,13 @@ int tiles_for(rd_schedule *s, int vec, const TileDesc **tiles, uint32_t *count)
     if (it == d.tiles.end()) {
         const std::vector<uint64_t> &off = s->sched.seg_off;
         std::vector<TileDesc> host;
-        if (vec == 4) {
-            // Streaming path.  Every segment is cut into equal tiles of at most one stage (whole 128-bit
-            // vectors of the buffers: where a segment starts or ends inside a vector the tile is padded to the
-            // vector and remembers how many elements are not its own).
+        if (vec == 4 || vec == kPairTiles) {
+            // Streaming path.  Every segment is cut into equal tiles of at most one stage, or half a stage when
+            // two operand tiles share a stage (whole 128-bit vectors of the buffers: where a segment starts or
+            // ends inside a vector the tile is padded to the vector and remembers how many elements are not its own).
             const uint64_t n = off.empty() ? 0 : off.back();
             d.stage_elems = stream_stage_elems(n / (uint64_t(d.sm_count) * 2) + 1);
-            const uint32_t cap = uint32_t(d.stage_elems);
+            const uint32_t cap = uint32_t(d.stage_elems) / (vec == kPairTiles ? 2u : 1u);
             const uint64_t n4 = n & ~uint64_t(3);          // the last n mod 4 elements go to the element kernel
             for (size_t seg = 0; seg + 1 < off.size(); seg++) {
                 const uint64_t b = std::min(off[seg], n4), e = std::min(off[seg + 1], n4);
@@ -331,16 +333,18 @@ int tiles_for(rd_schedule *s, int vec, const TileDesc **tiles, uint32_t *count)
 // NUMBER of tiles up to one (a tile costs a CTA about the same time however full it is, one ring hand-off
 // per operation, so for small messages the number of tiles per CTA, not the number of elements, sets the
 // kernel's duration; for large ones the two coincide).  acc_words: 2 for bf16, whose partial results are fp32.
-int stream_plan(rd_schedule *s, int acc_words, const DeviceTables::StreamPlan **out)
+int stream_plan(rd_schedule *s, int acc_words, int ops_per_stage, const DeviceTables::StreamPlan **out)
 {
     DeviceTables &d = s->dev;
-    auto it = d.plans.find(acc_words);
+    const int key = 4 * acc_words + ops_per_stage;
+    auto it = d.plans.find(key);
     if (it == d.plans.end()) {
         const TileDesc *tiles = nullptr;
         uint32_t nTiles = 0;
-        if (int rc = tiles_for(s, 4, &tiles, &nTiles)) return rc;
+        if (int rc = tiles_for(s, ops_per_stage == 2 ? kPairTiles : 4, &tiles, &nTiles)) return rc;
         DeviceTables::StreamPlan plan;
-        stream_shape(s->progs.stack_depth, acc_words, d.smem_per_sm, d.stage_elems, nTiles, d.sm_count, &plan.ctas_per_sm, &plan.stages);
+        stream_shape(s->progs.stack_depth, acc_words, ops_per_stage, d.smem_per_sm, d.stage_elems, nTiles, d.sm_count, &plan.ctas_per_sm,
+                     &plan.stages);
         const uint64_t ctas = std::min<uint64_t>(uint64_t(d.sm_count) * uint64_t(plan.ctas_per_sm), std::max<uint64_t>(nTiles, 1));
         std::vector<uint32_t> first(size_t(ctas) + 1, 0);
         for (uint64_t c = 0; c < ctas; c++) first[size_t(c)] = uint32_t(uint64_t(nTiles) * c / ctas);
@@ -351,7 +355,7 @@ int stream_plan(rd_schedule *s, int acc_words, const DeviceTables::StreamPlan **
             return RD_ERR_CUDA;
         }
         plan.n_ctas = uint32_t(ctas);
-        it = d.plans.emplace(acc_words, plan).first;
+        it = d.plans.emplace(key, plan).first;
     }
     *out = &it->second;
     return RD_OK;
@@ -360,6 +364,15 @@ int stream_plan(rd_schedule *s, int acc_words, const DeviceTables::StreamPlan **
 // Argument checks common to the reducing entry points.  On success *n_words is the message length
 // in 32-bit words, the unit in which the schedule's segment boundaries and the kernels count.
 bool is_half(rd_dtype_t dtype) { return dtype == RD_BF16 || dtype == RD_FP16; }
+// Operand tiles per ring stage of the streaming kernel.  The 16-bit types are combined in fp32, so a tile's
+// waiting partial results take twice the shared memory of its operand: they run on tiles of half a stage, two
+// to a stage, unless the schedule asks for one kind of stage or the other.
+int stage_ops(rd_dtype_t dtype, int tree_variant)
+{
+    if (tree_variant == RD_TREE_STREAM) return 1;
+    if (tree_variant == RD_TREE_STREAM_PAIRED) return 2;
+    return is_half(dtype) ? 2 : 1;
+}
 size_t elem_bytes(rd_dtype_t dtype) { return (dtype == RD_INT64 || dtype == RD_FP64) ? 8 : is_half(dtype) ? 2 : 4; }
 
 int check_reduce_args(const rd_schedule *s, const void *const *d_inputs, const void *d_out, size_t n_elems, rd_dtype_t dtype,
@@ -391,10 +404,11 @@ int reduce_tree(rd_schedule *s, const void *const *d_inputs, void *d_out, size_t
     for (int i = 0; i < s->p && wide; i++) wide = (reinterpret_cast<uintptr_t>(d_inputs[i]) & 15u) == 0;
     TreeLaunch l{};
     l.vec = wide ? 4 : 1;
-    if (int rc = tiles_for(s, l.vec, &l.tiles, &l.n_tiles)) return rc;
+    l.ops_per_stage = stage_ops(dtype, s->tree_variant);
+    if (int rc = tiles_for(s, wide ? (l.ops_per_stage == 2 ? kPairTiles : 4) : 1, &l.tiles, &l.n_tiles)) return rc;
     const DeviceTables::StreamPlan *plan = nullptr;
     if (wide)
-        if (int rc = stream_plan(s, is_half(dtype) ? 2 : 1, &plan)) return rc;
+        if (int rc = stream_plan(s, is_half(dtype) ? 2 : 1, l.ops_per_stage, &plan)) return rc;
     const TileDesc *tailTiles = nullptr;
     uint32_t nTail = 0;
     if (wide && (n & 3u) != 0)
@@ -595,11 +609,12 @@ int reduce_batch_fused(size_t n_jobs, rd_schedule_t *const *schedules, const voi
     uint64_t total = 0;
     size_t nPtrs = 0;
     int depth = 0;
+    const int opsPerStage = stage_ops(dtype, RD_TREE_AUTO);        // one kind of stage for the whole launch
     for (size_t j = 0; j < n_jobs; j++) {
         rd_schedule *s = schedules[j];
         const TileDesc *tiles = nullptr;
         uint32_t count = 0;
-        if (int rc = tiles_for(s, 4, &tiles, &count)) return rc;
+        if (int rc = tiles_for(s, opsPerStage == 2 ? kPairTiles : 4, &tiles, &count)) return rc;
         BatchJob &b = jobs[j];
         b.inputs = nullptr; b.out = static_cast<uint32_t *>(d_outs[j]); b.tiles = tiles; b.ops = s->dev.ops;
         b.tile_begin = uint32_t(total); b.p = s->p; b.ptr_base = 0;
@@ -613,11 +628,11 @@ int reduce_batch_fused(size_t n_jobs, rd_schedule_t *const *schedules, const voi
     DeviceTables &d0 = schedules[0]->dev;
     const int stageElems = d0.stage_elems;
     int ctasPerSm = 1, stages = 2;
-    stream_shape(depth, is_half(dtype) ? 2 : 1, d0.smem_per_sm, stageElems, total, d0.sm_count, &ctasPerSm, &stages);
+    stream_shape(depth, is_half(dtype) ? 2 : 1, opsPerStage, d0.smem_per_sm, stageElems, total, d0.sm_count, &ctasPerSm, &stages);
     const uint64_t ctas = std::min<uint64_t>(uint64_t(d0.sm_count) * uint64_t(ctasPerSm), total);
     BatchLaunch b{};
     b.n_jobs = uint32_t(n_jobs); b.n_tiles = uint32_t(total); b.n_ctas = uint32_t(ctas);
-    b.stages = stages; b.stack_depth = depth; b.stage_elems = stageElems;
+    b.stages = stages; b.stack_depth = depth; b.stage_elems = stageElems; b.ops_per_stage = opsPerStage;
     b.dtype = int(dtype); b.op = int(op); b.device = device; b.status = d0.status; b.stream = user;
     b.tile_counter = next_tile_counter(device, user);
     if (n_jobs <= size_t(kBatchPackJobs) && nPtrs <= size_t(kBatchPackPtrs)) {
@@ -923,7 +938,7 @@ int rd_schedule_set_wait_budget(rd_schedule_t *s, double seconds)
 
 int rd_schedule_set_tree_variant(rd_schedule_t *s, rd_tree_variant_t variant)
 {
-    if (!s || int(variant) < RD_TREE_AUTO || int(variant) > RD_TREE_DIRECT) return RD_ERR_INVALID_ARG;
+    if (!s || int(variant) < RD_TREE_AUTO || int(variant) > RD_TREE_STREAM_PAIRED) return RD_ERR_INVALID_ARG;
     if (variant == RD_TREE_DIRECT && !direct_applies(s->p, s->progs.stack_depth)) return RD_ERR_UNSUPPORTED;
     s->tree_variant = int(variant);
     return RD_OK;
@@ -964,12 +979,13 @@ int rd_schedule_tree_shape(rd_schedule_t *s, int *variant, int *blocks_per_sm, i
     return guarded([&] {
         if (int rc = upload(s)) return rc;
         TreeLaunch l{};
-        if (int rc = tiles_for(s, 4, &l.tiles, &l.n_tiles)) return rc;
+        const int opsPerStage = stage_ops(RD_FP32, s->tree_variant);
+        if (int rc = tiles_for(s, opsPerStage == 2 ? kPairTiles : 4, &l.tiles, &l.n_tiles)) return rc;
         const bool direct = direct_applies(s->p, s->progs.stack_depth) &&
                             (s->tree_variant == RD_TREE_DIRECT || (s->tree_variant == RD_TREE_AUTO && s->p <= kDirectAutoProcs));
-        if (variant) *variant = direct ? RD_TREE_DIRECT : RD_TREE_STREAM;
+        if (variant) *variant = direct ? RD_TREE_DIRECT : opsPerStage == 2 ? RD_TREE_STREAM_PAIRED : RD_TREE_STREAM;
         const DeviceTables::StreamPlan *plan = nullptr;
-        if (int rc = stream_plan(s, 1, &plan)) return rc;
+        if (int rc = stream_plan(s, 1, opsPerStage, &plan)) return rc;
         if (blocks_per_sm) *blocks_per_sm = direct ? direct_blocks_per_sm(s->p) : plan->ctas_per_sm;
         if (ring_stages) *ring_stages = direct ? 0 : plan->stages;
         if (n_tiles) *n_tiles = l.n_tiles;

@@ -17,6 +17,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdint>
+#include <map>
 #include <mutex>
 
 #include "rd_kernels.h"
@@ -30,19 +31,23 @@ namespace {
 // never moves again, so launches of different ring shapes from different threads cannot undercut each
 // other (setting it per launch to that launch's own size could leave it below what a concurrent launch
 // of a larger shape was about to ask for).
-template <typename K> cudaError_t opt_in_shared_memory(K kernel, int device)
+inline cudaError_t opt_in_shared_memory(const void *kernel, int device)
 {
     static std::mutex lock;
-    static bool done[64] = {};
+    static std::map<const void *, uint64_t> done;            // kernel -> devices it has been opted in on
     if (device < 0 || device >= 64) return cudaErrorInvalidDevice;
     std::lock_guard<std::mutex> hold(lock);
-    if (done[device]) return cudaSuccess;
+    uint64_t &mask = done[kernel];
+    if (mask >> device & 1u) return cudaSuccess;
     int most = 0;
     cudaError_t e = cudaDeviceGetAttribute(&most, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+    cudaFuncAttributes fa;
+    e = cudaFuncGetAttributes(&fa, kernel);                  // the limit covers static and dynamic shared memory together
     if (e != cudaSuccess) return e;
-    done[device] = true;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most - int(fa.sharedSizeBytes));
+    if (e != cudaSuccess) return e;
+    mask |= uint64_t(1) << device;
     return cudaSuccess;
 }
 
@@ -62,6 +67,7 @@ template <int DT> struct Wide {
     static constexpr int ADT = half ? DT_FP32 : DT;
 };
 enum { OPR_SUM = 0, OPR_MAX = 1, OPR_MIN = 2, OPR_PROD = 3 };
+enum { LAUNCH_STREAM = 0, LAUNCH_BATCH = 1, LAUNCH_DIRECT = 2, LAUNCH_ELEMENT = 3 };
 
 template <int V> struct Vec { uint32_t w[V]; };
 
@@ -554,71 +560,85 @@ struct TileSource {
     }
 };
 
-// What a consumer thread carries for its (up to) two 128-bit vectors of a stage: the vectors themselves,
-// or (bf16, fp16) their elements widened to fp32, twice as many words.
-template <int DT> struct StageAcc {
+// What a consumer thread carries for its N (one or two) 128-bit vectors of an operand tile: the vectors
+// themselves, or (bf16, fp16) their elements widened to fp32, twice as many words.
+template <int DT, int N> struct StageAcc {
     static constexpr int W = Wide<DT>::W;
     static constexpr int ADT = Wide<DT>::ADT;
-    Vec<4> v[2 * W];
+    Vec<4> v[N * W];
     __device__ __forceinline__ void clear()
     {
 #pragma unroll
-        for (int k = 0; k < 2 * W; k++)
+        for (int k = 0; k < N * W; k++)
 #pragma unroll
             for (int e = 0; e < 4; e++) v[k].w[e] = 0;
     }
-    __device__ __forceinline__ void load(const uint4 &r0, const uint4 &r1)
+    __device__ __forceinline__ void load(const uint4 (&r)[N])
     {
-        const Vec<4> m0 = {{r0.x, r0.y, r0.z, r0.w}}, m1 = {{r1.x, r1.y, r1.z, r1.w}};
-        const Vec<4 * W> a0 = widen<DT, 4>(m0), a1 = widen<DT, 4>(m1);
 #pragma unroll
-        for (int k = 0; k < W; k++)
+        for (int n = 0; n < N; n++) {
+            const Vec<4> m = {{r[n].x, r[n].y, r[n].z, r[n].w}};
+            const Vec<4 * W> a = widen<DT, 4>(m);
 #pragma unroll
-            for (int e = 0; e < 4; e++) { v[k].w[e] = a0.w[4 * k + e]; v[W + k].w[e] = a1.w[4 * k + e]; }
+            for (int k = 0; k < W; k++)
+#pragma unroll
+                for (int e = 0; e < 4; e++) v[n * W + k].w[e] = a.w[4 * k + e];
+        }
     }
     // *this = combine(held, in); *this may be either of them
     template <int OPR> __device__ __forceinline__ void combine(const StageAcc &held, const StageAcc &in)
     {
 #pragma unroll
-        for (int k = 0; k < 2 * W; k++) combine_vec<ADT, OPR, 4>(v[k], held.v[k], in.v[k]);
+        for (int k = 0; k < N * W; k++) combine_vec<ADT, OPR, 4>(v[k], held.v[k], in.v[k]);
     }
-    // one stack level: [vector][consumer thread], the first stage vector's words first
-    __device__ __forceinline__ void push(uint4 *level, uint32_t tid, bool two) const
+    // one stack level: [vector][consumer thread], the first vector's words first; `all` false: only the
+    // first vector of the thread is in use (tiles of at most 1024 words)
+    __device__ __forceinline__ void push(uint4 *level, uint32_t tid, bool all) const
     {
 #pragma unroll
-        for (int k = 0; k < 2 * W; k++)
-            if (k < W || two) level[k * kConsumers + tid] = make_uint4(v[k].w[0], v[k].w[1], v[k].w[2], v[k].w[3]);
+        for (int k = 0; k < N * W; k++)
+            if (k < W || all) level[k * kConsumers + tid] = make_uint4(v[k].w[0], v[k].w[1], v[k].w[2], v[k].w[3]);
     }
-    __device__ __forceinline__ void pop(const uint4 *level, uint32_t tid, bool two)
+    __device__ __forceinline__ void pop(const uint4 *level, uint32_t tid, bool all)
     {
 #pragma unroll
-        for (int k = 0; k < 2 * W; k++) {
-            const uint4 y = (k < W || two) ? level[k * kConsumers + tid] : make_uint4(0, 0, 0, 0);
+        for (int k = 0; k < N * W; k++) {
+            const uint4 y = (k < W || all) ? level[k * kConsumers + tid] : make_uint4(0, 0, 0, 0);
             v[k].w[0] = y.x; v[k].w[1] = y.y; v[k].w[2] = y.z; v[k].w[3] = y.w;
         }
     }
-    __device__ __forceinline__ void result(Vec<4> &o0, Vec<4> &o1) const
+    __device__ __forceinline__ void result(Vec<4> (&o)[N]) const
     {
-        Vec<4 * W> a0, a1;
 #pragma unroll
-        for (int k = 0; k < W; k++)
+        for (int n = 0; n < N; n++) {
+            Vec<4 * W> a;
 #pragma unroll
-            for (int e = 0; e < 4; e++) { a0.w[4 * k + e] = v[k].w[e]; a1.w[4 * k + e] = v[W + k].w[e]; }
-        o0 = narrow<DT, 4>(a0); o1 = narrow<DT, 4>(a1);
+            for (int k = 0; k < W; k++)
+#pragma unroll
+                for (int e = 0; e < 4; e++) a.w[4 * k + e] = v[n * W + k].w[e];
+            o[n] = narrow<DT, 4>(a);
+        }
     }
 };
 
-template <int DT, int OPR, typename PRM>
+// G = operand tiles per ring stage.  G = 1: a stage holds one tile of up to a whole stage (two vectors per
+// consumer thread).  G = 2: tiles are half as long (one vector per consumer thread), a stage holds the tiles of
+// two consecutive operations of the program, each brought by its own bulk copy, and is handed over once for
+// both: the partial results that wait in the stack are half as large per tile, while the bytes per stage
+// hand-over, which set the pace, stay the same.
+template <int DT, int OPR, typename PRM, int G>
 __global__ void __launch_bounds__(kStreamThreads, 3)
 rd_tree_stream_kernel(const __grid_constant__ PRM a)
 {
     using Jobs = typename PRM::Jobs;
+    constexpr int N = 2 / G;                                                                 // vectors per thread and operand
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int S = a.stages;
     const uint32_t stageVecs = uint32_t(a.stage_elems) / 4u;                                 // 128-bit vectors per stage
-    uint4 *ring = reinterpret_cast<uint4 *>(smem_raw);                                       // [S][stageVecs]
-    const bool two = a.stage_elems > 4 * kConsumers;                                         // a second vector per thread
-    const uint32_t levelVecs = (two ? 2u : 1u) * uint32_t(Wide<DT>::W) * kConsumers;
+    const uint32_t subVecs = stageVecs / uint32_t(G);                                        // ... per operand tile
+    uint4 *ring = reinterpret_cast<uint4 *>(smem_raw);                                       // [S][G][subVecs]
+    const bool all = subVecs > kConsumers;                                                   // a second vector per thread
+    const uint32_t levelVecs = (all ? 2u : 1u) * uint32_t(Wide<DT>::W) * kConsumers;
     uint4 *stack = ring + size_t(S) * stageVecs;                                              // [depth][(1 or 2) * W][256]
     uint64_t *full = reinterpret_cast<uint64_t *>(stack + size_t(a.depth) * levelVecs);
     uint64_t *empty = full + S;
@@ -641,11 +661,12 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
 
     if (tid >= kConsumers) {
         // ------------------------------------------------------------------ producers
-        // One lane in each of the kProducers producer warps.  Producer j owns the steps j, j + P,
-        // j + 2P, ... of this CTA's sequence of (tile, operation) pairs and issues them in order:
-        // stages are released by the consumers in that same order, so a producer never waits for a
-        // stage while a later one of its own is already free.  Being alone in its warp, a producer
-        // polls without divergence; the table look-ups of a step are issued before its wait.
+        // One lane in each of the kProducers producer warps.  A step is one ring stage: the operand tiles of
+        // G consecutive operations of a tile's program.  Producer j owns the steps j, j + P, j + 2P, ... of
+        // this CTA's sequence of steps and issues them in order: stages are released by the consumers in that
+        // same order, so a producer never waits for a stage while a later one of its own is already free.
+        // Being alone in its warp, a producer polls without divergence; the table look-ups of a step are
+        // issued before its wait.
         if ((tid & 31u) != 0) return;
         const int P = kProducers < S ? kProducers : S;
         const int j = int(tid - kConsumers) / 32;
@@ -659,12 +680,13 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
         uint32_t k = 0;                         // position in this CTA's sequence of tiles
         uint32_t tile = j == 0 ? source.get(0) : tile_at(&tileq, 0, &abort_flag, a.status);
         Jobs jobs(a, tile, tile != kNoTile);
-        int i = j;
+        int i = j;                              // step within the tile
         int p = jobs.p();                       // of the job `tile` belongs to
-        while (tile != kNoTile && i >= p) {
-            i -= p; k++;
+        int steps = (p + G - 1) / G;
+        while (tile != kNoTile && i >= steps) {
+            i -= steps; k++;
             tile = j == 0 ? source.get(k) : tile_at(&tileq, k, &abort_flag, a.status);
-            if (tile != kNoTile) { jobs.seek(tile); p = jobs.p(); }
+            if (tile != kNoTile) { jobs.seek(tile); p = jobs.p(); steps = (p + G - 1) / G; }
         }
         int stage = j % S;
         uint32_t laps = 0;                      // times this producer has gone round the ring
@@ -675,17 +697,25 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
         uint32_t lastLap = 0;
         while (tile != kNoTile) {
             if (tile != cur) { td = jobs.tile(tile); cur = tile; }
-            const uint32_t *src = jobs.input(__ldg(jobs.ops() + td.prog + i) & kIdxMask) + td.elem_off;
+            const int first = i * G;
+            const int cnt = p - first < G ? p - first : G;
+            const uint32_t *src[G];
+#pragma unroll
+            for (int g = 0; g < G; g++)
+                src[g] = g < cnt ? jobs.input(__ldg(jobs.ops() + td.prog + first + g) & kIdxMask) + td.elem_off : nullptr;
             if (laps >= 1u && !mbar_wait(empty + stage, (laps - 1u) & 1u, &abort_flag)) { ok = false; break; }
-            mbar_expect_tx(full + stage, (td.len & kLenMask) * 4u);
-            bulk_load(ring + size_t(stage) * stageVecs, src, (td.len & kLenMask) * 4u, full + stage);
+            const uint32_t bytes = (td.len & kLenMask) * 4u;
+            mbar_expect_tx(full + stage, bytes * uint32_t(cnt));
+#pragma unroll
+            for (int g = 0; g < G; g++)
+                if (g < cnt) bulk_load(ring + size_t(stage) * stageVecs + size_t(g) * subVecs, src[g], bytes, full + stage);
             any = true; lastStage = stage; lastLap = laps;
             if (j == 0) source.poke(k);
             i += P;
-            while (tile != kNoTile && i >= p) {
-                i -= p; k++;
+            while (tile != kNoTile && i >= steps) {
+                i -= steps; k++;
                 tile = j == 0 ? source.get(k) : tile_at(&tileq, k, &abort_flag, a.status);
-                if (tile != kNoTile) { jobs.seek(tile); p = jobs.p(); }
+                if (tile != kNoTile) { jobs.seek(tile); p = jobs.p(); steps = (p + G - 1) / G; }
             }
             stage += P;
             if (stage >= S) { stage -= S; laps++; }
@@ -693,7 +723,7 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
         if (j == 0) source.finish(gridDim.x);
         if (!ok) {
             if (!abort_flag) { atomicCAS(a.status, 0, -5); abort_flag = 1; }
-            // leave only after this producer's last copy has landed (bounded); its earlier ones were consumed
+            // leave only after this producer's last copies have landed (bounded); its earlier ones were consumed
             if (any) {
                 const long long start = clock64();
                 while (!mbar_try_wait(full + lastStage, lastLap & 1u) && clock64() - start < kWaitCycles) {}
@@ -715,60 +745,79 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
         const TileDesc td = jobs.tile(tile);
         const uint32_t *prog = jobs.ops() + td.prog;
         const uint32_t len = td.len & kLenMask;                       // padded to whole 128-bit vectors
-        const bool live0 = tid * 4u < len, live1 = (kConsumers + tid) * 4u < len;
-        StageAcc<DT> top;
+        bool live[N];
+#pragma unroll
+        for (int n = 0; n < N; n++) live[n] = (uint32_t(n) * kConsumers + tid) * 4u < len;
+        StageAcc<DT, N> top;
         top.clear();
         int sp = 0;
-        uint32_t w = __ldg(prog);
-        for (int i = 0; i < p; i++) {
-            const uint32_t wn = (i + 1 < p) ? __ldg(prog + i + 1) : 0u;
+        uint32_t w[G];
+#pragma unroll
+        for (int g = 0; g < G; g++) w[g] = g < p ? __ldg(prog + g) : 0u;
+        for (int i = 0; i < p; i += G) {
+            uint32_t wn[G];
+#pragma unroll
+            for (int g = 0; g < G; g++) wn[g] = (i + G + g < p) ? __ldg(prog + i + G + g) : 0u;
             if (!mbar_wait(full + stage, phase, &abort_flag)) {
                 if (!abort_flag) { atomicCAS(a.status, 0, -5); abort_flag = 1; }
                 return;
             }
             const uint4 *st = ring + size_t(stage) * stageVecs;
-            uint4 r0 = make_uint4(0, 0, 0, 0), r1 = make_uint4(0, 0, 0, 0);
-            if (live0) r0 = st[tid];
-            if (live1) r1 = st[kConsumers + tid];
-            StageAcc<DT> x;
-            x.load(r0, r1);
-            const uint32_t kind = (w >> kIdxBits) & 3u;
-            if (kind == 1u) {
-                top.push(stack + sp * levelVecs, tid, two);
-                sp++;
+            uint4 r[G][N];
+#pragma unroll
+            for (int g = 0; g < G; g++)
+#pragma unroll
+                for (int n = 0; n < N; n++)
+                    r[g][n] = (live[n] && i + g < p) ? st[uint32_t(g) * subVecs + uint32_t(n) * kConsumers + tid] : make_uint4(0, 0, 0, 0);
+#pragma unroll
+            for (int g = 0; g < G; g++) {
+                if (g > 0 && i + g >= p) break;
+                StageAcc<DT, N> x;
+                x.load(r[g]);
+                const uint32_t kind = (w[g] >> kIdxBits) & 3u;
+                if (kind == 1u) {
+                    top.push(stack + sp * levelVecs, tid, all);
+                    sp++;
+                }
+                if (kind <= 1u) {
+                    top = x;
+                } else if (kind == 2u || Commutes<OPR>::value) {
+                    top.template combine<OPR>(top, x);
+                } else {
+                    top.template combine<OPR>(x, top);
+                }
+                if (g == 0) {
+                    // the stage's data is in registers: hand the stage back to the producer
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(empty + stage);
+                    if (++stage == S) { stage = 0; phase ^= 1u; }
+                }
+                uint32_t npop = (w[g] >> (kIdxBits + 2)) & 0xFu;
+                uint32_t roles = w[g] >> (kIdxBits + 6);
+                while (npop--) {
+                    sp--;
+                    const bool poppedHeld = (roles & 1u) != 0;
+                    roles >>= 1;
+                    StageAcc<DT, N> y;
+                    y.pop(stack + sp * levelVecs, tid, all);
+                    if (poppedHeld || Commutes<OPR>::value) top.template combine<OPR>(y, top);
+                    else top.template combine<OPR>(top, y);
+                }
             }
-            if (kind <= 1u) {
-                top = x;
-            } else if (kind == 2u || Commutes<OPR>::value) {
-                top.template combine<OPR>(top, x);
-            } else {
-                top.template combine<OPR>(x, top);
-            }
-            // the stage's data is in registers: hand the stage back to the producer
-            __syncwarp();
-            if (lane == 0) mbar_arrive(empty + stage);
-            if (++stage == S) { stage = 0; phase ^= 1u; }
-            uint32_t npop = (w >> (kIdxBits + 2)) & 0xFu;
-            uint32_t roles = w >> (kIdxBits + 6);
-            while (npop--) {
-                sp--;
-                const bool poppedHeld = (roles & 1u) != 0;
-                roles >>= 1;
-                StageAcc<DT> y;
-                y.pop(stack + sp * levelVecs, tid, two);
-                if (poppedHeld || Commutes<OPR>::value) top.template combine<OPR>(y, top);
-                else top.template combine<OPR>(top, y);
-            }
-            w = wn;
+#pragma unroll
+            for (int g = 0; g < G; g++) w[g] = wn[g];
         }
-        Vec<4> top0, top1;
-        top.result(top0, top1);
+        Vec<4> res[N];
+        top.result(res);
         // A segment may begin or end inside a vector: the tile then starts / ends with a vector whose other
         // elements belong to the neighbouring segment (another tile writes those); only this tile's are stored.
         uint32_t *dst = jobs.out() + td.elem_off;
         const uint32_t head = (td.len >> 16) & 3u, tail = (td.len >> 18) & 3u, lastVec = len / 4u - 1u;
-        if (live0) store_part(dst + tid * 4u, top0, tid == 0 ? head : 0u, tid == lastVec ? tail : 0u);
-        if (live1) store_part(dst + (kConsumers + tid) * 4u, top1, 0u, kConsumers + tid == lastVec ? tail : 0u);
+#pragma unroll
+        for (int n = 0; n < N; n++) {
+            const uint32_t vec = uint32_t(n) * kConsumers + tid;
+            if (live[n]) store_part(dst + vec * 4u, res[n], vec == 0u ? head : 0u, vec == lastVec ? tail : 0u);
+        }
     }
 }
 
@@ -899,7 +948,7 @@ cudaError_t launch_one(const TreeLaunch &l)
     auto kernel = rd_tree_kernel<DT, OPR, V, kU, kK, PACKED>;
     const int depth = l.stack_depth > 0 ? l.stack_depth : 1;
     const size_t smem = size_t(depth) * kU * kTreeThreads * sizeof(Vec<V * Wide<DT>::W>);
-    cudaError_t e = opt_in_shared_memory(kernel, l.device);
+    cudaError_t e = opt_in_shared_memory(reinterpret_cast<const void *>(kernel), l.device);
     if (e != cudaSuccess) return e;
     int perSm = 0;
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&perSm, kernel, kTreeThreads, smem);
@@ -919,13 +968,13 @@ cudaError_t launch_dtop(const TreeLaunch &l)
 }
 
 // Launches the streaming kernel for one parameter type (one job with packed pointers, one job with a
-// pointer table, or a batch).
-template <int DT, int OPR, typename PRM>
+// pointer table, or a batch) and one number of operand tiles per ring stage.
+template <int DT, int OPR, int G, typename PRM>
 cudaError_t launch_stream_kernel(const PRM &prm, uint32_t n_ctas, int device, void *stream)
 {
-    auto kernel = rd_tree_stream_kernel<DT, OPR, PRM>;
-    const size_t smem = stream_smem_bytes(prm.stages, prm.depth, prm.stage_elems, Wide<DT>::W);
-    if (cudaError_t e = opt_in_shared_memory(kernel, device)) return e;
+    auto kernel = rd_tree_stream_kernel<DT, OPR, PRM, G>;
+    const size_t smem = stream_smem_bytes(prm.stages, prm.depth, prm.stage_elems, Wide<DT>::W, G);
+    if (cudaError_t e = opt_in_shared_memory(reinterpret_cast<const void *>(kernel), device)) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(n_ctas); cfg.blockDim = dim3(kStreamThreads); cfg.dynamicSmemBytes = smem;
     cfg.stream = static_cast<cudaStream_t>(stream);
@@ -934,6 +983,12 @@ cudaError_t launch_stream_kernel(const PRM &prm, uint32_t n_ctas, int device, vo
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, prm);
+}
+template <int DT, int OPR, typename PRM>
+cudaError_t launch_stream_kernel(const PRM &prm, int ops_per_stage, uint32_t n_ctas, int device, void *stream)
+{
+    return ops_per_stage == 2 ? launch_stream_kernel<DT, OPR, 2>(prm, n_ctas, device, stream)
+                              : launch_stream_kernel<DT, OPR, 1>(prm, n_ctas, device, stream);
 }
 
 template <int DT, int OPR, bool PACKED>
@@ -949,7 +1004,7 @@ cudaError_t launch_stream(const TreeLaunch &l)
     prm.t.tiles = l.tiles; prm.t.ops = l.ops; prm.t.n_tiles = l.n_tiles; prm.t.p = l.p;
     prm.cta_first = l.cta_first; prm.status = l.status; prm.tile_counter = l.tile_counter;
     prm.stages = l.stages; prm.depth = l.stack_depth > 0 ? l.stack_depth : 1; prm.stage_elems = l.stage_elems;
-    return launch_stream_kernel<DT, OPR>(prm, l.n_ctas, l.device, l.stream);
+    return launch_stream_kernel<DT, OPR>(prm, l.ops_per_stage, l.n_ctas, l.device, l.stream);
 }
 
 template <int DT, int OPR>
@@ -964,12 +1019,12 @@ cudaError_t launch_stream_batch(const BatchLaunch &b)
             prm.ptrs[i] = i < b.n_ptrs ? static_cast<const uint32_t *>(b.host_ptrs[i]) : nullptr;
         prm.n_jobs = b.n_jobs; prm.n_tiles = b.n_tiles; prm.status = b.status; prm.tile_counter = b.tile_counter;
         prm.stages = b.stages; prm.depth = depth; prm.stage_elems = b.stage_elems;
-        return launch_stream_kernel<DT, OPR>(prm, b.n_ctas, b.device, b.stream);
+        return launch_stream_kernel<DT, OPR>(prm, b.ops_per_stage, b.n_ctas, b.device, b.stream);
     }
     BatchStreamParams<false> prm;
     prm.jobs = b.jobs; prm.n_jobs = b.n_jobs; prm.n_tiles = b.n_tiles; prm.status = b.status; prm.tile_counter = b.tile_counter;
     prm.stages = b.stages; prm.depth = depth; prm.stage_elems = b.stage_elems;
-    return launch_stream_kernel<DT, OPR>(prm, b.n_ctas, b.device, b.stream);
+    return launch_stream_kernel<DT, OPR>(prm, b.ops_per_stage, b.n_ctas, b.device, b.stream);
 }
 
 template <int DT, int OPR>
@@ -1005,60 +1060,7 @@ cudaError_t launch_direct_dtop(const TreeLaunch &l)
     return launch_direct<DT, OPR, 8>(l);
 }
 
-}  // namespace
-
-uint32_t tree_tile_elems(int vec) { return uint32_t(kTreeThreads) * kU * uint32_t(vec); }
-
-// One stack level holds one 128-bit vector per consumer thread, two when a stage has more than 1024 elements.
-// (acc_words: words of partial result per message word, 2 for bf16 whose elements are combined in fp32, else 1)
-static int stack_level_bytes(int stage_elems, int acc_words) { return (stage_elems > 4 * kConsumers ? 2 : 1) * acc_words * kConsumers * 16; }
-
-size_t stream_smem_bytes(int stages, int depth, int stage_elems, int acc_words)
-{
-    return size_t(stages) * size_t(stage_elems) * 4 + size_t(depth) * stack_level_bytes(stage_elems, acc_words) + size_t(2 * stages) * sizeof(uint64_t);
-}
-
-int stream_stage_elems(uint64_t elems_per_cta)
-{
-    // Measured on B200: the time per bulk copy hardly depends on its size up to 8 KB, so smaller
-    // stages only lower the throughput, also for small messages.  The kernel accepts 512 and 1024.
-    (void)elems_per_cta;
-    return kMaxStageElems;
-}
-
-void stream_shape(int stack_depth, int acc_words, int smem_per_sm, int stage_elems, uint64_t n_tiles, int sm_count, int *ctas_per_sm, int *stages)
-{
-    const int depth = stack_depth > 0 ? stack_depth : 1;
-    const int stageBytes = stage_elems * 4;
-    // Stages that fit when `ctas` CTAs share an SM (room left for the per-CTA reserve and statics).
-    auto fit = [&](int ctas) { return (smem_per_sm / ctas - 2048 - depth * stack_level_bytes(stage_elems, acc_words) - 512) / stageBytes; };
-    // Measured on B200: with many tiles per CTA, three CTAs with 4 stages each stream 3-7 % more than two
-    // with 6 to 13 (6.8-7.0 TB/s for 3 to 256 processes); the bytes in flight are no more, the third set
-    // of consumers is what helps (three CTAs with 5 stages are behind 4, and 3 stages are too few to hide
-    // the hand-off).  With few tiles the count of tiles per CTA decides instead: every CTA of an SM gets
-    // 1 / ctas of its bandwidth, so a launch lasts about ceil(tiles / CTAs) * ctas tile times.  Three CTAs
-    // are chosen when their product is at most 8 % above that of two (512 tiles on 148 SMs: 2 * 3 against
-    // 2 * 2, two CTAs are 20 % faster; 768 tiles: 2 * 3 against 3 * 2, three are 4 % faster; 1024 tiles:
-    // 3 * 3 against 4 * 2, two are 3 % faster).  Two CTAs take all the stages that fit: a launch of one or
-    // two tiles per CTA is over sooner the more of it is in flight from the start.
-    const int s3 = fit(3), s2 = fit(2);
-    if (s3 >= 4 && s2 >= 3 && sm_count > 0) {
-        const uint64_t t = n_tiles > 0 ? n_tiles : 1;
-        const uint64_t cost3 = (t + 3u * uint64_t(sm_count) - 1) / (3u * uint64_t(sm_count)) * 3u;
-        const uint64_t cost2 = (t + 2u * uint64_t(sm_count) - 1) / (2u * uint64_t(sm_count)) * 2u;
-        if (cost3 * 100u <= cost2 * 108u) { *ctas_per_sm = 3; *stages = 4; return; }
-    }
-    // Two CTAs per SM whenever each still gets three stages (deep stacks, p = 512..1024: two CTAs with
-    // 4-5 stages stream 6.6 TB/s where one CTA with 19 stages reaches 5.3).
-    if (s2 >= 3) { *ctas_per_sm = 2; *stages = s2 > kMaxStages ? kMaxStages : s2; return; }
-    const int s1 = fit(1);
-    *ctas_per_sm = 1;
-    *stages = s1 > kMaxStages ? kMaxStages : s1 < 2 ? 2 : s1;
-}
-
-namespace {
-
-// Calls f.template operator()<DT, OPR>() for the run-time pair (dtype, op).
+// Calls f.template operator()<DT, OPR>() for the run-time operation.
 template <int DT, typename F> cudaError_t with_op(int op, F &&f)
 {
     switch (op) {
@@ -1066,17 +1068,6 @@ template <int DT, typename F> cudaError_t with_op(int op, F &&f)
     case OPR_MAX: return f.template operator()<DT, OPR_MAX>();
     case OPR_MIN: return f.template operator()<DT, OPR_MIN>();
     default: return f.template operator()<DT, OPR_PROD>();
-    }
-}
-template <typename F> cudaError_t with_type_and_op(int dtype, int op, F &&f)
-{
-    switch (dtype) {
-    case DT_INT32: return with_op<DT_INT32>(op, f);
-    case DT_FP32: return with_op<DT_FP32>(op, f);
-    case DT_INT64: return with_op<DT_INT64>(op, f);
-    case DT_BF16: return with_op<DT_BF16>(op, f);
-    case DT_FP16: return with_op<DT_FP16>(op, f);
-    default: return with_op<DT_FP64>(op, f);
     }
 }
 struct StreamLauncher {
@@ -1102,16 +1093,111 @@ struct ElementLauncher {
 
 }  // namespace
 
+// This file is compiled once per element type (RD_DT = 0..5: that type's kernels behind one entry point)
+// and once without RD_DT (launch shapes and the dispatch over the element types), so that the element
+// types build side by side.
+#ifdef RD_DT
+
+#define RD_CAT2(a, b) a##b
+#define RD_CAT(a, b) RD_CAT2(a, b)
+int RD_CAT(launch_for_dtype_, RD_DT)(int which, const void *launch, int op)
+{
+    switch (which) {
+    case LAUNCH_STREAM: return int(with_op<RD_DT>(op, StreamLauncher{*static_cast<const TreeLaunch *>(launch)}));
+    case LAUNCH_BATCH: return int(with_op<RD_DT>(op, BatchLauncher{*static_cast<const BatchLaunch *>(launch)}));
+    case LAUNCH_DIRECT: return int(with_op<RD_DT>(op, DirectLauncher{*static_cast<const TreeLaunch *>(launch)}));
+    default: return int(with_op<RD_DT>(op, ElementLauncher{*static_cast<const TreeLaunch *>(launch)}));
+    }
+}
+
+#else
+
+uint32_t tree_tile_elems(int vec) { return uint32_t(kTreeThreads) * kU * uint32_t(vec); }
+
+// One stack level holds one 128-bit vector per consumer thread and word of partial result, two when an operand
+// tile has more than 1024 words.  (acc_words: words of partial result per message word, 2 for the 16-bit types,
+// whose elements are combined in fp32, else 1; ops_per_stage: operand tiles that share a ring stage.)
+static int stack_level_bytes(int stage_elems, int acc_words, int ops_per_stage)
+{
+    return (stage_elems / ops_per_stage > 4 * kConsumers ? 2 : 1) * acc_words * kConsumers * 16;
+}
+
+size_t stream_smem_bytes(int stages, int depth, int stage_elems, int acc_words, int ops_per_stage)
+{
+    return size_t(stages) * size_t(stage_elems) * 4 + size_t(depth) * stack_level_bytes(stage_elems, acc_words, ops_per_stage) +
+           size_t(2 * stages) * sizeof(uint64_t);
+}
+
+int stream_stage_elems(uint64_t elems_per_cta)
+{
+    // Measured on B200: the time per stage hand-over hardly depends on the stage's size up to 8 KB, so smaller
+    // stages only lower the throughput, also for small messages.
+    (void)elems_per_cta;
+    return kMaxStageElems;
+}
+
+void stream_shape(int stack_depth, int acc_words, int ops_per_stage, int smem_per_sm, int stage_elems, uint64_t n_tiles, int sm_count,
+                  int *ctas_per_sm, int *stages)
+{
+    const int depth = stack_depth > 0 ? stack_depth : 1;
+    const int stageBytes = stage_elems * 4;
+    // Stages that fit when `ctas` CTAs share an SM (room left for the per-CTA reserve and statics).
+    auto fit = [&](int ctas) {
+        return (smem_per_sm / ctas - 2048 - depth * stack_level_bytes(stage_elems, acc_words, ops_per_stage) - 512) / stageBytes;
+    };
+    // Measured on B200: with many tiles per CTA, three CTAs with 4 stages each stream 3-7 % more than two
+    // with 6 to 13 (6.8-7.0 TB/s for 3 to 256 processes); the bytes in flight are no more, the third set
+    // of consumers is what helps (three CTAs with 5 stages are behind 4, and 3 stages are too few to hide
+    // the hand-off).  With few tiles the count of tiles per CTA decides instead: every CTA of an SM gets
+    // 1 / ctas of its bandwidth, so a launch lasts about ceil(tiles / CTAs) * ctas tile times.  Three CTAs
+    // are chosen when their product is at most 8 % above that of two (512 tiles on 148 SMs: 2 * 3 against
+    // 2 * 2, two CTAs are 20 % faster; 768 tiles: 2 * 3 against 3 * 2, three are 4 % faster; 1024 tiles:
+    // 3 * 3 against 4 * 2, two are 3 % faster).  Two CTAs take all the stages that fit: a launch of one or
+    // two tiles per CTA is over sooner the more of it is in flight from the start.
+    const int s3 = fit(3), s2 = fit(2);
+    if (s3 >= 4 && s2 >= 3 && sm_count > 0) {
+        const uint64_t t = n_tiles > 0 ? n_tiles : 1;
+        const uint64_t cost3 = (t + 3u * uint64_t(sm_count) - 1) / (3u * uint64_t(sm_count)) * 3u;
+        const uint64_t cost2 = (t + 2u * uint64_t(sm_count) - 1) / (2u * uint64_t(sm_count)) * 2u;
+        if (cost3 * 100u <= cost2 * 108u) { *ctas_per_sm = 3; *stages = 4; return; }
+    }
+    // Two CTAs per SM whenever each still gets three stages (deep stacks, p = 512..1024: two CTAs with
+    // 4-5 stages stream 6.6 TB/s where one CTA with 19 stages reaches 5.3).
+    if (s2 >= 3) { *ctas_per_sm = 2; *stages = s2 > kMaxStages ? kMaxStages : s2; return; }
+    const int s1 = fit(1);
+    *ctas_per_sm = 1;
+    *stages = s1 > kMaxStages ? kMaxStages : s1 < 2 ? 2 : s1;
+}
+
+int launch_for_dtype_0(int which, const void *launch, int op);
+int launch_for_dtype_1(int which, const void *launch, int op);
+int launch_for_dtype_2(int which, const void *launch, int op);
+int launch_for_dtype_3(int which, const void *launch, int op);
+int launch_for_dtype_4(int which, const void *launch, int op);
+int launch_for_dtype_5(int which, const void *launch, int op);
+
+static int launch_for(int dtype, int which, const void *launch, int op)
+{
+    switch (dtype) {
+    case DT_INT32: return launch_for_dtype_0(which, launch, op);
+    case DT_FP32: return launch_for_dtype_1(which, launch, op);
+    case DT_INT64: return launch_for_dtype_2(which, launch, op);
+    case DT_FP64: return launch_for_dtype_3(which, launch, op);
+    case DT_BF16: return launch_for_dtype_4(which, launch, op);
+    default: return launch_for_dtype_5(which, launch, op);
+    }
+}
+
 int launch_tree_stream(const TreeLaunch &l)
 {
     if (l.n_tiles == 0 || l.n_ctas == 0) return 0;
-    return int(with_type_and_op(l.dtype, l.op, StreamLauncher{l}));
+    return launch_for(l.dtype, LAUNCH_STREAM, &l, l.op);
 }
 
 int launch_tree_stream_batch(const BatchLaunch &b)
 {
     if (b.n_jobs == 0 || b.n_ctas == 0) return 0;
-    return int(with_type_and_op(b.dtype, b.op, BatchLauncher{b}));
+    return launch_for(b.dtype, LAUNCH_BATCH, &b, b.op);
 }
 
 bool direct_applies(int p, int stack_depth)
@@ -1125,13 +1211,15 @@ int direct_blocks_per_sm(int p) { return p <= 2 ? DirectShape<2>::B : p <= 4 ? D
 int launch_tree_direct(const TreeLaunch &l)
 {
     if (l.n_tiles == 0) return 0;
-    return int(with_type_and_op(l.dtype, l.op, DirectLauncher{l}));
+    return launch_for(l.dtype, LAUNCH_DIRECT, &l, l.op);
 }
 
 int launch_tree(const TreeLaunch &l)
 {
     if (l.n_tiles == 0) return 0;
-    return int(with_type_and_op(l.dtype, l.op, ElementLauncher{l}));
+    return launch_for(l.dtype, LAUNCH_ELEMENT, &l, l.op);
 }
+
+#endif  // RD_DT
 
 }  // namespace rd

@@ -36,6 +36,7 @@ struct TreeLaunch {
     uint32_t n_ctas;
     int stages;
     int stage_elems;
+    int ops_per_stage;                // operand tiles that share a ring stage (1 or 2); tiles hold stage_elems / ops_per_stage words
     int *status;                      // device word
     uint32_t *tile_counter;           // device: two words, both 0, for handing tiles out on demand; null: fixed ranges
 };
@@ -60,7 +61,7 @@ struct BatchLaunch {
     const BatchJob *jobs;             // device, n_jobs entries (when host_jobs is null)
     uint32_t n_jobs, n_tiles;
     uint32_t n_ctas;
-    int stages, stack_depth, stage_elems;
+    int stages, stack_depth, stage_elems, ops_per_stage;
     int dtype, op, device;
     int *status;                      // device word
     uint32_t *tile_counter;           // as in TreeLaunch
@@ -75,8 +76,9 @@ int launch_tree(const TreeLaunch &a);
 // Streaming variant (128-bit path): stage size for a CTA's share of the message, ring shape for a
 // stack depth and the SM's shared memory, launch.
 int stream_stage_elems(uint64_t elems_per_cta);
-void stream_shape(int stack_depth, int acc_words, int smem_per_sm, int stage_elems, uint64_t n_tiles, int sm_count, int *ctas_per_sm, int *stages);
-size_t stream_smem_bytes(int stages, int depth, int stage_elems, int acc_words);
+void stream_shape(int stack_depth, int acc_words, int ops_per_stage, int smem_per_sm, int stage_elems, uint64_t n_tiles, int sm_count,
+                  int *ctas_per_sm, int *stages);
+size_t stream_smem_bytes(int stages, int depth, int stage_elems, int acc_words, int ops_per_stage);
 int launch_tree_stream(const TreeLaunch &a);
 // Direct variant (128-bit path, at most kDirectMaxProcs processes): all operands of a thread's elements
 // are fetched into registers at once.  Uses the streaming variant's tiles.

@@ -89,6 +89,9 @@ def main(argv=None):
                     help="also run every schedule in schedule-faithful mode (fp32 sum) and record its makespan")
     ap.add_argument("--dtypes", nargs="*", default=["int32", "fp32"], choices=list(TORCH_DTYPES))
     ap.add_argument("--ops", nargs="*", default=["sum", "max"], choices=["sum", "max", "min"])
+    ap.add_argument("--schedules", nargs="*", default=[s[0] for s in SCHEDULES], choices=[s[0] for s in SCHEDULES])
+    ap.add_argument("--variant", default="auto", choices=["auto", "stream", "paired"],
+                    help="tree-mode kernel: the library's choice, or the streaming kernel with one / two operand tiles per ring stage")
     args = ap.parse_args(argv)
     dev = torch.device("cuda", torch.cuda.current_device())
     sink = sys.stdout if args.out == "-" else open(args.out, "w")
@@ -107,6 +110,8 @@ def main(argv=None):
                 continue
             n = m // 4
             for name, algo, port in SCHEDULES:
+                if name not in args.schedules:
+                    continue
                 t0 = time.perf_counter()
                 seg = rd.rd_optimal_segment(algo, port, p, m, ALPHA, BETA, GAMMA)
                 if any(ELEM_BYTES[dt] == 8 for dt in args.dtypes):
@@ -115,6 +120,8 @@ def main(argv=None):
                 create_ms = (time.perf_counter() - t0) * 1e3
                 info = rd.rd_schedule_info(h)
                 rd.rd_schedule_upload(h)
+                if args.variant != "auto":
+                    rd.rd_schedule_set_tree_variant(h, rd.RD_TREE_STREAM if args.variant == "stream" else rd.RD_TREE_STREAM_PAIRED)
                 try:
                     if args.faithful and p > 1:
                         x = arenas["fp32"][: p * n].view(p, n)

@@ -171,7 +171,7 @@ def test_tree_variant_is_checked_on_the_host():
                 rd.rd_schedule_set_tree_variant(h, rd.RD_TREE_DIRECT)
             else:
                 assert status_of(rd.rd_schedule_set_tree_variant, h, rd.RD_TREE_DIRECT) == rd.RD_ERR_UNSUPPORTED
-            assert status_of(rd.rd_schedule_set_tree_variant, h, 3) == rd.RD_ERR_INVALID_ARG
+            assert status_of(rd.rd_schedule_set_tree_variant, h, 4) == rd.RD_ERR_INVALID_ARG
             assert status_of(rd.rd_schedule_set_tree_variant, h, -1) == rd.RD_ERR_INVALID_ARG
         finally:
             rd.rd_destroy(h)

@@ -75,6 +75,36 @@ def test_parity_small_shapes_on_the_direct_kernel(name, algo, port, dist, op):
         check(algo, port, x, 4 * seg, op, variant=rd.RD_TREE_DIRECT)
 
 
+@pytest.mark.parametrize("name,algo,port", SCHEDULES)
+@pytest.mark.parametrize("dist,op", [("int_pm2p20", "sum"), ("normal", "sum"), ("normal", "max")])
+def test_parity_small_shapes_with_two_operand_tiles_per_stage(name, algo, port, dist, op):
+    """The streaming kernel on tiles of 1024 words, two operands to a ring stage (what the 16-bit types use
+    by default), asked for here with 4-byte elements: odd process counts leave the last stage of a tile half
+    full, p = 1 and p = 2 have a single stage per tile.  Same bits."""
+    for p, n, seg in SHAPES:
+        x = make_inputs(p, n, dist, seed=p * 1000 + n, device="cuda")
+        check(algo, port, x, 4 * seg, op, variant=rd.RD_TREE_STREAM_PAIRED)
+
+
+def test_two_operand_tiles_per_stage_deep_stacks_and_many_tiles():
+    """Many tiles per thread block, stacks up to depth 8 (binomial, p = 300), eight-byte elements."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    for p, n, seg, (name, algo, port) in [(9, 1024 * 7 * sms + 100, 3 * 1024 + 520, SCHEDULES[0]), (300, 1024 * 40 + 8, 4096, SCHEDULES[2]),
+                                          (128, 1024 * 5 * sms, 4096, SCHEDULES[1]), (3, 1024 * 9 * sms + 8, 2048 + 520, SCHEDULES[5])]:
+        x = make_inputs(p, n, "normal", seed=p + n, device="cuda")
+        h = rd.rd_schedule_create(algo, port, p, 4 * n, 4 * seg, *M1)
+        try:
+            rd.rd_schedule_set_tree_variant(h, rd.RD_TREE_STREAM_PAIRED)
+            shape = rd.rd_schedule_tree_shape(h)
+        finally:
+            rd.rd_destroy(h)
+        assert shape["variant"] == rd.RD_TREE_STREAM_PAIRED and shape["n_tiles"] >= n // 1024
+        check(algo, port, x, 4 * seg, "sum", variant=rd.RD_TREE_STREAM_PAIRED)
+    for kind, op in (("int64", "sum"), ("fp64", "sum"), ("fp64", "max")):
+        x = inputs64(13, 3 * 2048 + 36, kind, seed=21)
+        check64(rd.RD_BI_GREEDY, rd.RD_PORT_BI, x, 8 * (1024 + 260), op, variant=rd.RD_TREE_STREAM_PAIRED)
+
+
 def test_launch_shapes_two_and_three_blocks_per_sm():
     """The streaming kernel runs two or three thread blocks per SM depending on the number of tiles and on
     the stack depth; the direct kernel runs when asked for.  Every shape, element by element."""
@@ -777,10 +807,12 @@ def bits(t):
     return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
 
 
-def check_bf16(algo, port, x, seg_bytes, op, rows=None, out=None):
+def check_bf16(algo, port, x, seg_bytes, op, rows=None, out=None, variant=None):
     p, n = x.shape                                                   # n 16-bit elements = 2 n bytes
     h = rd.rd_schedule_create(algo, port, p, 2 * n, seg_bytes, *M1)
     try:
+        if variant is not None:
+            rd.rd_schedule_set_tree_variant(h, variant)
         out = torch.full((n,), 7.0, dtype=x.dtype, device="cuda") if out is None else out
         rd.rd_reduce(h, rows if rows is not None else x, out, OPS[op])
         torch.cuda.synchronize()
@@ -792,7 +824,7 @@ def check_bf16(algo, port, x, seg_bytes, op, rows=None, out=None):
     return out
 
 
-# (p, n bf16 elements, segment in bf16 elements): tiles hold 4096 of them; ragged tails; segments that
+# (p, n bf16 elements, segment in bf16 elements): tiles hold 2048 or 4096 of them; ragged tails; segments that
 # begin inside a 128-bit vector (multiples of 2 elements); lengths that are not whole vectors
 SHAPES_BF16 = [(8, 8192, 1024), (5, 20000, 5000), (13, 3 * 4096 + 72, 4096 + 1040), (64, 16384, 2048), (2, 8200, 8200),
                (33, 12000, 2000), (16, 256, 16), (1, 10000, 2000), (8, 6000, 666), (4, 128, 6), (32, 16384, 4098),
@@ -812,6 +844,17 @@ def test_bf16_parity(name, algo, port, kind, op, dtype):
             assert torch.equal(out.float(), x.float().sum(dim=0))
         elif op in ("max", "min"):
             assert torch.equal(out, x.amax(dim=0) if op == "max" else x.amin(dim=0))
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
+@pytest.mark.parametrize("name,algo,port", SCHEDULES)
+def test_bf16_parity_with_one_operand_tile_per_stage(name, algo, port, dtype):
+    """The 16-bit types run two operand tiles of 2048 elements per ring stage by default (the test above); on
+    request one tile of 4096 elements per stage, with stack levels twice as large.  Same bits."""
+    for p, n, seg in SHAPES_BF16:
+        x = bf16_inputs(p, n, "normal", seed=p * 1000 + n, dtype=dtype)
+        for op in ("sum", "max"):
+            check_bf16(algo, port, x, 2 * seg, op, variant=rd.RD_TREE_STREAM)
 
 
 def test_bf16_partial_results_stay_in_fp32_and_ties_round_to_even():

@@ -404,3 +404,22 @@ def test_fp16_small_integers_sum_exactly_and_extrema_are_order_free(p):
         assert (f16_value(O.reduce(ev, y, seg_off(sizes), "min", half="fp16")) == f16_value(y).min(axis=0)).all(), name
         wide = O.reduce(ev, f16_value(y), seg_off(sizes), "sum")
         assert (O.reduce(ev, y, seg_off(sizes), "sum", half="fp16") == f16_bits(wide)).all(), name
+
+
+def test_openmp_build_gives_the_bits_of_the_plain_build():
+    """The second build of the oracle (-fopenmp, timed by the benchmark on all cores) splits every segment's
+    elements over the threads; nothing else changes, so the results are identical bit for bit."""
+    rng = np.random.default_rng(7)
+    p, sizes = 13, [1000, 1000, 1000, 37]
+    n = sum(sizes)
+    assert O.threads(openmp=False) == 1 and O.threads(openmp=True) >= 1
+    xf = (rng.standard_normal((p, n)) * 10.0 ** rng.integers(-4, 5, size=(p, n))).astype(np.float32)
+    xi = rng.integers(-2**31, 2**31, size=(p, n), dtype=np.int64).astype(np.int32)
+    for name, ev in schedules(p, sizes):
+        for op in ("sum", "max", "min", "prod"):
+            for x in (xf, xi):
+                a = O.reduce(ev, x, seg_off(sizes), op)
+                b = O.reduce(ev, x, seg_off(sizes), op, openmp=True)
+                assert a.tobytes() == b.tobytes(), (name, op, x.dtype)
+    ev, off, _ = O.butterfly(p, n, 4, 3, 1, 1)
+    assert O.reduce(ev, xf, off, "sum").tobytes() == O.reduce(ev, xf, off, "sum", openmp=True).tobytes()
