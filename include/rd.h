@@ -17,9 +17,9 @@
  *     implementation makes the same restriction, Fig. 2 caption).  The system
  *     is homogeneous and fully connected (Section II), so a schedule does not
  *     care which buffer plays which process: to reduce towards another root,
- *     pass the pointer array permuted so that the root's buffer comes first.
- *     On one GPU every process can read the result buffer, so an all-reduce
- *     (Section III) needs no broadcast after the reduce.
+ *     pass the pointer array permuted so that the root's buffer comes first
+ *     (the combine order is then the schedule's with the processes relabelled
+ *     the same way).  rd_allreduce gives every process a copy of the result.
  *   - Sizes called "bytes" are bytes.  A schedule knows sizes in bytes only and reports segment
  *     boundaries in 4-byte words; n_elems of the reducing calls counts elements of the call's
  *     rd_dtype_t (4 or 8 bytes each).
@@ -176,7 +176,8 @@ RD_API int rd_optimal_segment(rd_algo_t algo, rd_port_t port, int p, size_t msg_
  * butterfly: p chunks), n_events the number of send/receive pairs
  * ((p-1)*q for the tree schedules), predicted_ticks / predicted_seconds the
  * completion time under the model, stack_depth the number of partial results
- * the combine programs keep besides the running one.                          */
+ * the combine programs keep besides the running one on a plain stack (with the
+ * hints of rd_schedule_program a kernel needs one level less).               */
 RD_API int rd_schedule_info(const rd_schedule_t *s, int *p, size_t *q, size_t *n_events,
                      double *predicted_seconds, int64_t *predicted_ticks, int *stack_depth);
 
@@ -202,7 +203,15 @@ RD_API int rd_schedule_segments(const rd_schedule_t *s, uint64_t *off, size_t ca
  *   bits 14-17  npop: number of pops that follow
  *   bits 18-29  bit k = role of the k-th pop: 1: top = combine(held = popped, incoming = top)
  *                                              0: top = combine(held = top, incoming = popped)
- * combine(held, incoming) = held + incoming, held * incoming, or incoming > held ? incoming : held
+ *   bit  30     the operation belongs to a sub-expression that needs no stack: it begins with a PUSH_LOAD,
+ *               continues with ACC operations and ends with the operation that has bit 31 set, whose
+ *               first pop takes back the entry the PUSH_LOAD pushed; nothing else is pushed or popped in
+ *               between.  An interpreter may evaluate such a sub-expression in a second accumulator
+ *               (PUSH_LOAD: second = x; ACC: second = combine(second, x) resp. combine(x, second)) and
+ *               leave top where it is; at the end the pop's two values are top (as "popped") and second.
+ *   bit  31     last operation of such a sub-expression
+ * Bits 30 and 31 are hints: an interpreter that pushes and pops everything on one stack gets the same
+ * result.  combine(held, incoming) = held + incoming, held * incoming, or incoming > held ? incoming : held
  * (min: <).
  * After the last operation top is the root's value (Section IV: the receiver
  * combines its segment with the one received).
@@ -240,6 +249,21 @@ RD_API int rd_schedule_program(const rd_schedule_t *s, size_t seg, uint32_t *ops
  */
 RD_API int rd_reduce(rd_schedule_t *s, const void *const *d_inputs, void *d_out, size_t n_elems,
               rd_dtype_t dtype, rd_op_t op, rd_exec_t exec, void *cuda_stream, rd_stats_t *stats);
+
+/*
+ * rd_allreduce -- Section III "All-reduce": every process ends up with the combined vector; as the paper
+ * states it, a reduce followed by a broadcast.  Tree mode: the reduction of rd_reduce into d_outs[0] (the
+ * root's copy, same kernel, same bits), then one more kernel that copies the root's result to the other
+ * p - 1 buffers (at most 256 destinations per launch).  Asynchronous on cuda_stream.
+ *   d_inputs  HOST array of p DEVICE pointers, as in rd_reduce.
+ *   d_outs    HOST array of p DEVICE pointers: d_outs[i] receives process i's copy, n_elems elements.
+ *             d_outs[i] may be d_inputs[i] itself (in-place all-reduce); otherwise no copy may overlap any
+ *             input or another copy (RD_ERR_INVALID_ARG).
+ *   stats     host or NULL: kernel_ms covers both kernels; bytes_moved = p*m + m for the reduce plus
+ *             m read and (p-1)*m written by the broadcast.
+ */
+RD_API int rd_allreduce(rd_schedule_t *s, const void *const *d_inputs, void *const *d_outs, size_t n_elems,
+                        rd_dtype_t dtype, rd_op_t op, void *cuda_stream, rd_stats_t *stats);
 
 /*
  * rd_reduce_batch -- several independent tree-mode reductions issued together (the paper has no

@@ -31,7 +31,7 @@ EXPORTS = ("rd_schedule_create", "rd_schedule_create_segments", "rd_optimal_segm
            "rd_schedule_events", "rd_schedule_segments", "rd_schedule_program", "rd_reduce",
            "rd_schedule_upload", "rd_reduce_host", "rd_destroy", "rd_strerror", "rd_schedule_set_wait_budget",
            "rd_schedule_trace", "rd_schedule_faithful_shape", "rd_schedule_actions", "rd_reduce_faithful_static", "rd_search_segmentation", "rd_schedule_status",
-           "rd_reduce_batch", "rd_schedule_set_tree_variant", "rd_schedule_tree_shape")
+           "rd_reduce_batch", "rd_schedule_set_tree_variant", "rd_schedule_tree_shape", "rd_allreduce")
 
 
 class rd_model_t(C.Structure):
@@ -80,6 +80,7 @@ def lib():
         L.rd_schedule_program.argtypes = [vp, sz, vp, sz]
         L.rd_reduce.argtypes = [vp, C.POINTER(vp), vp, sz, i32, i32, i32, vp, C.POINTER(rd_stats_t)]
         L.rd_schedule_upload.argtypes = [vp]
+        L.rd_allreduce.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), sz, i32, i32, vp, C.POINTER(rd_stats_t)]
         L.rd_reduce_host.argtypes = [vp, C.POINTER(vp), vp, vp, sz, i32, i32, vp]
         L.rd_schedule_set_wait_budget.argtypes = [vp, C.c_double]
         L.rd_schedule_set_tree_variant.argtypes = [vp, i32]
@@ -242,6 +243,22 @@ def rd_reduce(h, inputs, out, op, exec_mode=RD_EXEC_TREE, stream=None, want_stat
     finally:
         if out.device.index != prev:
             torch.cuda.set_device(prev)
+    return stats
+
+
+def rd_allreduce(h, inputs, outs, op, stream=None, want_stats=False):
+    """inputs, outs: each a PointerTable, a [p, n] CUDA tensor or a list of p CUDA tensors; outs[i] receives
+    process i's copy of the result and may be inputs[i] itself.  Returns rd_stats_t or None."""
+    import torch
+    tab = inputs if isinstance(inputs, PointerTable) else PointerTable(inputs)
+    otab = outs if isinstance(outs, PointerTable) else PointerTable(outs)
+    if not tab.is_cuda or not otab.is_cuda or tab.n != otab.n or tab.p != otab.p or tab.dtype != otab.dtype or tab.device != otab.device:
+        raise ValueError("inputs and outs must be p contiguous CUDA tensors each, of one dtype, length and device")
+    s = stream if stream is not None else torch.cuda.current_stream(tab.device)
+    stats = rd_stats_t() if want_stats else None
+    with torch.cuda.device(tab.device):
+        _check(lib().rd_allreduce(h, tab.array, otab.array, tab.n, _dtype_code(tab), int(op), s.cuda_stream,
+                                  C.byref(stats) if want_stats else None), "rd_allreduce")
     return stats
 
 

@@ -14,9 +14,10 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librd.so")
 SOURCES = ["rd_api.cpp", "rd_sched.cpp", "rd_compile.cpp", "rd_kernels.cu", "rd_faithful.cu"]
 HEADERS = ["rd_internal.h", "rd_kernels.h"]
-# rd_kernels.cu is compiled once per element type (-DRD_DT=k: that type's kernels) and once without
-# (launch shapes and dispatch), side by side
-KERNEL_DTYPES = 6
+# rd_kernels.cu is compiled once per element type (-DRD_DT=k: that type's kernels; the 16-bit types count
+# twice, once for sum and product and once for max and min) and once without (launch shapes and dispatch),
+# side by side
+KERNEL_DTYPES = 8
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC,-Wall,-Wextra,-fvisibility=hidden",

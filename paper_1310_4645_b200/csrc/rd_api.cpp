@@ -87,6 +87,13 @@ void reset_tile_counters(int device)
 constexpr int kDirectAutoProcs = 0;     // the direct kernel is never chosen by the library itself
 constexpr int kTailTiles = 5; // key of the tile table for the elements the 128-bit path leaves over
 constexpr int kPairTiles = 8; // key of the tile table of the 128-bit path with two operand tiles per ring stage
+int tiles_key(int ops_per_stage) { return ops_per_stage == 2 ? kPairTiles : 4; }
+// Levels the streaming kernel's shared-memory stack needs for a schedule's programs.
+int ring_depth(const Programs &progs, int acc_words_per_word, int ops_per_stage)
+{
+    return stream_second_accumulator(acc_words_per_word, ops_per_stage) ? progs.shared_depth : progs.stack_depth;
+}
+
 
 struct DeviceTables {
     int device = -1;
@@ -101,8 +108,8 @@ struct DeviceTables {
         int ctas_per_sm = 0;
         int stages = 0;
     };
-    std::map<int, StreamPlan> plans;        // key: 4 * (words of partial result per message word: 1, or 2 for 16-bit
-                                            // elements) + operand tiles per ring stage (1 or 2)
+    std::map<int, StreamPlan> plans;        // key: 64 * (words of partial result per message word: 1, or 2 for 16-bit
+                                            // elements) + 16 * operand tiles per ring stage + consumer warps
     int stage_elems = 0;
     int *status = nullptr;                                  // device word written by a kernel that gave up a wait
     // pointer tables for large p: pinned host ring + device ring, one event per slot
@@ -329,22 +336,30 @@ int tiles_for(rd_schedule *s, int vec, const TileDesc **tiles, uint32_t *count)
     return RD_OK;
 }
 
+// Whether the schedule's programs push a partial result on the stack for at least every tenth operand (trees like
+// the binomial one do for every fourth, the steady-state trees of uni-greedy for every fiftieth).
+bool many_pushes(const rd_schedule *s)
+{
+    const size_t operands = size_t(s->p) * s->progs.seg_prog.size();
+    return operands > 0 && s->progs.shared_pushes * 10 >= operands;
+}
+
 // Launch shape of a single reduction on the streaming path: CTAs get contiguous runs of tiles, the same
 // NUMBER of tiles up to one (a tile costs a CTA about the same time however full it is, one ring hand-off
 // per operation, so for small messages the number of tiles per CTA, not the number of elements, sets the
 // kernel's duration; for large ones the two coincide).  acc_words: 2 for bf16, whose partial results are fp32.
-int stream_plan(rd_schedule *s, int acc_words, int ops_per_stage, const DeviceTables::StreamPlan **out)
+int stream_plan(rd_schedule *s, int acc_words, int ops_per_stage, int consumer_warps, const DeviceTables::StreamPlan **out)
 {
     DeviceTables &d = s->dev;
-    const int key = 4 * acc_words + ops_per_stage;
+    const int key = 64 * acc_words + 16 * ops_per_stage + consumer_warps;
     auto it = d.plans.find(key);
     if (it == d.plans.end()) {
         const TileDesc *tiles = nullptr;
         uint32_t nTiles = 0;
-        if (int rc = tiles_for(s, ops_per_stage == 2 ? kPairTiles : 4, &tiles, &nTiles)) return rc;
+        if (int rc = tiles_for(s, tiles_key(ops_per_stage), &tiles, &nTiles)) return rc;
         DeviceTables::StreamPlan plan;
-        stream_shape(s->progs.stack_depth, acc_words, ops_per_stage, d.smem_per_sm, d.stage_elems, nTiles, d.sm_count, &plan.ctas_per_sm,
-                     &plan.stages);
+        stream_shape(ring_depth(s->progs, acc_words, ops_per_stage), acc_words, ops_per_stage, many_pushes(s), d.smem_per_sm, d.stage_elems,
+                     nTiles, d.sm_count, &plan.ctas_per_sm, &plan.stages);
         const uint64_t ctas = std::min<uint64_t>(uint64_t(d.sm_count) * uint64_t(plan.ctas_per_sm), std::max<uint64_t>(nTiles, 1));
         std::vector<uint32_t> first(size_t(ctas) + 1, 0);
         for (uint64_t c = 0; c < ctas; c++) first[size_t(c)] = uint32_t(uint64_t(nTiles) * c / ctas);
@@ -364,14 +379,28 @@ int stream_plan(rd_schedule *s, int acc_words, int ops_per_stage, const DeviceTa
 // Argument checks common to the reducing entry points.  On success *n_words is the message length
 // in 32-bit words, the unit in which the schedule's segment boundaries and the kernels count.
 bool is_half(rd_dtype_t dtype) { return dtype == RD_BF16 || dtype == RD_FP16; }
-// Operand tiles per ring stage of the streaming kernel.  The 16-bit types are combined in fp32, so a tile's
-// waiting partial results take twice the shared memory of its operand: they run on tiles of half a stage, two
-// to a stage, unless the schedule asks for one kind of stage or the other.
-int stage_ops(rd_dtype_t dtype, int tree_variant)
+// Words of partial result per message word: the 16-bit types are widened to fp32 for sum and product; their
+// max and min stay in 16 bits (the result of a combine is one of its operands).
+int acc_words(rd_dtype_t dtype, rd_op_t op) { return is_half(dtype) && (op == RD_SUM || op == RD_PROD) ? 2 : 1; }
+// Operand tiles per ring stage of the streaming kernel.  Where partial results are fp32 values of 16-bit elements
+// a tile's waiting partial results take twice the shared memory of its operand: from stack depth 2 on such
+// reductions run on tiles of half a stage, two to a stage (measured, bf16 sum, 64 MiB messages, GB/s, one tile
+// against two tiles per stage: p = 2 6197 / 4705, p = 4 6616 / 6396, p = 8 6801 / 6838, p = 64 uni-greedy
+// 6214 / 7174), unless the schedule asks for one kind of stage or the other.
+int stage_ops(int acc_words_per_word, int tree_variant, int stack_depth)
 {
     if (tree_variant == RD_TREE_STREAM) return 1;
     if (tree_variant == RD_TREE_STREAM_PAIRED) return 2;
-    return is_half(dtype) ? 2 : 1;
+    return acc_words_per_word > 1 && stack_depth >= 2 ? 2 : 1;
+}
+// Consumer warps of the streaming kernel: 8 with two vectors of a tile each, or 4 with four (two when two tiles
+// share a stage).  Fewer warps with more vectors each spend fewer issue slots per byte; that pays for the 16-bit
+// types, which have twice the elements per byte, and for deep stacks, where shared memory leaves room for two
+// thread blocks per SM only (measured, fp32 sum, p = 256, GB/s, 8 against 4 warps: binomial 6747 / 7104,
+// uni-greedy 7109 / 7321; p = 2 ... 64: equal within 1 %).
+int stage_warps(int acc_words_per_word, int ops_per_stage, int stack_depth)
+{
+    return ops_per_stage >= 2 || acc_words_per_word > 1 || stack_depth >= 6 ? 4 : 8;
 }
 size_t elem_bytes(rd_dtype_t dtype) { return (dtype == RD_INT64 || dtype == RD_FP64) ? 8 : is_half(dtype) ? 2 : 4; }
 
@@ -404,11 +433,12 @@ int reduce_tree(rd_schedule *s, const void *const *d_inputs, void *d_out, size_t
     for (int i = 0; i < s->p && wide; i++) wide = (reinterpret_cast<uintptr_t>(d_inputs[i]) & 15u) == 0;
     TreeLaunch l{};
     l.vec = wide ? 4 : 1;
-    l.ops_per_stage = stage_ops(dtype, s->tree_variant);
-    if (int rc = tiles_for(s, wide ? (l.ops_per_stage == 2 ? kPairTiles : 4) : 1, &l.tiles, &l.n_tiles)) return rc;
+    l.ops_per_stage = stage_ops(acc_words(dtype, op), s->tree_variant, s->progs.shared_depth);
+    l.consumer_warps = stage_warps(acc_words(dtype, op), l.ops_per_stage, s->progs.shared_depth);
+    if (int rc = tiles_for(s, wide ? tiles_key(l.ops_per_stage) : 1, &l.tiles, &l.n_tiles)) return rc;
     const DeviceTables::StreamPlan *plan = nullptr;
     if (wide)
-        if (int rc = stream_plan(s, is_half(dtype) ? 2 : 1, l.ops_per_stage, &plan)) return rc;
+        if (int rc = stream_plan(s, acc_words(dtype, op), l.ops_per_stage, l.consumer_warps, &plan)) return rc;
     const TileDesc *tailTiles = nullptr;
     uint32_t nTail = 0;
     if (wide && (n & 3u) != 0)
@@ -425,6 +455,7 @@ int reduce_tree(rd_schedule *s, const void *const *d_inputs, void *d_out, size_t
         l.dev_ptr_table = dv;
     }
     l.out = d_out; l.ops = d.ops; l.p = s->p; l.stack_depth = s->progs.stack_depth;
+    l.shared_depth = ring_depth(s->progs, acc_words(dtype, op), l.ops_per_stage);
     l.dtype = int(dtype); l.op = int(op); l.sm_count = d.sm_count; l.stream = stream;
     if (plan) { l.cta_first = plan->cta_first; l.n_ctas = plan->n_ctas; l.stages = plan->stages; }
     l.tile_counter = wide ? next_tile_counter(d.device, stream) : nullptr;
@@ -609,12 +640,15 @@ int reduce_batch_fused(size_t n_jobs, rd_schedule_t *const *schedules, const voi
     uint64_t total = 0;
     size_t nPtrs = 0;
     int depth = 0;
-    const int opsPerStage = stage_ops(dtype, RD_TREE_AUTO);        // one kind of stage for the whole launch
+    for (size_t j = 0; j < n_jobs; j++) depth = std::max(depth, schedules[j]->progs.shared_depth);
+    const int opsPerStage = stage_ops(acc_words(dtype, op), RD_TREE_AUTO, depth);  // one kind of stage for the whole launch
+    if (!stream_second_accumulator(acc_words(dtype, op), opsPerStage))             // levels in shared memory
+        for (size_t j = 0; j < n_jobs; j++) depth = std::max(depth, schedules[j]->progs.stack_depth);
     for (size_t j = 0; j < n_jobs; j++) {
         rd_schedule *s = schedules[j];
         const TileDesc *tiles = nullptr;
         uint32_t count = 0;
-        if (int rc = tiles_for(s, opsPerStage == 2 ? kPairTiles : 4, &tiles, &count)) return rc;
+        if (int rc = tiles_for(s, tiles_key(opsPerStage), &tiles, &count)) return rc;
         BatchJob &b = jobs[j];
         b.inputs = nullptr; b.out = static_cast<uint32_t *>(d_outs[j]); b.tiles = tiles; b.ops = s->dev.ops;
         b.tile_begin = uint32_t(total); b.p = s->p; b.ptr_base = 0;
@@ -622,17 +656,19 @@ int reduce_batch_fused(size_t n_jobs, rd_schedule_t *const *schedules, const voi
         if (total > 0xFFFFFFFFull) return RD_ERR_UNSUPPORTED;
         b.tile_end = uint32_t(total);
         nPtrs += size_t(s->p);
-        depth = std::max(depth, s->progs.stack_depth);
     }
     if (total == 0) return RD_OK;
     DeviceTables &d0 = schedules[0]->dev;
     const int stageElems = d0.stage_elems;
     int ctasPerSm = 1, stages = 2;
-    stream_shape(depth, is_half(dtype) ? 2 : 1, opsPerStage, d0.smem_per_sm, stageElems, total, d0.sm_count, &ctasPerSm, &stages);
+    const int consumerWarps = stage_warps(acc_words(dtype, op), opsPerStage, depth);
+    bool pushy = false;
+    for (size_t j = 0; j < n_jobs; j++) pushy = pushy || many_pushes(schedules[j]);
+    stream_shape(depth, acc_words(dtype, op), opsPerStage, pushy, d0.smem_per_sm, stageElems, total, d0.sm_count, &ctasPerSm, &stages);
     const uint64_t ctas = std::min<uint64_t>(uint64_t(d0.sm_count) * uint64_t(ctasPerSm), total);
     BatchLaunch b{};
     b.n_jobs = uint32_t(n_jobs); b.n_tiles = uint32_t(total); b.n_ctas = uint32_t(ctas);
-    b.stages = stages; b.stack_depth = depth; b.stage_elems = stageElems; b.ops_per_stage = opsPerStage;
+    b.stages = stages; b.stack_depth = depth; b.stage_elems = stageElems; b.ops_per_stage = opsPerStage; b.consumer_warps = consumerWarps;
     b.dtype = int(dtype); b.op = int(op); b.device = device; b.status = d0.status; b.stream = user;
     b.tile_counter = next_tile_counter(device, user);
     if (n_jobs <= size_t(kBatchPackJobs) && nPtrs <= size_t(kBatchPackPtrs)) {
@@ -830,6 +866,59 @@ int rd_reduce(rd_schedule_t *s, const void *const *d_inputs, void *d_out, size_t
     });
 }
 
+int rd_allreduce(rd_schedule_t *s, const void *const *d_inputs, void *const *d_outs, size_t n_elems, rd_dtype_t dtype, rd_op_t op,
+                 void *cuda_stream, rd_stats_t *stats)
+{
+    if (!s || !d_outs) return RD_ERR_INVALID_ARG;
+    size_t n_words = 0;
+    if (int rc = check_reduce_args(s, d_inputs, d_outs[0], n_elems, dtype, op, &n_words)) return rc;
+    const size_t bytes = n_words * 4;
+    const size_t align = elem_bytes(dtype) < 4 ? 4 : elem_bytes(dtype);
+    auto overlap = [bytes](const void *a, const void *b) {
+        const uintptr_t x = reinterpret_cast<uintptr_t>(a), y = reinterpret_cast<uintptr_t>(b);
+        return bytes > 0 && x < y + bytes && y < x + bytes;
+    };
+    bool wide = (n_words & 3u) == 0;
+    for (int i = 0; i < s->p; i++) {
+        if ((n_elems > 0 && !d_outs[i]) || (reinterpret_cast<uintptr_t>(d_outs[i]) & (align - 1))) return RD_ERR_INVALID_ARG;
+        wide = wide && (reinterpret_cast<uintptr_t>(d_outs[i]) & 15u) == 0;
+        // the copies are written while other processes' inputs may still be read: a copy may only coincide with
+        // its own process's input (the in-place all-reduce), and no two copies may overlap
+        for (int k = 0; k < s->p; k++) {
+            if (k != i && overlap(d_outs[i], d_inputs[k])) return RD_ERR_INVALID_ARG;
+            if (k > i && overlap(d_outs[i], d_outs[k])) return RD_ERR_INVALID_ARG;
+        }
+        if (d_outs[i] != d_inputs[i] && overlap(d_outs[i], d_inputs[i])) return RD_ERR_INVALID_ARG;
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    return guarded([&]() -> int {
+        if (int rc = upload(s)) return rc;
+        DeviceTables &d = s->dev;
+        if (stats && cudaEventRecord(d.ev_start, stream) != cudaSuccess) return RD_ERR_CUDA;
+        // Section III: a reduce to the root followed by a broadcast of the root's result
+        if (int rc = reduce_tree(s, d_inputs, d_outs[0], n_words, dtype, op, stream, nullptr)) return rc;
+        if (s->p > 1 && launch_broadcast(d_outs[0], d_outs + 1, s->p - 1, n_words, wide, d.sm_count, stream) != 0) return RD_ERR_CUDA;
+        if (stats) {
+            if (cudaEventRecord(d.ev_stop, stream) != cudaSuccess || cudaEventSynchronize(d.ev_stop) != cudaSuccess) return RD_ERR_CUDA;
+            float ms = 0;
+            if (cudaEventElapsedTime(&ms, d.ev_start, d.ev_stop) != cudaSuccess) return RD_ERR_CUDA;
+            std::memset(stats, 0, sizeof(*stats));
+            stats->kernel_ms = ms;
+            stats->bytes_moved = (uint64_t(s->p + 1) + uint64_t(s->p > 1 ? s->p : 0)) * uint64_t(bytes);
+            stats->gbytes_per_s = ms > 0 ? double(stats->bytes_moved) / (double(ms) * 1e6) : 0.0;
+            stats->predicted_s = double(s->sched.completion) * s->ticks.tick;
+            bool vectors = (reinterpret_cast<uintptr_t>(d_outs[0]) & 15u) == 0;      // the reduction took the 128-bit path
+            for (int i = 0; i < s->p && vectors; i++) vectors = (reinterpret_cast<uintptr_t>(d_inputs[i]) & 15u) == 0;
+            stats->n_launches = n_words ? 1 + (vectors && (n_words & 3u) ? 1 : 0) + (s->p > 1 ? (s->p - 2) / kBcastPackPtrs + 1 : 0) : 0;
+            int st = 0;
+            if (cudaMemcpy(&st, d.status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return RD_ERR_CUDA;
+            stats->device_status = st;
+            if (st != 0) return RD_ERR_TIMEOUT;
+        }
+        return RD_OK;
+    });
+}
+
 int rd_reduce_batch(size_t n_jobs, rd_schedule_t *const *schedules, const void *const *const *d_inputs, void *const *d_outs,
                     const size_t *n_elems, rd_dtype_t dtype, rd_op_t op, void *cuda_stream)
 {
@@ -979,13 +1068,13 @@ int rd_schedule_tree_shape(rd_schedule_t *s, int *variant, int *blocks_per_sm, i
     return guarded([&] {
         if (int rc = upload(s)) return rc;
         TreeLaunch l{};
-        const int opsPerStage = stage_ops(RD_FP32, s->tree_variant);
-        if (int rc = tiles_for(s, opsPerStage == 2 ? kPairTiles : 4, &l.tiles, &l.n_tiles)) return rc;
+        const int opsPerStage = stage_ops(1, s->tree_variant, s->progs.shared_depth);
+        if (int rc = tiles_for(s, tiles_key(opsPerStage), &l.tiles, &l.n_tiles)) return rc;
         const bool direct = direct_applies(s->p, s->progs.stack_depth) &&
                             (s->tree_variant == RD_TREE_DIRECT || (s->tree_variant == RD_TREE_AUTO && s->p <= kDirectAutoProcs));
         if (variant) *variant = direct ? RD_TREE_DIRECT : opsPerStage == 2 ? RD_TREE_STREAM_PAIRED : RD_TREE_STREAM;
         const DeviceTables::StreamPlan *plan = nullptr;
-        if (int rc = stream_plan(s, 1, opsPerStage, &plan)) return rc;
+        if (int rc = stream_plan(s, 1, opsPerStage, stage_warps(1, opsPerStage, s->progs.shared_depth), &plan)) return rc;
         if (blocks_per_sm) *blocks_per_sm = direct ? direct_blocks_per_sm(s->p) : plan->ctas_per_sm;
         if (ring_stages) *ring_stages = direct ? 0 : plan->stages;
         if (n_tiles) *n_tiles = l.n_tiles;

@@ -71,6 +71,8 @@ int compile_programs(int p, size_t q, const std::vector<rd_event_t> &events, Pro
     out.ops.clear();
     out.seg_prog.assign(q, 0);
     out.stack_depth = 0;
+    out.shared_depth = 0;
+    out.shared_pushes = 0;
     out.n_distinct = 0;
     // bucket the pairs by segment, keeping their start-time order
     std::vector<size_t> first(q + 1, 0);
@@ -138,6 +140,39 @@ int compile_programs(int p, size_t q, const std::vector<rd_event_t> &events, Pro
         if (prog.size() != size_t(p)) return RD_ERR_INTERNAL;
         if (need[size_t(root)] > kMaxPops) return RD_ERR_INTERNAL;
         out.stack_depth = std::max(out.stack_depth, need[size_t(root)]);
+        // A pushed value that is popped again before anything else is pushed never has another entry above it,
+        // and the sub-expression evaluated in between (the PUSH_LOAD, the combines that follow it, up to the
+        // operation whose first pop takes the entry back) needs no stack of its own: a kernel may evaluate it in a
+        // second accumulator and leave the running value where it is, instead of pushing and popping it.  Those
+        // operations are marked, and so is the one that ends the sub-expression; what remains is the depth a
+        // stack really needs then.
+        {
+            std::vector<std::pair<size_t, bool>> open;      // pushes not yet popped: (operation, still nothing above it)
+            int onStack = 0, deepest = 0;
+            size_t pushed = 0;                               // pushes that stay pushes
+            for (size_t k = 0; k < prog.size(); k++) {
+                if (((prog[k] >> kIdxBits) & 3u) == OP_PUSH_LOAD) {
+                    if (!open.empty() && open.back().second) { open.back().second = false; deepest = std::max(deepest, ++onStack); }
+                    open.emplace_back(k, true);
+                }
+                const uint32_t pops = (prog[k] >> (kIdxBits + 2)) & 0xFu;
+                for (uint32_t m = 0; m < pops; m++) {
+                    if (open.empty()) return RD_ERR_INTERNAL;
+                    if (open.back().second) {
+                        if (m != 0) return RD_ERR_INTERNAL;
+                        for (size_t t = open.back().first; t <= k; t++) prog[t] |= kOpSecondAccumulator;
+                        prog[k] |= kOpMergeSecond;
+                    } else {
+                        onStack--;
+                        pushed++;
+                    }
+                    open.pop_back();
+                }
+            }
+            if (!open.empty() || onStack != 0) return RD_ERR_INTERNAL;
+            out.shared_depth = std::max(out.shared_depth, deepest);
+            out.shared_pushes += pushed;
+        }
         std::string key(reinterpret_cast<const char *>(prog.data()), prog.size() * sizeof(uint32_t));
         auto it = seen.find(key);
         if (it == seen.end()) {

@@ -41,11 +41,15 @@ constexpr int kIdxBits = 12;           // process index field of an operation wo
 constexpr int kMaxProcs = 1 << kIdxBits;
 constexpr int kMaxPops = 12;
 enum OpKind : uint32_t { OP_LOAD = 0, OP_PUSH_LOAD = 1, OP_ACC_IN = 2, OP_ACC_HELD = 3 };
+constexpr uint32_t kOpSecondAccumulator = 1u << 30;   // the operation belongs to a sub-expression that needs no stack (see rd.h)
+constexpr uint32_t kOpMergeSecond = 1u << 31;         // ... and is its last one: its first pop joins it with the running value
 
 struct Programs {
     std::vector<uint32_t> ops;        // distinct programs, p words each, back to back
     std::vector<uint32_t> seg_prog;   // per segment: first word of its program in ops
     int stack_depth = 0;              // deepest stack any program needs (entries besides top)
+    int shared_depth = 0;             // ... when sub-expressions that need no stack run in a second accumulator
+    size_t shared_pushes = 0;         // pushes that remain then, summed over all segments
     size_t n_distinct = 0;
 };
 int compile_programs(int p, size_t q, const std::vector<rd_event_t> &events, Programs &out);

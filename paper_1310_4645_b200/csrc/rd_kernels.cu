@@ -54,7 +54,12 @@ inline cudaError_t opt_in_shared_memory(const void *kernel, int device)
 constexpr int kIdxBits = 12;
 constexpr uint32_t kIdxMask = (1u << kIdxBits) - 1;
 
-enum { DT_INT32 = 0, DT_FP32 = 1, DT_INT64 = 2, DT_FP64 = 3, DT_BF16 = 4, DT_FP16 = 5 };
+// DT_BF16_PICK, DT_FP16_PICK: the 16-bit types under max and min.  The result of such a combine is one of its
+// two operands, so nothing ever leaves the 16-bit format: the kernels work on the packed pairs of a word
+// directly (one packed comparison and one bit select per word), partial results are as large as the
+// operands, and the result equals, bit for bit, that of widening to fp32, comparing there and rounding at
+// the end (widening keeps the order, the selected value is representable).
+enum { DT_INT32 = 0, DT_FP32 = 1, DT_INT64 = 2, DT_FP64 = 3, DT_BF16 = 4, DT_FP16 = 5, DT_BF16_PICK = 6, DT_FP16_PICK = 7 };
 
 // The kernels move and index the message in 32-bit words; an element is one word or two, or (bf16, fp16)
 // half a word: a word then holds two elements, the lower-addressed one in its low half.
@@ -100,6 +105,17 @@ template <int DT, int OPR> __device__ __forceinline__ uint32_t combine(uint32_t 
         if (OPR == OPR_PROD) return held * in;                      // wraps modulo 2^32
         if (OPR == OPR_MAX) return (int32_t(in) > int32_t(held)) ? in : held;
         return (int32_t(in) < int32_t(held)) ? in : held;
+    } else if (DT == DT_BF16_PICK || DT == DT_FP16_PICK) {
+        // two elements per word: all ones in the half where the incoming element wins (never on a tie or a NaN)
+        unsigned wins;
+        if (DT == DT_BF16_PICK) {
+            const __nv_bfloat162 h = *reinterpret_cast<const __nv_bfloat162 *>(&held), i = *reinterpret_cast<const __nv_bfloat162 *>(&in);
+            wins = OPR == OPR_MAX ? __hgt2_mask(i, h) : __hlt2_mask(i, h);
+        } else {
+            const __half2 h = *reinterpret_cast<const __half2 *>(&held), i = *reinterpret_cast<const __half2 *>(&in);
+            wins = OPR == OPR_MAX ? __hgt2_mask(i, h) : __hlt2_mask(i, h);
+        }
+        return (in & wins) | (held & ~wins);
     } else {
         const float h = __uint_as_float(held), i = __uint_as_float(in);
         if (OPR == OPR_SUM) return __float_as_uint(__fadd_rn(h, i));   // one IEEE add, never contracted
@@ -309,11 +325,10 @@ rd_tree_kernel(const __grid_constant__ TreeParams<PACKED> a)
 // Every wait is bounded: on expiry the thread records an error code and the CTA winds down (a
 // producer lane first waits, again bounded, for the copy it has in flight).
 // ---------------------------------------------------------------------------------------------
-constexpr int kMaxStageElems = 2048;                    // largest stage = largest tile (8 KB)
+constexpr int kStageWords = 2048;                       // a ring stage: 8 KB; the largest tile
+constexpr int kStageVecs = kStageWords / 4;
 constexpr int kMaxStages = 32;
-constexpr int kConsumers = 256;
 constexpr int kProducers = 2;                            // producer warps per CTA (one active lane each)
-constexpr int kStreamThreads = kConsumers + 32 * kProducers;
 constexpr long long kWaitCycles = 4000000000ll;         // a wait gives up after about two seconds of SM clock
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p) { return uint32_t(__cvta_generic_to_shared(p)); }
@@ -337,15 +352,25 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
                  : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
+// The same on a barrier given by its shared-memory address.  The last operand is a hint: the thread may stay
+// suspended in hardware up to that many nanoseconds while the phase is not complete (it resumes when it is), so
+// a waiting thread spends few issue slots.
+__device__ __forceinline__ bool mbar_try_wait_at(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity), "r"(20000u) : "memory");
+    return ok != 0;
+}
 // Bounded wait; false when it gave up or another thread of the CTA already did.  try_wait suspends
 // the thread in hardware for a while, so the loop turns slowly; the clock and the abort flag are
 // only looked at every 64 turns.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+__device__ __forceinline__ bool mbar_wait_at(uint32_t bar, uint32_t parity, volatile int *abort_flag)
 {
-    if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait_at(bar, parity)) return true;
     long long start = 0;
     for (uint32_t turns = 1;; turns++) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait_at(bar, parity)) return true;
         if ((turns & 63u) == 0u) {
             if (*abort_flag) return false;
             const long long now = clock64();
@@ -354,10 +379,28 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
         }
     }
 }
-__device__ __forceinline__ void bulk_load(void *smem_dst, const void *gmem_src, uint32_t bytes, uint64_t *bar)
+__device__ __forceinline__ void mbar_arrive_at(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr)
+{
+    uint4 r;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr) : "memory");
+    return r;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, const uint4 &v)
+{
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void bulk_load_at(uint32_t smem_dst, const void *gmem_src, uint32_t bytes, uint32_t bar)
 {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_addr(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+                 ::"r"(smem_dst), "l"(gmem_src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx_at(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 
 constexpr uint32_t kLenMask = 0xFFFFu;   // TileDesc::len: bits 0-15 padded length, 16-17 elements to skip at the head, 18-19 at the tail
@@ -384,7 +427,7 @@ template <bool PACKED> struct StreamParams {
     int *status;                 // device word: 0, or the first error code
     uint32_t *tile_counter;      // two device words (next tile, CTAs done), both 0 at launch: tiles are handed out
                                  // on demand; null: every CTA works through its own range
-    int stages, depth, stage_elems;
+    int stages, depth;
     __device__ __forceinline__ void tile_range(uint32_t cta, uint32_t &t0, uint32_t &t1) const { t0 = cta_first[cta]; t1 = cta_first[cta + 1]; }
     __device__ __forceinline__ uint32_t total_tiles() const { return t.n_tiles; }
 };
@@ -400,7 +443,7 @@ template <> struct BatchStreamParams<true> {
     uint32_t n_jobs, n_tiles;
     int *status;
     uint32_t *tile_counter;
-    int stages, depth, stage_elems;
+    int stages, depth;
     __device__ __forceinline__ uint32_t total_tiles() const { return n_tiles; }
     __device__ __forceinline__ BatchJob job(uint32_t j) const { return jobs[j]; }
     __device__ __forceinline__ uint32_t job_end(uint32_t j) const { return jobs[j].tile_end; }
@@ -416,7 +459,7 @@ template <> struct BatchStreamParams<false> {
     uint32_t n_jobs, n_tiles;
     int *status;
     uint32_t *tile_counter;
-    int stages, depth, stage_elems;
+    int stages, depth;
     __device__ __forceinline__ uint32_t total_tiles() const { return n_tiles; }
     __device__ __forceinline__ BatchJob job(uint32_t j) const { return jobs[j]; }
     __device__ __forceinline__ uint32_t job_end(uint32_t j) const { return jobs[j].tile_end; }
@@ -560,8 +603,8 @@ struct TileSource {
     }
 };
 
-// What a consumer thread carries for its N (one or two) 128-bit vectors of an operand tile: the vectors
-// themselves, or (bf16, fp16) their elements widened to fp32, twice as many words.
+// What a consumer thread carries for its N 128-bit vectors of an operand tile: the vectors themselves, or
+// (bf16, fp16) their elements widened to fp32, twice as many words.
 template <int DT, int N> struct StageAcc {
     static constexpr int W = Wide<DT>::W;
     static constexpr int ADT = Wide<DT>::ADT;
@@ -591,19 +634,17 @@ template <int DT, int N> struct StageAcc {
 #pragma unroll
         for (int k = 0; k < N * W; k++) combine_vec<ADT, OPR, 4>(v[k], held.v[k], in.v[k]);
     }
-    // one stack level: [vector][consumer thread], the first vector's words first; `all` false: only the
-    // first vector of the thread is in use (tiles of at most 1024 words)
-    __device__ __forceinline__ void push(uint4 *level, uint32_t tid, bool all) const
+    // one stack level (shared-memory address): [vector][consumer thread]
+    __device__ __forceinline__ void push(uint32_t level, uint32_t tid, uint32_t threads) const
     {
 #pragma unroll
-        for (int k = 0; k < N * W; k++)
-            if (k < W || all) level[k * kConsumers + tid] = make_uint4(v[k].w[0], v[k].w[1], v[k].w[2], v[k].w[3]);
+        for (int k = 0; k < N * W; k++) sts128(level + (uint32_t(k) * threads + tid) * 16u, make_uint4(v[k].w[0], v[k].w[1], v[k].w[2], v[k].w[3]));
     }
-    __device__ __forceinline__ void pop(const uint4 *level, uint32_t tid, bool all)
+    __device__ __forceinline__ void pop(uint32_t level, uint32_t tid, uint32_t threads)
     {
 #pragma unroll
         for (int k = 0; k < N * W; k++) {
-            const uint4 y = (k < W || all) ? level[k * kConsumers + tid] : make_uint4(0, 0, 0, 0);
+            const uint4 y = lds128(level + (uint32_t(k) * threads + tid) * 16u);
             v[k].w[0] = y.x; v[k].w[1] = y.y; v[k].w[2] = y.z; v[k].w[3] = y.w;
         }
     }
@@ -621,27 +662,47 @@ template <int DT, int N> struct StageAcc {
     }
 };
 
-// G = operand tiles per ring stage.  G = 1: a stage holds one tile of up to a whole stage (two vectors per
-// consumer thread).  G = 2: tiles are half as long (one vector per consumer thread), a stage holds the tiles of
-// two consecutive operations of the program, each brought by its own bulk copy, and is handed over once for
-// both: the partial results that wait in the stack are half as large per tile, while the bytes per stage
-// hand-over, which set the pace, stay the same.
-template <int DT, int OPR, typename PRM, int G>
-__global__ void __launch_bounds__(kStreamThreads, 3)
+// Shape of a streaming launch.  G = operand tiles per ring stage: G = 1, a stage holds one tile of up to a whole
+// stage; G = 2, tiles are half as long, a stage holds the tiles of two consecutive operations of the program,
+// each brought by its own bulk copy, and is handed over once for both, so that the partial results that wait
+// in the stack are half as large per tile while the bytes per stage hand-over stay the same.  CW = consumer
+// warps: the 512 / G vectors of a tile are spread over CW * 32 threads, N = 16 / (G * CW) vectors each.  The
+// path is bound by instruction issue as much as by HBM (the waits, releases and the decoding of an operation
+// cost a warp about as many issue slots as the combines of two vectors), so fewer warps with more vectors
+// each spend fewer slots per byte.
+template <int G, int CW> struct StreamShape {
+    static constexpr int CT = CW * 32;                       // consumer threads
+    static constexpr int N = kStageVecs / (G * CT);          // vectors per thread and operand
+    static constexpr int THREADS = CT + 32 * kProducers;
+    static_assert(N >= 1 && N * G * CT == kStageVecs, "a tile is a whole number of vectors per consumer thread");
+};
+// Thread blocks per SM the registers must leave room for (shared memory decides how many actually run).
+template <int DT, int CW> struct StreamBlocks { static constexpr int value = 3; };
+// Whether the kernel evaluates the sub-expressions marked in the programs (bit 30) in a second accumulator, which
+// saves their pushes and pops and one level of the shared-memory stack.  Not where a thread's accumulator is
+// 32 registers already (16-bit elements on whole-stage tiles: these serve shallow programs only).
+template <int DT, int G> struct SecondAccumulator { static constexpr bool value = !(Wide<DT>::half && G == 1); };
+
+template <int DT, int OPR, typename PRM, int G, int CW>
+__global__ void __launch_bounds__(StreamShape<G, CW>::THREADS, StreamBlocks<DT, CW>::value)
 rd_tree_stream_kernel(const __grid_constant__ PRM a)
 {
     using Jobs = typename PRM::Jobs;
-    constexpr int N = 2 / G;                                                                 // vectors per thread and operand
+    using Shape = StreamShape<G, CW>;
+    constexpr int N = Shape::N;
+    constexpr uint32_t CT = Shape::CT;
+    constexpr uint32_t kStageBytes = kStageWords * 4u, kSubBytes = kStageBytes / uint32_t(G);
+    constexpr uint32_t kLevelBytes = uint32_t(N) * uint32_t(Wide<DT>::W) * CT * 16u;          // one stack level
+    constexpr uint32_t kSecondBit = 1u << (30 - kIdxBits), kMergeBit = 1u << (31 - kIdxBits); // in an operation word >> kIdxBits
+    constexpr bool AUX = SecondAccumulator<DT, G>::value;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int S = a.stages;
-    const uint32_t stageVecs = uint32_t(a.stage_elems) / 4u;                                 // 128-bit vectors per stage
-    const uint32_t subVecs = stageVecs / uint32_t(G);                                        // ... per operand tile
-    uint4 *ring = reinterpret_cast<uint4 *>(smem_raw);                                       // [S][G][subVecs]
-    const bool all = subVecs > kConsumers;                                                   // a second vector per thread
-    const uint32_t levelVecs = (all ? 2u : 1u) * uint32_t(Wide<DT>::W) * kConsumers;
-    uint4 *stack = ring + size_t(S) * stageVecs;                                              // [depth][(1 or 2) * W][256]
-    uint64_t *full = reinterpret_cast<uint64_t *>(stack + size_t(a.depth) * levelVecs);
-    uint64_t *empty = full + S;
+    // dynamic shared memory: ring [S][G][kSubBytes] | stack [depth][N * W][CT] vectors | full[S] | empty[S] | steps [S][G]
+    const uint32_t ring = smem_addr(smem_raw);
+    const uint32_t stack = ring + uint32_t(S) * kStageBytes;
+    const uint32_t full = stack + uint32_t(a.depth) * kLevelBytes;
+    const uint32_t empty = full + uint32_t(S) * 8u;
+    const uint32_t stepWords = empty + uint32_t(S) * 8u;             // per stage: the operation words of its G operands
     __shared__ int abort_flag;
     __shared__ TileQueue tileq;
     const uint32_t tid = threadIdx.x;
@@ -649,7 +710,10 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
     if (tid == 0) {
         abort_flag = 0;
         tileq.published = 0;
-        for (int s = 0; s < S; s++) { mbar_init(full + s, 1); mbar_init(empty + s, kConsumers / 32); }
+        for (int s = 0; s < S; s++) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full + uint32_t(s) * 8u), "r"(1u) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty + uint32_t(s) * 8u), "r"(uint32_t(CW)) : "memory");
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -659,17 +723,17 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    if (tid >= kConsumers) {
+    if (tid >= CT) {
         // ------------------------------------------------------------------ producers
         // One lane in each of the kProducers producer warps.  A step is one ring stage: the operand tiles of
         // G consecutive operations of a tile's program.  Producer j owns the steps j, j + P, j + 2P, ... of
         // this CTA's sequence of steps and issues them in order: stages are released by the consumers in that
         // same order, so a producer never waits for a stage while a later one of its own is already free.
         // Being alone in its warp, a producer polls without divergence; the table look-ups of a step are
-        // issued before its wait.
+        // issued before its wait.  The step's operation words travel to the consumers beside the stage.
         if ((tid & 31u) != 0) return;
         const int P = kProducers < S ? kProducers : S;
-        const int j = int(tid - kConsumers) / 32;
+        const int j = int(tid - CT) / 32;
         if (j >= P) return;
         TileSource source;                      // used by producer 0 only
         if (j == 0) {
@@ -699,16 +763,23 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
             if (tile != cur) { td = jobs.tile(tile); cur = tile; }
             const int first = i * G;
             const int cnt = p - first < G ? p - first : G;
+            uint32_t wv[G];
             const uint32_t *src[G];
 #pragma unroll
-            for (int g = 0; g < G; g++)
-                src[g] = g < cnt ? jobs.input(__ldg(jobs.ops() + td.prog + first + g) & kIdxMask) + td.elem_off : nullptr;
-            if (laps >= 1u && !mbar_wait(empty + stage, (laps - 1u) & 1u, &abort_flag)) { ok = false; break; }
+            for (int g = 0; g < G; g++) {
+                wv[g] = g < cnt ? __ldg(jobs.ops() + td.prog + first + g) : 0u;
+                src[g] = g < cnt ? jobs.input(wv[g] & kIdxMask) + td.elem_off : nullptr;
+            }
+            if (laps >= 1u && !mbar_wait_at(empty + uint32_t(stage) * 8u, (laps - 1u) & 1u, &abort_flag)) { ok = false; break; }
             const uint32_t bytes = (td.len & kLenMask) * 4u;
-            mbar_expect_tx(full + stage, bytes * uint32_t(cnt));
+            const uint32_t bar = full + uint32_t(stage) * 8u;
 #pragma unroll
             for (int g = 0; g < G; g++)
-                if (g < cnt) bulk_load(ring + size_t(stage) * stageVecs + size_t(g) * subVecs, src[g], bytes, full + stage);
+                asm volatile("st.shared.u32 [%0], %1;" ::"r"(stepWords + uint32_t(stage * G + g) * 4u), "r"(wv[g]) : "memory");
+            mbar_expect_tx_at(bar, bytes * uint32_t(cnt));             // (release: the words above are visible with the data)
+#pragma unroll
+            for (int g = 0; g < G; g++)
+                if (g < cnt) bulk_load_at(ring + uint32_t(stage) * kStageBytes + uint32_t(g) * kSubBytes, src[g], bytes, bar);
             any = true; lastStage = stage; lastLap = laps;
             if (j == 0) source.poke(k);
             i += P;
@@ -726,7 +797,7 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
             // leave only after this producer's last copies have landed (bounded); its earlier ones were consumed
             if (any) {
                 const long long start = clock64();
-                while (!mbar_try_wait(full + lastStage, lastLap & 1u) && clock64() - start < kWaitCycles) {}
+                while (!mbar_try_wait_at(full + uint32_t(lastStage) * 8u, lastLap & 1u) && clock64() - start < kWaitCycles) {}
             }
         }
         return;
@@ -743,70 +814,96 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
         jobs.seek(tile);
         const int p = jobs.p();
         const TileDesc td = jobs.tile(tile);
-        const uint32_t *prog = jobs.ops() + td.prog;
         const uint32_t len = td.len & kLenMask;                       // padded to whole 128-bit vectors
-        bool live[N];
-#pragma unroll
-        for (int n = 0; n < N; n++) live[n] = (uint32_t(n) * kConsumers + tid) * 4u < len;
-        StageAcc<DT, N> top;
+        StageAcc<DT, N> top, side;                                    // the running value; a sub-expression that needs no stack
         top.clear();
-        int sp = 0;
-        uint32_t w[G];
-#pragma unroll
-        for (int g = 0; g < G; g++) w[g] = g < p ? __ldg(prog + g) : 0u;
+        side.clear();
+        uint32_t sp = stack;                                          // address of the next free stack level
         for (int i = 0; i < p; i += G) {
-            uint32_t wn[G];
-#pragma unroll
-            for (int g = 0; g < G; g++) wn[g] = (i + G + g < p) ? __ldg(prog + i + G + g) : 0u;
-            if (!mbar_wait(full + stage, phase, &abort_flag)) {
+            if (!mbar_wait_at(full + uint32_t(stage) * 8u, phase, &abort_flag)) {
                 if (!abort_flag) { atomicCAS(a.status, 0, -5); abort_flag = 1; }
                 return;
             }
-            const uint4 *st = ring + size_t(stage) * stageVecs;
+            // the step's operation words, then its data: every thread reads its N vectors of each operand (threads
+            // beyond a short tile's end read stale bytes of the stage and never store their results)
+            uint32_t w[G];
+#pragma unroll
+            for (int g = 0; g < G; g++)
+                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w[g]) : "r"(stepWords + uint32_t(stage * G + g) * 4u) : "memory");
+            const uint32_t stageAddr = ring + uint32_t(stage) * kStageBytes + tid * 16u;
             uint4 r[G][N];
 #pragma unroll
             for (int g = 0; g < G; g++)
 #pragma unroll
-                for (int n = 0; n < N; n++)
-                    r[g][n] = (live[n] && i + g < p) ? st[uint32_t(g) * subVecs + uint32_t(n) * kConsumers + tid] : make_uint4(0, 0, 0, 0);
+                for (int n = 0; n < N; n++) r[g][n] = lds128(stageAddr + uint32_t(g) * kSubBytes + uint32_t(n) * CT * 16u);
+            // the stage's data is in registers: hand the stage back to the producer
+            __syncwarp();
+            if (lane == 0) mbar_arrive_at(empty + uint32_t(stage) * 8u);
+            if (++stage == S) { stage = 0; phase ^= 1u; }
 #pragma unroll
             for (int g = 0; g < G; g++) {
                 if (g > 0 && i + g >= p) break;
-                StageAcc<DT, N> x;
-                x.load(r[g]);
-                const uint32_t kind = (w[g] >> kIdxBits) & 3u;
-                if (kind == 1u) {
-                    top.push(stack + sp * levelVecs, tid, all);
-                    sp++;
-                }
-                if (kind <= 1u) {
-                    top = x;
-                } else if (kind == 2u || Commutes<OPR>::value) {
+                const uint32_t ctl = w[g] >> kIdxBits;                // kind | pops << 2 | roles of the pops << 6 | hints << 18
+                if (Commutes<OPR>::value ? (ctl | 1u) == 3u : ctl == 2u) {
+                    StageAcc<DT, N> x;                                // the common step: combine into the running value, no pops
+                    x.load(r[g]);
                     top.template combine<OPR>(top, x);
+                    continue;
+                }
+                if (AUX && (Commutes<OPR>::value ? (ctl | 1u) == (3u | kSecondBit) : ctl == (2u | kSecondBit))) {
+                    StageAcc<DT, N> x;                                // the same inside a sub-expression that needs no stack
+                    x.load(r[g]);
+                    side.template combine<OPR>(side, x);
+                    continue;
+                }
+                const uint32_t kind = ctl & 3u;
+                uint32_t npop = (ctl >> 2) & 0xFu;
+                uint32_t roles = ctl >> 6;
+                if (AUX && (ctl & kSecondBit)) {
+                    // a sub-expression that needs no stack: it is evaluated in `side`, the running value stays put
+                    if (kind == 1u) {
+                        side.load(r[g]);
+                    } else {
+                        StageAcc<DT, N> x;
+                        x.load(r[g]);
+                        if (kind == 2u || Commutes<OPR>::value) side.template combine<OPR>(side, x);
+                        else side.template combine<OPR>(x, side);
+                    }
+                    if (!(ctl & kMergeBit)) continue;
+                    // its end: what a stack machine would pop first is the running value, its current value is `side`
+                    npop--;
+                    const bool poppedHeld = (roles & 1u) != 0;
+                    roles >>= 1;
+                    if (poppedHeld || Commutes<OPR>::value) top.template combine<OPR>(top, side);
+                    else top.template combine<OPR>(side, top);
                 } else {
-                    top.template combine<OPR>(x, top);
+                    if (kind == 1u) {
+                        top.push(sp, tid, CT);
+                        sp += kLevelBytes;
+                    }
+                    if (kind <= 1u) {
+                        top.load(r[g]);
+                    } else {
+                        StageAcc<DT, N> x;
+                        x.load(r[g]);
+                        if (kind == 2u || Commutes<OPR>::value) top.template combine<OPR>(top, x);
+                        else top.template combine<OPR>(x, top);
+                    }
                 }
-                if (g == 0) {
-                    // the stage's data is in registers: hand the stage back to the producer
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(empty + stage);
-                    if (++stage == S) { stage = 0; phase ^= 1u; }
-                }
-                uint32_t npop = (w[g] >> (kIdxBits + 2)) & 0xFu;
-                uint32_t roles = w[g] >> (kIdxBits + 6);
                 while (npop--) {
-                    sp--;
+                    sp -= kLevelBytes;
                     const bool poppedHeld = (roles & 1u) != 0;
                     roles >>= 1;
                     StageAcc<DT, N> y;
-                    y.pop(stack + sp * levelVecs, tid, all);
+                    y.pop(sp, tid, CT);
                     if (poppedHeld || Commutes<OPR>::value) top.template combine<OPR>(y, top);
                     else top.template combine<OPR>(top, y);
                 }
             }
-#pragma unroll
-            for (int g = 0; g < G; g++) w[g] = wn[g];
         }
+        bool live[N];
+#pragma unroll
+        for (int n = 0; n < N; n++) live[n] = (uint32_t(n) * CT + tid) * 4u < len;
         Vec<4> res[N];
         top.result(res);
         // A segment may begin or end inside a vector: the tile then starts / ends with a vector whose other
@@ -815,7 +912,7 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
         const uint32_t head = (td.len >> 16) & 3u, tail = (td.len >> 18) & 3u, lastVec = len / 4u - 1u;
 #pragma unroll
         for (int n = 0; n < N; n++) {
-            const uint32_t vec = uint32_t(n) * kConsumers + tid;
+            const uint32_t vec = uint32_t(n) * CT + tid;
             if (live[n]) store_part(dst + vec * 4u, res[n], vec == 0u ? head : 0u, vec == lastVec ? tail : 0u);
         }
     }
@@ -968,15 +1065,15 @@ cudaError_t launch_dtop(const TreeLaunch &l)
 }
 
 // Launches the streaming kernel for one parameter type (one job with packed pointers, one job with a
-// pointer table, or a batch) and one number of operand tiles per ring stage.
-template <int DT, int OPR, int G, typename PRM>
+// pointer table, or a batch) and one shape (operand tiles per ring stage, consumer warps).
+template <int DT, int OPR, int G, int CW, typename PRM>
 cudaError_t launch_stream_kernel(const PRM &prm, uint32_t n_ctas, int device, void *stream)
 {
-    auto kernel = rd_tree_stream_kernel<DT, OPR, PRM, G>;
-    const size_t smem = stream_smem_bytes(prm.stages, prm.depth, prm.stage_elems, Wide<DT>::W, G);
+    auto kernel = rd_tree_stream_kernel<DT, OPR, PRM, G, CW>;
+    const size_t smem = stream_smem_bytes(prm.stages, prm.depth, kStageWords, Wide<DT>::W, G);
     if (cudaError_t e = opt_in_shared_memory(reinterpret_cast<const void *>(kernel), device)) return e;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(n_ctas); cfg.blockDim = dim3(kStreamThreads); cfg.dynamicSmemBytes = smem;
+    cfg.gridDim = dim3(n_ctas); cfg.blockDim = dim3(StreamShape<G, CW>::THREADS); cfg.dynamicSmemBytes = smem;
     cfg.stream = static_cast<cudaStream_t>(stream);
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -985,10 +1082,12 @@ cudaError_t launch_stream_kernel(const PRM &prm, uint32_t n_ctas, int device, vo
     return cudaLaunchKernelEx(&cfg, kernel, prm);
 }
 template <int DT, int OPR, typename PRM>
-cudaError_t launch_stream_kernel(const PRM &prm, int ops_per_stage, uint32_t n_ctas, int device, void *stream)
+cudaError_t launch_stream_kernel(const PRM &prm, int ops_per_stage, int consumer_warps, uint32_t n_ctas, int device, void *stream)
 {
-    return ops_per_stage == 2 ? launch_stream_kernel<DT, OPR, 2>(prm, n_ctas, device, stream)
-                              : launch_stream_kernel<DT, OPR, 1>(prm, n_ctas, device, stream);
+    if (ops_per_stage == 2 && consumer_warps == 4) return launch_stream_kernel<DT, OPR, 2, 4>(prm, n_ctas, device, stream);
+    if (ops_per_stage == 1 && consumer_warps == 4) return launch_stream_kernel<DT, OPR, 1, 4>(prm, n_ctas, device, stream);
+    if (ops_per_stage == 1 && consumer_warps == 8) return launch_stream_kernel<DT, OPR, 1, 8>(prm, n_ctas, device, stream);
+    return cudaErrorInvalidValue;
 }
 
 template <int DT, int OPR, bool PACKED>
@@ -1003,8 +1102,8 @@ cudaError_t launch_stream(const TreeLaunch &l)
     prm.t.out = static_cast<uint32_t *>(l.out);
     prm.t.tiles = l.tiles; prm.t.ops = l.ops; prm.t.n_tiles = l.n_tiles; prm.t.p = l.p;
     prm.cta_first = l.cta_first; prm.status = l.status; prm.tile_counter = l.tile_counter;
-    prm.stages = l.stages; prm.depth = l.stack_depth > 0 ? l.stack_depth : 1; prm.stage_elems = l.stage_elems;
-    return launch_stream_kernel<DT, OPR>(prm, l.ops_per_stage, l.n_ctas, l.device, l.stream);
+    prm.stages = l.stages; prm.depth = l.shared_depth > 0 ? l.shared_depth : 1;
+    return launch_stream_kernel<DT, OPR>(prm, l.ops_per_stage, l.consumer_warps, l.n_ctas, l.device, l.stream);
 }
 
 template <int DT, int OPR>
@@ -1018,13 +1117,13 @@ cudaError_t launch_stream_batch(const BatchLaunch &b)
         for (uint32_t i = 0; i < uint32_t(kBatchPackPtrs); i++)
             prm.ptrs[i] = i < b.n_ptrs ? static_cast<const uint32_t *>(b.host_ptrs[i]) : nullptr;
         prm.n_jobs = b.n_jobs; prm.n_tiles = b.n_tiles; prm.status = b.status; prm.tile_counter = b.tile_counter;
-        prm.stages = b.stages; prm.depth = depth; prm.stage_elems = b.stage_elems;
-        return launch_stream_kernel<DT, OPR>(prm, b.ops_per_stage, b.n_ctas, b.device, b.stream);
+        prm.stages = b.stages; prm.depth = depth;
+        return launch_stream_kernel<DT, OPR>(prm, b.ops_per_stage, b.consumer_warps, b.n_ctas, b.device, b.stream);
     }
     BatchStreamParams<false> prm;
     prm.jobs = b.jobs; prm.n_jobs = b.n_jobs; prm.n_tiles = b.n_tiles; prm.status = b.status; prm.tile_counter = b.tile_counter;
-    prm.stages = b.stages; prm.depth = depth; prm.stage_elems = b.stage_elems;
-    return launch_stream_kernel<DT, OPR>(prm, b.ops_per_stage, b.n_ctas, b.device, b.stream);
+    prm.stages = b.stages; prm.depth = depth;
+    return launch_stream_kernel<DT, OPR>(prm, b.ops_per_stage, b.consumer_warps, b.n_ctas, b.device, b.stream);
 }
 
 template <int DT, int OPR>
@@ -1063,6 +1162,9 @@ cudaError_t launch_direct_dtop(const TreeLaunch &l)
 // Calls f.template operator()<DT, OPR>() for the run-time operation.
 template <int DT, typename F> cudaError_t with_op(int op, F &&f)
 {
+    if constexpr (DT == DT_BF16_PICK || DT == DT_FP16_PICK) {        // these serve max and min only
+        return op == OPR_MAX ? f.template operator()<DT, OPR_MAX>() : op == OPR_MIN ? f.template operator()<DT, OPR_MIN>() : cudaErrorInvalidValue;
+    }
     switch (op) {
     case OPR_SUM: return f.template operator()<DT, OPR_SUM>();
     case OPR_MAX: return f.template operator()<DT, OPR_MAX>();
@@ -1082,7 +1184,7 @@ struct DirectLauncher {
     const TreeLaunch &l;
     template <int DT, int OPR> cudaError_t operator()() const
     {
-        if constexpr (Wide<DT>::half) return cudaErrorInvalidValue;     // 16-bit types go through the streaming kernel
+        if constexpr (DT >= DT_BF16) return cudaErrorInvalidValue;       // 16-bit types go through the streaming kernel
         else return launch_direct_dtop<DT, OPR>(l);
     }
 };
@@ -1112,20 +1214,98 @@ int RD_CAT(launch_for_dtype_, RD_DT)(int which, const void *launch, int op)
 
 #else
 
+// ---------------------------------------------------------------------------------------------
+// Broadcast of the root's result (all-reduce = reduce, then broadcast): every thread reads U vectors of
+// the source and writes them to each of the n_dst destinations.  Bound by HBM writes: m bytes read,
+// n_dst * m written.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kBcastThreads = 256;
+constexpr int kBcastU = 4;               // vectors in flight per thread
+
+struct BcastParams {
+    uint32_t *dst[kBcastPackPtrs];
+    const uint32_t *src;
+    uint64_t n_vec;                      // vectors (of V words) to copy
+    int n_dst;
+};
+
+template <int V>
+__global__ void __launch_bounds__(kBcastThreads, 4)
+rd_broadcast_kernel(const __grid_constant__ BcastParams a)
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");           // the reduction that produced src has finished
+    const uint64_t stride = uint64_t(gridDim.x) * kBcastThreads;
+    for (uint64_t v0 = uint64_t(blockIdx.x) * kBcastThreads + threadIdx.x; v0 < a.n_vec; v0 += stride * kBcastU) {
+        Vec<V> x[kBcastU];
+#pragma unroll
+        for (int u = 0; u < kBcastU; u++) {
+            const uint64_t v = v0 + uint64_t(u) * stride;
+            if (v < a.n_vec) {
+                if constexpr (V == 4) {
+                    const uint4 t = __ldcs(reinterpret_cast<const uint4 *>(a.src) + v);
+                    x[u].w[0] = t.x; x[u].w[1] = t.y; x[u].w[2] = t.z; x[u].w[3] = t.w;
+                } else {
+                    x[u].w[0] = __ldcs(a.src + v);
+                }
+            }
+        }
+        for (int d = 0; d < a.n_dst; d++) {
+#pragma unroll
+            for (int u = 0; u < kBcastU; u++) {
+                const uint64_t v = v0 + uint64_t(u) * stride;
+                if (v < a.n_vec) store_stream<V>(a.dst[d] + v * V, x[u]);
+            }
+        }
+    }
+}
+
+}  // namespace
+
+int launch_broadcast(const void *src, void *const *dsts, int n_dst, uint64_t n_words, bool wide, int sm_count, void *stream)
+{
+    if (n_words == 0) return 0;
+    for (int base = 0; base < n_dst; base += kBcastPackPtrs) {
+        BcastParams prm;
+        const int cnt = n_dst - base < kBcastPackPtrs ? n_dst - base : kBcastPackPtrs;
+        for (int i = 0; i < kBcastPackPtrs; i++) prm.dst[i] = i < cnt ? static_cast<uint32_t *>(dsts[base + i]) : nullptr;
+        prm.src = static_cast<const uint32_t *>(src);
+        prm.n_vec = wide ? n_words / 4 : n_words;
+        prm.n_dst = cnt;
+        const uint64_t perBlock = uint64_t(kBcastThreads) * kBcastU;
+        uint64_t blocks = (prm.n_vec + perBlock - 1) / perBlock;
+        const uint64_t most = uint64_t(sm_count > 0 ? sm_count : 1) * 8u;
+        if (blocks > most) blocks = most;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(unsigned(blocks)); cfg.blockDim = dim3(kBcastThreads); cfg.dynamicSmemBytes = 0;
+        cfg.stream = static_cast<cudaStream_t>(stream);
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        const cudaError_t e = wide ? cudaLaunchKernelEx(&cfg, rd_broadcast_kernel<4>, prm) : cudaLaunchKernelEx(&cfg, rd_broadcast_kernel<1>, prm);
+        if (e != cudaSuccess) return int(e);
+    }
+    return 0;
+}
+
 uint32_t tree_tile_elems(int vec) { return uint32_t(kTreeThreads) * kU * uint32_t(vec); }
 
-// One stack level holds one 128-bit vector per consumer thread and word of partial result, two when an operand
-// tile has more than 1024 words.  (acc_words: words of partial result per message word, 2 for the 16-bit types,
-// whose elements are combined in fp32, else 1; ops_per_stage: operand tiles that share a ring stage.)
+// One stack level holds the partial results of one tile.  (acc_words: words of partial result per message word,
+// 2 for the 16-bit types, whose elements are combined in fp32, else 1; ops_per_stage: operand tiles that share a
+// ring stage, each stage_elems / ops_per_stage words long.)
 static int stack_level_bytes(int stage_elems, int acc_words, int ops_per_stage)
 {
-    return (stage_elems / ops_per_stage > 4 * kConsumers ? 2 : 1) * acc_words * kConsumers * 16;
+    return stage_elems / ops_per_stage * acc_words * 4;
 }
 
 size_t stream_smem_bytes(int stages, int depth, int stage_elems, int acc_words, int ops_per_stage)
 {
+    // ring | stack | two barriers per stage | the operation words of a stage's operands
     return size_t(stages) * size_t(stage_elems) * 4 + size_t(depth) * stack_level_bytes(stage_elems, acc_words, ops_per_stage) +
-           size_t(2 * stages) * sizeof(uint64_t);
+           size_t(2 * stages) * sizeof(uint64_t) + size_t(stages) * size_t(ops_per_stage) * sizeof(uint32_t);
 }
 
 int stream_stage_elems(uint64_t elems_per_cta)
@@ -1133,11 +1313,13 @@ int stream_stage_elems(uint64_t elems_per_cta)
     // Measured on B200: the time per stage hand-over hardly depends on the stage's size up to 8 KB, so smaller
     // stages only lower the throughput, also for small messages.
     (void)elems_per_cta;
-    return kMaxStageElems;
+    return kStageWords;
 }
 
-void stream_shape(int stack_depth, int acc_words, int ops_per_stage, int smem_per_sm, int stage_elems, uint64_t n_tiles, int sm_count,
-                  int *ctas_per_sm, int *stages)
+bool stream_second_accumulator(int acc_words, int ops_per_stage) { return !(acc_words > 1 && ops_per_stage == 1); }
+
+void stream_shape(int stack_depth, int acc_words, int ops_per_stage, bool many_pushes, int smem_per_sm, int stage_elems, uint64_t n_tiles,
+                  int sm_count, int *ctas_per_sm, int *stages)
 {
     const int depth = stack_depth > 0 ? stack_depth : 1;
     const int stageBytes = stage_elems * 4;
@@ -1155,6 +1337,12 @@ void stream_shape(int stack_depth, int acc_words, int ops_per_stage, int smem_pe
     // 3 * 3 against 4 * 2, two are 3 % faster).  Two CTAs take all the stages that fit: a launch of one or
     // two tiles per CTA is over sooner the more of it is in flight from the start.
     const int s3 = fit(3), s2 = fit(2);
+    // The 16-bit types under sum and product (fp32 partial results, two tiles per stage) spend the most issue slots
+    // per byte and gain from a third thread block even when it leaves only three stages each, or two where the
+    // programs push often (binomial-like trees).  Measured, bf16 sum, 64 MiB messages, GB/s: three blocks x 3
+    // stages against two x 6, p = 256 (six levels of stack): uni-greedy 7035 / 6828, binomial 6294 / 5473; three
+    // blocks x 2 stages against two x 6, p = 512 (seven levels): uni-greedy 6318 / 6599, binomial 6005 / 5418.
+    if (acc_words > 1 && sm_count > 0 && (s3 == 3 || (s3 == 2 && many_pushes))) { *ctas_per_sm = 3; *stages = s3; return; }
     if (s3 >= 4 && s2 >= 3 && sm_count > 0) {
         const uint64_t t = n_tiles > 0 ? n_tiles : 1;
         const uint64_t cost3 = (t + 3u * uint64_t(sm_count) - 1) / (3u * uint64_t(sm_count)) * 3u;
@@ -1175,16 +1363,21 @@ int launch_for_dtype_2(int which, const void *launch, int op);
 int launch_for_dtype_3(int which, const void *launch, int op);
 int launch_for_dtype_4(int which, const void *launch, int op);
 int launch_for_dtype_5(int which, const void *launch, int op);
+int launch_for_dtype_6(int which, const void *launch, int op);
+int launch_for_dtype_7(int which, const void *launch, int op);
 
 static int launch_for(int dtype, int which, const void *launch, int op)
 {
+    if ((dtype == DT_BF16 || dtype == DT_FP16) && (op == OPR_MAX || op == OPR_MIN)) dtype += DT_BF16_PICK - DT_BF16;
     switch (dtype) {
     case DT_INT32: return launch_for_dtype_0(which, launch, op);
     case DT_FP32: return launch_for_dtype_1(which, launch, op);
     case DT_INT64: return launch_for_dtype_2(which, launch, op);
     case DT_FP64: return launch_for_dtype_3(which, launch, op);
     case DT_BF16: return launch_for_dtype_4(which, launch, op);
-    default: return launch_for_dtype_5(which, launch, op);
+    case DT_FP16: return launch_for_dtype_5(which, launch, op);
+    case DT_BF16_PICK: return launch_for_dtype_6(which, launch, op);
+    default: return launch_for_dtype_7(which, launch, op);
     }
 }
 

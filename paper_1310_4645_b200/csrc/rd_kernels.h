@@ -25,7 +25,8 @@ struct TreeLaunch {
     const uint32_t *ops;              // device
     uint32_t n_tiles;
     int p;
-    int stack_depth;
+    int stack_depth;                  // partial results a program keeps besides the running one
+    int shared_depth;                 // levels the streaming kernel's shared-memory stack needs in this launch
     int dtype, op;                    // rd_dtype_t, rd_op_t
     int vec;                          // 4: 128-bit path, 1: element path
     int sm_count;
@@ -37,6 +38,7 @@ struct TreeLaunch {
     int stages;
     int stage_elems;
     int ops_per_stage;                // operand tiles that share a ring stage (1 or 2); tiles hold stage_elems / ops_per_stage words
+    int consumer_warps;               // 8, 4 or 2 (two tiles per stage: 4 or 2)
     int *status;                      // device word
     uint32_t *tile_counter;           // device: two words, both 0, for handing tiles out on demand; null: fixed ranges
 };
@@ -61,7 +63,7 @@ struct BatchLaunch {
     const BatchJob *jobs;             // device, n_jobs entries (when host_jobs is null)
     uint32_t n_jobs, n_tiles;
     uint32_t n_ctas;
-    int stages, stack_depth, stage_elems, ops_per_stage;
+    int stages, stack_depth, stage_elems, ops_per_stage, consumer_warps;   // stack_depth: levels in shared memory
     int dtype, op, device;
     int *status;                      // device word
     uint32_t *tile_counter;           // as in TreeLaunch
@@ -76,8 +78,12 @@ int launch_tree(const TreeLaunch &a);
 // Streaming variant (128-bit path): stage size for a CTA's share of the message, ring shape for a
 // stack depth and the SM's shared memory, launch.
 int stream_stage_elems(uint64_t elems_per_cta);
-void stream_shape(int stack_depth, int acc_words, int ops_per_stage, int smem_per_sm, int stage_elems, uint64_t n_tiles, int sm_count,
-                  int *ctas_per_sm, int *stages);
+// many_pushes: the programs push a partial result on the shared-memory stack for at least every tenth operand.
+void stream_shape(int stack_depth, int acc_words, int ops_per_stage, bool many_pushes, int smem_per_sm, int stage_elems, uint64_t n_tiles,
+                  int sm_count, int *ctas_per_sm, int *stages);
+// Whether the streaming kernel of this shape runs the marked sub-expressions of a program in a second accumulator
+// (its shared-memory stack then needs Programs::shared_depth levels, else Programs::stack_depth).
+bool stream_second_accumulator(int acc_words, int ops_per_stage);
 size_t stream_smem_bytes(int stages, int depth, int stage_elems, int acc_words, int ops_per_stage);
 int launch_tree_stream(const TreeLaunch &a);
 // Direct variant (128-bit path, at most kDirectMaxProcs processes): all operands of a thread's elements
@@ -86,6 +92,11 @@ constexpr int kDirectMaxProcs = 8;
 bool direct_applies(int p, int stack_depth);
 int direct_blocks_per_sm(int p);
 int launch_tree_direct(const TreeLaunch &a);
+
+// Broadcast (all-reduce = reduce + broadcast): copies n_words 32-bit words from src to each of the n_dst
+// destinations (device pointers in a host array); wide: all buffers 16-byte aligned and n_words a multiple of 4.
+constexpr int kBcastPackPtrs = 256;   // destinations per launch (they travel as kernel parameters)
+int launch_broadcast(const void *src, void *const *dsts, int n_dst, uint64_t n_words, bool wide, int sm_count, void *stream);
 
 // ---- schedule-faithful execution (rd_faithful.cu)
 constexpr int kFaithfulThreads = 128;

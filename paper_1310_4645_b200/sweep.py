@@ -9,6 +9,8 @@ under the linear model, measured microseconds and GB/s ((p+1)*m bytes per reduct
 result passed its check (integers, max and min: exact against torch's order-free result; fp32 sum:
 |r - r64| <= 1e-5 * sum|x| against an fp64 sum, fp64 sum: the same with 1e-14, bf16 sum: the fp32 bound plus
 one rounding, 2^-8 |r64|; on the whole message or on sampled slices of it).
+These checks are order free and run on every one of the thousands of cases; the bit-for-bit comparison with the CPU
+checker at these same tuned segment sizes is made by the test suite on a thinned grid of the cells.
 Inputs: uniform random numbers from seed 4 (integers in [-2^20, 2^20], floating point in [-1, 1)), one
 arena per element type (--dtypes), every case a view of its first p*n elements.
 """

@@ -37,9 +37,11 @@ def oracle_schedule(algo, port, p, msg_bytes, seg_bytes, alpha, beta, gamma, siz
     return np.sort(ev, order=ORDER), off, comp
 
 
-def run_program(ops, x, op):
+def run_program(ops, x, op, use_hints=True, depth_out=None):
     """Reference interpreter of one compiled combine program (format documented in include/rd.h).
-    x: [p, len] array; returns the root's value.  Written from the header's description only."""
+    x: [p, len] array; returns the root's value.  Written from the header's description only.
+    use_hints: honour bits 30 / 31 (sub-expressions that need no stack run in a second accumulator);
+    depth_out: a list that receives the deepest the stack got."""
     x = np.asarray(x)
 
     def combine(held, incoming):
@@ -55,26 +57,46 @@ def run_program(ops, x, op):
             return np.where(incoming < held, incoming, held)
         return np.where(incoming > held, incoming, held)
 
-    stack, top = [], None
-    loads = 0
+    stack, top, second = [], None, None
+    loads = deepest = 0
     for w in ops:
         w = int(w)
-        proc, kind, npop, roles = w & 0xFFF, (w >> 12) & 3, (w >> 14) & 0xF, w >> 18
+        proc, kind, npop, roles = w & 0xFFF, (w >> 12) & 3, (w >> 14) & 0xF, (w >> 18) & 0xFFF
+        aside, last = (w >> 30) & 1, (w >> 31) & 1
         v = x[proc]
         loads += 1
-        if kind == 0:
-            top = v.copy()
-        elif kind == 1:
-            stack.append(top)
-            top = v.copy()
-        elif kind == 2:
-            top = combine(top, v)
+        assert not last or (aside and npop >= 1)
+        first_pop = 0
+        if aside and use_hints:
+            # a sub-expression that needs no stack, evaluated in a second accumulator
+            if kind == 1:
+                assert second is None
+                second = v.copy()
+            else:
+                assert kind in (2, 3) and second is not None
+                second = combine(second, v) if kind == 2 else combine(v, second)
+            assert npop == 0 or last                         # nothing is popped inside it
+            if last:
+                top = combine(top, second) if roles & 1 else combine(second, top)
+                second, first_pop = None, 1
         else:
-            top = combine(v, top)
-        for k in range(npop):
+            assert second is None or not use_hints           # nothing else happens while one is under way
+            if kind == 0:
+                top = v.copy()
+            elif kind == 1:
+                stack.append(top)
+                deepest = max(deepest, len(stack))
+                top = v.copy()
+            elif kind == 2:
+                top = combine(top, v)
+            else:
+                top = combine(v, top)
+        for k in range(first_pop, npop):
             y = stack.pop()
             top = combine(y, top) if (roles >> k) & 1 else combine(top, y)
-    assert not stack and loads == x.shape[0]
+    assert not stack and second is None and loads == x.shape[0]
+    if depth_out is not None:
+        depth_out.append(deepest)
     return top
 
 

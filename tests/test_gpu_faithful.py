@@ -144,6 +144,27 @@ def test_calibration_tool_fits_positive_parameters(capsys):
     assert set(d["schedules"]) == {"uni_greedy", "binomial", "pipeline", "binary"}
     assert d["rank_by_model"][0] == "uni_greedy"          # Theorem 5: optimal among in-order one-port schedules
     assert all(v["measured_us"] > 0 for v in d["schedules"].values())
+    # the second fit separates the combine from the hand-off (one-port against two-port pipeline periods)
+    two = d.get("two_port_fit")
+    if two is not None:
+        assert two["alpha_s"] > 0 and two["beta_s_per_byte"] >= 0 and two["gamma_s_per_byte"] >= 0
+        assert two["beta_s_per_byte"] + two["gamma_s_per_byte"] > 0
+        assert two["rank_by_model"][0] == "uni_greedy"
+
+
+def test_tuning_tool_runs_every_schedule_at_every_power_of_two_segment(tmp_path, capsys):
+    """Section VII's procedure on a small case: every schedule, every segment size 2^i, best of a few runs."""
+    import json
+    from paper_1310_4645_b200 import tune
+    out = tmp_path / "tune.jsonl"
+    assert tune.main(["--p", "8", "--min-log2-bytes", "16", "--max-log2-bytes", "17", "--reps", "2", "--out", str(out)]) == 0
+    rows = [json.loads(ln) for ln in out.read_text().splitlines() if ln.strip()]
+    sized = [r for r in rows if "msg_bytes" in r]
+    assert {r["msg_bytes"] for r in sized} == {1 << 16, 1 << 17}
+    for r in sized:
+        assert set(r["schedules"]) == {"uni_greedy", "bi_greedy", "pipeline", "binary", "binomial", "butterfly"}
+        for v in r["schedules"].values():
+            assert v["best_us"] > 0
 
 
 def test_randomized_shapes_order_free_results():

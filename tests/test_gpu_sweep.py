@@ -5,8 +5,10 @@ A thinned grid of the sweep: p in {2, 16, 128, 1024} x message in {8 B, 4 KiB, 1
 schedules x {int32, fp32} x {sum, max}.  The library is asked for `seg_bytes = 0`, i.e. the segment size
 rd_optimal_segment returns for the schedule; the oracle's own simulator then builds the schedule for that
 segment size and its evaluator gives the expected bytes.  Where p * m is at most 256 MiB the whole message is
-compared; above that, at least eight whole segments (the first two, the last three -- the last one is the
-ragged one whenever the segment size does not divide the message -- and three in between) are.
+compared; above that, at least eight segments (the first two, the last three -- the last one is the
+ragged one whenever the segment size does not divide the message -- and three in between) are: whole when
+the segment's p operands fit in 64 MiB, else on its first, middle and last 16 MiB / 4p elements (the oracle
+replays the segment's events on those element ranges; elements do not depend on each other).
 Inputs: uniform random numbers from seed 4 (integers in [-2^20, 2^20], floats in [-1, 1)), as in the sweep.
 """
 import numpy as np
@@ -23,6 +25,8 @@ pytestmark = pytest.mark.gpu
 MODEL = (ALPHA, BETA, GAMMA)
 OPS = {"sum": rd.RD_SUM, "max": rd.RD_MAX}
 WHOLE_LIMIT = 256 << 20
+SEGMENT_LIMIT = 64 << 20          # a picked segment is checked whole when its p operands are at most this many bytes
+SLICE_BYTES = 16 << 20            # ... else on three slices of this many operand bytes each
 
 
 def picked_segments(q):
@@ -58,8 +62,15 @@ def run_case(p, m, x, out, name, algo, port, ops):
                 lo, hi = int(off[j]), int(off[j + 1])
                 sel = ev[ev["seg"] == j].copy()
                 sel["seg"] = 0
-                want = O.reduce(sel, x[:, lo:hi].cpu().numpy(), [0, hi - lo], opname)
-                assert out[lo:hi].cpu().numpy().tobytes() == want.tobytes(), (name, p, m, seg, opname, j)
+                if (hi - lo) * p * 4 <= SEGMENT_LIMIT:
+                    spans = [(lo, hi)]
+                else:
+                    w = max(4, SLICE_BYTES // (4 * p))
+                    mid = lo + (hi - lo - w) // 2
+                    spans = [(lo, lo + w), (mid, mid + w), (hi - w, hi)]
+                for a, b in spans:
+                    want = O.reduce(sel, x[:, a:b].cpu().numpy(), [0, b - a], opname)
+                    assert out[a:b].cpu().numpy().tobytes() == want.tobytes(), (name, p, m, seg, opname, j, a)
             # and order free over the whole message: the maximum is the maximum
             if opname == "max":
                 assert torch.equal(out, x.amax(dim=0))

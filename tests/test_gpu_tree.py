@@ -406,57 +406,109 @@ def test_unequal_segmentation_end_to_end(mode):
             assert out.cpu().numpy().tobytes() == want.tobytes(), (parts, algo)
 
 
-def _sampled_parity(wname, schedules, ops, n_samples=5):
-    """Full-size workload in the launch configuration the benchmark uses; the oracle checks whole sampled
-    segments bit for bit and slabs of the message against the fp64 reference."""
+def _device_fp64_bound(x, out):
+    """|r - r64| <= 1e-5 * sum_i |x_i| on EVERY element, the fp64 sums taken on the device slab by slab; returns
+    the largest error relative to the largest |r64| as well."""
+    n = out.numel()
+    slab = max(1 << 16, (1 << 27) // x.shape[0])          # 1 GiB of fp64 operands at a time
+    worst, biggest = 0.0, 0.0
+    for lo in range(0, n, slab):
+        xs = x[:, lo:lo + slab].double()
+        ref, mag = xs.sum(dim=0), xs.abs().sum(dim=0)
+        err = (out[lo:lo + slab].double() - ref).abs()
+        assert bool((err <= 1e-5 * mag).all()), lo
+        worst, biggest = max(worst, float(err.max())), max(biggest, float(ref.abs().max()))
+    assert worst / biggest <= 1e-5
+    return worst / biggest
+
+
+def _full_size_parity(wname, schedules, ops, n_samples=16, whole_message_for=()):
+    """A full-size workload in the launch configuration the benchmark uses (one rd_reduce call per schedule and
+    operation on the resident arena).  What is compared, and on which fraction of the output elements:
+      * bit for bit against the oracle -- its own simulator's schedule, its evaluator -- on n_samples whole
+        segments per schedule and operation (the first two, the last four, which are the tiles handed out last,
+        and others spread evenly): n_samples / q of the elements; for the schedules in `whole_message_for`
+        on every element (fraction 1.0);
+      * `max`: equal to the order-free maximum taken on the device, on every element (fraction 1.0);
+      * `sum`: within 1e-5 * sum|x_i| of the fp64 sum taken on the device, on every element (fraction 1.0).
+    Returns the fractions so that the callers can state them."""
     w = WORKLOADS[wname]
     model = (w["alpha"], w["beta"], w["gamma"])
     p, n = w["p"], w["n"]
     x = make_inputs(p, n, w["dist"], w["seed"], device="cuda")
     tab = rd.PointerTable(x)
     out = torch.empty(n, device="cuda")
+    want_max = x.amax(dim=0) if "max" in ops else None
+    fractions = {}
     for algo, port in schedules:
         h = rd.rd_schedule_create(algo, port, p, 4 * n, w["seg_bytes"], *model)
-        ev = rd.rd_schedule_events(h)
-        off = rd.rd_schedule_segments(h).astype(np.int64)
-        oev = np.zeros(len(ev), dtype=O.EVENT_DTYPE)
-        for f in ("t_start", "seg", "src", "dst", "kind"):
-            oev[f] = ev[f]                       # identical to the oracle's own list (tests/test_scheduler_vs_oracle.py)
+        oev, off, comp = oracle_schedule(algo, port, p, 4 * n, w["seg_bytes"], *model)     # the oracle's own events
+        assert rd.rd_schedule_info(h)["predicted_ticks"] == comp
+        assert (rd.rd_schedule_segments(h).astype(np.int64) == off).all()
         q = len(off) - 1
-        picks = sorted({0, 1, q // 3, q // 2, q - 2, q - 1})[:n_samples + 1]
+        picks = {0, 1, q - 4, q - 3, q - 2, q - 1} & set(range(q))
+        for j in np.linspace(2, q - 5, max(n_samples - 6, 0) * 2).astype(int):     # others, spread evenly
+            if len(picks) < min(n_samples, q) and 0 <= j < q:
+                picks.add(int(j))
+        picks = sorted(picks)
+        assert len(picks) >= min(n_samples, q)
+        xh = x.cpu().numpy() if algo in whole_message_for else None
         for op in ops:
+            out.fill_(7.0)
             rd.rd_reduce(h, tab, out, OPS[op])
             torch.cuda.synchronize()
-            for j in picks:
-                lo, hi = int(off[j]), int(off[j + 1])
-                if hi == lo:
-                    continue
-                xs = x[:, lo:hi].cpu().numpy()
-                sel = oev[oev["seg"] == j].copy()
-                sel["seg"] = 0
-                want = O.reduce(sel, xs, [0, hi - lo], op)
-                got = out[lo:hi].cpu().numpy()
-                assert got.tobytes() == want.tobytes(), (wname, algo, op, j)
-                if op == "sum":
-                    ref, mag = O.reference_f64(xs, "sum")
-                    assert (np.abs(got.astype(np.float64) - ref) <= 1e-5 * mag).all()
+            covered = 0
+            if xh is not None:
+                want = O.reduce(oev, xh, off, op)
+                assert out.cpu().numpy().tobytes() == want.tobytes(), (wname, algo, op)
+                covered = n
+            else:
+                for j in picks:
+                    lo, hi = int(off[j]), int(off[j + 1])
+                    if hi == lo:
+                        continue
+                    sel = oev[oev["seg"] == j].copy()
+                    sel["seg"] = 0
+                    want = O.reduce(sel, x[:, lo:hi].cpu().numpy(), [0, hi - lo], op)
+                    assert out[lo:hi].cpu().numpy().tobytes() == want.tobytes(), (wname, algo, op, j)
+                    covered += hi - lo
+            fractions[(algo, op, "oracle")] = covered / n
+            if op == "max":
+                assert torch.equal(out, want_max), (wname, algo)
+                fractions[(algo, op, "order_free")] = 1.0
+            if op == "sum":
+                _device_fp64_bound(x, out)
+                fractions[(algo, op, "fp64_bound")] = 1.0
+        del xh
         rd.rd_destroy(h)
+    return fractions
 
 
-def test_config3_full_size_sampled():
-    """p = 256, n = 2^22 fp32 uniform [-1, 1), 64 KiB segments, two ports: bi-greedy, butterfly and the trees."""
-    _sampled_parity("config3", [(rd.RD_BI_GREEDY, rd.RD_PORT_BI), (rd.RD_BUTTERFLY, rd.RD_PORT_BI),
-                                (rd.RD_BINOMIAL, rd.RD_PORT_BI), (rd.RD_PIPELINE, rd.RD_PORT_BI),
-                                (rd.RD_BINARY, rd.RD_PORT_BI)], ["sum"], n_samples=3)
+def test_config3_full_size():
+    """p = 256, n = 2^22 fp32 uniform [-1, 1), 64 KiB segments, two ports: bi-greedy, butterfly and the trees.
+    bi-greedy is evaluated by the oracle end to end (every element, 4 GiB of inputs on the host); the other
+    four schedules on 16 of their 256 segments (butterfly: of its 256 chunks); the fp64 bound on every element
+    for all five."""
+    fr = _full_size_parity("config3", [(rd.RD_BI_GREEDY, rd.RD_PORT_BI), (rd.RD_BUTTERFLY, rd.RD_PORT_BI),
+                                        (rd.RD_BINOMIAL, rd.RD_PORT_BI), (rd.RD_PIPELINE, rd.RD_PORT_BI),
+                                        (rd.RD_BINARY, rd.RD_PORT_BI)], ["sum"], n_samples=16,
+                            whole_message_for=(rd.RD_BI_GREEDY,))
+    assert fr[(rd.RD_BI_GREEDY, "sum", "oracle")] == 1.0
+    assert all(v >= 16 / 256 for k, v in fr.items() if k[2] == "oracle")
+    assert all(v == 1.0 for k, v in fr.items() if k[2] != "oracle")
 
 
-def test_config4_full_size_sampled():
-    """p = 32, n = 2^28 fp32 N(0,1) (32 GiB), 1 MiB segments: uni- and bi-greedy, sum and max."""
+def test_config4_full_size():
+    """p = 32, n = 2^28 fp32 N(0,1) (32 GiB), 1 MiB segments: uni- and bi-greedy, sum and max.  The oracle sees
+    16 of the 1024 segments per schedule and operation (1/64 of the elements, among them the last four);
+    the maximum and the fp64 bound are checked on every element."""
     free_b, _ = torch.cuda.mem_get_info()
-    if free_b < (40 << 30):
-        pytest.skip("needs 33 GiB of device memory")
-    _sampled_parity("config4", [(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI), (rd.RD_BI_GREEDY, rd.RD_PORT_BI)], ["sum", "max"],
-                    n_samples=3)
+    if free_b < (48 << 30):
+        pytest.skip("needs 40 GiB of device memory")
+    fr = _full_size_parity("config4", [(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI), (rd.RD_BI_GREEDY, rd.RD_PORT_BI)], ["sum", "max"],
+                            n_samples=16)
+    assert all(v >= 16 / 1024 for k, v in fr.items() if k[2] == "oracle")
+    assert all(v == 1.0 for k, v in fr.items() if k[2] != "oracle")
 
 
 def test_tree_mode_launches_can_be_replayed_from_a_cuda_graph():
@@ -855,6 +907,34 @@ def test_bf16_parity_with_one_operand_tile_per_stage(name, algo, port, dtype):
         x = bf16_inputs(p, n, "normal", seed=p * 1000 + n, dtype=dtype)
         for op in ("sum", "max"):
             check_bf16(algo, port, x, 2 * seg, op, variant=rd.RD_TREE_STREAM)
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
+def test_sixteen_bit_extrema_of_zeros_subnormals_and_infinities(dtype):
+    """max and min of 16-bit elements are taken on the packed 16-bit values themselves; the oracle widens to fp32,
+    compares there and rounds at the end.  Same bits, also where it is delicate: +0 against -0 (the held value
+    survives a tie, so the order of the schedule decides the sign), subnormals (never flushed), infinities, and
+    neighbouring values that differ in the last bit."""
+    info = torch.finfo(dtype)
+    tiny_sub = 2.0 ** (-133 if dtype == torch.bfloat16 else -24)                   # the smallest subnormal
+    palette = torch.tensor([0.0, -0.0, tiny_sub, -tiny_sub, 3 * tiny_sub, -3 * tiny_sub, info.tiny, -info.tiny,
+                            info.tiny * (1 - info.eps), 1.0, 1.0 + info.eps, -1.0, -1.0 - info.eps, info.max, -info.max,
+                            float("inf"), float("-inf"), 0.5, -0.5], dtype=torch.float64).to(dtype).cuda()
+    assert (palette[2].float() > 0) and (palette[2].float() < info.tiny)            # really a subnormal of the type
+    g = torch.Generator("cuda").manual_seed(11)
+    for p, n, seg in [(8, 8192, 1024), (13, 3 * 4096 + 72, 4096 + 1040), (64, 16384, 2048), (5, 14, 4), (200, 4096, 4096)]:
+        idx = torch.randint(0, len(palette), (p, n), device="cuda", generator=g)
+        idx[:, : n // 4] = torch.randint(0, 2, (p, n // 4), device="cuda", generator=g)       # a stretch of nothing but +0 and -0
+        x = palette[idx]
+        for name, algo, port in SCHEDULES:
+            for op in ("max", "min"):
+                out = check_bf16(algo, port, x, 2 * seg, op)
+                assert torch.equal(out.float(), (x.float().amax(dim=0) if op == "max" else x.float().amin(dim=0)))  # as numbers
+        rows = [x[i, 2:] for i in range(p)]                                        # 4 bytes off a vector: the element kernel
+        if n > 16:
+            check_bf16(rd.RD_BI_GREEDY, rd.RD_PORT_BI, x[:, 2:].contiguous(), 2 * 1000, "max")
+            big_out = torch.zeros(n, dtype=dtype, device="cuda")
+            check_bf16(rd.RD_BI_GREEDY, rd.RD_PORT_BI, x[:, 2:], 2 * 1000, "max", rows=rows, out=big_out[2:])
 
 
 def test_bf16_partial_results_stay_in_fp32_and_ties_round_to_even():

@@ -40,7 +40,12 @@ def test_programs_reproduce_the_oracle(algo, port, p):
                 for j in range(info["q"]):
                     ops = rd.rd_schedule_program(h, j)
                     assert sorted(int(w) & 0xFFF for w in ops) == list(range(p))     # every process exactly once
-                    got[off[j]:off[j + 1]] = run_program(ops, x[:, off[j]:off[j + 1]], op)
+                    depth, depth_plain = [], []
+                    got[off[j]:off[j + 1]] = run_program(ops, x[:, off[j]:off[j + 1]], op, depth_out=depth)
+                    # bits 30 / 31 are hints: one plain stack gives the same bits, one level deeper at most
+                    plain = run_program(ops, x[:, off[j]:off[j + 1]], op, use_hints=False, depth_out=depth_plain)
+                    assert plain.tobytes() == got[off[j]:off[j + 1]].tobytes()
+                    assert depth_plain[0] <= info["stack_depth"] and depth[0] <= max(depth_plain[0] - 1, 0)
                 assert got.tobytes() == want.tobytes(), (op, x.dtype)
     finally:
         rd.rd_destroy(h)
