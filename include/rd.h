@@ -92,7 +92,8 @@ typedef enum { RD_SUM = 0, RD_MAX = 1, RD_MIN = 2, RD_PROD = 3 } rd_op_t;
  * accumulation"; the paper fixes nothing here).  Every input is widened exactly, partial results are fp32
  * values combined by one IEEE fp32 operation per combine in the schedule's order, and only what the root
  * holds at the end is rounded to 16 bits, once, to nearest with ties to even (fp16: overflow to infinity,
- * gradual underflow).  n_elems counts 16-bit elements (msg_bytes / 2, always even); buffers must be aligned
+ * gradual underflow).  (Max and min select one of their operands, so the kernels take them on the 16-bit values
+ * directly; the bits are the same.)  n_elems counts 16-bit elements (msg_bytes / 2, always even); buffers must be aligned
  * to 4 bytes.  Tree mode only: the schedule-faithful execution would have to hand fp32 partial segments
  * between processes and returns RD_ERR_UNSUPPORTED. */
 typedef enum { RD_INT32 = 0, RD_FP32 = 1, RD_INT64 = 2, RD_FP64 = 3, RD_BF16 = 4, RD_FP16 = 5 } rd_dtype_t;
@@ -329,7 +330,8 @@ RD_API int rd_schedule_set_wait_budget(rd_schedule_t *s, double seconds);
  *   RD_TREE_STREAM_PAIRED  the streaming kernel on tiles of half the length (1024 words), a ring stage
  *                   holding the tiles of two consecutive operands: the partial results that wait in the
  *                   stack take half the shared memory per tile, the bytes per stage hand-over stay the same.
- *                   What RD_TREE_AUTO picks for the 16-bit element types, whose partial results are fp32.
+ *                   What RD_TREE_AUTO picks for sums and products of the 16-bit element types (whose partial
+ *                   results are fp32) when the programs keep two or more partial results waiting.
  */
 typedef enum { RD_TREE_AUTO = 0, RD_TREE_STREAM = 1, RD_TREE_DIRECT = 2, RD_TREE_STREAM_PAIRED = 3 } rd_tree_variant_t;
 RD_API int rd_schedule_set_tree_variant(rd_schedule_t *s, rd_tree_variant_t variant);

@@ -7,6 +7,7 @@
 //   rd_tree_stream_kernel  the throughput path (128-bit aligned buffers): operand tiles are streamed
 //                          into a shared-memory ring by bulk asynchronous copies issued by producer
 //                          threads, consumers execute the program on them;
+//   rd_tree_direct_kernel  few processes, on request: all operands of an element in registers at once;
 //   rd_tree_kernel         the element path (buffers aligned to the element only): operands are fetched K
 //                          operations ahead, in program order, into a register ring that is
 //                          statically indexed by unrolling the interpreter K times.
@@ -317,11 +318,11 @@ rd_tree_kernel(const __grid_constant__ TreeParams<PACKED> a)
 // Streaming variant (128-bit path).  Two producer threads per CTA (one per producer warp) walk the
 // CTA's (tile, operation) pairs in program order and issue one bulk asynchronous copy
 // (cp.async.bulk, global -> shared, completion counted in bytes on an mbarrier) per operand tile
-// into a ring of shared-memory stages; they run ahead across tile boundaries, so the number of
-// bytes in flight per SM is set by the ring, not by registers or scoreboards.  256 consumer
-// threads take the stages in the same order, each reading its (up to) two 128-bit vectors of the
-// stage, and execute the program on them.  The stage size is a launch parameter (up to 2048
-// elements).
+// into a ring of 8 KB shared-memory stages; they run ahead across tile boundaries, so the number of
+// bytes in flight per SM is set by the ring, not by registers or scoreboards.  The consumer warps
+// (8 or 4) take the stages in the same order, each thread reading its vectors of the stage, and
+// execute the program on them.  A stage holds one operand tile of up to 2048 words, or two of up to
+// 1024 (see StreamShape).
 // Every wait is bounded: on expiry the thread records an error code and the CTA winds down (a
 // producer lane first waits, again bounded, for the copy it has in flight).
 // ---------------------------------------------------------------------------------------------
@@ -333,26 +334,7 @@ constexpr long long kWaitCycles = 4000000000ll;         // a wait gives up after
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p) { return uint32_t(__cvta_generic_to_shared(p)); }
 
-__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-// The same on a barrier given by its shared-memory address.  The last operand is a hint: the thread may stay
+// Waits on a barrier given by its shared-memory address.  The last operand is a hint: the thread may stay
 // suspended in hardware up to that many nanoseconds while the phase is not complete (it resumes when it is), so
 // a waiting thread spends few issue slots.
 __device__ __forceinline__ bool mbar_try_wait_at(uint32_t bar, uint32_t parity)
@@ -717,11 +699,13 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    // Programmatic dependent launch: the next launch on the stream may begin its own set-up (barriers, table
-    // look-ups above) while this grid is still running; before it touches message data it waits here for
-    // the grid before it to have finished completely.
+    // Programmatic dependent launch: the next launch on the stream may begin while this grid is still running,
+    // as soon as an SM has room for one of its thread blocks.  What does not depend on the grid before (barriers,
+    // the tile counter, tile descriptors, operation words, source addresses: tables the host wrote) is done
+    // right away; each thread waits for the grid before it to have finished completely just before its first
+    // access to message data: the producers before their first copy, the consumers before their first store.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    bool waited = false;
 
     if (tid >= CT) {
         // ------------------------------------------------------------------ producers
@@ -773,6 +757,7 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
             if (laps >= 1u && !mbar_wait_at(empty + uint32_t(stage) * 8u, (laps - 1u) & 1u, &abort_flag)) { ok = false; break; }
             const uint32_t bytes = (td.len & kLenMask) * 4u;
             const uint32_t bar = full + uint32_t(stage) * 8u;
+            if (!waited) { asm volatile("griddepcontrol.wait;" ::: "memory"); waited = true; }
 #pragma unroll
             for (int g = 0; g < G; g++)
                 asm volatile("st.shared.u32 [%0], %1;" ::"r"(stepWords + uint32_t(stage * G + g) * 4u), "r"(wv[g]) : "memory");
@@ -910,6 +895,7 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
         // elements belong to the neighbouring segment (another tile writes those); only this tile's are stored.
         uint32_t *dst = jobs.out() + td.elem_off;
         const uint32_t head = (td.len >> 16) & 3u, tail = (td.len >> 18) & 3u, lastVec = len / 4u - 1u;
+        if (!waited) { asm volatile("griddepcontrol.wait;" ::: "memory"); waited = true; }
 #pragma unroll
         for (int n = 0; n < N; n++) {
             const uint32_t vec = uint32_t(n) * CT + tid;
