@@ -841,6 +841,13 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
                     side.template combine<OPR>(side, x);
                     continue;
                 }
+                if (!Commutes<OPR>::value && (ctl == 3u || (AUX && ctl == (3u | kSecondBit)))) {
+                    StageAcc<DT, N> x;                                // max, min: the operand is the held value, nothing popped
+                    x.load(r[g]);
+                    if (ctl == 3u) top.template combine<OPR>(x, top);
+                    else side.template combine<OPR>(x, side);
+                    continue;
+                }
                 const uint32_t kind = ctl & 3u;
                 uint32_t npop = (ctl >> 2) & 0xFu;
                 uint32_t roles = ctl >> 6;

@@ -79,6 +79,37 @@ def check(x, out, op, max_check_elems=1 << 22):
     return True
 
 
+def copy_reference(args, dev, sink):
+    """What a kernel that only copies reaches at the launch sizes of the sweep's largest messages: one JSON line per
+    p with the median and best GB/s (bytes read plus bytes written) of 5 loops of 20 back-to-back copies that rotate
+    over three destinations."""
+    m = 1 << args.max_log2_bytes
+    for p in args.p:
+        nbytes = (p + 1) * m // 2 // 4 * 4
+        if 4 * nbytes > int(args.max_total_gib * (1 << 30)):
+            continue
+        src = torch.empty(nbytes // 4, dtype=torch.float32, device=dev).normal_()
+        dst = [torch.empty_like(src) for _ in range(3)]
+        for i in range(5):
+            dst[i % 3].copy_(src)
+        torch.cuda.synchronize()
+        rates = []
+        for _ in range(5):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for i in range(20):
+                dst[i % 3].copy_(src)
+            b.record()
+            torch.cuda.synchronize()
+            rates.append(2 * nbytes * 20 / (a.elapsed_time(b) * 1e-3) / 1e9)
+        rates.sort()
+        sink.write(json.dumps({"copy_reference": True, "p": p, "msg_bytes": m, "traffic_bytes": 2 * nbytes,
+                               "gbs_median": rates[2], "gbs_best": rates[-1]}) + "\n")
+        sink.flush()
+        del src, dst
+        torch.cuda.empty_cache()
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     ap.add_argument("--out", default="-")
@@ -92,11 +123,19 @@ def main(argv=None):
     ap.add_argument("--dtypes", nargs="*", default=["int32", "fp32"], choices=list(TORCH_DTYPES))
     ap.add_argument("--ops", nargs="*", default=["sum", "max"], choices=["sum", "max", "min"])
     ap.add_argument("--schedules", nargs="*", default=[s[0] for s in SCHEDULES], choices=[s[0] for s in SCHEDULES])
+    ap.add_argument("--copy-reference", action="store_true",
+                    help="instead of the sweep: time a plain device-to-device copy (torch copy_) whose traffic, read plus written, "
+                         "is that of a reduction of p messages of the largest size, (p + 1) * m bytes, for every p")
     ap.add_argument("--variant", default="auto", choices=["auto", "stream", "paired"],
                     help="tree-mode kernel: the library's choice, or the streaming kernel with one / two operand tiles per ring stage")
     args = ap.parse_args(argv)
     dev = torch.device("cuda", torch.cuda.current_device())
     sink = sys.stdout if args.out == "-" else open(args.out, "w")
+    if args.copy_reference:
+        copy_reference(args, dev, sink)
+        if sink is not sys.stdout:
+            sink.close()
+        return 0
     sizes = [1 << k for k in range(args.min_log2_bytes, args.max_log2_bytes + 1)]
     limit = int(args.max_total_gib * (1 << 30))
     biggest = max(p * m for p in args.p for m in sizes if p * m <= limit)
