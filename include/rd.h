@@ -254,8 +254,12 @@ RD_API int rd_reduce(rd_schedule_t *s, const void *const *d_inputs, void *d_out,
 /*
  * rd_allreduce -- Section III "All-reduce": every process ends up with the combined vector; as the paper
  * states it, a reduce followed by a broadcast.  Tree mode: the reduction of rd_reduce into d_outs[0] (the
- * root's copy, same kernel, same bits), then one more kernel that copies the root's result to the other
- * p - 1 buffers (at most 256 destinations per launch).  Asynchronous on cuda_stream.
+ * root's copy, same kernel, same bits), then a broadcast kernel that copies the root's result to the other
+ * p - 1 buffers.  When every copy is 16-byte aligned: for up to 16 destinations tiles of 4 KB travel through
+ * shared memory by bulk asynchronous copies (one in, p - 1 out), for more every thread carries 128-bit vectors
+ * through registers; the last n mod 4 words of a ragged message go by a second, word-wise launch.  Otherwise
+ * word by word.  At most 256 destinations per launch.  Asynchronous on cuda_stream; a bounded wait that gives
+ * up is reported as for rd_reduce (rd_schedule_status).
  *   d_inputs  HOST array of p DEVICE pointers, as in rd_reduce.
  *   d_outs    HOST array of p DEVICE pointers: d_outs[i] receives process i's copy, n_elems elements.
  *             d_outs[i] may be d_inputs[i] itself (in-place all-reduce); otherwise no copy may overlap any

@@ -12,7 +12,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librd.so")
-SOURCES = ["rd_api.cpp", "rd_sched.cpp", "rd_compile.cpp", "rd_kernels.cu", "rd_faithful.cu"]
+SOURCES = ["rd_api.cpp", "rd_sched.cpp", "rd_compile.cpp", "rd_kernels.cu", "rd_faithful.cu", "rd_broadcast.cu"]
 HEADERS = ["rd_internal.h", "rd_kernels.h"]
 # rd_kernels.cu is compiled once per element type (-DRD_DT=k: that type's kernels; the 16-bit types count
 # twice, once for sum and product and once for max and min) and once without (launch shapes and dispatch),

@@ -878,7 +878,7 @@ int rd_allreduce(rd_schedule_t *s, const void *const *d_inputs, void *const *d_o
         const uintptr_t x = reinterpret_cast<uintptr_t>(a), y = reinterpret_cast<uintptr_t>(b);
         return bytes > 0 && x < y + bytes && y < x + bytes;
     };
-    bool wide = (n_words & 3u) == 0;
+    bool wide = true;                                  // every copy 16-byte aligned
     for (int i = 0; i < s->p; i++) {
         if ((n_elems > 0 && !d_outs[i]) || (reinterpret_cast<uintptr_t>(d_outs[i]) & (align - 1))) return RD_ERR_INVALID_ARG;
         wide = wide && (reinterpret_cast<uintptr_t>(d_outs[i]) & 15u) == 0;
@@ -897,7 +897,7 @@ int rd_allreduce(rd_schedule_t *s, const void *const *d_inputs, void *const *d_o
         if (stats && cudaEventRecord(d.ev_start, stream) != cudaSuccess) return RD_ERR_CUDA;
         // Section III: a reduce to the root followed by a broadcast of the root's result
         if (int rc = reduce_tree(s, d_inputs, d_outs[0], n_words, dtype, op, stream, nullptr)) return rc;
-        if (s->p > 1 && launch_broadcast(d_outs[0], d_outs + 1, s->p - 1, n_words, wide, d.sm_count, stream) != 0) return RD_ERR_CUDA;
+        if (s->p > 1 && launch_broadcast(d_outs[0], d_outs + 1, s->p - 1, n_words, wide, d.sm_count, d.status, stream) != 0) return RD_ERR_CUDA;
         if (stats) {
             if (cudaEventRecord(d.ev_stop, stream) != cudaSuccess || cudaEventSynchronize(d.ev_stop) != cudaSuccess) return RD_ERR_CUDA;
             float ms = 0;
@@ -909,7 +909,7 @@ int rd_allreduce(rd_schedule_t *s, const void *const *d_inputs, void *const *d_o
             stats->predicted_s = double(s->sched.completion) * s->ticks.tick;
             bool vectors = (reinterpret_cast<uintptr_t>(d_outs[0]) & 15u) == 0;      // the reduction took the 128-bit path
             for (int i = 0; i < s->p && vectors; i++) vectors = (reinterpret_cast<uintptr_t>(d_inputs[i]) & 15u) == 0;
-            stats->n_launches = n_words ? 1 + (vectors && (n_words & 3u) ? 1 : 0) + (s->p > 1 ? (s->p - 2) / kBcastPackPtrs + 1 : 0) : 0;
+            stats->n_launches = n_words ? 1 + (vectors && (n_words & 3u) ? 1 : 0) + broadcast_launches(s->p - 1, n_words, wide) : 0;
             int st = 0;
             if (cudaMemcpy(&st, d.status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return RD_ERR_CUDA;
             stats->device_status = st;

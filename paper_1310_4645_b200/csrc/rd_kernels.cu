@@ -658,15 +658,14 @@ template <int G, int CW> struct StreamShape {
     static constexpr int THREADS = CT + 32 * kProducers;
     static_assert(N >= 1 && N * G * CT == kStageVecs, "a tile is a whole number of vectors per consumer thread");
 };
-// Thread blocks per SM the registers must leave room for (shared memory decides how many actually run).
-template <int DT, int CW> struct StreamBlocks { static constexpr int value = 3; };
+constexpr int kStreamBlocks = 3;    // thread blocks per SM the registers must leave room for (shared memory decides how many run)
 // Whether the kernel evaluates the sub-expressions marked in the programs (bit 30) in a second accumulator, which
 // saves their pushes and pops and one level of the shared-memory stack.  Not where a thread's accumulator is
 // 32 registers already (16-bit elements on whole-stage tiles: these serve shallow programs only).
 template <int DT, int G> struct SecondAccumulator { static constexpr bool value = !(Wide<DT>::half && G == 1); };
 
 template <int DT, int OPR, typename PRM, int G, int CW>
-__global__ void __launch_bounds__(StreamShape<G, CW>::THREADS, StreamBlocks<DT, CW>::value)
+__global__ void __launch_bounds__(StreamShape<G, CW>::THREADS, kStreamBlocks)
 rd_tree_stream_kernel(const __grid_constant__ PRM a)
 {
     using Jobs = typename PRM::Jobs;
@@ -1206,83 +1205,6 @@ int RD_CAT(launch_for_dtype_, RD_DT)(int which, const void *launch, int op)
 }
 
 #else
-
-// ---------------------------------------------------------------------------------------------
-// Broadcast of the root's result (all-reduce = reduce, then broadcast): every thread reads U vectors of
-// the source and writes them to each of the n_dst destinations.  Bound by HBM writes: m bytes read,
-// n_dst * m written.
-// ---------------------------------------------------------------------------------------------
-namespace {
-
-constexpr int kBcastThreads = 256;
-constexpr int kBcastU = 4;               // vectors in flight per thread
-
-struct BcastParams {
-    uint32_t *dst[kBcastPackPtrs];
-    const uint32_t *src;
-    uint64_t n_vec;                      // vectors (of V words) to copy
-    int n_dst;
-};
-
-template <int V>
-__global__ void __launch_bounds__(kBcastThreads, 4)
-rd_broadcast_kernel(const __grid_constant__ BcastParams a)
-{
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    asm volatile("griddepcontrol.wait;" ::: "memory");           // the reduction that produced src has finished
-    const uint64_t stride = uint64_t(gridDim.x) * kBcastThreads;
-    for (uint64_t v0 = uint64_t(blockIdx.x) * kBcastThreads + threadIdx.x; v0 < a.n_vec; v0 += stride * kBcastU) {
-        Vec<V> x[kBcastU];
-#pragma unroll
-        for (int u = 0; u < kBcastU; u++) {
-            const uint64_t v = v0 + uint64_t(u) * stride;
-            if (v < a.n_vec) {
-                if constexpr (V == 4) {
-                    const uint4 t = __ldcs(reinterpret_cast<const uint4 *>(a.src) + v);
-                    x[u].w[0] = t.x; x[u].w[1] = t.y; x[u].w[2] = t.z; x[u].w[3] = t.w;
-                } else {
-                    x[u].w[0] = __ldcs(a.src + v);
-                }
-            }
-        }
-        for (int d = 0; d < a.n_dst; d++) {
-#pragma unroll
-            for (int u = 0; u < kBcastU; u++) {
-                const uint64_t v = v0 + uint64_t(u) * stride;
-                if (v < a.n_vec) store_stream<V>(a.dst[d] + v * V, x[u]);
-            }
-        }
-    }
-}
-
-}  // namespace
-
-int launch_broadcast(const void *src, void *const *dsts, int n_dst, uint64_t n_words, bool wide, int sm_count, void *stream)
-{
-    if (n_words == 0) return 0;
-    for (int base = 0; base < n_dst; base += kBcastPackPtrs) {
-        BcastParams prm;
-        const int cnt = n_dst - base < kBcastPackPtrs ? n_dst - base : kBcastPackPtrs;
-        for (int i = 0; i < kBcastPackPtrs; i++) prm.dst[i] = i < cnt ? static_cast<uint32_t *>(dsts[base + i]) : nullptr;
-        prm.src = static_cast<const uint32_t *>(src);
-        prm.n_vec = wide ? n_words / 4 : n_words;
-        prm.n_dst = cnt;
-        const uint64_t perBlock = uint64_t(kBcastThreads) * kBcastU;
-        uint64_t blocks = (prm.n_vec + perBlock - 1) / perBlock;
-        const uint64_t most = uint64_t(sm_count > 0 ? sm_count : 1) * 8u;
-        if (blocks > most) blocks = most;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(unsigned(blocks)); cfg.blockDim = dim3(kBcastThreads); cfg.dynamicSmemBytes = 0;
-        cfg.stream = static_cast<cudaStream_t>(stream);
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr; cfg.numAttrs = 1;
-        const cudaError_t e = wide ? cudaLaunchKernelEx(&cfg, rd_broadcast_kernel<4>, prm) : cudaLaunchKernelEx(&cfg, rd_broadcast_kernel<1>, prm);
-        if (e != cudaSuccess) return int(e);
-    }
-    return 0;
-}
 
 uint32_t tree_tile_elems(int vec) { return uint32_t(kTreeThreads) * kU * uint32_t(vec); }
 

@@ -93,10 +93,15 @@ bool direct_applies(int p, int stack_depth);
 int direct_blocks_per_sm(int p);
 int launch_tree_direct(const TreeLaunch &a);
 
-// Broadcast (all-reduce = reduce + broadcast): copies n_words 32-bit words from src to each of the n_dst
-// destinations (device pointers in a host array); wide: all buffers 16-byte aligned and n_words a multiple of 4.
+// Broadcast (all-reduce = reduce + broadcast; rd_broadcast.cu): copies n_words 32-bit words from src to each of the
+// n_dst destinations (device pointers in a host array).  aligned: all buffers 16-byte aligned; the whole 128-bit
+// vectors then go through bulk asynchronous copies, the last n_words mod 4 words (or, unaligned, everything) through a
+// word-wise kernel.  status: device word that receives an error code when a bounded wait gives up.
+// broadcast_launches: how many kernels launch_broadcast launches for these arguments.
 constexpr int kBcastPackPtrs = 256;   // destinations per launch (they travel as kernel parameters)
-int launch_broadcast(const void *src, void *const *dsts, int n_dst, uint64_t n_words, bool wide, int sm_count, void *stream);
+int launch_broadcast(const void *src, void *const *dsts, int n_dst, uint64_t n_words, bool aligned, int sm_count, int *status,
+                     void *stream);
+int broadcast_launches(int n_dst, uint64_t n_words, bool aligned);
 
 // ---- schedule-faithful execution (rd_faithful.cu)
 constexpr int kFaithfulThreads = 128;

@@ -110,6 +110,40 @@ def copy_reference(args, dev, sink):
         torch.cuda.empty_cache()
 
 
+def allreduce_timing(args, dev, sink):
+    """rd_allreduce for every p at the largest message size: one JSON line per p with the time of both kernels together,
+    GB/s counting (p + 1) m bytes for the reduce plus m read and (p - 1) m written by the broadcast, and a check that
+    every process's copy equals the root's and the root's passes the order-free check."""
+    m = 1 << args.max_log2_bytes
+    n = m // 4
+    for p in args.p:
+        if 2 * p * m > int(args.max_total_gib * (1 << 30)):
+            continue
+        x = fill_arena(p * n, torch.float32, dev).view(p, n)
+        outs = torch.empty_like(x)
+        seg = rd.rd_optimal_segment(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, p, m, ALPHA, BETA, GAMMA)
+        h = rd.rd_schedule_create(rd.RD_UNI_GREEDY, rd.RD_PORT_UNI, p, m, seg, ALPHA, BETA, GAMMA)
+        try:
+            tin, tout = rd.PointerTable(x), rd.PointerTable(outs)
+            rd.rd_allreduce(h, tin, tout, rd.RD_SUM)
+            ok = check(x, outs[0], "sum") and all(torch.equal(outs[i], outs[0]) for i in range(1, p))
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(args.reps):
+                rd.rd_allreduce(h, tin, tout, rd.RD_SUM)
+            b.record()
+            torch.cuda.synchronize()
+            us = a.elapsed_time(b) * 1e3 / args.reps
+            moved = (p + 1) * m + (p * m if p > 1 else 0)
+            sink.write(json.dumps({"allreduce": True, "p": p, "msg_bytes": m, "seg_bytes": seg, "measured_us": us,
+                                   "bytes_moved": moved, "gbs": moved / us / 1e3, "ok": ok}) + "\n")
+            sink.flush()
+        finally:
+            rd.rd_destroy(h)
+        del x, outs
+        torch.cuda.empty_cache()
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     ap.add_argument("--out", default="-")
@@ -126,13 +160,16 @@ def main(argv=None):
     ap.add_argument("--copy-reference", action="store_true",
                     help="instead of the sweep: time a plain device-to-device copy (torch copy_) whose traffic, read plus written, "
                          "is that of a reduction of p messages of the largest size, (p + 1) * m bytes, for every p")
+    ap.add_argument("--allreduce", action="store_true",
+                    help="instead of the sweep: time rd_allreduce (the reduce, then the broadcast of the root's result to every "
+                         "process) for every p at the largest message size, uni-greedy at its tuned segment size, fp32 sum")
     ap.add_argument("--variant", default="auto", choices=["auto", "stream", "paired"],
                     help="tree-mode kernel: the library's choice, or the streaming kernel with one / two operand tiles per ring stage")
     args = ap.parse_args(argv)
     dev = torch.device("cuda", torch.cuda.current_device())
     sink = sys.stdout if args.out == "-" else open(args.out, "w")
-    if args.copy_reference:
-        copy_reference(args, dev, sink)
+    if args.copy_reference or args.allreduce:
+        (copy_reference if args.copy_reference else allreduce_timing)(args, dev, sink)
         if sink is not sys.stdout:
             sink.close()
         return 0

@@ -47,14 +47,21 @@ def test_every_process_receives_the_roots_result(algo, port):
             assert st.bytes_moved == ((p + 1) + (p if p > 1 else 0)) * 4 * n
             vectors = all(x[i].data_ptr() % 16 == 0 for i in range(p)) and outs.data_ptr() % 16 == 0
             tail = 1 if vectors and n % 4 else 0             # the 128-bit path leaves the last n mod 4 elements to a second, tiny launch
-            assert st.n_launches == 1 + tail + (0 if p == 1 else (p - 2) // 256 + 1)
+            # the broadcast: at most 256 destinations per launch; aligned copies go through the bulk-copy kernel (whole
+            # 128-bit vectors) and a word-wise launch for the last n mod 4 words, other copies through the word-wise one
+            groups = 0 if p == 1 else (p - 2) // 256 + 1
+            aligned = all(outs[i].data_ptr() % 16 == 0 for i in range(p))
+            per_group = (1 if n >= 4 else 0) + (1 if n % 4 else 0) if aligned else 1
+            assert st.n_launches == 1 + tail + groups * per_group
 
 
 def test_in_place_and_unaligned_buffers():
     p = 16
     wide = make_inputs(p, 6000, "normal", seed=8, device="cuda")                             # every row 16-byte aligned
     big = make_inputs(p, 6002, "normal", seed=9, device="cuda")
-    for rows in ([wide[i] for i in range(p)], [big[i, :6001] for i in range(p)], [big[i, 1:] for i in range(p)]):
+    ragged = make_inputs(p, 6004, "normal", seed=11, device="cuda")                          # aligned rows, n mod 4 = 2
+    for rows in ([wide[i] for i in range(p)], [big[i, :6001] for i in range(p)], [big[i, 1:] for i in range(p)],
+                 [ragged[i, :6002] for i in range(p)]):
         n = rows[0].numel()
         keep = torch.stack(rows).cpu().numpy()
         h = rd.rd_schedule_create(rd.RD_BI_GREEDY, rd.RD_PORT_BI, p, 4 * n, 4 * 1000, *M1)
