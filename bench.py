@@ -375,8 +375,14 @@ class TreeBench:
         for st in streams:
             if st is not self.main_stream:
                 st.wait_event(e0)
+        self.step_marks = [e0]
         for _ in range(steps):
             self.step(streams)
+            if len(streams) == 1:
+                # one stream: an event after every step gives the spread over the steps (median, best)
+                mark = torch.cuda.Event(enable_timing=True)
+                mark.record(self.main_stream)
+                self.step_marks.append(mark)
         for st in streams:
             if st is not self.main_stream:
                 done = torch.cuda.Event()
@@ -384,6 +390,14 @@ class TreeBench:
                 self.main_stream.wait_event(done)
         e1.record(self.main_stream)
         return e0, e1
+
+    def step_spread(self):
+        """Median and best step time (ms) of the last one-stream timed region, or None."""
+        marks = getattr(self, "step_marks", [])
+        if len(marks) < 2:
+            return None
+        t = sorted(a.elapsed_time(b) for a, b in zip(marks[:-1], marks[1:]))
+        return {"median": t[len(t) // 2], "best": t[0], "worst": t[-1]}
 
     def per_schedule(self, reps):
         rd, torch = self.rd, self.torch
@@ -474,6 +488,7 @@ def measure(tb, steps, warmup, barrier, dev, world, sample_clocks, local_rank):
     barrier()
     clocks = sampler.stop() if sampler else None
     ms = max_over_ranks(e0.elapsed_time(e1), dev)
+    spread = tb.step_spread()
     value = replica_throughput(steps * tb.reduces_per_step * tb.bytes_per_reduce, ms, world)
     if tb.n_streams > 1:
         k_steps = max(3, steps // 2)
@@ -487,7 +502,7 @@ def measure(tb, steps, warmup, barrier, dev, world, sample_clocks, local_rank):
     else:
         kernel_ms = ms / (steps * tb.launches_per_step)
         timed_over = "the %d launches of the timed region (one stream, CUDA events around it), %.2f us each" % (steps * tb.launches_per_step, kernel_ms * 1e3)
-    return value, ms, kernel_ms, timed_over, clocks
+    return value, ms, kernel_ms, timed_over, clocks, spread
 
 
 def roofline_block(tb, kernel_ms, timed_over):
@@ -613,7 +628,7 @@ def main():
         torch.cuda.synchronize()
 
     tb = TreeBench(rd, torch, wname, w, dev, args.issue, args.streams)
-    value, ms, kernel_ms, timed_over, clocks = measure(tb, args.steps, args.warmup, barrier, dev, world, True, local_rank)
+    value, ms, kernel_ms, timed_over, clocks, spread = measure(tb, args.steps, args.warmup, barrier, dev, world, True, local_rank)
     per_schedule = tb.per_schedule(max(5, min(10, args.steps // 2)))
     e2e = None if args.no_e2e else end_to_end(rd, torch, tb, dev, world, barrier, args.steps)
     faithful = None
@@ -631,7 +646,7 @@ def main():
         w2 = WORKLOADS["config2"]
         tb2 = TreeBench(rd, torch, "config2", w2, dev, "batch", 2)
         steps2 = 200
-        v2, ms2, k2, over2, _ = measure(tb2, steps2, 10, barrier, dev, world, False, local_rank)
+        v2, ms2, k2, over2, _, _ = measure(tb2, steps2, 10, barrier, dev, world, False, local_rank)
         small = {"config": tb2.describe(world), "value": v2, "unit": "GB/s", "steps": steps2, "ms_per_step": ms2 / steps2,
                  "roofline": roofline_block(tb2, k2, over2), "per_schedule_gbs": tb2.per_schedule(20),
                  "schedule_create_ms": tb2.create_ms,
@@ -645,7 +660,7 @@ def main():
         peak = roof["peak"]
         line = {
             "metric": "reduction_throughput", "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "ms_per_step_spread": spread, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "i32" if w["dist"].startswith("int") else "f32", "data": "synthetic",
             "config": config, "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": gpu_launches, "clocks": clocks,
             "reductions_per_step": reductions_per_step, "per_schedule_gbs": per_schedule, "schedule_create_ms": create_ms,

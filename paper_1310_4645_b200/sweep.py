@@ -127,13 +127,15 @@ def allreduce_timing(args, dev, sink):
             tin, tout = rd.PointerTable(x), rd.PointerTable(outs)
             rd.rd_allreduce(h, tin, tout, rd.RD_SUM)
             ok = check(x, outs[0], "sum") and all(torch.equal(outs[i], outs[0]) for i in range(1, p))
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            for _ in range(args.reps):
-                rd.rd_allreduce(h, tin, tout, rd.RD_SUM)
-            b.record()
-            torch.cuda.synchronize()
-            us = a.elapsed_time(b) * 1e3 / args.reps
+            us = float("inf")
+            for _ in range(3):                                   # the best of three runs of 4 * reps calls each
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                for _ in range(4 * args.reps):
+                    rd.rd_allreduce(h, tin, tout, rd.RD_SUM)
+                b.record()
+                torch.cuda.synchronize()
+                us = min(us, a.elapsed_time(b) * 1e3 / (4 * args.reps))
             moved = (p + 1) * m + (p * m if p > 1 else 0)
             sink.write(json.dumps({"allreduce": True, "p": p, "msg_bytes": m, "seg_bytes": seg, "measured_us": us,
                                    "bytes_moved": moved, "gbs": moved / us / 1e3, "ok": ok}) + "\n")

@@ -55,8 +55,8 @@ def test_every_process_receives_the_roots_result(algo, port):
             assert st.n_launches == 1 + tail + groups * per_group
 
 
-def test_in_place_and_unaligned_buffers():
-    p = 16
+@pytest.mark.parametrize("p", [16, 40])      # up to 16 destinations: bulk copies through shared memory; more: registers
+def test_in_place_and_unaligned_buffers(p):
     wide = make_inputs(p, 6000, "normal", seed=8, device="cuda")                             # every row 16-byte aligned
     big = make_inputs(p, 6002, "normal", seed=9, device="cuda")
     ragged = make_inputs(p, 6004, "normal", seed=11, device="cuda")                          # aligned rows, n mod 4 = 2
