@@ -92,7 +92,21 @@ int compile_programs(int p, size_t q, const std::vector<rd_event_t> &events, Pro
     std::vector<int> expr(P, 0), need, leafSeen(P, 0);
     std::vector<uint32_t> prog;
     std::vector<int> walk;
+    size_t pushedBefore = 0;                 // pushes that remain in the segment before this one
     for (size_t j = 0; j < q; j++) {
+        // The program depends only on who sends to whom, in which order: a segment whose pairs repeat those of the
+        // segment before it (every segment of a fixed tree, most segments of a greedy schedule's steady state)
+        // shares that segment's program.
+        if (j > 0 && first[j + 1] - first[j] == first[j] - first[j - 1]) {
+            bool same = true;
+            for (size_t k = first[j], k0 = first[j - 1]; k < first[j + 1] && same; k++, k0++)
+                same = bySeg[k].src == bySeg[k0].src && bySeg[k].dst == bySeg[k0].dst && bySeg[k].kind == bySeg[k0].kind;
+            if (same) {
+                out.seg_prog[j] = out.seg_prog[j - 1];
+                out.shared_pushes += pushedBefore;
+                continue;
+            }
+        }
         nodes.clear();
         for (int i = 0; i < p; i++) expr[size_t(i)] = i;
         for (size_t k = first[j]; k < first[j + 1]; k++) {
@@ -172,6 +186,7 @@ int compile_programs(int p, size_t q, const std::vector<rd_event_t> &events, Pro
             if (!open.empty() || onStack != 0) return RD_ERR_INTERNAL;
             out.shared_depth = std::max(out.shared_depth, deepest);
             out.shared_pushes += pushed;
+            pushedBefore = pushed;
         }
         std::string key(reinterpret_cast<const char *>(prog.data()), prog.size() * sizeof(uint32_t));
         auto it = seen.find(key);

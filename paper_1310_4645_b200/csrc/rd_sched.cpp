@@ -28,6 +28,37 @@ void sort_events(std::vector<rd_event_t> &ev)
     });
 }
 
+static bool event_before(const rd_event_t &a, const rd_event_t &b)
+{
+    if (a.t_start != b.t_start) return a.t_start < b.t_start;
+    if (a.seg != b.seg) return a.seg < b.seg;
+    if (a.src != b.src) return a.src < b.src;
+    return a.dst < b.dst;
+}
+
+// Lock-step schedules: every pair starts at a multiple of the round length, and the generators emit the pairs
+// segment by segment, process by process, so a stable counting sort on the round leaves each round in
+// (segment, source) order: linear time where the comparison sort of a few million pairs takes longer than everything
+// else together.  Falls back to the comparison sort when the rounds are too sparse or the order is not reached.
+static void order_by_round(std::vector<rd_event_t> &ev, int64_t len)
+{
+    if (ev.size() < 2) return;
+    if (std::is_sorted(ev.begin(), ev.end(), event_before)) return;
+    int64_t last = -1;
+    if (len > 0) {
+        last = 0;
+        for (const rd_event_t &e : ev) last = std::max(last, e.t_start / len);
+    }
+    if (last < 0 || uint64_t(last) > 8 * uint64_t(ev.size()) + 1024) { sort_events(ev); return; }
+    std::vector<size_t> first(size_t(last) + 2, 0);
+    for (const rd_event_t &e : ev) first[size_t(e.t_start / len) + 1]++;
+    for (size_t r = 0; r + 1 < first.size(); r++) first[r + 1] += first[r];
+    std::vector<rd_event_t> sorted(ev.size());
+    for (const rd_event_t &e : ev) sorted[first[size_t(e.t_start / len)]++] = e;
+    ev.swap(sorted);
+    if (!std::is_sorted(ev.begin(), ev.end(), event_before)) sort_events(ev);
+}
+
 static void set_offsets(const std::vector<int64_t> &seg_bytes, Schedule &out)
 {
     out.seg_off.assign(1, 0);
@@ -90,22 +121,33 @@ int gen_bi_greedy(int p, const std::vector<int64_t> &seg_bytes, const Ticks &c, 
     std::vector<uint8_t> sent(P * q, 0);              // sent[i*q + j]: i has sent j (root: j complete)
     std::vector<int64_t> lastSendEnd(q, 0);
     std::vector<uint32_t> holders(q, uint32_t(p));    // processes (root included) not yet done with j
-    std::vector<int> sendOnly, recvOnly, both, sendList, recvList;
+    std::vector<int> sendOnly, recvOnly, both, sendList, recvList, idle;
+    std::vector<int64_t> fruitless;                   // segment lengths that cannot be paired at the current instant
     size_t rootNext = 0;                              // first segment the root has not completed
     int64_t t = 0;
     while (rootNext < q) {
+        // the processes with a free port at this instant, in process order: only they can be paired now
         int freeSend = 0, freeRecv = 0, freeSendNonRoot = 0;
+        idle.clear();
+        fruitless.clear();
         for (int i = 0; i < p; i++) {
-            if (sendFreeAt[size_t(i)] <= t) { freeSend++; if (i != 0) freeSendNonRoot++; }
-            if (recvFreeAt[size_t(i)] <= t) freeRecv++;
+            const bool s = sendFreeAt[size_t(i)] <= t, r = recvFreeAt[size_t(i)] <= t;
+            if (s) { freeSend++; if (i != 0) freeSendNonRoot++; }
+            if (r) freeRecv++;
+            if ((s && i != 0) || r) idle.push_back(i);
         }
         for (size_t j = rootNext; j < q; j++) {
             if (freeSendNonRoot == 0 || freeRecv == 0) break;   // nothing can be paired from here on
+            // A segment that none of the idle processes has sent yet and that still found no pair (ports free on one
+            // side only, or combines in the way) settles every later segment of its length at this instant: their
+            // candidates are a subset of its, and fewer candidates never make a pair where more made none.
+            if (std::find(fruitless.begin(), fruitless.end(), seg_bytes[j]) != fruitless.end()) continue;
             const int64_t tc = c.comm(seg_bytes[j]), tp = c.comp(seg_bytes[j]);
             sendOnly.clear(); recvOnly.clear(); both.clear();
-            for (int i = 0; i < p; i++) {
+            bool allHold = true;
+            for (int i : idle) {
                 const size_t I = size_t(i);
-                if (sent[I * q + j]) continue;
+                if (sent[I * q + j]) { allHold = false; continue; }
                 if (t < compEnd[I] && compBegin[I] < t + tc) continue;        // would meet its combine
                 const bool canSend = i != 0 && sendFreeAt[I] <= t;
                 const bool canRecv = recvFreeAt[I] <= t;
@@ -128,6 +170,7 @@ int gen_bi_greedy(int p, const std::vector<int64_t> &seg_bytes, const Ticks &c, 
             recvList.insert(recvList.end(), both.begin(), both.begin() + toRecv);
             std::sort(recvList.begin(), recvList.end());
             const size_t pairs = std::min(sendList.size(), recvList.size());
+            if (pairs == 0 && allHold) fruitless.push_back(seg_bytes[j]);
             for (size_t k = 0; k < pairs; k++) {
                 const int a = sendList[k], b = recvList[k];
                 const size_t Ia = size_t(a), Ib = size_t(b);
@@ -177,6 +220,7 @@ int gen_binomial(int p, const std::vector<int64_t> &seg_bytes, const Ticks &c, S
     const int rounds = ceil_log2(uint64_t(p));
     const int64_t len = round_length(seg_bytes, c);
     out.events.clear();
+    out.events.reserve(size_t(p > 0 ? p - 1 : 0) * seg_bytes.size());
     for (size_t j = 0; j < seg_bytes.size(); j++)
         for (int r = 0; r < rounds; r++)
             for (int64_t k = int64_t(1) << r; k < p; k += int64_t(2) << r)
@@ -184,7 +228,7 @@ int gen_binomial(int p, const std::vector<int64_t> &seg_bytes, const Ticks &c, S
                                                 (int64_t(j) * rounds + r) * len});
     out.completion = int64_t(seg_bytes.size()) * rounds * len;
     set_offsets(seg_bytes, out);
-    sort_events(out.events);
+    order_by_round(out.events, len);
     return RD_OK;
 }
 
@@ -194,12 +238,20 @@ int gen_pipeline(int p, const std::vector<int64_t> &seg_bytes, const Ticks &c, b
     const int64_t q = int64_t(seg_bytes.size());
     const int64_t perSegment = bidir ? 1 : 2;   // a one-port process alternates receive and send
     out.events.clear();
-    for (int64_t j = 0; j < q; j++)
-        for (int k = 1; k < p; k++)
-            out.events.push_back(rd_event_t{int32_t(j), k, k - 1, 0, (int64_t(p - 1 - k) + perSegment * j) * len});
     out.completion = (p < 2 || q == 0) ? 0 : (int64_t(p - 1) + perSegment * (q - 1)) * len;
     set_offsets(seg_bytes, out);
-    sort_events(out.events);
+    if (p < 2 || q == 0) return RD_OK;
+    // process k sends segment j in round (p - 1 - k) + perSegment * j; emitted round by round, in a round by segment
+    out.events.reserve(size_t(p - 1) * size_t(q));
+    const int64_t lastRound = int64_t(p - 2) + perSegment * (q - 1);
+    for (int64_t round = 0; round <= lastRound; round++) {
+        const int64_t over = round - int64_t(p - 2);                         // segments before this one are through
+        int64_t j = over > 0 ? (over + perSegment - 1) / perSegment : 0;
+        for (; j < q && perSegment * j <= round; j++) {
+            const int k = int(int64_t(p - 1) - (round - perSegment * j));
+            out.events.push_back(rd_event_t{int32_t(j), k, k - 1, 0, round * len});
+        }
+    }
     return RD_OK;
 }
 
@@ -211,6 +263,7 @@ int gen_binary(int p, const std::vector<int64_t> &seg_bytes, const Ticks &c, boo
     const int64_t perSegment = bidir ? 2 : 4;
     int64_t rounds = 0;
     out.events.clear();
+    out.events.reserve(size_t(p > 0 ? p - 1 : 0) * seg_bytes.size());
     for (int64_t j = 0; j < q; j++) {
         for (int k = 1; k < p; k++) {
             const int d = ceil_log2(uint64_t(k) + 2) - 1;    // depth of node k = floor(log2(k+1))
@@ -221,7 +274,7 @@ int gen_binary(int p, const std::vector<int64_t> &seg_bytes, const Ticks &c, boo
     }
     out.completion = rounds * len;
     set_offsets(seg_bytes, out);
-    sort_events(out.events);
+    order_by_round(out.events, len);
     return RD_OK;
 }
 

@@ -76,6 +76,30 @@ def test_unequal_segmentation():
             compare(rd.RD_PIPELINE, rd.RD_PORT_UNI, p, sum(sizes), 0, model, sizes=sizes)
 
 
+def test_random_models_and_segmentations():
+    """Seeded random cases: process counts around powers of two, equal, ragged and arbitrary segment sizes, models
+    with zero terms (many ties).  The library's generators skip work the simulators do (bi-greedy stops visiting
+    segments of a length that found no pair at an instant, the fixed trees are emitted or bucketed by round instead
+    of sorted), so every shortcut has to reproduce the simulators' pairs exactly."""
+    rng = np.random.default_rng(20131017)
+    kinds = [(a, port) for a in PORTS if a != rd.RD_BUTTERFLY for port in PORTS[a]] + [(rd.RD_BI_GREEDY, rd.RD_PORT_BI)] * 3
+    for _ in range(250):
+        algo, port = kinds[int(rng.integers(len(kinds)))]
+        p = int(rng.choice([1, 2, 3, 4, 5, 7, 8, 13, 16, 31, 32, 33, 64, 100, 257]))
+        q = int(rng.choice([1, 2, 3, 5, 8, 17, 40, 129]))
+        how = rng.random()
+        if how < 0.4:
+            sizes = [4 * int(rng.integers(1, 51))] * q
+        elif how < 0.7:
+            sizes = [4 * int(rng.integers(1, 51))] * (q - 1) + [4 * int(rng.integers(1, 51))]
+        else:
+            sizes = [4 * int(s) for s in rng.integers(1, 51, size=q)]
+        A, B, G = int(rng.choice([0, 1, 3, 10, 1000, 12345])), int(rng.choice([0, 1, 2, 7, 100])), int(rng.choice([0, 0, 1, 3, 50]))
+        if A == 0 and B == 0:
+            B = 1
+        compare(algo, port, p, sum(sizes), 0, (A * 1e-15, B * 1e-15, G * 1e-15), sizes=sizes)
+
+
 def test_library_schedules_pass_the_oracle_validator():
     for algo in PORTS:
         for port in PORTS[algo]:
