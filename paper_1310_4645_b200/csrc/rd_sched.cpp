@@ -66,37 +66,57 @@ static void set_offsets(const std::vector<int64_t> &seg_bytes, Schedule &out)
 }
 
 // ---------------------------------------------------------------------------------------------
-// Algorithm 1 (uni-greedy).  Per segment a min-heap of (state, process) over the processes that
-// still hold the segment: the two smallest are paired at t = the larger of their states; the root
-// never sends (Lemma 1), so it is the receiver whenever it is one of the two.
+// Algorithm 1 (uni-greedy).  Per segment the two processes with the smallest states (ties: the smaller
+// process index) among those that still hold the segment are paired at t = the larger of the two states;
+// the root never sends (Lemma 1), so it is the receiver whenever it is one of the two.
+// The pairing instants of a segment never decrease, so the receivers' new states come out in
+// non-decreasing order: as in the two-queue construction of a Huffman tree, the smallest state is always
+// at the head of one of two sorted queues (the states the segment started with; the states of receivers),
+// and a segment costs O(p) once its initial states are in order.  They are: the senders' states after a
+// segment, taken in pairing order, are sorted already, and the root, the last receiver, has the largest.
+// Equal states are put in process order where they meet (runs of equal states are short).
 // ---------------------------------------------------------------------------------------------
 int gen_uni_greedy(int p, const std::vector<int64_t> &seg_bytes, const Ticks &c, Schedule &out, bool want_events)
 {
-    typedef std::pair<int64_t, int> Key;
-    std::vector<int64_t> state(size_t(p), 0);
+    typedef std::pair<int64_t, int> Key;                 // (state, process)
     out.events.clear();
-    if (want_events) out.events.reserve(size_t(p > 0 ? p - 1 : 0) * seg_bytes.size());
-    std::vector<Key> init;
+    out.completion = 0;
+    set_offsets(seg_bytes, out);
+    if (p < 1) return RD_OK;
+    if (want_events) out.events.reserve(size_t(p - 1) * seg_bytes.size());
+    std::vector<Key> start, next, received;
+    for (int i = 0; i < p; i++) start.push_back(Key(0, i));
     for (size_t j = 0; j < seg_bytes.size(); j++) {
         const int64_t tc = c.comm(seg_bytes[j]), tp = c.comp(seg_bytes[j]);
-        init.clear();
-        for (int i = 0; i < p; i++) init.push_back(Key(state[size_t(i)], i));
-        std::priority_queue<Key, std::vector<Key>, std::greater<Key>> heap(std::greater<Key>(), std::move(init));
-        init = std::vector<Key>();
-        while (heap.size() >= 2) {
-            const Key first = heap.top(); heap.pop();
-            const Key second = heap.top(); heap.pop();
+        size_t h1 = 0, h2 = 0;
+        received.clear();
+        next.clear();
+        auto take = [&]() {
+            if (h1 < start.size() && (h2 >= received.size() || start[h1] < received[h2])) return start[h1++];
+            return received[h2++];
+        };
+        for (int k = 0; k + 1 < p; k++) {
+            const Key first = take(), second = take();
             const int64_t t = second.first;
             int sender = first.second, receiver = second.second;
             if (sender == 0) std::swap(sender, receiver);
             if (want_events) out.events.push_back(rd_event_t{int32_t(j), sender, receiver, 0, t});
-            state[size_t(sender)] = t + tc;
-            state[size_t(receiver)] = t + tc + tp;
-            heap.push(Key(t + tc + tp, receiver));
+            next.push_back(Key(t + tc, sender));
+            // no state in the queue is larger than the new one: it joins the run of equal states at the end
+            const Key key(t + tc + tp, receiver);
+            received.insert(std::upper_bound(received.begin() + std::ptrdiff_t(h2), received.end(), key), key);
         }
+        next.push_back(take());                          // the root, with the largest state
+        for (size_t a = 0; a < next.size();) {           // runs of equal states in process order
+            size_t b = a + 1;
+            while (b < next.size() && next[b].first == next[a].first) b++;
+            if (b - a > 1) std::sort(next.begin() + std::ptrdiff_t(a), next.begin() + std::ptrdiff_t(b));
+            a = b;
+        }
+        start.swap(next);
     }
-    out.completion = p > 0 ? state[0] : 0;
-    set_offsets(seg_bytes, out);
+    for (const Key &k : start)
+        if (k.second == 0) out.completion = k.first;
     if (want_events) sort_events(out.events);
     return RD_OK;
 }
