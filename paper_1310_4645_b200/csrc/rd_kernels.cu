@@ -205,8 +205,12 @@ template <int DT, int V> __device__ __forceinline__ Vec<V> narrow(const Vec<V * 
     return m;
 }
 
-// Sum and product give the same bits whichever operand was held (IEEE add and multiply commute).
-template <int OPR> struct Commutes { static constexpr bool value = OPR == OPR_SUM || OPR == OPR_PROD; };
+// Sum and product give the same bits whichever operand was held (IEEE add and multiply commute), and so do max and
+// min of integers (equal integers are the same bits; floating-point zeros of either sign compare equal, so there the
+// held operand has to be known).
+template <int DT, int OPR> struct Commutes {
+    static constexpr bool value = OPR == OPR_SUM || OPR == OPR_PROD || DT == DT_INT32 || DT == DT_INT64;
+};
 
 struct PtrPack { const uint32_t *ptr[kPackedPtrs]; };
 struct PtrRef { const uint32_t *const *table; };
@@ -285,7 +289,7 @@ rd_tree_kernel(const __grid_constant__ TreeParams<PACKED> a)
                     if (kind <= 1u) {                      // LOAD / PUSH_LOAD
 #pragma unroll
                         for (int u = 0; u < U; u++) top[u] = x[u];
-                    } else if (kind == 2u || Commutes<OPR>::value) {   // ACC_IN (a sum does not care who held what)
+                    } else if (kind == 2u || Commutes<DT, OPR>::value) {   // ACC_IN (a sum does not care who held what)
 #pragma unroll
                         for (int u = 0; u < U; u++) combine_vec<ADT, OPR, AV>(top[u], top[u], x[u]);
                     } else {                               // ACC_HELD
@@ -301,7 +305,7 @@ rd_tree_kernel(const __grid_constant__ TreeParams<PACKED> a)
 #pragma unroll
                         for (int u = 0; u < U; u++) {
                             const Vec<AV> y = stack[(sp * U + u) * kTreeThreads + tid];
-                            if (poppedHeld || Commutes<OPR>::value) combine_vec<ADT, OPR, AV>(top[u], y, top[u]);
+                            if (poppedHeld || Commutes<DT, OPR>::value) combine_vec<ADT, OPR, AV>(top[u], y, top[u]);
                             else combine_vec<ADT, OPR, AV>(top[u], top[u], y);
                         }
                     }
@@ -828,19 +832,19 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
             for (int g = 0; g < G; g++) {
                 if (g > 0 && i + g >= p) break;
                 const uint32_t ctl = w[g] >> kIdxBits;                // kind | pops << 2 | roles of the pops << 6 | hints << 18
-                if (Commutes<OPR>::value ? (ctl | 1u) == 3u : ctl == 2u) {
+                if (Commutes<DT, OPR>::value ? (ctl | 1u) == 3u : ctl == 2u) {
                     StageAcc<DT, N> x;                                // the common step: combine into the running value, no pops
                     x.load(r[g]);
                     top.template combine<OPR>(top, x);
                     continue;
                 }
-                if (AUX && (Commutes<OPR>::value ? (ctl | 1u) == (3u | kSecondBit) : ctl == (2u | kSecondBit))) {
+                if (AUX && (Commutes<DT, OPR>::value ? (ctl | 1u) == (3u | kSecondBit) : ctl == (2u | kSecondBit))) {
                     StageAcc<DT, N> x;                                // the same inside a sub-expression that needs no stack
                     x.load(r[g]);
                     side.template combine<OPR>(side, x);
                     continue;
                 }
-                if (!Commutes<OPR>::value && (ctl == 3u || (AUX && ctl == (3u | kSecondBit)))) {
+                if (!Commutes<DT, OPR>::value && (ctl == 3u || (AUX && ctl == (3u | kSecondBit)))) {
                     StageAcc<DT, N> x;                                // max, min: the operand is the held value, nothing popped
                     x.load(r[g]);
                     if (ctl == 3u) top.template combine<OPR>(x, top);
@@ -857,7 +861,7 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
                     } else {
                         StageAcc<DT, N> x;
                         x.load(r[g]);
-                        if (kind == 2u || Commutes<OPR>::value) side.template combine<OPR>(side, x);
+                        if (kind == 2u || Commutes<DT, OPR>::value) side.template combine<OPR>(side, x);
                         else side.template combine<OPR>(x, side);
                     }
                     if (!(ctl & kMergeBit)) continue;
@@ -865,7 +869,7 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
                     npop--;
                     const bool poppedHeld = (roles & 1u) != 0;
                     roles >>= 1;
-                    if (poppedHeld || Commutes<OPR>::value) top.template combine<OPR>(top, side);
+                    if (poppedHeld || Commutes<DT, OPR>::value) top.template combine<OPR>(top, side);
                     else top.template combine<OPR>(side, top);
                 } else {
                     if (kind == 1u) {
@@ -877,7 +881,7 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
                     } else {
                         StageAcc<DT, N> x;
                         x.load(r[g]);
-                        if (kind == 2u || Commutes<OPR>::value) top.template combine<OPR>(top, x);
+                        if (kind == 2u || Commutes<DT, OPR>::value) top.template combine<OPR>(top, x);
                         else top.template combine<OPR>(x, top);
                     }
                 }
@@ -887,7 +891,7 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
                     roles >>= 1;
                     StageAcc<DT, N> y;
                     y.pop(sp, tid, CT);
-                    if (poppedHeld || Commutes<OPR>::value) top.template combine<OPR>(y, top);
+                    if (poppedHeld || Commutes<DT, OPR>::value) top.template combine<OPR>(y, top);
                     else top.template combine<OPR>(top, y);
                 }
             }
@@ -989,7 +993,7 @@ rd_tree_direct_kernel(const __grid_constant__ TreeParams<true> a)
                     if (kind <= 1u) {
 #pragma unroll
                         for (int u = 0; u < U; u++) top[u] = x[k][u];
-                    } else if (kind == 2u || Commutes<OPR>::value) {
+                    } else if (kind == 2u || Commutes<DT, OPR>::value) {
 #pragma unroll
                         for (int u = 0; u < U; u++) combine_vec<DT, OPR, 4>(top[u], top[u], x[k][u]);
                     } else {
@@ -1006,7 +1010,7 @@ rd_tree_direct_kernel(const __grid_constant__ TreeParams<true> a)
                             const Vec<4> y = st[0][u];
 #pragma unroll
                             for (int d = 0; d + 1 < D; d++) st[d][u] = st[d + 1][u];
-                            if (poppedHeld || Commutes<OPR>::value) combine_vec<DT, OPR, 4>(top[u], y, top[u]);
+                            if (poppedHeld || Commutes<DT, OPR>::value) combine_vec<DT, OPR, 4>(top[u], y, top[u]);
                             else combine_vec<DT, OPR, 4>(top[u], top[u], y);
                         }
                     }
