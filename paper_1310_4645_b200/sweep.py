@@ -165,8 +165,9 @@ def main(argv=None):
     ap.add_argument("--allreduce", action="store_true",
                     help="instead of the sweep: time rd_allreduce (the reduce, then the broadcast of the root's result to every "
                          "process) for every p at the largest message size, uni-greedy at its tuned segment size, fp32 sum")
-    ap.add_argument("--variant", default="auto", choices=["auto", "stream", "paired"],
-                    help="tree-mode kernel: the library's choice, or the streaming kernel with one / two operand tiles per ring stage")
+    ap.add_argument("--variant", default="auto", choices=["auto", "stream", "paired", "direct"],
+                    help="tree-mode kernel: the library's choice, the streaming kernel with one / two operand tiles per ring stage, or "
+                         "the direct kernel (at most 8 processes; the library falls back to the streaming kernel where it does not apply)")
     args = ap.parse_args(argv)
     dev = torch.device("cuda", torch.cuda.current_device())
     sink = sys.stdout if args.out == "-" else open(args.out, "w")
@@ -201,7 +202,8 @@ def main(argv=None):
                 info = rd.rd_schedule_info(h)
                 rd.rd_schedule_upload(h)
                 if args.variant != "auto":
-                    rd.rd_schedule_set_tree_variant(h, rd.RD_TREE_STREAM if args.variant == "stream" else rd.RD_TREE_STREAM_PAIRED)
+                    rd.rd_schedule_set_tree_variant(h, {"stream": rd.RD_TREE_STREAM, "paired": rd.RD_TREE_STREAM_PAIRED,
+                                                        "direct": rd.RD_TREE_DIRECT}[args.variant])
                 try:
                     if args.faithful and p > 1:
                         x = arenas["fp32"][: p * n].view(p, n)
