@@ -143,10 +143,25 @@ template <int DT, int OPR> __device__ __forceinline__ unsigned long long combine
     }
 }
 
+// Two fp32 sums (products) in one instruction: sm_100's packed single-precision add (multiply) works on a pair of
+// registers, each half one IEEE operation rounded to nearest even like the scalar one, subnormals kept.
+template <int OPR> __device__ __forceinline__ void combine_pair_f32(uint32_t &r0, uint32_t &r1, uint32_t h0, uint32_t h1, uint32_t i0, uint32_t i1)
+{
+    if (OPR == OPR_SUM)
+        asm("{\n\t.reg .b64 a, b, c;\n\tmov.b64 a, {%2, %3};\n\tmov.b64 b, {%4, %5};\n\tadd.rn.f32x2 c, a, b;\n\tmov.b64 {%0, %1}, c;\n\t}"
+            : "=r"(r0), "=r"(r1) : "r"(h0), "r"(h1), "r"(i0), "r"(i1));
+    else
+        asm("{\n\t.reg .b64 a, b, c;\n\tmov.b64 a, {%2, %3};\n\tmov.b64 b, {%4, %5};\n\tmul.rn.f32x2 c, a, b;\n\tmov.b64 {%0, %1}, c;\n\t}"
+            : "=r"(r0), "=r"(r1) : "r"(h0), "r"(h1), "r"(i0), "r"(i1));
+}
+
 // A vector of V words: V elements of a 4-byte type, V / 2 of an 8-byte type.  r may be held or in.
 template <int DT, int OPR, int V> __device__ __forceinline__ void combine_vec(Vec<V> &r, const Vec<V> &held, const Vec<V> &in)
 {
-    if constexpr (ElemWords<DT>::value == 1) {
+    if constexpr (DT == DT_FP32 && (OPR == OPR_SUM || OPR == OPR_PROD) && V % 2 == 0) {
+#pragma unroll
+        for (int v = 0; v < V; v += 2) combine_pair_f32<OPR>(r.w[v], r.w[v + 1], held.w[v], held.w[v + 1], in.w[v], in.w[v + 1]);
+    } else if constexpr (ElemWords<DT>::value == 1) {
 #pragma unroll
         for (int v = 0; v < V; v++) r.w[v] = combine<DT, OPR>(held.w[v], in.w[v]);
     } else {
@@ -1082,7 +1097,8 @@ cudaError_t launch_stream_kernel(const PRM &prm, int ops_per_stage, int consumer
 {
     if (ops_per_stage == 2 && consumer_warps == 4) return launch_stream_kernel<DT, OPR, 2, 4>(prm, n_ctas, device, stream);
     if (ops_per_stage == 1 && consumer_warps == 4) return launch_stream_kernel<DT, OPR, 1, 4>(prm, n_ctas, device, stream);
-    if (ops_per_stage == 1 && consumer_warps == 8) return launch_stream_kernel<DT, OPR, 1, 8>(prm, n_ctas, device, stream);
+    if constexpr (!Wide<DT>::half)       // (elements widened to fp32 always run with four consumer warps)
+        if (ops_per_stage == 1 && consumer_warps == 8) return launch_stream_kernel<DT, OPR, 1, 8>(prm, n_ctas, device, stream);
     return cudaErrorInvalidValue;
 }
 
