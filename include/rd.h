@@ -81,7 +81,8 @@ typedef enum { RD_PORT_UNI = 0, RD_PORT_BI = 1 } rd_port_t;   /* Section II */
  * settles the sign of a zero result; fp32 and fp64 sum and product are one IEEE
  * round-to-nearest operation per combine (subnormals kept, infinities as IEEE has them).  A NaN, whether an
  * input or born of inf - inf or inf * 0, comes out as a NaN of the GPU's own bit pattern (0x7fffffff), which
- * need not be the pattern another machine produces; under max and min a NaN never wins a comparison. */
+ * need not be the pattern another machine produces; under max and min every comparison with a NaN is false,
+ * so an incoming NaN never replaces the held value and a held NaN is never replaced. */
 typedef enum { RD_SUM = 0, RD_MAX = 1, RD_MIN = 2, RD_PROD = 3 } rd_op_t;
 /* Element type.  The paper's implementation is restricted to int and notes that the restriction is
  * not a consequence of the algorithm (Fig. 2 caption).  With an 8-byte type no segment may begin
