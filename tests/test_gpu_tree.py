@@ -608,6 +608,71 @@ def test_randomized_shapes_order_free_results():
             rd.rd_destroy(h)
 
 
+def test_randomized_shapes_types_and_operations_against_the_oracle():
+    """150 seeded random cases over every element type, operation and schedule, with process counts, message
+    lengths and segment sizes that respect no vector or tile boundary: the oracle's bytes, exactly.  A third of the
+    fp32 cases carry signed zeros, subnormals and the smallest normal number among their inputs (no infinities:
+    inf - inf would be a NaN, whose bit pattern is the machine's own)."""
+    rng = np.random.default_rng(4645)
+    special = torch.tensor([0.0, -0.0, 1.0, -1.0, 2.0 ** -149, -(2.0 ** -149), 2.0 ** -126, 0.5, 1.5, -2.5], device="cuda")
+    esizes = {"fp32": 4, "int32": 4, "bf16": 2, "fp16": 2, "fp64": 8, "int64": 8}
+    done = 0
+    for case in range(150):
+        _, algo, port = SCHEDULES[int(rng.integers(len(SCHEDULES)))]
+        p = int(rng.choice([1, 2, 3, 4, 5, 8, 9, 16, 17, 33, 64, 100, 128, 257, 300]))
+        dt = str(rng.choice(list(esizes)))
+        esize = esizes[dt]
+        words = int(rng.integers(1, 20000))                       # 4-byte words of a message
+        n = words * (4 // esize) if esize <= 4 else words // 2 + 1
+        seg_words = int(rng.integers(1, words + 1)) if rng.random() < 0.5 else int(rng.integers(1, 700))
+        if esize == 8:
+            seg_words = max(2, seg_words // 2 * 2)                # no segment may begin inside an element
+        msg_bytes, op = n * esize, str(rng.choice(list(OPS)))
+        seg_bytes = min(seg_words * 4, msg_bytes)
+        g = torch.Generator("cuda").manual_seed(case)
+        if dt in ("int32", "int64"):
+            x = torch.randint(-(1 << 20), 1 << 20, (p, n), device="cuda", generator=g, dtype=torch.int32 if dt == "int32" else torch.int64)
+            if op == "prod":
+                x = x % 7 - 3
+        else:
+            x = torch.randn(p, n, device="cuda", generator=g, dtype=torch.float64 if dt == "fp64" else torch.float32)
+            if op == "prod":
+                x = x.abs() * 0.5 + 0.75                           # magnitudes around 1: no overflow, no inf * 0
+            else:
+                x = x * 10.0 ** torch.randint(-4, 5, x.shape, device="cuda", generator=g)
+                if dt == "fp32" and rng.random() < 0.33:
+                    pick = torch.rand(x.shape, device="cuda", generator=g) < 0.3
+                    x = torch.where(pick, special[torch.randint(0, len(special), x.shape, device="cuda", generator=g)], x)
+            if dt == "bf16":
+                x = x.to(torch.bfloat16)
+            if dt == "fp16":
+                x = x.clamp(-6e4, 6e4).to(torch.float16)
+        x = x.contiguous()
+        out = torch.empty(n, dtype=x.dtype, device="cuda")
+        try:
+            h = rd.rd_schedule_create(algo, port, p, msg_bytes, seg_bytes, *M1)
+        except rd.RdError:
+            continue                                               # (a butterfly whose halving would cut an 8-byte element)
+        try:
+            rd.rd_reduce(h, x, out, OPS[op])
+            torch.cuda.synchronize()
+        except rd.RdError as e:
+            assert e.status == rd.RD_ERR_INVALID_ARG and esize == 8, (case, e.status)
+            continue
+        finally:
+            rd.rd_destroy(h)
+        ev, off, _ = oracle_schedule(algo, port, p, msg_bytes, seg_bytes, *M1)
+        off = off // 2 if esize == 8 else off * (4 // esize)       # boundaries in elements of the type
+        if dt in ("bf16", "fp16"):
+            want = O.reduce(ev, x.view(torch.int16).cpu().numpy().view(np.uint16), off, op, half=dt)
+            got = out.view(torch.int16).cpu().numpy().view(np.uint16)
+        else:
+            want, got = O.reduce(ev, x.cpu().numpy(), off, op), out.cpu().numpy()
+        assert got.tobytes() == want.tobytes(), (case, algo, p, dt, op, n, seg_bytes)
+        done += 1
+    assert done >= 130
+
+
 def test_batch_equals_separate_calls_and_keeps_stream_order():
     """Independent jobs issued together: bit-identical to one rd_reduce per job; what follows the batch on
     the stream sees every result, what precedes it is seen by every job."""
