@@ -394,13 +394,17 @@ int stage_ops(int acc_words_per_word, int tree_variant, int stack_depth)
     return acc_words_per_word > 1 && stack_depth >= 2 ? 2 : 1;
 }
 // Consumer warps of the streaming kernel: 8 with two vectors of a tile each, or 4 with four (two when two tiles
-// share a stage).  Fewer warps with more vectors each spend fewer issue slots per byte; that pays for the 16-bit
-// types, which have twice the elements per byte, and for deep stacks, where shared memory leaves room for two
-// thread blocks per SM only (measured, fp32 sum, p = 256, GB/s, 8 against 4 warps: binomial 6747 / 7104,
-// uni-greedy 7109 / 7321; p = 2 ... 64: equal within 1 %).
-int stage_warps(int acc_words_per_word, int ops_per_stage, int stack_depth)
+// share a stage).  Fewer warps with more vectors each spend fewer issue slots per byte, and with fewer instructions
+// the SM clock settles higher under the board's power cap.  That pays for the 16-bit types, which have twice the
+// elements per byte, for deep stacks, where shared memory leaves room for two thread blocks per SM only (measured,
+// fp32 sum, p = 256, GB/s, 8 against 4 warps: binomial 6747 / 7104, uni-greedy 7109 / 7321), and from 16 processes
+// on (p = 32, 1 GiB messages, a box whose SM clock is 1.6 GHz under the cap: uni- and bi-greedy, sum and max together
+// 7092 / 7171, bi-greedy max 6882 / 7017; the batch of p = 64 with 4 MiB messages 7141 / 7172; at 1.85 GHz the two are
+// level).  Fewer processes keep 8 warps: their launches are short, and a tile is finished sooner by more threads
+// (p = 8, 64 KiB ... 1 MiB messages: 4 warps 4-5 % behind).
+int stage_warps(int acc_words_per_word, int ops_per_stage, int stack_depth, int p)
 {
-    return ops_per_stage >= 2 || acc_words_per_word > 1 || stack_depth >= 6 ? 4 : 8;
+    return ops_per_stage >= 2 || acc_words_per_word > 1 || stack_depth >= 6 || p >= 16 ? 4 : 8;
 }
 size_t elem_bytes(rd_dtype_t dtype) { return (dtype == RD_INT64 || dtype == RD_FP64) ? 8 : is_half(dtype) ? 2 : 4; }
 
@@ -434,7 +438,7 @@ int reduce_tree(rd_schedule *s, const void *const *d_inputs, void *d_out, size_t
     TreeLaunch l{};
     l.vec = wide ? 4 : 1;
     l.ops_per_stage = stage_ops(acc_words(dtype, op), s->tree_variant, s->progs.shared_depth);
-    l.consumer_warps = stage_warps(acc_words(dtype, op), l.ops_per_stage, s->progs.shared_depth);
+    l.consumer_warps = stage_warps(acc_words(dtype, op), l.ops_per_stage, s->progs.shared_depth, s->p);
     if (int rc = tiles_for(s, wide ? tiles_key(l.ops_per_stage) : 1, &l.tiles, &l.n_tiles)) return rc;
     const DeviceTables::StreamPlan *plan = nullptr;
     if (wide)
@@ -661,7 +665,9 @@ int reduce_batch_fused(size_t n_jobs, rd_schedule_t *const *schedules, const voi
     DeviceTables &d0 = schedules[0]->dev;
     const int stageElems = d0.stage_elems;
     int ctasPerSm = 1, stages = 2;
-    const int consumerWarps = stage_warps(acc_words(dtype, op), opsPerStage, depth);
+    int mostProcs = 0;
+    for (size_t j = 0; j < n_jobs; j++) mostProcs = std::max(mostProcs, schedules[j]->p);
+    const int consumerWarps = stage_warps(acc_words(dtype, op), opsPerStage, depth, mostProcs);
     bool pushy = false;
     for (size_t j = 0; j < n_jobs; j++) pushy = pushy || many_pushes(schedules[j]);
     stream_shape(depth, acc_words(dtype, op), opsPerStage, pushy, d0.smem_per_sm, stageElems, total, d0.sm_count, &ctasPerSm, &stages);
@@ -1074,7 +1080,7 @@ int rd_schedule_tree_shape(rd_schedule_t *s, int *variant, int *blocks_per_sm, i
                             (s->tree_variant == RD_TREE_DIRECT || (s->tree_variant == RD_TREE_AUTO && s->p <= kDirectAutoProcs));
         if (variant) *variant = direct ? RD_TREE_DIRECT : opsPerStage == 2 ? RD_TREE_STREAM_PAIRED : RD_TREE_STREAM;
         const DeviceTables::StreamPlan *plan = nullptr;
-        if (int rc = stream_plan(s, 1, opsPerStage, stage_warps(1, opsPerStage, s->progs.shared_depth), &plan)) return rc;
+        if (int rc = stream_plan(s, 1, opsPerStage, stage_warps(1, opsPerStage, s->progs.shared_depth, s->p), &plan)) return rc;
         if (blocks_per_sm) *blocks_per_sm = direct ? direct_blocks_per_sm(s->p) : plan->ctas_per_sm;
         if (ring_stages) *ring_stages = direct ? 0 : plan->stages;
         if (n_tiles) *n_tiles = l.n_tiles;
