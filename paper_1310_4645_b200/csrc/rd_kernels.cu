@@ -604,8 +604,88 @@ struct TileSource {
     }
 };
 
+// ---- arithmetic of the streaming kernel's accumulators.
+// A consumer thread's running value lives in registers for the whole life of the thread, across the branches of the
+// interpreter.  Written as ordinary assignments, every branch that leaves it alone (or changes it) ends in a block of
+// register-to-register copies that bring "the new value" to the place the join expects (a third of all executed
+// instructions were such copies).  So every write to an accumulator is one instruction whose destination is tied to
+// the accumulator's own register (an asm operand that is input and output at once): the value never changes place.
+//   acc_word<ADT, OPR, HELD>(t, x)          t = combine(t, x) (HELD: t is the held operand) or combine(x, t); one word
+//   acc_pair<ADT, OPR, HELD>(t0, t1, x0, x1)  the same for two words: one 8-byte element, or two fp32 values under sum
+//                                           and product (sm_100's packed add and multiply: two IEEE operations, each
+//                                           rounded to nearest even like the scalar one, subnormals kept)
+__device__ __forceinline__ void set_word(uint32_t &t, uint32_t x) { asm("mov.b32 %0, %1;" : "+r"(t) : "r"(x)); }
+
+template <int ADT, int OPR, bool HELD> __device__ __forceinline__ void acc_word(uint32_t &t, uint32_t x)
+{
+    if constexpr (ADT == DT_INT32) {
+        if (OPR == OPR_SUM) asm("add.s32 %0, %0, %1;" : "+r"(t) : "r"(x));                  // wraps modulo 2^32
+        else if (OPR == OPR_PROD) asm("mul.lo.s32 %0, %0, %1;" : "+r"(t) : "r"(x));
+        else if (OPR == OPR_MAX) asm("max.s32 %0, %0, %1;" : "+r"(t) : "r"(x));
+        else asm("min.s32 %0, %0, %1;" : "+r"(t) : "r"(x));
+    } else if constexpr (ADT == DT_BF16_PICK || ADT == DT_FP16_PICK) {
+        // two 16-bit elements per word; `wins`: all ones in the half where the incoming element wins (never on a tie)
+        const uint32_t held = HELD ? t : x, in = HELD ? x : t;
+        unsigned wins;
+        if (ADT == DT_BF16_PICK) {
+            const __nv_bfloat162 h = *reinterpret_cast<const __nv_bfloat162 *>(&held), i = *reinterpret_cast<const __nv_bfloat162 *>(&in);
+            wins = OPR == OPR_MAX ? __hgt2_mask(i, h) : __hlt2_mask(i, h);
+        } else {
+            const __half2 h = *reinterpret_cast<const __half2 *>(&held), i = *reinterpret_cast<const __half2 *>(&in);
+            wins = OPR == OPR_MAX ? __hgt2_mask(i, h) : __hlt2_mask(i, h);
+        }
+        // t = wins ? in : held, bit by bit (lop3 0xCA: a ? b : c)
+        if (HELD) asm("lop3.b32 %0, %1, %2, %0, 0xCA;" : "+r"(t) : "r"(wins), "r"(x));
+        else asm("lop3.b32 %0, %1, %0, %2, 0xCA;" : "+r"(t) : "r"(wins), "r"(x));
+    } else {
+        static_assert(ADT == DT_FP32, "a 4-byte type");
+        if (OPR == OPR_SUM) asm("add.rn.f32 %0, %0, %1;" : "+r"(t) : "r"(x));               // one IEEE add, never contracted
+        else if (OPR == OPR_PROD) asm("mul.rn.f32 %0, %0, %1;" : "+r"(t) : "r"(x));
+        else if (HELD) {                                                                    // (x > t) ? x : t   (min: <)
+            if (OPR == OPR_MAX) asm("{\n\t.reg .pred p;\n\tsetp.gt.f32 p, %1, %0;\n\tselp.b32 %0, %1, %0, p;\n\t}" : "+r"(t) : "r"(x));
+            else asm("{\n\t.reg .pred p;\n\tsetp.lt.f32 p, %1, %0;\n\tselp.b32 %0, %1, %0, p;\n\t}" : "+r"(t) : "r"(x));
+        } else {                                                                            // (t > x) ? t : x
+            if (OPR == OPR_MAX) asm("{\n\t.reg .pred p;\n\tsetp.gt.f32 p, %0, %1;\n\tselp.b32 %0, %0, %1, p;\n\t}" : "+r"(t) : "r"(x));
+            else asm("{\n\t.reg .pred p;\n\tsetp.lt.f32 p, %0, %1;\n\tselp.b32 %0, %0, %1, p;\n\t}" : "+r"(t) : "r"(x));
+        }
+    }
+}
+
+#define RD_PAIR_ASM(body) asm("{\n\t.reg .b64 a, b;\n\t.reg .pred p;\n\tmov.b64 a, {%0, %1};\n\tmov.b64 b, {%2, %3};\n\t" body "\n\tmov.b64 {%0, %1}, a;\n\t}" \
+                              : "+r"(t0), "+r"(t1) : "r"(x0), "r"(x1))
+#define RD_PAIR_ASM_F64(body) asm("{\n\t.reg .f64 a, b;\n\t.reg .pred p;\n\tmov.b64 a, {%0, %1};\n\tmov.b64 b, {%2, %3};\n\t" body "\n\tmov.b64 {%0, %1}, a;\n\t}" \
+                                  : "+r"(t0), "+r"(t1) : "r"(x0), "r"(x1))
+template <int ADT, int OPR, bool HELD>
+__device__ __forceinline__ void acc_pair(uint32_t &t0, uint32_t &t1, uint32_t x0, uint32_t x1)
+{
+    if constexpr (ADT == DT_FP32) {
+        static_assert(OPR == OPR_SUM || OPR == OPR_PROD, "packed single precision: add and multiply");
+        if (OPR == OPR_SUM) RD_PAIR_ASM("add.rn.f32x2 a, a, b;");
+        else RD_PAIR_ASM("mul.rn.f32x2 a, a, b;");
+    } else if constexpr (ADT == DT_INT64) {                    // low word first
+        if (OPR == OPR_SUM) RD_PAIR_ASM("add.s64 a, a, b;");                              // wraps modulo 2^64
+        else if (OPR == OPR_PROD) RD_PAIR_ASM("mul.lo.s64 a, a, b;");
+        else if (OPR == OPR_MAX) RD_PAIR_ASM("max.s64 a, a, b;");
+        else RD_PAIR_ASM("min.s64 a, a, b;");
+    } else {
+        static_assert(ADT == DT_FP64, "an 8-byte type");
+        if (OPR == OPR_SUM) RD_PAIR_ASM_F64("add.rn.f64 a, a, b;");
+        else if (OPR == OPR_PROD) RD_PAIR_ASM_F64("mul.rn.f64 a, a, b;");
+        else if (HELD) {                                                                    // (x > t) ? x : t   (min: <)
+            if (OPR == OPR_MAX) RD_PAIR_ASM_F64("setp.gt.f64 p, b, a;\n\tselp.f64 a, b, a, p;");
+            else RD_PAIR_ASM_F64("setp.lt.f64 p, b, a;\n\tselp.f64 a, b, a, p;");
+        } else {                                                                            // (t > x) ? t : x
+            if (OPR == OPR_MAX) RD_PAIR_ASM_F64("setp.gt.f64 p, a, b;\n\tselp.f64 a, a, b, p;");
+            else RD_PAIR_ASM_F64("setp.lt.f64 p, a, b;\n\tselp.f64 a, a, b, p;");
+        }
+    }
+}
+#undef RD_PAIR_ASM
+#undef RD_PAIR_ASM_F64
+
 // What a consumer thread carries for its N 128-bit vectors of an operand tile: the vectors themselves, or
-// (bf16, fp16) their elements widened to fp32, twice as many words.
+// (bf16, fp16) their elements widened to fp32, twice as many words.  Created once per thread (zero), then only
+// written through the tied-operand instructions above.
 template <int DT, int N> struct StageAcc {
     static constexpr int W = Wide<DT>::W;
     static constexpr int ADT = Wide<DT>::ADT;
@@ -617,6 +697,7 @@ template <int DT, int N> struct StageAcc {
 #pragma unroll
             for (int e = 0; e < 4; e++) v[k].w[e] = 0;
     }
+    // *this = the operand whose vectors are r
     __device__ __forceinline__ void load(const uint4 (&r)[N])
     {
 #pragma unroll
@@ -626,14 +707,39 @@ template <int DT, int N> struct StageAcc {
 #pragma unroll
             for (int k = 0; k < W; k++)
 #pragma unroll
-                for (int e = 0; e < 4; e++) v[n * W + k].w[e] = a.w[4 * k + e];
+                for (int e = 0; e < 4; e++) set_word(v[n * W + k].w[e], a.w[4 * k + e]);
         }
     }
-    // *this = combine(held, in); *this may be either of them
-    template <int OPR> __device__ __forceinline__ void combine(const StageAcc &held, const StageAcc &in)
+    // one 128-bit vector of operand words: *this[k] = combine(*this[k], x) (HELD) or combine(x, *this[k])
+    template <int OPR, bool HELD> __device__ __forceinline__ void accumulate_vec(int k, const Vec<4> &x)
+    {
+        if constexpr (ElemWords<ADT>::value == 2 || (ADT == DT_FP32 && (OPR == OPR_SUM || OPR == OPR_PROD))) {
+#pragma unroll
+            for (int e = 0; e < 4; e += 2) acc_pair<ADT, OPR, HELD>(v[k].w[e], v[k].w[e + 1], x.w[e], x.w[e + 1]);
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; e++) acc_word<ADT, OPR, HELD>(v[k].w[e], x.w[e]);
+        }
+    }
+    // *this = combine(*this, operand) (HELD: *this is the held one) or combine(operand, *this); the operand as it
+    // comes from the ring, or another accumulator
+    template <int OPR, bool HELD> __device__ __forceinline__ void accumulate(const uint4 (&r)[N])
     {
 #pragma unroll
-        for (int k = 0; k < N * W; k++) combine_vec<ADT, OPR, 4>(v[k], held.v[k], in.v[k]);
+        for (int n = 0; n < N; n++) {
+            const Vec<4> m = {{r[n].x, r[n].y, r[n].z, r[n].w}};
+            const Vec<4 * W> a = widen<DT, 4>(m);
+#pragma unroll
+            for (int k = 0; k < W; k++) {
+                const Vec<4> x = {{a.w[4 * k], a.w[4 * k + 1], a.w[4 * k + 2], a.w[4 * k + 3]}};
+                accumulate_vec<OPR, HELD>(n * W + k, x);
+            }
+        }
+    }
+    template <int OPR, bool HELD> __device__ __forceinline__ void accumulate(const StageAcc &in)
+    {
+#pragma unroll
+        for (int k = 0; k < N * W; k++) accumulate_vec<OPR, HELD>(k, in.v[k]);
     }
     // one stack level (shared-memory address): [vector][consumer thread]
     __device__ __forceinline__ void push(uint32_t level, uint32_t tid, uint32_t threads) const
@@ -641,12 +747,14 @@ template <int DT, int N> struct StageAcc {
 #pragma unroll
         for (int k = 0; k < N * W; k++) sts128(level + (uint32_t(k) * threads + tid) * 16u, make_uint4(v[k].w[0], v[k].w[1], v[k].w[2], v[k].w[3]));
     }
-    __device__ __forceinline__ void pop(uint32_t level, uint32_t tid, uint32_t threads)
+    // *this = combine(popped, *this) (POPPED_HELD) or combine(*this, popped), the popped value read from a stack level
+    template <int OPR, bool POPPED_HELD> __device__ __forceinline__ void pop_accumulate(uint32_t level, uint32_t tid, uint32_t threads)
     {
 #pragma unroll
         for (int k = 0; k < N * W; k++) {
             const uint4 y = lds128(level + (uint32_t(k) * threads + tid) * 16u);
-            v[k].w[0] = y.x; v[k].w[1] = y.y; v[k].w[2] = y.z; v[k].w[3] = y.w;
+            const Vec<4> x = {{y.x, y.y, y.z, y.w}};
+            accumulate_vec<OPR, !POPPED_HELD>(k, x);
         }
     }
     __device__ __forceinline__ void result(Vec<4> (&o)[N]) const
@@ -813,57 +921,80 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
     uint32_t k = 0;
     uint32_t tile = tile_at(&tileq, 0, &abort_flag, a.status);
     Jobs jobs(a, tile, tile != kNoTile);
+    StageAcc<DT, N> top, side;      // the running value; the value of a sub-expression that needs no stack.  Every tile's
+    top.clear();                    // program begins with a load, so nothing of a tile's values outlives the tile
+    side.clear();
     for (; tile != kNoTile; tile = tile_at(&tileq, ++k, &abort_flag, a.status)) {
         jobs.seek(tile);
         const int p = jobs.p();
         const TileDesc td = jobs.tile(tile);
         const uint32_t len = td.len & kLenMask;                       // padded to whole 128-bit vectors
-        StageAcc<DT, N> top, side;                                    // the running value; a sub-expression that needs no stack
-        top.clear();
-        side.clear();
         uint32_t sp = stack;                                          // address of the next free stack level
-        for (int i = 0; i < p; i += G) {
-            if (!mbar_wait_at(full + uint32_t(stage) * 8u, phase, &abort_flag)) {
-                if (!abort_flag) { atomicCAS(a.status, 0, -5); abort_flag = 1; }
-                return;
-            }
-            // the step's operation words, then its data: every thread reads its N vectors of each operand (threads
-            // beyond a short tile's end read stale bytes of the stage and never store their results)
+        // The operations of a tile, G to a ring stage.  Most of them only combine their operand into the running value
+        // (in the steady state of a pipelined schedule all but a few per tile do): those are taken by the inner loop,
+        // which changes nothing but one of the two accumulators and the ring position; an operation that loads, pushes
+        // or pops leaves the inner loop with its stage already in registers and is done by the general code below it.
+        int i = 0;
+        while (i < p) {
             uint32_t w[G];
-#pragma unroll
-            for (int g = 0; g < G; g++)
-                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w[g]) : "r"(stepWords + uint32_t(stage * G + g) * 4u) : "memory");
-            const uint32_t stageAddr = ring + uint32_t(stage) * kStageBytes + tid * 16u;
             uint4 r[G][N];
+            bool general = false;
+            do {
+                if (!mbar_wait_at(full + uint32_t(stage) * 8u, phase, &abort_flag)) {
+                    if (!abort_flag) { atomicCAS(a.status, 0, -5); abort_flag = 1; }
+                    return;
+                }
+                // the step's operation words, then its data: every thread reads its N vectors of each operand (threads
+                // beyond a short tile's end read stale bytes of the stage and never store their results)
 #pragma unroll
-            for (int g = 0; g < G; g++)
+                for (int g = 0; g < G; g++)
+                    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w[g]) : "r"(stepWords + uint32_t(stage * G + g) * 4u) : "memory");
+                const uint32_t stageAddr = ring + uint32_t(stage) * kStageBytes + tid * 16u;
 #pragma unroll
-                for (int n = 0; n < N; n++) r[g][n] = lds128(stageAddr + uint32_t(g) * kSubBytes + uint32_t(n) * CT * 16u);
-            // the stage's data is in registers: hand the stage back to the producer
-            __syncwarp();
-            if (lane == 0) mbar_arrive_at(empty + uint32_t(stage) * 8u);
-            if (++stage == S) { stage = 0; phase ^= 1u; }
+                for (int g = 0; g < G; g++)
+#pragma unroll
+                    for (int n = 0; n < N; n++) r[g][n] = lds128(stageAddr + uint32_t(g) * kSubBytes + uint32_t(n) * CT * 16u);
+                // the stage's data is in registers: hand the stage back to the producer
+                __syncwarp();
+                if (lane == 0) mbar_arrive_at(empty + uint32_t(stage) * 8u);
+                if (++stage == S) { stage = 0; phase ^= 1u; }
+                bool simple = G == 1;           // (two operations to a stage: the general code takes them, one after the other)
+#pragma unroll
+                for (int g = 0; g < G; g++) {
+                    if (g > 0 && i + g >= p) break;
+                    // combine the operand (incoming or held) into the running value, or into the sub-expression's, nothing popped
+                    simple = simple && (((w[g] >> kIdxBits) & ~(AUX ? kSecondBit : 0u)) | 1u) == 3u;
+                }
+                if (!simple) { general = true; break; }
+#pragma unroll
+                for (int g = 0; g < G; g++) {
+                    if (g > 0 && i + g >= p) break;
+                    const bool held = Commutes<DT, OPR>::value || ((w[g] >> kIdxBits) & 1u) == 0u;   // max, min: else the operand is the held value
+                    if (AUX && ((w[g] >> kIdxBits) & kSecondBit)) {
+                        if (held) side.template accumulate<OPR, true>(r[g]);
+                        else side.template accumulate<OPR, false>(r[g]);
+                    } else {
+                        if (held) top.template accumulate<OPR, true>(r[g]);
+                        else top.template accumulate<OPR, false>(r[g]);
+                    }
+                }
+                i += G;
+            } while (i < p);
+            if (!general) break;
 #pragma unroll
             for (int g = 0; g < G; g++) {
                 if (g > 0 && i + g >= p) break;
                 const uint32_t ctl = w[g] >> kIdxBits;                // kind | pops << 2 | roles of the pops << 6 | hints << 18
-                if (Commutes<DT, OPR>::value ? (ctl | 1u) == 3u : ctl == 2u) {
-                    StageAcc<DT, N> x;                                // the common step: combine into the running value, no pops
-                    x.load(r[g]);
-                    top.template combine<OPR>(top, x);
-                    continue;
-                }
-                if (AUX && (Commutes<DT, OPR>::value ? (ctl | 1u) == (3u | kSecondBit) : ctl == (2u | kSecondBit))) {
-                    StageAcc<DT, N> x;                                // the same inside a sub-expression that needs no stack
-                    x.load(r[g]);
-                    side.template combine<OPR>(side, x);
-                    continue;
-                }
-                if (!Commutes<DT, OPR>::value && (ctl == 3u || (AUX && ctl == (3u | kSecondBit)))) {
-                    StageAcc<DT, N> x;                                // max, min: the operand is the held value, nothing popped
-                    x.load(r[g]);
-                    if (ctl == 3u) top.template combine<OPR>(x, top);
-                    else side.template combine<OPR>(x, side);
+                if (G > 1 && ((ctl & ~(AUX ? kSecondBit : 0u)) | 1u) == 3u) {
+                    // the common step: combine into the running value, or into the sub-expression's, no pops
+                    const bool held = Commutes<DT, OPR>::value || (ctl & 1u) == 0u;
+                    if (AUX && (ctl & kSecondBit)) {
+                        if (held) side.template accumulate<OPR, true>(r[g]);
+                        else side.template accumulate<OPR, false>(r[g]);
+                    } else {
+                        if (held) top.template accumulate<OPR, true>(r[g]);
+                        else top.template accumulate<OPR, false>(r[g]);
+                    }
                     continue;
                 }
                 const uint32_t kind = ctl & 3u;
@@ -871,45 +1002,34 @@ rd_tree_stream_kernel(const __grid_constant__ PRM a)
                 uint32_t roles = ctl >> 6;
                 if (AUX && (ctl & kSecondBit)) {
                     // a sub-expression that needs no stack: it is evaluated in `side`, the running value stays put
-                    if (kind == 1u) {
-                        side.load(r[g]);
-                    } else {
-                        StageAcc<DT, N> x;
-                        x.load(r[g]);
-                        if (kind == 2u || Commutes<DT, OPR>::value) side.template combine<OPR>(side, x);
-                        else side.template combine<OPR>(x, side);
-                    }
+                    if (kind == 1u) side.load(r[g]);
+                    else if (kind == 2u || Commutes<DT, OPR>::value) side.template accumulate<OPR, true>(r[g]);
+                    else side.template accumulate<OPR, false>(r[g]);
                     if (!(ctl & kMergeBit)) continue;
                     // its end: what a stack machine would pop first is the running value, its current value is `side`
                     npop--;
                     const bool poppedHeld = (roles & 1u) != 0;
                     roles >>= 1;
-                    if (poppedHeld || Commutes<DT, OPR>::value) top.template combine<OPR>(top, side);
-                    else top.template combine<OPR>(side, top);
+                    if (poppedHeld || Commutes<DT, OPR>::value) top.template accumulate<OPR, true>(side);
+                    else top.template accumulate<OPR, false>(side);
                 } else {
                     if (kind == 1u) {
                         top.push(sp, tid, CT);
                         sp += kLevelBytes;
                     }
-                    if (kind <= 1u) {
-                        top.load(r[g]);
-                    } else {
-                        StageAcc<DT, N> x;
-                        x.load(r[g]);
-                        if (kind == 2u || Commutes<DT, OPR>::value) top.template combine<OPR>(top, x);
-                        else top.template combine<OPR>(x, top);
-                    }
+                    if (kind <= 1u) top.load(r[g]);
+                    else if (kind == 2u || Commutes<DT, OPR>::value) top.template accumulate<OPR, true>(r[g]);
+                    else top.template accumulate<OPR, false>(r[g]);
                 }
                 while (npop--) {
                     sp -= kLevelBytes;
                     const bool poppedHeld = (roles & 1u) != 0;
                     roles >>= 1;
-                    StageAcc<DT, N> y;
-                    y.pop(sp, tid, CT);
-                    if (poppedHeld || Commutes<DT, OPR>::value) top.template combine<OPR>(y, top);
-                    else top.template combine<OPR>(top, y);
+                    if (poppedHeld || Commutes<DT, OPR>::value) top.template pop_accumulate<OPR, true>(sp, tid, CT);
+                    else top.template pop_accumulate<OPR, false>(sp, tid, CT);
                 }
             }
+            i += G;
         }
         bool live[N];
 #pragma unroll
